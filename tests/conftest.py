@@ -1,0 +1,64 @@
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def pytest_configure(config):
+    config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+
+
+def pytest_collection_modifyitems(config, items):
+    try:
+        import torch
+
+        have_gpu = torch.cuda.is_available()
+    except Exception:  # pragma: no cover
+        have_gpu = False
+    if have_gpu:
+        return
+    skip = pytest.mark.skip(reason="no CUDA device")
+    for item in items:
+        if "gpu" in item.keywords:
+            item.add_marker(skip)
+
+
+def read_golden(path):
+    """Parse tests/golden/*.txt blocks into dicts (name, shape, sampling, mask, sq)."""
+    import numpy as np
+
+    cases, cur = [], {}
+    with open(path) as fh:
+        for raw in fh:
+            line = raw.strip()
+            if line.startswith("#"):
+                continue
+            if not line:
+                if cur:
+                    cases.append(cur)
+                    cur = {}
+                continue
+            key, *vals = line.split()
+            if key == "name":
+                cur["name"] = vals[0]
+            elif key == "shape":
+                cur["shape"] = tuple(int(v) for v in vals)
+            elif key == "sampling":
+                cur["sampling"] = tuple(float(v) for v in vals)
+            elif key == "mask":
+                cur["mask"] = np.array([int(v) for v in vals], dtype=np.uint8)
+            elif key == "sq":
+                cur["sq"] = np.array([float(v) for v in vals], dtype=np.float64)
+    if cur:
+        cases.append(cur)
+    for c in cases:
+        c["mask"] = c["mask"].reshape((1, 1) + c["shape"])
+        c["sq"] = c["sq"].reshape((1, 1) + c["shape"])
+    return cases
+
+
+GOLDEN_DIR = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
