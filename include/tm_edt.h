@@ -1,0 +1,127 @@
+/*
+ * tm_edt -- exact Euclidean distance transform on one NVIDIA B200 (sm_100a), C ABI.
+ *
+ * Operation (paper, Section 2.1 "Covered transforms", paragraph "Distance transforms", and
+ * Section 2.3.2 "Distance-transform kernels"): every nonzero (foreground) element of a batched
+ * mask is labelled with its Euclidean distance to the nearest zero (background) element of the
+ * same image, with scipy.ndimage.distance_transform_edt semantics: per-axis sampling, optional
+ * nearest-background index map (Section 2.3.2, "indices are propagated through the passes on
+ * request"), inputs shaped (B, C, Spatial...) with 1 <= spatial rank <= 8 (Section 2.2.1
+ * "API surface"), pre-allocated outputs, work issued on the caller's stream (Section 2.2.4,
+ * runtime tests).
+ *
+ * For every image (b, c), with Z the set of its zero voxels and w_k the sampling of spatial axis k:
+ *
+ *     sq(x)   = min over z in Z of  sum_k ( w_k * (x_k - z_k) )^2
+ *     dist(x) = sqrt(sq(x))                      -> out_dist   (float32)
+ *     sq(x) with every w_k == 1                  -> out_sqdist (int64, exact)
+ *     some z attaining the minimum               -> out_indices (int64, one plane per spatial axis)
+ *
+ * An image with no zero voxel has no nearest background: its out_dist is +inf, its out_sqdist is
+ * INT64_MAX and every component of out_indices is -1.  This is decided per image.  (The paper
+ * mentions SciPy's virtual out-of-bounds convention for that case; this library defines the
+ * result as infinite instead.)  When several background voxels are equally near, which one
+ * out_indices names is unspecified; it always names one at the minimal distance, and a background
+ * voxel names itself.
+ *
+ * All entry points are thread-safe and keep no state between calls apart from cached device
+ * attributes.  Nothing is thrown and no device trap is ever raised: every problem is a return code,
+ * and every argument check happens before any work is enqueued.
+ */
+#ifndef TM_EDT_H_
+#define TM_EDT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define TM_EDT_API __attribute__((visibility("default")))
+#else
+#define TM_EDT_API
+#endif
+
+#define TM_EDT_MAX_DIMS 8      /* spatial rank bound (Section 2.2.1 / 2.2.2: compile-time bound of eight) */
+#define TM_EDT_MAX_EXTENT 8192 /* largest supported extent of one spatial axis */
+
+typedef enum {
+    TM_EDT_OK = 0,
+    TM_EDT_ERR_INVALID_ARG = 1, /* NULL input/shape, ndim outside 1..8, negative extent, sampling not finite
+                                   and > 0, no output requested, outputs overlapping each other or the input */
+    TM_EDT_ERR_UNSUPPORTED = 2, /* extent > TM_EDT_MAX_EXTENT, out_sqdist with non-unit sampling, more than
+                                   2^40 elements, or more than 2^31 - 1 voxels per image */
+    TM_EDT_ERR_BAD_POINTER = 3, /* a device buffer is not device-accessible memory of the current device
+                                   (or a host buffer of tm_edt_host is device memory) */
+    TM_EDT_ERR_ALLOC = 4,       /* scratch allocation failed, or the supplied workspace is too small */
+    TM_EDT_ERR_CUDA = 5         /* a CUDA runtime call or launch failed; see tm_edt_last_cuda_error() */
+} tm_edt_status;
+
+/* The stream argument is a cudaStream_t (NULL = the legacy default stream). */
+typedef struct CUstream_st* tm_edt_stream_t;
+
+/*
+ * The transform.  Enqueues all work on `stream` of the current device and returns without
+ * synchronising; outputs are complete once the stream reaches the end of that work.
+ *
+ *   input        device, uint8, contiguous row-major (B, C, n_0 .. n_{ndim-1}); nonzero = foreground
+ *                (a bool tensor is passed as its bytes).  Read only.
+ *   ndim         number of SPATIAL dimensions, 1..8.
+ *   shape        host, ndim + 2 entries: B, C, n_0 .. n_{ndim-1}.  Any entry may be 0 (nothing is
+ *                written, TM_EDT_OK); extents of 1 are legal.  Copied during the call.
+ *   sampling     host, ndim entries, each finite and > 0, or NULL for 1.0 on every axis.  Copied.
+ *   out_dist     device float32 (B, C, n...), or NULL.
+ *   out_sqdist   device int64 (B, C, n...), or NULL.  Requires unit sampling (else UNSUPPORTED).
+ *   out_indices  device int64 (B, C, ndim, n...), or NULL.  out_indices[b, c, a, x] is the coordinate
+ *                along spatial axis a of the background voxel chosen for voxel x.
+ *   At least one output must be non-NULL.  The caller owns every buffer; the library keeps no
+ *   pointer once the enqueued work has run.  Scratch memory is taken from the stream-ordered
+ *   allocator of the device (allocation and release are both ordered on `stream`).
+ *
+ * Returns a tm_edt_status.  On any error other than TM_EDT_ERR_CUDA nothing has been enqueued.
+ */
+TM_EDT_API int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+           int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
+
+/*
+ * Scratch bytes tm_edt_ws needs for a call with this geometry (0 for empty problems, and (size_t)-1
+ * if ndim/shape are invalid or unsupported).  Depends only on ndim and shape.
+ */
+TM_EDT_API size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape);
+
+/*
+ * Same transform with caller-provided scratch: `workspace` is device memory of at least
+ * tm_edt_workspace_bytes(ndim, shape) bytes, 256-byte aligned, private to this call until the
+ * enqueued work has run.  Allocates nothing.  A too-small workspace gives TM_EDT_ERR_ALLOC.
+ */
+TM_EDT_API int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+              int64_t* out_sqdist, int64_t* out_indices, void* workspace, size_t workspace_bytes,
+              tm_edt_stream_t stream);
+
+/*
+ * Host-buffer convenience: `input` and the outputs are HOST memory (pinned memory makes the copies
+ * asynchronous).  Device buffers come from the stream-ordered allocator; the input is copied to the
+ * device, the transform runs, and the requested outputs are copied back, all ordered on `stream`.
+ * Does not synchronise: the host outputs are valid after the caller synchronises the stream.
+ */
+TM_EDT_API int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
+
+/* Static description of a status code. Never NULL. */
+TM_EDT_API const char* tm_edt_strerror(int status);
+
+/* The cudaError_t value behind the calling thread's most recent TM_EDT_ERR_CUDA / TM_EDT_ERR_ALLOC (0 if none). */
+TM_EDT_API int tm_edt_last_cuda_error(void);
+
+/* Library version string, e.g. "tm_edt 0.1 (sm_100a)". */
+TM_EDT_API const char* tm_edt_version(void);
+
+/* Number of kernels the calling thread's most recent successful tm_edt* call enqueued. */
+TM_EDT_API int tm_edt_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TM_EDT_H_ */

@@ -1,0 +1,187 @@
+"""ctypes binding of the C-ABI library ``libtm_edt.so`` -- argument marshalling only.
+
+Every step of the transform runs inside the CUDA library; PyTorch is used here for device memory and
+streams.  There is no fallback: if the library cannot be loaded, or a call fails, an exception is
+raised.  Entry points carry the names of the C functions declared in ``include/tm_edt.h``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtm_edt.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_POINTER, ERR_ALLOC, ERR_CUDA = range(6)
+MAX_DIMS = 8
+MAX_EXTENT = 8192
+
+EXPORTS = (
+    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_workspace_bytes", "tm_edt_strerror",
+    "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count",
+)
+
+_lock = threading.Lock()
+_lib = None
+
+
+class TmEdtError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("tm_edt failed: %s (status %d)" % (message, status))
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Open the CUDA library (once).  Raises if it has not been built: there is no other code path."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(LIB_PATH):
+                raise RuntimeError(
+                    "CUDA library %s is missing; build it with `python -m paper_2608_24738_b200.buildlib`" % LIB_PATH
+                )
+            L = ctypes.CDLL(LIB_PATH)
+            vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+            L.tm_edt.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
+            L.tm_edt.restype = i
+            L.tm_edt_ws.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp]
+            L.tm_edt_ws.restype = i
+            L.tm_edt_host.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
+            L.tm_edt_host.restype = i
+            L.tm_edt_workspace_bytes.argtypes = [i, vp]
+            L.tm_edt_workspace_bytes.restype = sz
+            L.tm_edt_strerror.argtypes = [i]
+            L.tm_edt_strerror.restype = ctypes.c_char_p
+            L.tm_edt_last_cuda_error.restype = i
+            L.tm_edt_last_launch_count.restype = i
+            L.tm_edt_version.restype = ctypes.c_char_p
+            _lib = L
+    return _lib
+
+
+def tm_edt_strerror(status: int) -> str:
+    return lib().tm_edt_strerror(int(status)).decode()
+
+
+def tm_edt_version() -> str:
+    return lib().tm_edt_version().decode()
+
+
+def tm_edt_last_cuda_error() -> int:
+    return int(lib().tm_edt_last_cuda_error())
+
+
+def tm_edt_last_launch_count() -> int:
+    return int(lib().tm_edt_last_launch_count())
+
+
+def _shape_array(shape: Sequence[int]):
+    return (ctypes.c_int64 * len(shape))(*[int(s) for s in shape])
+
+
+def _sampling_array(sampling, ndim):
+    if sampling is None:
+        return None
+    vals = [float(s) for s in sampling]
+    if len(vals) != ndim:
+        raise ValueError("sampling needs one entry per spatial axis")
+    return (ctypes.c_double * ndim)(*vals)
+
+
+def tm_edt_workspace_bytes(shape: Sequence[int]) -> int:
+    """shape = (B, C, n_0 .. n_{d-1})."""
+    n = int(lib().tm_edt_workspace_bytes(len(shape) - 2, _shape_array(shape)))
+    if n == ctypes.c_size_t(-1).value:
+        raise TmEdtError(ERR_INVALID_ARG, "invalid or unsupported shape")
+    return n
+
+
+def _raw_stream(stream) -> Optional[int]:
+    import torch
+
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(status: int) -> None:
+    if status != OK:
+        raise TmEdtError(status, tm_edt_strerror(status))
+
+
+def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, device):
+    import torch
+
+    if mask.dim() < 3:
+        raise ValueError("mask must be shaped (B, C, spatial...)")
+    if mask.dtype == torch.bool:
+        mask = mask.view(torch.uint8)
+    if mask.dtype != torch.uint8:
+        raise TypeError("mask must be uint8 or bool")
+    if not mask.is_contiguous():
+        mask = mask.contiguous()
+    shape = tuple(mask.shape)
+    ndim = len(shape) - 2
+
+    def out(buf, want, dtype, shp):
+        if buf is not None:
+            if buf.dtype != dtype or tuple(buf.shape) != tuple(shp) or not buf.is_contiguous():
+                raise ValueError("pre-allocated output has the wrong dtype, shape or layout")
+            return buf
+        return torch.empty(shp, dtype=dtype, device=device, pin_memory=(device == "cpu_pinned")) if want else None
+
+    dev = mask.device if device is None else device
+    if dev == "cpu_pinned":
+        mk = lambda want, dtype, shp, buf: buf if buf is not None else (
+            torch.empty(shp, dtype=dtype, pin_memory=True) if want else None)
+    else:
+        mk = lambda want, dtype, shp, buf: out(buf, want, dtype, shp)
+    d = mk(return_distances, torch.float32, shape, distances)
+    s = mk(return_sqdist, torch.int64, shape, sqdist)
+    x = mk(return_indices, torch.int64, shape[:2] + (ndim,) + shape[2:], indices)
+    return mask, shape, ndim, d, s, x
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def tm_edt(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
+           distances=None, indices=None, sqdist=None, workspace=None, stream=None):
+    """Distance transform of a CUDA mask tensor (B, C, spatial...), uint8 or bool.
+
+    Returns a dict with the requested tensors among ``dist`` (float32), ``sq`` (int64, unit sampling
+    only) and ``idx`` (int64, (B, C, ndim, spatial...)).  With ``workspace`` (a CUDA uint8 tensor of at
+    least ``tm_edt_workspace_bytes(mask.shape)`` bytes) the call goes through ``tm_edt_ws`` and allocates
+    nothing; otherwise through ``tm_edt``.  Work is enqueued on ``stream`` (default: current stream).
+    """
+    L = lib()
+    if not mask.is_cuda:
+        raise ValueError("mask must be a CUDA tensor (use tm_edt_host for host buffers)")
+    mask, shape, ndim, d, s, x = _prepare(
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+    shp, smp, st = _shape_array(shape), _sampling_array(sampling, ndim), _raw_stream(stream)
+    if workspace is None:
+        rc = L.tm_edt(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), st)
+    else:
+        rc = L.tm_edt_ws(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), _p(workspace),
+                         ctypes.c_size_t(workspace.numel() * workspace.element_size()), st)
+    _check(rc)
+    return {"dist": d, "sq": s, "idx": x}
+
+
+def tm_edt_host(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
+                distances=None, indices=None, sqdist=None, stream=None):
+    """Same transform for HOST tensors (pinned for asynchronous copies): the C library copies the mask to
+    the device, runs, and copies the outputs back, all on ``stream``; the caller synchronises."""
+    L = lib()
+    if mask.is_cuda:
+        raise ValueError("tm_edt_host takes host tensors")
+    mask, shape, ndim, d, s, x = _prepare(
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, "cpu_pinned")
+    rc = L.tm_edt_host(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
+                       _raw_stream(stream))
+    _check(rc)
+    return {"dist": d, "sq": s, "idx": x}

@@ -1,0 +1,353 @@
+// C ABI of the distance-transform library: argument validation, the host-side plan
+// (all geometry is resolved on the host: paper, Section 2.2.2 "Three layers") and kernel launches.
+#include "../../include/tm_edt.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "edt_common.cuh"
+#include "edt_generic.cuh"
+
+namespace tmedt {
+
+static thread_local int g_last_cuda_error = 0;
+static thread_local int g_last_launches = 0;
+
+// The contiguous (B, C, n_0 .. n_{d-1}) array is, for the pass along spatial axis a, a
+// (outer, n_a, inner) array.  Axes of extent 1 are never processed (their pass is the identity).
+// Processing order: last spatial axis first ("plane" p = p-th processed axis).
+struct Plan {
+    int ndim = 0;
+    int64_t images = 0, V = 0, N = 0;
+    int E = 0;
+    int axis[kMaxDims];
+    int plane_of_axis[kMaxDims];
+    int ext[kMaxDims];
+    int64_t inner[kMaxDims];
+    double w[kMaxDims];
+    bool unit = true;
+    bool use_double = false;  // arithmetic type of the envelope passes
+    bool wide = false;        // int16 offsets instead of int8
+    size_t ws_bytes = 0;
+    size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
+};
+
+static int make_plan(int ndim, const int64_t* shape, const double* sampling, Plan& pl) {
+    if (!shape || ndim < 1 || ndim > kMaxDims) return TM_EDT_ERR_INVALID_ARG;
+    for (int k = 0; k < ndim + 2; ++k)
+        if (shape[k] < 0) return TM_EDT_ERR_INVALID_ARG;
+    if (sampling)
+        for (int k = 0; k < ndim; ++k)
+            if (!(sampling[k] > 0.0) || isinf(sampling[k])) return TM_EDT_ERR_INVALID_ARG;
+    pl.ndim = ndim;
+    // element counts, guarding against overflow
+    const int64_t kMaxElems = (int64_t)1 << 40;
+    int64_t V = 1;
+    bool empty = shape[0] == 0 || shape[1] == 0;
+    for (int k = 0; k < ndim; ++k) {
+        if (shape[2 + k] == 0) empty = true;
+        if (shape[2 + k] > TM_EDT_MAX_EXTENT) return TM_EDT_ERR_UNSUPPORTED;
+    }
+    if (empty) { pl.images = 0; pl.V = 0; pl.N = 0; pl.E = 0; pl.ws_bytes = 0; return TM_EDT_OK; }
+    for (int k = 0; k < ndim; ++k) {
+        V *= shape[2 + k];
+        if (V > (int64_t)INT32_MAX) return TM_EDT_ERR_UNSUPPORTED;
+    }
+    if (shape[0] > kMaxElems || shape[1] > kMaxElems) return TM_EDT_ERR_UNSUPPORTED;
+    const int64_t images = shape[0] * shape[1];
+    if (images > kMaxElems || images * V > kMaxElems) return TM_EDT_ERR_UNSUPPORTED;
+    pl.images = images; pl.V = V; pl.N = images * V;
+
+    pl.unit = true;
+    if (sampling)
+        for (int k = 0; k < ndim; ++k)
+            if (sampling[k] != 1.0) pl.unit = false;
+
+    for (int a = 0; a < ndim; ++a) pl.plane_of_axis[a] = -1;
+    int E = 0;
+    int64_t inner = 1;
+    for (int a = ndim - 1; a >= 0; --a) {
+        const int64_t n = shape[2 + a];
+        if (n > 1) {
+            pl.axis[E] = a; pl.ext[E] = (int)n; pl.inner[E] = inner;
+            pl.w[E] = sampling ? sampling[a] : 1.0;
+            pl.plane_of_axis[a] = E;
+            ++E;
+        }
+        inner *= n;
+    }
+    if (E == 0) {  // a single voxel per image: keep the last axis so that one pass runs
+        pl.axis[0] = ndim - 1; pl.ext[0] = 1; pl.inner[0] = 1;
+        pl.w[0] = sampling ? sampling[ndim - 1] : 1.0;
+        pl.plane_of_axis[ndim - 1] = 0;
+        E = 1;
+    }
+    pl.E = E;
+    int nmax = 1;
+    double sumsq = 0.0;
+    for (int p = 0; p < E; ++p) {
+        nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
+        sumsq += (double)(pl.ext[p] - 1) * (double)(pl.ext[p] - 1);
+    }
+    pl.wide = nmax > 128;
+    // float32 envelope arithmetic is exact for unit sampling while every value stays below 2^24 and the
+    // interval starts keep a safe margin to the next integer; otherwise switch to float64.  Sampled
+    // transforms are float32 throughout (their results are only defined up to rounding).
+    pl.use_double = pl.unit && !(sumsq + (double)nmax * nmax < 16777216.0 && nmax <= 512);
+    const size_t elem = pl.wide ? 2 : 1;
+    pl.plane_bytes = (((size_t)pl.N * elem) + 255) & ~(size_t)255;
+    pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
+    return TM_EDT_OK;
+}
+
+static void fill_epilogue(const Plan& pl, float* dist, int64_t* sq, int64_t* idx, EpilogueParams& ep) {
+    memset(&ep, 0, sizeof(ep));
+    ep.dist = dist; ep.sq = sq; ep.idx = idx;
+    ep.V = pl.V; ep.ndim = pl.ndim; ep.E = pl.E;
+    for (int p = 0; p < kMaxDims; ++p) {
+        ep.axis[p] = p < pl.E ? pl.axis[p] : 0;
+        ep.ext[p] = p < pl.E ? pl.ext[p] : 1;
+        ep.w2[p] = p < pl.E ? pl.w[p] * pl.w[p] : 0.0;
+    }
+    for (int a = 0; a < kMaxDims; ++a) ep.plane_of_axis[a] = a < pl.ndim ? pl.plane_of_axis[a] : -1;
+}
+
+template <typename OT>
+static cudaError_t launch_pass0(const Plan& pl, const uint8_t* in, void* out, bool final_pass,
+                                const EpilogueParams& ep, cudaStream_t st) {
+    Pass0Params P;
+    P.in = in; P.out = out; P.n = pl.ext[0]; P.lines = pl.N / pl.ext[0]; P.w = pl.w[0];
+    if (P.n <= 32) {
+        const int per_warp = 32 / P.n;
+        const int64_t warps = (P.lines + per_warp - 1) / per_warp;
+        const int64_t blocks = (warps + 7) / 8;
+        if (final_pass) pass0_short_kernel<OT, true><<<(unsigned)blocks, 256, 0, st>>>(P, ep);
+        else pass0_short_kernel<OT, false><<<(unsigned)blocks, 256, 0, st>>>(P, ep);
+    } else {
+        const int nw = (P.n + 31) / 32;
+        const size_t smem = (size_t)4 * 3 * nw * sizeof(int);
+        const int64_t blocks = (P.lines + 3) / 4;
+        if (final_pass) pass0_long_kernel<OT, true><<<(unsigned)blocks, 128, smem, st>>>(P, ep);
+        else pass0_long_kernel<OT, false><<<(unsigned)blocks, 128, smem, st>>>(P, ep);
+    }
+    return cudaGetLastError();
+}
+
+template <typename CT, typename OT, int K, bool FINAL>
+static cudaError_t launch_axis_k(const AxisParams& P, const EpilogueParams& ep, cudaStream_t st) {
+    const int nw = (P.n + 31) / 32;
+    const size_t per_thread = (size_t)2 * nw * sizeof(unsigned);
+    int threads = 128;
+    while (threads > 32 && per_thread * threads > 64 * 1024) threads >>= 1;
+    const size_t smem = per_thread * threads;
+    auto kern = axis_pass_kernel<CT, OT, K, FINAL>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const int64_t blocks = (P.lines + threads - 1) / threads;
+    kern<<<(unsigned)blocks, threads, smem, st>>>(P, ep);
+    return cudaGetLastError();
+}
+
+template <typename CT, typename OT, bool FINAL>
+static cudaError_t launch_axis(int K, const AxisParams& P, const EpilogueParams& ep, cudaStream_t st) {
+    switch (K) {
+        case 1: return launch_axis_k<CT, OT, 1, FINAL>(P, ep, st);
+        case 2: return launch_axis_k<CT, OT, 2, FINAL>(P, ep, st);
+        case 3: return launch_axis_k<CT, OT, 3, FINAL>(P, ep, st);
+        case 4: return launch_axis_k<CT, OT, 4, FINAL>(P, ep, st);
+        case 5: return launch_axis_k<CT, OT, 5, FINAL>(P, ep, st);
+        case 6: return launch_axis_k<CT, OT, 6, FINAL>(P, ep, st);
+        case 7: return launch_axis_k<CT, OT, 7, FINAL>(P, ep, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+template <typename CT, typename OT>
+static cudaError_t run_generic(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws,
+                               cudaStream_t st, int& launches) {
+    cudaError_t e;
+    char* bufA = static_cast<char*>(ws);
+    char* bufB = bufA + (size_t)(pl.E > 1 ? pl.E - 1 : 0) * pl.plane_bytes;
+    e = launch_pass0<OT>(pl, in, bufA, pl.E == 1, ep, st);
+    ++launches;
+    if (e != cudaSuccess) return e;
+    char* src = bufA;
+    char* dst = bufB;
+    for (int k = 1; k < pl.E; ++k) {
+        AxisParams P;
+        memset(&P, 0, sizeof(P));
+        P.in = src; P.out = dst;
+        P.plane_elems = (int64_t)(pl.plane_bytes / sizeof(OT));
+        P.n = pl.ext[k]; P.inner = pl.inner[k]; P.lines = pl.N / pl.ext[k];
+        P.w2 = pl.w[k] * pl.w[k];
+        for (int p = 0; p < k; ++p) P.w2p[p] = pl.w[p] * pl.w[p];
+        const bool fin = k == pl.E - 1;
+        e = fin ? launch_axis<CT, OT, true>(k, P, ep, st) : launch_axis<CT, OT, false>(k, P, ep, st);
+        ++launches;
+        if (e != cudaSuccess) return e;
+        char* t = src; src = dst; dst = t;
+    }
+    return cudaSuccess;
+}
+
+static bool is_device_ptr(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (at.type == cudaMemoryTypeManaged) return true;
+    return at.type == cudaMemoryTypeDevice && at.device == dev;
+}
+
+static bool is_host_ptr(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return true; }
+    return at.type != cudaMemoryTypeDevice;
+}
+
+static bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// Argument checks common to every entry point (no CUDA work).
+static int check_call(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                      int64_t* out_sq, int64_t* out_idx, Plan& pl) {
+    if (!input) return TM_EDT_ERR_INVALID_ARG;
+    const int rc = make_plan(ndim, shape, sampling, pl);
+    if (rc != TM_EDT_OK) return rc;
+    if (!out_dist && !out_sq && !out_idx) return TM_EDT_ERR_INVALID_ARG;
+    if (out_sq && !pl.unit) return TM_EDT_ERR_UNSUPPORTED;
+    const size_t N = (size_t)pl.N;
+    const size_t bi = N, bd = N * 4, bs = N * 8, bx = N * 8 * (size_t)ndim;
+    if (overlap(input, bi, out_dist, bd) || overlap(input, bi, out_sq, bs) || overlap(input, bi, out_idx, bx) ||
+        overlap(out_dist, bd, out_sq, bs) || overlap(out_dist, bd, out_idx, bx) || overlap(out_sq, bs, out_idx, bx))
+        return TM_EDT_ERR_INVALID_ARG;
+    return TM_EDT_OK;
+}
+
+static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int64_t* out_sq, int64_t* out_idx,
+                      void* ws, cudaStream_t st) {
+    EpilogueParams ep;
+    fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
+    int launches = 0;
+    cudaError_t e;
+    if (pl.use_double)
+        e = pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
+                    : run_generic<double, int8_t>(pl, input, ep, ws, st, launches);
+    else
+        e = pl.wide ? run_generic<float, int16_t>(pl, input, ep, ws, st, launches)
+                    : run_generic<float, int8_t>(pl, input, ep, ws, st, launches);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    g_last_launches = launches;
+    return TM_EDT_OK;
+}
+
+}  // namespace tmedt
+
+using namespace tmedt;
+
+extern "C" {
+
+size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape) {
+    Plan pl;
+    if (make_plan(ndim, shape, nullptr, pl) != TM_EDT_OK) return (size_t)-1;
+    return pl.ws_bytes;
+}
+
+int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+              int64_t* out_sqdist, int64_t* out_indices, void* workspace, size_t workspace_bytes,
+              tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl);
+    if (rc != TM_EDT_OK) return rc;
+    if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (pl.ws_bytes > 0) {
+        if (!workspace || workspace_bytes < pl.ws_bytes) return TM_EDT_ERR_ALLOC;
+        if (((uintptr_t)workspace & 255u) != 0) return TM_EDT_ERR_INVALID_ARG;
+        if (!is_device_ptr(workspace)) return TM_EDT_ERR_BAD_POINTER;
+    }
+    if (!is_device_ptr(input) || (out_dist && !is_device_ptr(out_dist)) || (out_sqdist && !is_device_ptr(out_sqdist)) ||
+        (out_indices && !is_device_ptr(out_indices)))
+        return TM_EDT_ERR_BAD_POINTER;
+    return run_device(pl, input, out_dist, out_sqdist, out_indices, workspace, (cudaStream_t)stream);
+}
+
+int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+           int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl);
+    if (rc != TM_EDT_OK) return rc;
+    if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (!is_device_ptr(input) || (out_dist && !is_device_ptr(out_dist)) || (out_sqdist && !is_device_ptr(out_sqdist)) ||
+        (out_indices && !is_device_ptr(out_indices)))
+        return TM_EDT_ERR_BAD_POINTER;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* ws = nullptr;
+    if (pl.ws_bytes > 0) {
+        cudaError_t e = cudaMallocAsync(&ws, pl.ws_bytes, st);
+        if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
+    }
+    rc = run_device(pl, input, out_dist, out_sqdist, out_indices, ws, st);
+    if (ws) cudaFreeAsync(ws, st);
+    return rc;
+}
+
+int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl);
+    if (rc != TM_EDT_OK) return rc;
+    if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (!is_host_ptr(input) || (out_dist && !is_host_ptr(out_dist)) || (out_sqdist && !is_host_ptr(out_sqdist)) ||
+        (out_indices && !is_host_ptr(out_indices)))
+        return TM_EDT_ERR_BAD_POINTER;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t N = (size_t)pl.N;
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t b_in = up(N), b_d = out_dist ? up(N * 4) : 0, b_s = out_sqdist ? up(N * 8) : 0,
+                 b_x = out_indices ? up(N * 8 * (size_t)ndim) : 0, b_ws = up(pl.ws_bytes);
+    char* dev = nullptr;
+    cudaError_t e = cudaMallocAsync((void**)&dev, b_in + b_d + b_s + b_x + b_ws, st);
+    if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
+    uint8_t* d_in = (uint8_t*)dev;
+    float* d_d = out_dist ? (float*)(dev + b_in) : nullptr;
+    int64_t* d_s = out_sqdist ? (int64_t*)(dev + b_in + b_d) : nullptr;
+    int64_t* d_x = out_indices ? (int64_t*)(dev + b_in + b_d + b_s) : nullptr;
+    void* d_ws = pl.ws_bytes ? (void*)(dev + b_in + b_d + b_s + b_x) : nullptr;
+    e = cudaMemcpyAsync(d_in, input, N, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) {
+        rc = run_device(pl, d_in, d_d, d_s, d_x, d_ws, st);
+        if (rc == TM_EDT_OK && out_dist) e = cudaMemcpyAsync(out_dist, d_d, N * 4, cudaMemcpyDeviceToHost, st);
+        if (rc == TM_EDT_OK && e == cudaSuccess && out_sqdist)
+            e = cudaMemcpyAsync(out_sqdist, d_s, N * 8, cudaMemcpyDeviceToHost, st);
+        if (rc == TM_EDT_OK && e == cudaSuccess && out_indices)
+            e = cudaMemcpyAsync(out_indices, d_x, N * 8 * (size_t)ndim, cudaMemcpyDeviceToHost, st);
+    }
+    cudaFreeAsync(dev, st);
+    if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    return rc;
+}
+
+const char* tm_edt_strerror(int status) {
+    switch (status) {
+        case TM_EDT_OK: return "ok";
+        case TM_EDT_ERR_INVALID_ARG: return "invalid argument";
+        case TM_EDT_ERR_UNSUPPORTED: return "unsupported size or option";
+        case TM_EDT_ERR_BAD_POINTER: return "buffer is not in the expected memory space";
+        case TM_EDT_ERR_ALLOC: return "scratch allocation failed or workspace too small";
+        case TM_EDT_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+int tm_edt_last_cuda_error(void) { return g_last_cuda_error; }
+int tm_edt_last_launch_count(void) { return g_last_launches; }
+const char* tm_edt_version(void) { return "tm_edt 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,101 @@
+"""The C-ABI library loads, exports every symbol the header declares, and rejects bad arguments
+before doing any device work (these checks need no GPU)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2608_24738_b200 import binding, buildlib
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    buildlib.build()
+    return binding.lib()
+
+
+def test_header_symbols_are_exported(L):
+    header = open(os.path.join(ROOT, "include", "tm_edt.h")).read()
+    declared = set(re.findall(r"TM_EDT_API[^;(]*?\b(tm_edt\w*)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_version_and_strerror(L):
+    assert "sm_100a" in binding.tm_edt_version()
+    for s in range(6):
+        assert binding.tm_edt_strerror(s)
+    assert binding.tm_edt_strerror(99) == "unknown status"
+
+
+def _call(L, inp=1, ndim=2, shape=(1, 1, 4, 4), sampling=None, d=1, s=0, x=0):
+    shp = (ctypes.c_int64 * len(shape))(*shape) if shape is not None else None
+    smp = (ctypes.c_double * len(sampling))(*sampling) if sampling is not None else None
+    fake = lambda v: ctypes.c_void_p(0x1000 * v) if v else None  # never dereferenced on these paths
+    return L.tm_edt(fake(inp), ndim, shp, smp, fake(2 * d), fake(3 * s), fake(4 * x), None)
+
+
+def test_invalid_arguments_return_before_any_device_work(L):
+    E = binding
+    assert _call(L, inp=0) == E.ERR_INVALID_ARG
+    assert _call(L, shape=None) == E.ERR_INVALID_ARG
+    assert _call(L, ndim=0, shape=(1, 1)) == E.ERR_INVALID_ARG
+    assert _call(L, ndim=9, shape=(1, 1) + (2,) * 9) == E.ERR_INVALID_ARG
+    assert _call(L, shape=(1, 1, -1, 4)) == E.ERR_INVALID_ARG
+    assert _call(L, shape=(-1, 1, 4, 4)) == E.ERR_INVALID_ARG
+    assert _call(L, sampling=(1.0, 0.0)) == E.ERR_INVALID_ARG
+    assert _call(L, sampling=(1.0, -2.0)) == E.ERR_INVALID_ARG
+    assert _call(L, sampling=(float("nan"), 1.0)) == E.ERR_INVALID_ARG
+    assert _call(L, sampling=(float("inf"), 1.0)) == E.ERR_INVALID_ARG
+    assert _call(L, d=0, s=0, x=0) == E.ERR_INVALID_ARG
+
+
+def test_unsupported(L):
+    E = binding
+    assert _call(L, shape=(1, 1, E.MAX_EXTENT + 1, 4)) == E.ERR_UNSUPPORTED
+    assert _call(L, sampling=(1.0, 2.0), s=1) == E.ERR_UNSUPPORTED
+    assert _call(L, shape=(1, 1, 8192, 8192, 64), ndim=3) == E.ERR_UNSUPPORTED  # > 2^31 - 1 voxels per image
+    assert _call(L, shape=(1 << 20, 1 << 10, 8192, 8192), ndim=2) == E.ERR_UNSUPPORTED  # > 2^40 elements
+
+
+def test_empty_problem_is_ok_without_touching_pointers(L):
+    assert _call(L, shape=(0, 1, 4, 4)) == binding.OK
+    assert _call(L, shape=(1, 1, 4, 0)) == binding.OK
+    assert binding.tm_edt_last_launch_count() == 0
+
+
+def test_overlapping_buffers_are_rejected(L):
+    shp = (ctypes.c_int64 * 4)(1, 1, 4, 4)
+    a = ctypes.c_void_p(0x10000)
+    b = ctypes.c_void_p(0x10008)  # overlaps a 64-byte float output starting at 0x10000
+    assert L.tm_edt(a, 2, shp, None, b, None, None, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt(ctypes.c_void_p(0x20000), 2, shp, None, a, b, None, None) == binding.ERR_INVALID_ARG
+
+
+def test_host_memory_is_not_accepted_as_device_memory(L):
+    # Valid arguments, but the buffers are ordinary host arrays: BAD_POINTER (with or without a GPU present).
+    m = np.ones((1, 1, 4, 4), dtype=np.uint8)
+    out = np.zeros((1, 1, 4, 4), dtype=np.float32)
+    shp = (ctypes.c_int64 * 4)(1, 1, 4, 4)
+    rc = L.tm_edt(m.ctypes.data_as(ctypes.c_void_p), 2, shp, None, out.ctypes.data_as(ctypes.c_void_p), None, None, None)
+    assert rc == binding.ERR_BAD_POINTER
+
+
+def test_workspace_bytes(L):
+    assert binding.tm_edt_workspace_bytes((1, 1, 0, 4)) == 0
+    assert binding.tm_edt_workspace_bytes((1, 1, 64)) == 0  # a single pass needs no scratch
+    assert binding.tm_edt_workspace_bytes((2, 3, 64, 64)) >= 2 * 3 * 64 * 64
+    with pytest.raises(binding.TmEdtError):
+        binding.tm_edt_workspace_bytes((1, 1, binding.MAX_EXTENT + 1))
+
+
+def test_binding_refuses_host_tensor():
+    import torch
+
+    with pytest.raises(ValueError):
+        binding.tm_edt(torch.ones((1, 1, 4, 4), dtype=torch.uint8))

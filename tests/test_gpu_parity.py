@@ -1,0 +1,214 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bars: int64 squared distances bit-exact; float32 distances |d - d_ref| <= 1e-5 * max(1, d_ref);
+indices name a background voxel at the minimal distance (ties may differ from the oracle's pick)."""
+import zlib
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_24738_b200 import binding, buildlib, workloads
+from tests import checker
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    buildlib.build()
+    binding.lib()
+
+
+def run_gpu(mask, sampling=None, dist=True, sq=False, idx=False, **kw):
+    import torch
+
+    t = torch.from_numpy(np.ascontiguousarray(mask)).cuda()
+    r = binding.tm_edt(t, sampling, return_distances=dist, return_sqdist=sq, return_indices=idx, **kw)
+    torch.cuda.synchronize()
+    return {k: (None if v is None else v.cpu().numpy()) for k, v in r.items()}
+
+
+def compare(mask, sampling, res, ref, dist=True, sq=False, idx=False):
+    if dist:
+        assert res["dist"].dtype == np.float32
+        checker.check_dist(res["dist"], ref["dist"])
+    if sq:
+        checker.check_sq_exact(res["sq"], ref["sq"])
+    if idx:
+        checker.check_indices(res["idx"], mask, ref, sampling)
+
+
+def full_check(mask, sampling=None):
+    unit = sampling is None or all(float(s) == 1.0 for s in sampling)
+    ref = oracle.sep(mask, sampling, want_idx=False)
+    res = run_gpu(mask, sampling, dist=True, sq=unit, idx=True)
+    compare(mask, sampling, res, ref, True, unit, True)
+    return res, ref
+
+
+SMALL = [
+    (1, 1, 1), (1, 1, 5), (2, 3, 32), (1, 1, 33), (3, 1, 100), (1, 1, 129), (1, 1, 600), (1, 1, 1500),
+    (1, 1, 7, 5), (2, 2, 33, 65), (1, 1, 1, 40), (1, 1, 40, 1), (1, 1, 130, 67), (1, 1, 67, 130), (1, 2, 64, 64),
+    (1, 1, 9, 10, 11), (2, 1, 33, 17, 40), (1, 1, 5, 1, 6), (1, 1, 1, 1, 1), (1, 1, 140, 9, 12),
+    (1, 1, 6, 5, 4, 7), (1, 1, 3, 4, 5, 3, 4), (1, 1, 2, 3, 4, 3, 2, 3), (1, 1, 3, 2, 3, 2, 3, 2, 3),
+    (2, 1, 3, 2, 3, 2, 3, 2, 3, 4), (1, 1, 6, 6, 6, 6, 6, 6, 6, 6),
+]
+
+
+def _sampling(ndim, kind):
+    if kind == "unit":
+        return None
+    return tuple(0.5 + 0.37 * ((3 * k + 1) % 5) for k in range(ndim))
+
+
+@pytest.mark.parametrize("shape", SMALL, ids=["x".join(map(str, s)) for s in SMALL])
+@pytest.mark.parametrize("p_fg", [0.3, 0.9, 0.995])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_small_shapes_every_rank(shape, p_fg, kind):
+    seed = zlib.crc32(repr((shape, p_fg, kind)).encode())
+    mask = workloads.random_mask(seed, shape, p_fg)
+    full_check(mask, _sampling(len(shape) - 2, kind))
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 64), (2, 1, 20, 30), (1, 2, 8, 9, 10), (1, 1, 200, 40)])
+def test_degenerate_masks(shape):
+    ndim = len(shape) - 2
+    allfg = np.ones(shape, dtype=np.uint8)
+    r = run_gpu(allfg, None, True, True, True)
+    assert np.isinf(r["dist"]).all() and (r["dist"] > 0).all()
+    assert (r["sq"] == np.iinfo(np.int64).max).all()
+    assert (r["idx"] == -1).all()
+    allbg = np.zeros(shape, dtype=np.uint8)
+    r = run_gpu(allbg, None, True, True, True)
+    assert (r["dist"] == 0).all() and (r["sq"] == 0).all()
+    full_check(allbg, None)
+    one = np.ones(shape, dtype=np.uint8)
+    z = tuple(n // 3 for n in shape[2:])
+    one[(0, 0) + z] = 0
+    if shape[0] * shape[1] > 1:
+        one[-1, -1] = 1  # last image keeps no background at all
+        one[(-1, -1) + tuple(n - 1 for n in shape[2:])] = 0 if shape[0] * shape[1] > 2 else 1
+    samp = tuple(1.0 + 0.25 * k for k in range(ndim))
+    full_check(one, samp)
+    full_check(one, None)
+    # values above one are foreground too
+    m = workloads.random_mask(5, shape, 0.7) * 200
+    full_check(m.astype(np.uint8), None)
+
+
+def test_mixed_batch_with_image_without_background():
+    mask = workloads.random_mask(77, (3, 2, 20, 21, 22), 0.9)
+    mask[1, 1] = 1
+    res, ref = full_check(mask, (2.5, 0.8, 1.0))
+    assert np.isinf(res["dist"][1, 1]).all()
+    assert np.isfinite(res["dist"][0, 0]).all()
+
+
+def test_half_space_and_far_sites():
+    mask = np.ones((1, 1, 128, 96), dtype=np.uint8)
+    mask[0, 0, :3] = 0
+    full_check(mask, None)
+    full_check(mask, (0.3, 1.9))
+    mask = np.ones((1, 1, 100, 128, 128), dtype=np.uint8)
+    mask[0, 0, 99, 127, 0] = 0
+    full_check(mask, None)  # largest offsets an int8 carry can hold
+    full_check(mask, (2.5, 0.8, 1.0))
+
+
+@pytest.mark.parametrize("n", [512, 513, 1100, 2048])
+def test_long_lines(n):
+    """Extents above 128 use 16-bit offsets; unit sampling beyond 512 switches the envelope to float64."""
+    mask = workloads.random_mask(n, (1, 1, 24, n), 0.97)
+    mask[0, 0, :, : n // 2] |= workloads.random_mask(n + 1, (24, n // 2), 0.9995)
+    full_check(mask, None)
+    full_check(np.ascontiguousarray(mask.transpose(0, 1, 3, 2)), None)
+    full_check(mask, (1.7, 0.6))
+
+
+def test_sparse_background_long_axis_exactness():
+    """Few background voxels and large extents: squared distances up to ~1e7 must stay exact."""
+    mask = np.ones((1, 1, 2048, 300), dtype=np.uint8)
+    rng = np.random.default_rng(3)
+    for _ in range(12):
+        mask[0, 0, rng.integers(0, 2048), rng.integers(0, 300)] = 0
+    full_check(mask, None)
+
+
+def test_workspace_variant_and_preallocated_outputs():
+    import torch
+
+    mask = workloads.random_mask(9, (2, 2, 30, 31, 32), 0.8)
+    ref = oracle.sep(mask, None, want_idx=False)
+    t = torch.from_numpy(mask).cuda()
+    ws = torch.empty(binding.tm_edt_workspace_bytes(mask.shape), dtype=torch.uint8, device="cuda")
+    d = torch.full(mask.shape, -1.0, dtype=torch.float32, device="cuda")
+    x = torch.full((2, 2, 3, 30, 31, 32), -7, dtype=torch.int64, device="cuda")
+    r = binding.tm_edt(t, None, return_distances=True, return_indices=True, distances=d, indices=x, workspace=ws)
+    torch.cuda.synchronize()
+    assert r["dist"] is d and r["idx"] is x
+    checker.check_dist(d.cpu().numpy(), ref["dist"])
+    checker.check_indices(x.cpu().numpy(), mask, ref, None)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.TmEdtError) as ei:
+        binding.tm_edt(t, None, workspace=small)
+    assert ei.value.status == binding.ERR_ALLOC
+
+
+def test_side_stream_is_honoured():
+    import torch
+
+    mask = workloads.random_mask(10, (4, 1, 96, 96, 96), 0.8)
+    ref = oracle.sep(mask, None, want_idx=False)
+    t = torch.from_numpy(mask).cuda()
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        r = binding.tm_edt(t, None, return_distances=True, return_sqdist=True)
+        done = torch.cuda.Event()
+        done.record(s)
+    done.synchronize()
+    checker.check_sq_exact(r["sq"].cpu().numpy(), ref["sq"])
+    # explicit stream argument
+    r = binding.tm_edt(t, None, return_distances=True, stream=s)
+    s.synchronize()
+    checker.check_dist(r["dist"].cpu().numpy(), ref["dist"])
+
+
+def test_host_buffer_entry_point():
+    import torch
+
+    mask = workloads.random_mask(12, (2, 1, 40, 50), 0.85)
+    ref = oracle.sep(mask, (1.5, 1.0), want_idx=False)
+    t = torch.from_numpy(mask).pin_memory()
+    r = binding.tm_edt_host(t, (1.5, 1.0), return_distances=True, return_indices=True)
+    torch.cuda.synchronize()
+    checker.check_dist(r["dist"].numpy(), ref["dist"])
+    checker.check_indices(r["idx"].numpy(), mask, ref, (1.5, 1.0))
+    with pytest.raises(binding.TmEdtError) as ei:
+        binding.lib()  # keep the library loaded
+        d = torch.empty(mask.shape, dtype=torch.float32, device="cuda")
+        import ctypes
+
+        shp = (ctypes.c_int64 * 4)(*mask.shape)
+        rc = binding.lib().tm_edt_host(ctypes.c_void_p(t.data_ptr()), 2, shp, None, ctypes.c_void_p(d.data_ptr()),
+                                       None, None, None)
+        binding._check(rc)
+    assert ei.value.status == binding.ERR_BAD_POINTER
+
+
+def test_config1_brute_force_every_voxel():
+    w = workloads.config1()
+    ref = oracle.brute(w.mask, w.sampling)
+    res = run_gpu(w.mask, None, True, True, True)
+    compare(w.mask, None, res, ref, True, True, True)
+
+
+@pytest.mark.parametrize("number", [2, 3, 4, 5])
+def test_full_size_configs(number):
+    w = workloads.CONFIGS[number]()
+    ref = oracle.sep(w.mask, w.sampling, want_idx=False)
+    res = run_gpu(w.mask, w.sampling, dist=w.want_dist, sq=w.want_sq, idx=w.want_idx)
+    compare(w.mask, w.sampling, res, ref, w.want_dist, w.want_sq, w.want_idx)
+    if number == 5:
+        assert np.isinf(res["dist"][1]).all() and np.isfinite(res["dist"][0]).all()
