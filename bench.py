@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the distance-transform hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+A step is one full transform (every pass plus the fused epilogue) of one seeded synthetic workload.
+Prints ONE JSON line.  `value` is Gvoxel/s with the mask already resident in device memory; `e2e` is
+the same metric through the host-buffer entry point (pinned host memory, copies inside the timed
+region).  With N > 1 (torchrun) every rank transforms its own copy of the workload on its own GPU --
+the images of a batch are independent, so there is no data-path collective -- and the time is the
+maximum over ranks.  `--impl reference` times the CPU oracle instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "edt_gvoxels_per_s"
+UNIT = "Gvoxel/s"
+L2_BYTES = 126 * 1024 * 1024
+REASON_BITS = {
+    0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+    0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+    0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.01):
+        self.period = period_s
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        self.max_mhz = None
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as exc:  # pragma: no cover - depends on the box
+            self.err = repr(exc)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, rs))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not inside and self.samples:  # region shorter than a sampling period: nearest samples
+            inside = sorted(self.samples, key=lambda s: abs(s[0] - 0.5 * (t0 + t1)))[:3]
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        reasons = [name for bit, name in REASON_BITS.items() if bits & bit and name != "gpu_idle"]
+        return {
+            "sm_mhz": statistics.median([s[1] for s in inside]) if inside else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": reasons,
+            "samples": len(inside),
+        }
+
+
+def dist_env():
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Largest `value` over all ranks (the process group must exist when world > 1)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, seconds_max: float) -> float:
+    """Aggregate rate of a weak-scaling job: every rank did `units_per_rank` in at most `seconds_max`."""
+    return units_per_rank * world / seconds_max
+
+
+def sample_images(w, max_voxels: int):
+    """First images of the workload, as many as fit in max_voxels (at least one)."""
+    B, C = w.mask.shape[:2]
+    per = w.voxels // (B * C)
+    flat = w.mask.reshape((B * C, 1) + w.mask.shape[2:])
+    k = max(1, min(B * C, max_voxels // per))
+    return flat[:k], k, B * C
+
+
+def time_oracle(w, max_voxels: int, repeats: int = 1):
+    import oracle
+
+    sub, k, total = sample_images(w, max_voxels)
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.sep(sub, w.sampling, want_idx=w.want_idx)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return sub.size / best / 1e9, best, "%d of %d images (%d voxels), full oracle incl. index decode" % (k, total, sub.size)
+
+
+def run_reference(args, w, world, rank):
+    """The CPU oracle as the reference arm: rank 0 only, bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+
+    # size the per-step sample so that the whole run stays near a minute
+    one, _, total = sample_images(w, 1)
+    t0 = time.perf_counter()
+    oracle.sep(one, w.sampling, want_idx=w.want_idx)
+    t_img = max(time.perf_counter() - t0, 1e-6)
+    budget_imgs = int(60.0 / (args.steps + args.warmup) / t_img)
+    sub, k, total = sample_images(w, min(args.ref_voxels, max(1, budget_imgs) * one.size))
+    for _ in range(args.warmup):
+        oracle.sep(sub, w.sampling, want_idx=w.want_idx)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.sep(sub, w.sampling, want_idx=w.want_idx)
+    dt = time.perf_counter() - t0
+    val = sub.size * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64" if w.sampling is not None else "int64", "data": "synthetic",
+        "config": {"workload": w.name, "voxels_per_step": int(sub.size)},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": "%d of %d images per step" % (k, total)},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-voxels", type=int, default=8 << 20, help="voxels per step of the reference arm")
+    ap.add_argument("--cpu-voxels", type=int, default=64 << 20, help="sample size of the cpu_baseline leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile-steps", type=int, default=20)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    world, rank, local = dist_env()
+
+    from paper_2608_24738_b200 import workloads
+
+    w = workloads.CONFIGS[args.config]()
+    if args.impl == "reference":
+        run_reference(args, w, world, rank)
+        return
+
+    import torch
+
+    from paper_2608_24738_b200 import binding, buildlib
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the transform has no CPU path")
+    buildlib.build()
+    binding.lib()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- buffers: rotate over enough independent sets that one lap exceeds twice the L2 ----
+    io = w.io_bytes()
+    sets = max(2, min(16, -(-2 * L2_BYTES // io)))
+    host_mask = torch.from_numpy(w.mask)
+    shape = tuple(w.mask.shape)
+    calls = []
+    for _ in range(sets):
+        m = host_mask.to(dev)
+        d = torch.empty(shape, dtype=torch.float32, device=dev) if w.want_dist else None
+        s = torch.empty(shape, dtype=torch.int64, device=dev) if w.want_sq else None
+        x = torch.empty(shape[:2] + (w.ndim,) + shape[2:], dtype=torch.int64, device=dev) if w.want_idx else None
+        calls.append(binding.PreparedCall(m, w.sampling, d, s, x))
+    stream = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(stream.cuda_stream)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(args.warmup):
+        calls[i % sets](sp)
+    launches_per_step = binding.tm_edt_last_launch_count()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+        torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for i in range(args.steps):
+        calls[i % sets](sp)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+        torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    seconds = ev0.elapsed_time(ev1) / 1e3
+    seconds = max_over_ranks(seconds, world, dev)
+    clocks = sampler.summary(t0, t1)
+    value = whole_job_rate(w.voxels * args.steps, world, seconds) / 1e9
+
+    # ---- per-kernel times (events between launches), same buffers, right after the timed region ----
+    ksum = {}
+    korder = []
+    for i in range(max(1, args.profile_steps)):
+        c = calls[i % sets]
+        _, ks = binding.tm_edt_profile(c.mask, w.sampling, distances=c.d, sqdist=c.s, indices=c.x, workspace=c.ws,
+                                       return_distances=w.want_dist, return_sqdist=w.want_sq,
+                                       return_indices=w.want_idx)
+        for j, (name, ms, nbytes) in enumerate(ks):
+            key = (j, name)
+            if key not in ksum:
+                ksum[key] = [0.0, nbytes, 0]
+                korder.append(key)
+            ksum[key][0] += ms
+            ksum[key][2] += 1
+    peak, peak_kind = measured_peak_gbs()
+    kernels = []
+    for key in korder:
+        tot, nbytes, cnt = ksum[key]
+        avg_ms = tot / cnt
+        kernels.append({"kernel": "%d:%s" % key, "avg_ms": avg_ms, "bytes": nbytes,
+                        "gbs": nbytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else None})
+    dom = max(kernels, key=lambda k: k["avg_ms"])
+    path_gbs = io * args.steps * 1.0 / seconds / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
+        "frac": dom["gbs"] / peak, "traffic": None, "peak_kind": peak_kind,
+        "path": {"io_bytes_per_step": io, "achieved": path_gbs, "frac": path_gbs / peak},
+        "kernels": kernels,
+    }
+
+    # ---- end to end: host buffers in, host buffers out, through tm_edt_host ----
+    e2e = None
+    if not args.no_e2e:
+        hm = host_mask.pin_memory()
+        hd = torch.empty(shape, dtype=torch.float32, pin_memory=True) if w.want_dist else None
+        hs = torch.empty(shape, dtype=torch.int64, pin_memory=True) if w.want_sq else None
+        hx = torch.empty(shape[:2] + (w.ndim,) + shape[2:], dtype=torch.int64, pin_memory=True) if w.want_idx else None
+        e2e_steps = max(3, min(args.steps, int(2e9 // max(io, 1)) or 3))
+        kw = dict(return_distances=w.want_dist, return_sqdist=w.want_sq, return_indices=w.want_idx,
+                  distances=hd, sqdist=hs, indices=hx)
+        for _ in range(2):
+            binding.tm_edt_host(hm, w.sampling, **kw)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            binding.tm_edt_host(hm, w.sampling, **kw)
+            stream.synchronize()  # the caller reads the host result every step
+        e1.record(stream)
+        torch.cuda.synchronize()
+        es = max_over_ranks(e0.elapsed_time(e1) / 1e3, world, dev)
+        e2e = {"value": whole_job_rate(w.voxels * e2e_steps, world, es) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": w.voxels, "d2h_bytes_per_step": io - w.voxels, "steps": e2e_steps}
+    sampler.stop()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+
+        v, secs, what = time_oracle(w, args.cpu_voxels)
+        cpu = {"value": v, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": what,
+               "seconds": secs}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.sampling is not None else "f32 (exact integers)", "data": "synthetic",
+            "config": {"workload": w.name, "shape": list(shape), "sampling": w.sampling,
+                       "outputs": [n for n, f in (("dist_f32", w.want_dist), ("sqdist_i64", w.want_sq),
+                                                   ("indices_i64", w.want_idx)) if f],
+                       "voxels_per_step": w.voxels, "l2": "rotating %d buffer sets, %d MB per set" % (sets, io >> 20),
+                       "sha256": w.sha256()[:16]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

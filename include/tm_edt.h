@@ -109,6 +109,21 @@ TM_EDT_API int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, c
 TM_EDT_API int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
                 int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
 
+/*
+ * Measurement aid: tm_edt_ws with a CUDA event recorded on `stream` before every kernel and after the
+ * last, then a wait for the last event (this entry point DOES block the calling thread).  On return
+ * kernel_ms[i] is the device time from the start of kernel i to the start of kernel i + 1 (or to the end
+ * of the call) in milliseconds, kernel_bytes[i] the bytes that launch has to read and write once (its
+ * inputs plus its outputs), kernel_names + 48 * i a NUL-terminated label, and *n_kernels how many
+ * entries were written (at most max_kernels).  kernel_bytes and kernel_names may be NULL.  The transform's outputs are
+ * written as by tm_edt_ws (same operation: Section 2.3.2; the timing protocol follows the paper's
+ * Results, "Protocol": explicit synchronisation inside the timed region).
+ */
+TM_EDT_API int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling,
+                              float* out_dist, int64_t* out_sqdist, int64_t* out_indices, void* workspace,
+                              size_t workspace_bytes, tm_edt_stream_t stream, int max_kernels, float* kernel_ms,
+                              double* kernel_bytes, char* kernel_names, int* n_kernels);
+
 /* Static description of a status code. Never NULL. */
 TM_EDT_API const char* tm_edt_strerror(int status);
 

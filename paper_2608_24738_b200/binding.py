@@ -19,7 +19,7 @@ MAX_DIMS = 8
 MAX_EXTENT = 8192
 
 EXPORTS = (
-    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_workspace_bytes", "tm_edt_strerror",
+    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_profile", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count",
 )
 
@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_ws.restype = i
             L.tm_edt_host.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
             L.tm_edt_host.restype = i
+            L.tm_edt_profile.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp, i, vp, vp, vp, vp]
+            L.tm_edt_profile.restype = i
             L.tm_edt_workspace_bytes.argtypes = [i, vp]
             L.tm_edt_workspace_bytes.restype = sz
             L.tm_edt_strerror.argtypes = [i]
@@ -185,3 +187,51 @@ def tm_edt_host(mask, sampling=None, return_distances=True, return_indices=False
                        _raw_stream(stream))
     _check(rc)
     return {"dist": d, "sq": s, "idx": x}
+
+
+def tm_edt_profile(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
+                   distances=None, indices=None, sqdist=None, workspace=None, stream=None):
+    """tm_edt_ws with per-kernel device times: returns (outputs dict, [(kernel label, milliseconds, bytes the launch must move), ...]).
+    Blocks until the work is done.  ``workspace`` is required when the shape needs scratch."""
+    import torch
+
+    L = lib()
+    mask, shape, ndim, d, s, x = _prepare(
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+    if workspace is None:
+        workspace = torch.empty(max(1, tm_edt_workspace_bytes(shape)), dtype=torch.uint8, device=mask.device)
+    kmax = 32
+    ms = (ctypes.c_float * kmax)()
+    nbytes = (ctypes.c_double * kmax)()
+    names = ctypes.create_string_buffer(48 * kmax)
+    n = ctypes.c_int(0)
+    rc = L.tm_edt_profile(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
+                          _p(workspace), ctypes.c_size_t(workspace.numel()), _raw_stream(stream), kmax, ms, nbytes, names,
+                          ctypes.byref(n))
+    _check(rc)
+    out = [(names.raw[48 * k: 48 * k + 48].split(b"\0", 1)[0].decode(), float(ms[k]), float(nbytes[k]))
+           for k in range(n.value)]
+    return {"dist": d, "sq": s, "idx": x}, out
+
+
+class PreparedCall:
+    """A tm_edt_ws call with its arguments marshalled once, for callers that repeat it (benchmarks, loops)."""
+
+    def __init__(self, mask, sampling=None, distances=None, sqdist=None, indices=None, workspace=None):
+        import torch
+
+        self._L = lib()
+        self.mask, self.shape, self.ndim, self.d, self.s, self.x = _prepare(
+            mask, sampling, distances is not None, sqdist is not None, indices is not None, distances, sqdist,
+            indices, mask.device)
+        need = tm_edt_workspace_bytes(self.shape)
+        if workspace is None:
+            workspace = torch.empty(max(1, need), dtype=torch.uint8, device=mask.device)
+        self.ws = workspace
+        self._args = (_p(self.mask), self.ndim, _shape_array(self.shape), _sampling_array(sampling, self.ndim),
+                      _p(self.d), _p(self.s), _p(self.x), _p(self.ws), ctypes.c_size_t(self.ws.numel()))
+
+    def __call__(self, stream_ptr):
+        rc = self._L.tm_edt_ws(*self._args, stream_ptr)
+        if rc != OK:
+            _check(rc)

@@ -15,6 +15,27 @@ namespace tmedt {
 static thread_local int g_last_cuda_error = 0;
 static thread_local int g_last_launches = 0;
 
+// Optional per-kernel timing (tm_edt_profile): an event is recorded on the stream before every launch
+// and once after the last one.
+constexpr int kProfMax = 32;
+struct Profiler {
+    bool active = false;
+    int count = 0;
+    cudaEvent_t ev[kProfMax + 1];
+    const char* name[kProfMax];
+    double bytes[kProfMax];
+};
+static thread_local Profiler g_prof;
+
+// `bytes`: what this launch has to read and write once (its inputs plus its outputs).
+static void prof_mark(cudaStream_t st, const char* name, double bytes) {
+    if (!g_prof.active || g_prof.count >= kProfMax) return;
+    cudaEventRecord(g_prof.ev[g_prof.count], st);
+    g_prof.name[g_prof.count] = name;
+    g_prof.bytes[g_prof.count] = bytes;
+    ++g_prof.count;
+}
+
 // The contiguous (B, C, n_0 .. n_{d-1}) array is, for the pass along spatial axis a, a
 // (outer, n_a, inner) array.  Axes of extent 1 are never processed (their pass is the identity).
 // Processing order: last spatial axis first ("plane" p = p-th processed axis).
@@ -114,11 +135,17 @@ static void fill_epilogue(const Plan& pl, float* dist, int64_t* sq, int64_t* idx
     for (int a = 0; a < kMaxDims; ++a) ep.plane_of_axis[a] = a < pl.ndim ? pl.plane_of_axis[a] : -1;
 }
 
+static double out_bytes_per_voxel(const EpilogueParams& ep) {
+    return (ep.dist ? 4.0 : 0.0) + (ep.sq ? 8.0 : 0.0) + (ep.idx ? 8.0 * ep.ndim : 0.0);
+}
+
 template <typename OT>
 static cudaError_t launch_pass0(const Plan& pl, const uint8_t* in, void* out, bool final_pass,
                                 const EpilogueParams& ep, cudaStream_t st) {
     Pass0Params P;
     P.in = in; P.out = out; P.n = pl.ext[0]; P.lines = pl.N / pl.ext[0]; P.w = pl.w[0];
+    prof_mark(st, P.n <= 32 ? "pass0_short" : "pass0_long",
+              (double)pl.N * (1.0 + (final_pass ? out_bytes_per_voxel(ep) : (double)sizeof(OT))));
     if (P.n <= 32) {
         const int per_warp = 32 / P.n;
         const int64_t warps = (P.lines + per_warp - 1) / per_warp;
@@ -148,6 +175,8 @@ static cudaError_t launch_axis_k(const AxisParams& P, const EpilogueParams& ep, 
         if (e != cudaSuccess) return e;
     }
     const int64_t blocks = (P.lines + threads - 1) / threads;
+    prof_mark(st, FINAL ? "axis_pass_final" : "axis_pass",
+              (double)P.lines * P.n * (K * (double)sizeof(OT) + (FINAL ? out_bytes_per_voxel(ep) : (K + 1.0) * sizeof(OT))));
     kern<<<(unsigned)blocks, threads, smem, st>>>(P, ep);
     return cudaGetLastError();
 }
@@ -344,6 +373,45 @@ const char* tm_edt_strerror(int status) {
         case TM_EDT_ERR_CUDA: return "CUDA runtime error";
     }
     return "unknown status";
+}
+
+int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                   int64_t* out_sqdist, int64_t* out_indices, void* workspace, size_t workspace_bytes,
+                   tm_edt_stream_t stream, int max_kernels, float* kernel_ms, double* kernel_bytes, char* kernel_names,
+                   int* n_kernels) {
+    if (!kernel_ms || !n_kernels || max_kernels < 1) return TM_EDT_ERR_INVALID_ARG;
+    *n_kernels = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    g_prof.count = 0;
+    for (int i = 0; i <= kProfMax; ++i)
+        if (cudaEventCreate(&g_prof.ev[i]) != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(g_prof.ev[j]);
+            g_last_cuda_error = (int)cudaGetLastError();
+            return TM_EDT_ERR_CUDA;
+        }
+    g_prof.active = true;
+    int rc = tm_edt_ws(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, workspace, workspace_bytes,
+                       stream);
+    g_prof.active = false;
+    const int cnt = g_prof.count;
+    if (rc == TM_EDT_OK && cnt > 0) {
+        cudaEventRecord(g_prof.ev[cnt], st);
+        cudaError_t e = cudaEventSynchronize(g_prof.ev[cnt]);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = TM_EDT_ERR_CUDA; }
+        for (int i = 0; rc == TM_EDT_OK && i < cnt && i < max_kernels; ++i) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, g_prof.ev[i], g_prof.ev[i + 1]);
+            kernel_ms[i] = ms;
+            if (kernel_bytes) kernel_bytes[i] = g_prof.bytes[i];
+            if (kernel_names) {
+                strncpy(kernel_names + (size_t)i * 48, g_prof.name[i], 47);
+                kernel_names[(size_t)i * 48 + 47] = 0;
+            }
+        }
+        if (rc == TM_EDT_OK) *n_kernels = cnt < max_kernels ? cnt : max_kernels;
+    }
+    for (int i = 0; i <= kProfMax; ++i) cudaEventDestroy(g_prof.ev[i]);
+    return rc;
 }
 
 int tm_edt_last_cuda_error(void) { return g_last_cuda_error; }
