@@ -9,6 +9,8 @@
 
 #include "edt_common.cuh"
 #include "edt_generic.cuh"
+#include "edt_fast.cuh"
+#include <stdlib.h>
 
 namespace tmedt {
 
@@ -51,6 +53,7 @@ struct Plan {
     bool unit = true;
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
+    bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
 };
@@ -120,6 +123,14 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     const size_t elem = pl.wide ? 2 : 1;
     pl.plane_bytes = (((size_t)pl.N * elem) + 255) & ~(size_t)255;
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
+    const char* force = getenv("TM_EDT_FORCE_GENERIC");
+    pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
+    if (pl.fast) {
+        auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+        const size_t a = E >= 3 ? up((size_t)pl.N * (E >= 5 ? 4 : 2)) : 0;
+        const size_t b = E >= 4 ? up((size_t)pl.N * 4) : 0;
+        pl.ws_bytes = a + b;
+    }
     return TM_EDT_OK;
 }
 
@@ -223,6 +234,79 @@ static cudaError_t run_generic(const Plan& pl, const uint8_t* in, const Epilogue
     return cudaSuccess;
 }
 
+template <int K, bool FINAL>
+static cudaError_t launch_column(const FastParams& P, const EpilogueParams& ep, cudaStream_t st, double out_bpv) {
+    const size_t eb = (size_t)entry_bytes(K);
+    int TX = 128;
+    while (TX > 32 && ((size_t)P.n * TX * eb + (size_t)(3 * P.n / 2 + 2) * TX > 56 * 1024 || TX / 2 >= P.inner)) TX >>= 1;
+    const size_t smem = (size_t)P.n * TX * eb + (size_t)(3 * P.n / 2 + 2) * TX;
+    auto kern = column_kernel<K, FINAL>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const int tiles = (int)((P.inner + TX - 1) / TX);
+    const int64_t blocks = P.outer * tiles;
+    const double vox = (double)P.outer * P.n * (double)P.inner;
+    prof_mark(st, FINAL ? "column_final" : "column", vox * ((double)eb + (FINAL ? out_bpv : (double)entry_bytes(K + 1))));
+    kern<<<(unsigned)blocks, TX, smem, st>>>(P, ep, tiles);
+    return cudaGetLastError();
+}
+
+template <bool FINAL>
+static cudaError_t launch_column_any(int K, const FastParams& P, const EpilogueParams& ep, cudaStream_t st,
+                                     double out_bpv) {
+    switch (K) {
+        case 2: return launch_column<2, FINAL>(P, ep, st, out_bpv);
+        case 3: return launch_column<3, FINAL>(P, ep, st, out_bpv);
+        case 4: if (FINAL) return launch_column<4, true>(P, ep, st, out_bpv);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// Packed-entry path: fused first + second axis, then one column kernel per further axis.
+static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                            int& launches) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    char* bufA = static_cast<char*>(ws);
+    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * (pl.E >= 5 ? 4 : 2)) : 0);
+    const double out_bpv = out_bytes_per_voxel(ep);
+    auto fill = [&](FastParams& P, int k) {
+        memset(&P, 0, sizeof(P));
+        P.n = pl.ext[k]; P.inner = pl.inner[k]; P.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+        P.w2 = (float)(pl.w[k] * pl.w[k]); P.inv2w2 = (float)(0.5 / (pl.w[k] * pl.w[k]));
+        for (int p = 0; p < k && p < 4; ++p) P.w2p[p] = (float)(pl.w[p] * pl.w[p]);
+        P.unit = pl.unit ? 1 : 0;
+    };
+    FastParams P;
+    fill(P, 1);
+    P.in = in; P.out = bufA; P.n0 = pl.ext[0];
+    {
+        const int threads = (pl.ext[0] + 31) & ~31;
+        const int tstride = (pl.ext[0] + 15) & ~15;
+        const size_t smem = (size_t)pl.ext[1] * tstride + (size_t)(3 * pl.ext[1] / 2 + 2) * threads;
+        const bool fin = pl.E == 2;
+        prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
+        if (fin) plane_kernel<true><<<(unsigned)P.outer, threads, smem, st>>>(P, ep);
+        else plane_kernel<false><<<(unsigned)P.outer, threads, smem, st>>>(P, ep);
+        ++launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    char* src = bufA;
+    char* dst = bufB;
+    for (int k = 2; k < pl.E; ++k) {
+        fill(P, k);
+        P.in = src; P.out = dst;
+        const bool fin = k == pl.E - 1;
+        cudaError_t e = fin ? launch_column_any<true>(k, P, ep, st, out_bpv) : launch_column_any<false>(k, P, ep, st, out_bpv);
+        ++launches;
+        if (e != cudaSuccess) return e;
+        char* t = src; src = dst; dst = t;
+    }
+    return cudaSuccess;
+}
+
 static bool is_device_ptr(const void* p) {
     cudaPointerAttributes at;
     if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
@@ -266,7 +350,9 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     int launches = 0;
     cudaError_t e;
-    if (pl.use_double)
+    if (pl.fast)
+        e = run_fast(pl, input, ep, ws, st, launches);
+    else if (pl.use_double)
         e = pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
                     : run_generic<double, int8_t>(pl, input, ep, ws, st, launches);
     else

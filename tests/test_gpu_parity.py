@@ -20,6 +20,16 @@ def _built():
     binding.lib()
 
 
+@pytest.fixture(params=["default", "generic"])
+def path(request, monkeypatch):
+    """Both kernel families: the planner's own choice, and the rank-/extent-generic kernels forced."""
+    if request.param == "generic":
+        monkeypatch.setenv("TM_EDT_FORCE_GENERIC", "1")
+    else:
+        monkeypatch.delenv("TM_EDT_FORCE_GENERIC", raising=False)
+    return request.param
+
+
 def run_gpu(mask, sampling=None, dist=True, sq=False, idx=False, **kw):
     import torch
 
@@ -53,6 +63,8 @@ SMALL = [
     (1, 1, 9, 10, 11), (2, 1, 33, 17, 40), (1, 1, 5, 1, 6), (1, 1, 1, 1, 1), (1, 1, 140, 9, 12),
     (1, 1, 6, 5, 4, 7), (1, 1, 3, 4, 5, 3, 4), (1, 1, 2, 3, 4, 3, 2, 3), (1, 1, 3, 2, 3, 2, 3, 2, 3),
     (2, 1, 3, 2, 3, 2, 3, 2, 3, 4), (1, 1, 6, 6, 6, 6, 6, 6, 6, 6),
+    (1, 1, 128, 128), (2, 1, 127, 128), (1, 1, 128, 100), (1, 2, 50, 128, 64), (1, 1, 128, 20, 48),
+    (1, 1, 16, 40, 24, 32), (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128),
 ]
 
 
@@ -65,14 +77,14 @@ def _sampling(ndim, kind):
 @pytest.mark.parametrize("shape", SMALL, ids=["x".join(map(str, s)) for s in SMALL])
 @pytest.mark.parametrize("p_fg", [0.3, 0.9, 0.995])
 @pytest.mark.parametrize("kind", ["unit", "sampled"])
-def test_small_shapes_every_rank(shape, p_fg, kind):
+def test_small_shapes_every_rank(shape, p_fg, kind, path):
     seed = zlib.crc32(repr((shape, p_fg, kind)).encode())
     mask = workloads.random_mask(seed, shape, p_fg)
     full_check(mask, _sampling(len(shape) - 2, kind))
 
 
 @pytest.mark.parametrize("shape", [(1, 1, 64), (2, 1, 20, 30), (1, 2, 8, 9, 10), (1, 1, 200, 40)])
-def test_degenerate_masks(shape):
+def test_degenerate_masks(shape, path):
     ndim = len(shape) - 2
     allfg = np.ones(shape, dtype=np.uint8)
     r = run_gpu(allfg, None, True, True, True)
@@ -97,7 +109,7 @@ def test_degenerate_masks(shape):
     full_check(m.astype(np.uint8), None)
 
 
-def test_mixed_batch_with_image_without_background():
+def test_mixed_batch_with_image_without_background(path):
     mask = workloads.random_mask(77, (3, 2, 20, 21, 22), 0.9)
     mask[1, 1] = 1
     res, ref = full_check(mask, (2.5, 0.8, 1.0))
@@ -105,7 +117,7 @@ def test_mixed_batch_with_image_without_background():
     assert np.isfinite(res["dist"][0, 0]).all()
 
 
-def test_half_space_and_far_sites():
+def test_half_space_and_far_sites(path):
     mask = np.ones((1, 1, 128, 96), dtype=np.uint8)
     mask[0, 0, :3] = 0
     full_check(mask, None)
@@ -197,7 +209,7 @@ def test_host_buffer_entry_point():
     assert ei.value.status == binding.ERR_BAD_POINTER
 
 
-def test_config1_brute_force_every_voxel():
+def test_config1_brute_force_every_voxel(path):
     w = workloads.config1()
     ref = oracle.brute(w.mask, w.sampling)
     res = run_gpu(w.mask, None, True, True, True)
