@@ -205,6 +205,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-steps", type=int, default=20)
+    ap.add_argument("--unit-sampling", action="store_true", help="override the workload's sampling with 1.0 per axis")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()
@@ -212,6 +213,9 @@ def main():
     from paper_2608_24738_b200 import workloads
 
     w = workloads.CONFIGS[args.config]()
+    if args.unit_sampling:
+        w.sampling = None
+        w.name += " (unit sampling)"
     if args.impl == "reference":
         run_reference(args, w, world, rank)
         return

@@ -1,30 +1,30 @@
 // Fast path for extents up to 128 and at most five processed axes.
 //
-// Carry layout ("entries"): after p + 1 processed axes every voxel holds one little packed entry whose
-// byte q (q <= p) is the signed offset  site_q - x_q  along processed axis q (plane order: contiguous
-// axis first); 1, 2, 4 bytes for 1, 2, 3..4 axes.  Byte 0 == 0x80 marks "no site yet".  An entry of
-// all zeros is a background voxel.  Entries make every load, gather and store of a voxel one access.
+// Carry layout ("entries"): after p + 1 processed axes every voxel holds one packed entry whose byte q
+// (q <= p) is the signed offset  site_q - x_q  along processed axis q (plane order: contiguous axis
+// first); 1, 2, 4 bytes for 1, 2, 3..4 axes.  Byte 0 == 0x80 marks "no site yet".  An entry of all
+// zeros is a background voxel.  Entries make every load, gather and store of a voxel one access.
 //
 // Kernels:
 //   plane_kernel   first axis + second axis fused: one thread block per (n_1 x n_0) plane.  The rows
 //                  of the raw mask are bit-packed with warp ballots and turned into 1-byte offsets in
-//                  shared memory (first-axis pass), then one thread per column runs the envelope pass
-//                  along axis 1 on the shared tile and writes 2-byte entries or the final outputs.
+//                  shared memory (first-axis pass); then the pass along axis 1 runs on that tile and
+//                  writes 2-byte entries or the final outputs.
 //   column_kernel  one further axis: a block stages an (n x TX) tile of entries in shared memory
-//                  (TX consecutive positions of the contiguous `inner` index), one thread per column
-//                  runs the envelope pass, outputs go straight to global memory (a warp writes one
-//                  contiguous run per row).
+//                  (TX consecutive positions of the contiguous `inner` index) and runs the pass on it.
 //
-// Envelope pass of one column (lower envelope of parabolas, paper Section 2.3.2; here split at
-// background voxels).  A background voxel has height 0, so no site beyond it can matter to the voxels
-// before it: the column falls apart into independent runs of foreground voxels, each bounded by the
-// background voxels next to it.  Background rows cost a load and a store.  Within a run the sites are
-// pushed on a stack of row numbers (one byte each, in shared memory); site v between u and w is dropped
-// when the parabola intersections are out of order, tested without division:
-//     (H_v - H_u) (w - v) >= (H_w - H_v) (v - u),   H_s = h_s + w^2 s^2.
-// The two top entries are cached in registers.  The query walks the surviving sites upward and moves
-// to the next one past their intersection  x* = (H_next - H_cur) / (2 w^2 (next - cur)).
-// All arithmetic is float32; for unit sampling every value is an integer below 2^24, hence exact.
+// The pass along an axis (g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (w_k (x_k - j))^2 ], paper
+// Section 2.3.2) is taken voxel by voxel as an exact bounded scan instead of a sequential envelope
+// sweep: starting from the voxel's own height, rows at distance d = 1, 2, .. on both sides are tried
+// and the scan stops as soon as w^2 d^2 >= best, because no farther row can then be smaller.  The
+// scan length is about the voxel's distance to the background along the axis -- short on real masks,
+// and never more than the extent (<= 128).  Every voxel is independent, a warp works on 32 neighbouring
+// columns of the same row (loads and stores are contiguous runs, neighbouring voxels have similar scan
+// lengths), and background voxels (height 0) leave the loop at once.
+//
+// Unit sampling: heights are integers; the tile holds keys (height << 8 | row) so that one fused
+// add-and-min instruction per candidate tracks value and site together, exactly.  Other sampling:
+// heights are float32, the site is tracked by a compare and select.
 #pragma once
 #include "edt_common.cuh"
 
@@ -44,77 +44,90 @@ struct FastParams {
     int n;               // extent of the axis of this pass
     int n0;              // plane kernel: extent of the contiguous axis (== inner)
     float w2;            // squared sampling of this axis
-    float inv2w2;        // 1 / (2 w2)
     float w2p[4];        // squared sampling of the earlier axes (plane order)
-    int unit;            // all sampling == 1
 };
+
+// add[d] = w^2 d^2 for the axis of the pass: float32 bits (sampled) or d^2 << shift (unit sampling keys).
+struct ScanTab { uint32_t add[132]; };
+
+constexpr uint32_t kNoneKey = 0xF0000000u;
+#define TMEDT_INF (__int_as_float(0x7f800000))
 
 __device__ __forceinline__ float small_int_to_float(int v) {  // exact for 0 <= v < 2^23, two full-rate ops
     return __int_as_float(v | 0x4B000000) - 8388608.0f;
 }
 
-template <int K> __device__ __forceinline__ bool entry_none(uint32_t e) { return (e & 0xffu) == 0x80u; }
+__device__ __forceinline__ bool entry_none(uint32_t e) { return (e & 0xffu) == 0x80u; }
 
-template <int K>
-__device__ __forceinline__ float entry_height(uint32_t e, const float* w2p, bool unit) {
-    int o0 = (int)(int8_t)(e & 0xff);
-    if (unit) {
-        int s = o0 * o0;
-        if (K > 1) { int o = (int)(int8_t)((e >> 8) & 0xff); s += o * o; }
-        if (K > 2) { int o = (int)(int8_t)((e >> 16) & 0xff); s += o * o; }
-        if (K > 3) { int o = (int)(int8_t)((e >> 24) & 0xff); s += o * o; }
-        return small_int_to_float(s);
-    }
-    float h = w2p[0] * small_int_to_float(o0 * o0);
-    if (K > 1) { int o = (int)(int8_t)((e >> 8) & 0xff); h = fmaf(w2p[1], small_int_to_float(o * o), h); }
-    if (K > 2) { int o = (int)(int8_t)((e >> 16) & 0xff); h = fmaf(w2p[2], small_int_to_float(o * o), h); }
-    if (K > 3) { int o = (int)(int8_t)((e >> 24) & 0xff); h = fmaf(w2p[3], small_int_to_float(o * o), h); }
-    return h;
+template <int K> __device__ __forceinline__ int entry_sumsq(uint32_t e) {
+    int o = (int)(int8_t)(e & 0xff);
+    int s = o * o;
+    if (K > 1) { o = (int)(int8_t)((e >> 8) & 0xff); s += o * o; }
+    if (K > 2) { o = (int)(int8_t)((e >> 16) & 0xff); s += o * o; }
+    if (K > 3) { o = (int)(int8_t)((e >> 24) & 0xff); s += o * o; }
+    return s;
 }
 
-// Per-column output sink.
+// Tile value the scan works on: unit sampling -> key (sum of squared offsets << 8 | row), none -> kNoneKey;
+// otherwise the bits of the float32 height sum_q w_q^2 off_q^2, none -> +inf.
+template <int K, bool UNIT>
+__device__ __forceinline__ uint32_t scan_value(uint32_t e, int row, const float* w2p) {
+    if (UNIT) return entry_none(e) ? kNoneKey : (((uint32_t)entry_sumsq<K>(e) << 8) | (uint32_t)row);
+    if (entry_none(e)) return 0x7f800000u;
+    int o = (int)(int8_t)(e & 0xff);
+    float h = w2p[0] * small_int_to_float(o * o);
+    if (K > 1) { o = (int)(int8_t)((e >> 8) & 0xff); h = fmaf(w2p[1], small_int_to_float(o * o), h); }
+    if (K > 2) { o = (int)(int8_t)((e >> 16) & 0xff); h = fmaf(w2p[2], small_int_to_float(o * o), h); }
+    if (K > 3) { o = (int)(int8_t)((e >> 24) & 0xff); h = fmaf(w2p[3], small_int_to_float(o * o), h); }
+    return __float_as_uint(h);
+}
+
+// Where the results of one column (fixed thread <-> column) go.
 template <int K, bool FINAL>
 struct ColumnOut {
-    // non-final
-    typename EntryType<entry_bytes(K + 1)>::type* out;  // &out[first voxel of the column]
-    // final
-    float* dist; int64_t* sq; int64_t* idx;  // &buf[image base + first voxel of the column]; idx: plane 0 of image
+    typename EntryType<entry_bytes(K + 1)>::type* out;  // non-final: &out[row 0 of the column]
+    float* dist; int64_t* sq; int64_t* idx;             // final: &buf[row 0 of the column] (idx: plane 0 of image)
     int64_t stride;      // distance between consecutive rows of the column, in voxels
     int64_t V;           // voxels per image (index-plane stride)
     int coord[4];        // own coordinates along the earlier planes
-    int axis[5];         // spatial axis of plane p
+    int axis[5];         // spatial axis of plane q
     int ndim;
-    bool unit;
+    bool dist_only;      // final: only out_dist was requested
 };
 
-template <int K, bool FINAL>
-__device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, uint32_t e, int offk, float h, bool none) {
+__device__ __forceinline__ float fast_sqrt(float v) {
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+
+// Emits row y of a column given the chosen site row j (or none), the site's entry and the squared distance.
+template <int K, bool FINAL, bool UNIT>
+__device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j, uint32_t e, float sqv, bool none) {
+    const int64_t p = (int64_t)y * o.stride;
     if (!FINAL) {
         using EO = typename EntryType<entry_bytes(K + 1)>::type;
-        uint32_t v = none ? 0x80u : (e | ((uint32_t)(uint8_t)(int8_t)offk << (8 * (K & 3))));
-        o.out[(int64_t)y * o.stride] = (EO)v;
+        const uint32_t v = none ? 0x80u : (e | ((uint32_t)((j - y) & 0xff) << (8 * (K & 3))));
+        o.out[p] = (EO)v;
         return;
     }
-    const int64_t p = (int64_t)y * o.stride;
+    // unit sampling: sqv is an exact integer below 2^24 and the root is correctly rounded; otherwise the
+    // approximate root (relative error about 1e-7) is far inside the float32 result's own rounding.
+    const float dv = none ? TMEDT_INF : (UNIT ? __fsqrt_rn(sqv) : fast_sqrt(sqv));
+    if (o.dist_only) { o.dist[p] = dv; return; }
+    if (o.dist) o.dist[p] = dv;
     if (none) {
-        if (o.dist) o.dist[p] = __int_as_float(0x7f800000);
         if (o.sq) o.sq[p] = INT64_MAX;
         if (o.idx)
             for (int a = 0; a < o.ndim; ++a) o.idx[(int64_t)a * o.V + p] = -1;
         return;
     }
-    if (o.dist) o.dist[p] = o.unit ? __fsqrt_rn(h) : sqrtf(h);
-    int off[5];
-#pragma unroll
-    for (int q = 0; q < K; ++q) off[q] = (int)(int8_t)((e >> (8 * q)) & 0xff);
-    off[K] = offk;
-    if (o.sq) {
-        int s = 0;
-#pragma unroll
-        for (int q = 0; q <= K; ++q) s += off[q] * off[q];
-        o.sq[p] = (int64_t)s;
-    }
+    if (o.sq) o.sq[p] = (int64_t)sqv;  // unit sampling only
     if (o.idx) {
+        int off[5];
+#pragma unroll
+        for (int q = 0; q < K; ++q) off[q] = (int)(int8_t)((e >> (8 * q)) & 0xff);
+        off[K] = j - y;
         // axes of extent 1 keep index 0; processed axes get own coordinate + offset
         for (int a = 0; a < o.ndim; ++a) {
             int64_t val = 0;
@@ -126,129 +139,139 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, uint32
     }
 }
 
-// One column of a shared-memory tile.  tile[y * tstride] is the entry of row y (ET = tile element type),
-// stk[k * sstride] the k-th stack slot of this column (3n/2 + 2 slots).
-//
-// Two sweeps, both with all lanes of a warp on the same row, so that the row's loads and stores are one
-// contiguous run per warp.  Sweep 1 builds, run by run, the surviving sites; the segments of successive
-// runs follow one another on the stack, each run's last slot carrying an end mark (bit 7; rows are
-// below 128).  Background rows that do not touch a run are not on the stack at all.  Sweep 2 emits the
-// outputs: background rows directly, foreground rows by walking the segment of their run.
-template <int K, bool FINAL, typename ET>
-__device__ __forceinline__ void column_pass(const ET* __restrict__ tile, int tstride, uint8_t* __restrict__ stk,
-                                            int sstride, int n, const FastParams& P,
-                                            const ColumnOut<K, FINAL>& out) {
-    const float w2 = P.w2, inv2w2 = P.inv2w2;
-    const bool unit = P.unit != 0;
-    float w2p[4] = {P.w2p[0], P.w2p[1], P.w2p[2], P.w2p[3]};
-
-    // ---- sweep 1: build ----
-    int k = -1;                 // top slot
-    int base = 0;               // first slot of the open run
-    int s1 = 0, s0 = 0;         // rows of the top and below-top entries of the open run
-    float fs1 = 0.f, fs0 = 0.f, H1 = 0.f, H0 = 0.f, D10 = 0.f, d10 = 0.f;
-    bool open = false;          // a run of foreground rows is open
-    int lastbg = -1;            // most recent background row
-
-    auto push = [&](int u, float fu, float Hu) {
-        while (k > base) {
-            if (D10 * (fu - fs1) >= (Hu - H1) * d10) {  // top is nowhere the minimum: pop
-                --k; s1 = s0; fs1 = fs0; H1 = H0;
-                if (k > base) {
-                    s0 = stk[(k - 1) * sstride];
-                    fs0 = small_int_to_float(s0);
-                    H0 = fmaf(w2 * fs0, fs0, entry_height<K>((uint32_t)tile[s0 * tstride], w2p, unit));
-                    D10 = H1 - H0; d10 = fs1 - fs0;
-                }
-            } else break;
+// ---------------------------------------------------------------------------------------------
+// Bounded scans of one voxel (row y of the column col[row * VS]).  All lanes of a warp share y, so the
+// loop bounds are warp-uniform; lanes leave individually once add[d] >= best.
+// ---------------------------------------------------------------------------------------------
+// Unit sampling: keys carry the site, one fused add-min per candidate.
+template <int VS>
+__device__ __forceinline__ uint32_t scan_keys(const uint32_t* __restrict__ col, int n, int y, const ScanTab& tab) {
+    uint32_t best = col[y * VS];
+    const int up = y, dn = n - 1 - y, m = min(up, dn);
+    const uint32_t* plo = col + (y - 1) * VS;
+    const uint32_t* phi = col + (y + 1) * VS;
+    int d = 1;
+    for (; d + 1 <= m; d += 2) {
+        const uint32_t a0 = tab.add[d], a1 = tab.add[d + 1];
+        if (a0 >= best) return best;
+        best = __viaddmin_u32(plo[0], a0, best);
+        best = __viaddmin_u32(phi[0], a0, best);
+        best = __viaddmin_u32(plo[-VS], a1, best);
+        best = __viaddmin_u32(phi[VS], a1, best);
+        plo -= 2 * VS; phi += 2 * VS;
+    }
+    if (d <= m) {
+        const uint32_t a0 = tab.add[d];
+        if (a0 >= best) return best;
+        best = __viaddmin_u32(plo[0], a0, best);
+        best = __viaddmin_u32(phi[0], a0, best);
+        plo -= VS; phi += VS; ++d;
+    }
+    if (up > dn) {
+        for (; d <= up; ++d, plo -= VS) {
+            const uint32_t a0 = tab.add[d];
+            if (a0 >= best) return best;
+            best = __viaddmin_u32(plo[0], a0, best);
         }
-        ++k;
-        stk[k * sstride] = (uint8_t)u;
-        s0 = s1; fs0 = fs1; H0 = H1;
-        s1 = u; fs1 = fu; H1 = Hu;
-        D10 = H1 - H0; d10 = fs1 - fs0;
-    };
-
-    {
-        float fy = 0.f;
-        for (int y = 0; y < n; ++y, fy += 1.0f) {
-            const uint32_t e = (uint32_t)tile[y * tstride];
-            if (e == 0u) {  // background voxel
-                if (open) {  // closes the run: it is the run's last site
-                    push(y, fy, w2 * fy * fy);
-                    stk[k * sstride] = (uint8_t)(y | 0x80);
-                    open = false;
-                }
-                lastbg = y;
-                continue;
-            }
-            if (!open) {  // first foreground row after background (or row 0): start a run
-                open = true;
-                base = k + 1;
-                if (lastbg >= 0) {
-                    k = base;
-                    stk[k * sstride] = (uint8_t)lastbg;
-                    s1 = lastbg; fs1 = small_int_to_float(lastbg); H1 = w2 * fs1 * fs1;
-                }
-            }
-            if (entry_none<K>(e)) continue;  // foreground without a site so far: no site, still in the run
-            push(y, fy, fmaf(w2 * fy, fy, entry_height<K>(e, w2p, unit)));
+    } else {
+        for (; d <= dn; ++d, phi += VS) {
+            const uint32_t a0 = tab.add[d];
+            if (a0 >= best) return best;
+            best = __viaddmin_u32(phi[0], a0, best);
         }
     }
-    const int ktop = k;  // last slot in use (-1: the column has no site at all)
+    return best;
+}
 
-    // ---- sweep 2: emit ----
-    int kc = -1;                // slot of the current site
-    bool in_run = false, last = true;   // `last`: the current site is the last of its run
-    int sc = 0; uint32_t ec = 0; float fsc = 0.f, hc = 0.f, Hc = 0.f;
-    int sn = 0; uint32_t en = 0; float fsn = 0.f, hn = 0.f, Hn = 0.f;
-    bool nlast = true;
-    float xb = __int_as_float(0x7f800000);
-    auto load_site = [&](int slot, int& s, uint32_t& e, float& fs, float& h, float& H, bool& is_last) {
-        const int raw = stk[slot * sstride];
-        is_last = (raw & 0x80) != 0 || slot == ktop;
-        s = raw & 0x7f;
-        e = (uint32_t)tile[s * tstride];
-        fs = small_int_to_float(s);
-        h = entry_height<K>(e, w2p, unit);
-        H = fmaf(w2 * fs, fs, h);
-    };
-    auto load_next = [&]() {
-        if (!last) {
-            load_site(kc + 1, sn, en, fsn, hn, Hn, nlast);
-            xb = __fdividef((Hn - Hc) * inv2w2, fsn - fsc);
+// Float heights.  ARG: also returns the distance bd (0 = own row) at which the minimum was found.
+template <int VS, bool ARG>
+__device__ __forceinline__ float scan_heights(const uint32_t* __restrict__ col, int n, int y, const ScanTab& tab,
+                                              int& bd) {
+    float best = __uint_as_float(col[y * VS]);
+    bd = 0;
+    const int up = y, dn = n - 1 - y, m = min(up, dn);
+    const uint32_t* plo = col + (y - 1) * VS;
+    const uint32_t* phi = col + (y + 1) * VS;
+    int d = 1;
+    for (; d + 1 <= m; d += 2) {
+        const float a0 = __uint_as_float(tab.add[d]), a1 = __uint_as_float(tab.add[d + 1]);
+        if (a0 >= best) return best;
+        const float c0 = fminf(__uint_as_float(plo[0]), __uint_as_float(phi[0])) + a0;
+        const float c1 = fminf(__uint_as_float(plo[-VS]), __uint_as_float(phi[VS])) + a1;
+        if (ARG) {
+            if (c0 < best) { best = c0; bd = d; }
+            if (c1 < best) { best = c1; bd = d + 1; }
         } else {
-            xb = __int_as_float(0x7f800000);
+            best = fminf(best, fminf(c0, c1));
         }
-    };
-    float fy = 0.f;
-    for (int y = 0; y < n; ++y, fy += 1.0f) {
-        const uint32_t e = (uint32_t)tile[y * tstride];
-        if (e == 0u) {
-            emit<K, FINAL>(out, y, 0u, 0, 0.f, false);
-            in_run = false;
-            continue;
-        }
-        if (ktop < 0) {  // no site in the whole column
-            emit<K, FINAL>(out, y, 0u, 0, 0.f, true);
-            continue;
-        }
-        if (!in_run) {  // first row of a run: move to the first slot of its segment
-            in_run = true;
-            if (kc >= 0) {
-                while (!last) { ++kc; last = (stk[kc * sstride] & 0x80) != 0 || kc == ktop; }
-            }
-            ++kc;
-            load_site(kc, sc, ec, fsc, hc, Hc, last);
-            load_next();
-        }
-        while (fy > xb) {
-            ++kc; sc = sn; ec = en; fsc = fsn; hc = hn; Hc = Hn; last = nlast;
-            load_next();
-        }
-        const float d = fsc - fy;
-        emit<K, FINAL>(out, y, ec, sc - y, fmaf(w2 * d, d, hc), false);
+        plo -= 2 * VS; phi += 2 * VS;
     }
+    if (d <= m) {
+        const float a0 = __uint_as_float(tab.add[d]);
+        if (a0 >= best) return best;
+        const float c0 = fminf(__uint_as_float(plo[0]), __uint_as_float(phi[0])) + a0;
+        if (ARG) { if (c0 < best) { best = c0; bd = d; } } else best = fminf(best, c0);
+        plo -= VS; phi += VS; ++d;
+    }
+    if (up > dn) {
+        for (; d <= up; ++d, plo -= VS) {
+            const float a0 = __uint_as_float(tab.add[d]);
+            if (a0 >= best) return best;
+            const float c0 = __uint_as_float(plo[0]) + a0;
+            if (ARG) { if (c0 < best) { best = c0; bd = d; } } else best = fminf(best, c0);
+        }
+    } else {
+        for (; d <= dn; ++d, phi += VS) {
+            const float a0 = __uint_as_float(tab.add[d]);
+            if (a0 >= best) return best;
+            const float c0 = __uint_as_float(phi[0]) + a0;
+            if (ARG) { if (c0 < best) { best = c0; bd = d; } } else best = fminf(best, c0);
+        }
+    }
+    return best;
+}
+
+// Scan of one voxel followed by its output.  ent[row * ES] are the entries of the column.
+template <int K, bool FINAL, bool UNIT, int VS, typename ET>
+__device__ __forceinline__ void scan_voxel(const uint32_t* __restrict__ col, const ET* __restrict__ ent, int ES, int n,
+                                           int y, const ScanTab& tab, const ColumnOut<K, FINAL>& out) {
+    int j;
+    float sqv;
+    bool none;
+    if (UNIT) {
+        const uint32_t best = scan_keys<VS>(col, n, y, tab);
+        none = best >= kNoneKey;
+        j = (int)(best & 0xffu);
+        sqv = small_int_to_float((int)(best >> 8));
+    } else if (FINAL) {
+        // the site itself is only needed for index output: find it only then
+        int bd;
+        if (out.dist_only) {
+            sqv = scan_heights<VS, false>(col, n, y, tab, bd);
+            emit<K, FINAL, UNIT>(out, y, y, 0u, sqv, sqv == TMEDT_INF);
+            return;
+        }
+        sqv = scan_heights<VS, true>(col, n, y, tab, bd);
+        none = sqv == TMEDT_INF;
+        j = y;
+        if (bd > 0) {
+            const float lo = bd <= y ? __uint_as_float(col[(y - bd) * VS]) : TMEDT_INF;
+            const float hi = y + bd < n ? __uint_as_float(col[(y + bd) * VS]) : TMEDT_INF;
+            j = lo <= hi ? y - bd : y + bd;
+        }
+    } else {
+        int bd;
+        sqv = scan_heights<VS, true>(col, n, y, tab, bd);
+        none = sqv == TMEDT_INF;
+        j = y;
+        if (bd > 0) {
+            const float lo = bd <= y ? __uint_as_float(col[(y - bd) * VS]) : TMEDT_INF;
+            const float hi = y + bd < n ? __uint_as_float(col[(y + bd) * VS]) : TMEDT_INF;
+            j = lo <= hi ? y - bd : y + bd;
+        }
+    }
+    const uint32_t e = none ? 0u : (uint32_t)ent[j * ES];
+    emit<K, FINAL, UNIT>(out, y, j, e, sqv, none);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -295,67 +318,99 @@ __device__ __forceinline__ void pass0_row_to_tile(const uint8_t* __restrict__ ro
     }
 }
 
-template <bool FINAL>
-__global__ void __launch_bounds__(128) plane_kernel(const __grid_constant__ FastParams P,
-                                                    const __grid_constant__ EpilogueParams ep) {
+template <bool FINAL, bool UNIT>
+__global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ FastParams P,
+                                                    const __grid_constant__ EpilogueParams ep,
+                                                    const __grid_constant__ ScanTab tab) {
     extern __shared__ __align__(16) uint8_t sm_plane[];
     const int n0 = P.n0, n1 = P.n;
     const int tstride = (n0 + 15) & ~15;
-    uint8_t* tile = sm_plane;                       // [n1][tstride]
-    uint8_t* stk = sm_plane + (size_t)n1 * tstride; // [3 n1 / 2 + 2][blockDim]
-    const int64_t plane = blockIdx.x;               // planes = outer
+    uint8_t* tile = sm_plane;                                                      // [n1][tstride] offsets
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_plane + (((size_t)n1 * tstride + 15) & ~(size_t)15));  // [n1][32]
+    const int64_t plane = blockIdx.x;  // planes = outer
     const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (int y = warp; y < n1; y += nwarps) pass0_row_to_tile(src + (int64_t)y * n0, n0, tile + y * tstride, lane);
     __syncthreads();
-    const int c = threadIdx.x;
-    if (c >= n0) return;
-    ColumnOut<1, FINAL> out;
-    out.stride = n0;
-    if (!FINAL) {
-        out.out = reinterpret_cast<uint16_t*>(P.out) + plane * (int64_t)n1 * n0 + c;
-    } else {
-        // two processed axes: the plane is the image
-        out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
-        out.sq = ep.sq ? ep.sq + plane * ep.V + c : nullptr;
-        out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
-        out.V = ep.V; out.ndim = ep.ndim; out.unit = P.unit != 0;
-        out.coord[0] = c;
-        out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+    const float w2p[4] = {P.w2p[0], 0.f, 0.f, 0.f};
+    const int ngroups = (n0 + 31) >> 5;
+    for (int g = 0; g < ngroups; ++g) {
+        const int c = g * 32 + lane;
+        const bool live = c < n0;
+        for (int y = warp; y < n1; y += nwarps)
+            val[y * 32 + lane] = scan_value<1, UNIT>(live ? (uint32_t)tile[y * tstride + c] : 0x80u, y, w2p);
+        __syncthreads();
+        if (live) {
+            ColumnOut<1, FINAL> out;
+            out.stride = n0;
+            if (!FINAL) {
+                out.out = reinterpret_cast<uint16_t*>(P.out) + plane * (int64_t)n1 * n0 + c;
+            } else {  // two processed axes: the plane is the image
+                out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
+                out.sq = ep.sq ? ep.sq + plane * ep.V + c : nullptr;
+                out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+                out.V = ep.V; out.ndim = ep.ndim;
+                out.dist_only = ep.dist && !ep.sq && !ep.idx;
+                out.coord[0] = c;
+                out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+            }
+            for (int y = warp; y < n1; y += nwarps)
+                scan_voxel<1, FINAL, UNIT, 32, uint8_t>(val + lane, tile + c, tstride, n1, y, tab, out);
+        }
+        __syncthreads();
     }
-    column_pass<1, FINAL, uint8_t>(tile + c, tstride, stk + c, blockDim.x, n1, P, out);
 }
 
-template <int K, bool FINAL>
-__global__ void __launch_bounds__(128) column_kernel(const __grid_constant__ FastParams P,
+template <int K, bool FINAL, bool UNIT, int TX>
+__global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ FastParams P,
                                                      const __grid_constant__ EpilogueParams ep,
+                                                     const __grid_constant__ ScanTab tab,
                                                      const int tiles_per_slab) {
     using EI = typename EntryType<entry_bytes(K)>::type;
     extern __shared__ __align__(16) uint8_t sm_col[];
-    const int TX = blockDim.x, n = P.n;
-    EI* tile = reinterpret_cast<EI*>(sm_col);                                  // [n][TX]
-    uint8_t* stk = sm_col + (size_t)n * TX * sizeof(EI);                       // [3 n / 2 + 2][TX]
+    constexpr int G = TX / 32;
+    const int n = P.n;
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_col);                  // [n][TX]
+    EI* tile = reinterpret_cast<EI*>(sm_col + (size_t)n * TX * 4);        // [n][TX]
     const int64_t slab = blockIdx.x / tiles_per_slab;
     const int64_t i0 = (int64_t)(blockIdx.x - slab * tiles_per_slab) * TX;
     const int width = (int)min((int64_t)TX, P.inner - i0);
     const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
-    // stage the tile: 16-byte chunks when rows are 16-byte aligned, single entries otherwise
+    const float w2p[4] = {P.w2p[0], P.w2p[1], P.w2p[2], P.w2p[3]};
+    // stage entries and scan values: 16-byte chunks when rows are 16-byte aligned, single entries otherwise
     constexpr int PER16 = 16 / (int)sizeof(EI);
     if ((P.inner % PER16) == 0 && (width % PER16) == 0) {
         const int chunks = width / PER16;
-        for (int t = threadIdx.x; t < n * chunks; t += TX) {
+        for (int t = threadIdx.x; t < n * chunks; t += blockDim.x) {
             const int y = t / chunks, ch = t - y * chunks;
             const uint4 v = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + ch * PER16);
             *reinterpret_cast<uint4*>(tile + y * TX + ch * PER16) = v;
+            const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+            uint32_t sv[PER16];
+#pragma unroll
+            for (int i = 0; i < PER16; ++i) {
+                const uint32_t word = wv[(i * (int)sizeof(EI)) >> 2];
+                const uint32_t e = sizeof(EI) == 4 ? word
+                                 : sizeof(EI) == 2 ? ((word >> (16 * (i & 1))) & 0xffffu)
+                                                   : ((word >> (8 * (i & 3))) & 0xffu);
+                sv[i] = scan_value<K, UNIT>(e, y, w2p);
+            }
+#pragma unroll
+            for (int i = 0; i < PER16; i += 4)
+                *reinterpret_cast<uint4*>(val + y * TX + ch * PER16 + i) = make_uint4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
         }
     } else {
-        for (int t = threadIdx.x; t < n * width; t += TX) {
+        for (int t = threadIdx.x; t < n * width; t += blockDim.x) {
             const int y = t / width, x = t - y * width;
-            tile[y * TX + x] = src[(int64_t)y * P.inner + x];
+            const EI e = src[(int64_t)y * P.inner + x];
+            tile[y * TX + x] = e;
+            val[y * TX + x] = scan_value<K, UNIT>((uint32_t)e, y, w2p);
         }
     }
     __syncthreads();
-    const int c = threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = warp % G, r0 = warp / G, rstep = nwarps / G;
+    const int c = g * 32 + lane;
     if (c >= width) return;
     ColumnOut<K, FINAL> out;
     out.stride = P.inner;
@@ -368,14 +423,16 @@ __global__ void __launch_bounds__(128) column_kernel(const __grid_constant__ Fas
         out.dist = ep.dist ? ep.dist + slab * ep.V + v0 : nullptr;
         out.sq = ep.sq ? ep.sq + slab * ep.V + v0 : nullptr;
         out.idx = ep.idx ? ep.idx + slab * ep.ndim * ep.V + v0 : nullptr;
-        out.V = ep.V; out.ndim = ep.ndim; out.unit = P.unit != 0;
+        out.V = ep.V; out.ndim = ep.ndim;
+        out.dist_only = ep.dist && !ep.sq && !ep.idx;
         int64_t rr = v0;
 #pragma unroll
         for (int q = 0; q < K; ++q) { out.coord[q] = (int)(rr % ep.ext[q]); rr /= ep.ext[q]; }
 #pragma unroll
         for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
     }
-    column_pass<K, FINAL, EI>(tile + c, TX, stk + c, TX, n, P, out);
+    for (int y = r0; y < n; y += rstep)
+        scan_voxel<K, FINAL, UNIT, TX, EI>(val + c, tile + c, TX, n, y, tab, out);
 }
 
 }  // namespace tmedt

@@ -234,13 +234,20 @@ static cudaError_t run_generic(const Plan& pl, const uint8_t* in, const Epilogue
     return cudaSuccess;
 }
 
-template <int K, bool FINAL>
-static cudaError_t launch_column(const FastParams& P, const EpilogueParams& ep, cudaStream_t st, double out_bpv) {
+template <bool UNIT>
+static void fill_scan_tab(ScanTab& tab, double w, int shift) {
+    for (int d = 0; d < 132; ++d) {
+        if (UNIT) tab.add[d] = (uint32_t)(d * d) << shift;
+        else { const float f = (float)(w * w) * (float)d * (float)d; memcpy(&tab.add[d], &f, 4); }
+    }
+}
+
+template <int K, bool FINAL, bool UNIT, int TX>
+static cudaError_t launch_column_tx(const FastParams& P, const EpilogueParams& ep, const ScanTab& tab, cudaStream_t st,
+                                    double out_bpv) {
     const size_t eb = (size_t)entry_bytes(K);
-    int TX = 128;
-    while (TX > 32 && ((size_t)P.n * TX * eb + (size_t)(3 * P.n / 2 + 2) * TX > 56 * 1024 || TX / 2 >= P.inner)) TX >>= 1;
-    const size_t smem = (size_t)P.n * TX * eb + (size_t)(3 * P.n / 2 + 2) * TX;
-    auto kern = column_kernel<K, FINAL>;
+    const size_t smem = (size_t)P.n * TX * (4 + eb);
+    auto kern = column_kernel<K, FINAL, UNIT, TX>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -249,22 +256,34 @@ static cudaError_t launch_column(const FastParams& P, const EpilogueParams& ep, 
     const int64_t blocks = P.outer * tiles;
     const double vox = (double)P.outer * P.n * (double)P.inner;
     prof_mark(st, FINAL ? "column_final" : "column", vox * ((double)eb + (FINAL ? out_bpv : (double)entry_bytes(K + 1))));
-    kern<<<(unsigned)blocks, TX, smem, st>>>(P, ep, tiles);
+    kern<<<(unsigned)blocks, 256, smem, st>>>(P, ep, tab, tiles);
     return cudaGetLastError();
 }
 
-template <bool FINAL>
-static cudaError_t launch_column_any(int K, const FastParams& P, const EpilogueParams& ep, cudaStream_t st,
-                                     double out_bpv) {
+template <int K, bool FINAL, bool UNIT>
+static cudaError_t launch_column(const FastParams& P, const EpilogueParams& ep, const ScanTab& tab, cudaStream_t st,
+                                 double out_bpv) {
+    // tile = n rows x (32 * G) columns, about 4096 voxels
+    int G = 1;
+    while (G < 4 && P.n * 32 * G * 2 <= 4096 && 32 * G < P.inner) G <<= 1;
+    if (G == 1) return launch_column_tx<K, FINAL, UNIT, 32>(P, ep, tab, st, out_bpv);
+    if (G == 2) return launch_column_tx<K, FINAL, UNIT, 64>(P, ep, tab, st, out_bpv);
+    return launch_column_tx<K, FINAL, UNIT, 128>(P, ep, tab, st, out_bpv);
+}
+
+template <bool FINAL, bool UNIT>
+static cudaError_t launch_column_any(int K, const FastParams& P, const EpilogueParams& ep, const ScanTab& tab,
+                                     cudaStream_t st, double out_bpv) {
     switch (K) {
-        case 2: return launch_column<2, FINAL>(P, ep, st, out_bpv);
-        case 3: return launch_column<3, FINAL>(P, ep, st, out_bpv);
-        case 4: if (FINAL) return launch_column<4, true>(P, ep, st, out_bpv);
+        case 2: return launch_column<2, FINAL, UNIT>(P, ep, tab, st, out_bpv);
+        case 3: return launch_column<3, FINAL, UNIT>(P, ep, tab, st, out_bpv);
+        case 4: if (FINAL) return launch_column<4, true, UNIT>(P, ep, tab, st, out_bpv);
     }
     return cudaErrorInvalidValue;
 }
 
 // Packed-entry path: fused first + second axis, then one column kernel per further axis.
+template <bool UNIT>
 static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
                             int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
@@ -274,21 +293,22 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     auto fill = [&](FastParams& P, int k) {
         memset(&P, 0, sizeof(P));
         P.n = pl.ext[k]; P.inner = pl.inner[k]; P.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
-        P.w2 = (float)(pl.w[k] * pl.w[k]); P.inv2w2 = (float)(0.5 / (pl.w[k] * pl.w[k]));
+        P.w2 = (float)(pl.w[k] * pl.w[k]);
         for (int p = 0; p < k && p < 4; ++p) P.w2p[p] = (float)(pl.w[p] * pl.w[p]);
-        P.unit = pl.unit ? 1 : 0;
     };
     FastParams P;
+    ScanTab tab;
     fill(P, 1);
+    fill_scan_tab<UNIT>(tab, pl.w[1], 8);
     P.in = in; P.out = bufA; P.n0 = pl.ext[0];
     {
-        const int threads = (pl.ext[0] + 31) & ~31;
+        const int threads = 256;
         const int tstride = (pl.ext[0] + 15) & ~15;
-        const size_t smem = (size_t)pl.ext[1] * tstride + (size_t)(3 * pl.ext[1] / 2 + 2) * threads;
+        const size_t smem = (((size_t)pl.ext[1] * tstride + 15) & ~(size_t)15) + (size_t)pl.ext[1] * 32 * 4;
         const bool fin = pl.E == 2;
         prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
-        if (fin) plane_kernel<true><<<(unsigned)P.outer, threads, smem, st>>>(P, ep);
-        else plane_kernel<false><<<(unsigned)P.outer, threads, smem, st>>>(P, ep);
+        if (fin) plane_kernel<true, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
+        else plane_kernel<false, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
         ++launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -297,9 +317,11 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     char* dst = bufB;
     for (int k = 2; k < pl.E; ++k) {
         fill(P, k);
+        fill_scan_tab<UNIT>(tab, pl.w[k], 8);
         P.in = src; P.out = dst;
         const bool fin = k == pl.E - 1;
-        cudaError_t e = fin ? launch_column_any<true>(k, P, ep, st, out_bpv) : launch_column_any<false>(k, P, ep, st, out_bpv);
+        cudaError_t e = fin ? launch_column_any<true, UNIT>(k, P, ep, tab, st, out_bpv)
+                            : launch_column_any<false, UNIT>(k, P, ep, tab, st, out_bpv);
         ++launches;
         if (e != cudaSuccess) return e;
         char* t = src; src = dst; dst = t;
@@ -351,7 +373,7 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
     int launches = 0;
     cudaError_t e;
     if (pl.fast)
-        e = run_fast(pl, input, ep, ws, st, launches);
+        e = pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
     else if (pl.use_double)
         e = pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
                     : run_generic<double, int8_t>(pl, input, ep, ws, st, launches);
