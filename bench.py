@@ -206,6 +206,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-steps", type=int, default=20)
     ap.add_argument("--unit-sampling", action="store_true", help="override the workload's sampling with 1.0 per axis")
+    ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()
@@ -216,6 +217,10 @@ def main():
     if args.unit_sampling:
         w.sampling = None
         w.name += " (unit sampling)"
+    if args.outputs:
+        want = set(args.outputs.split(","))
+        w.want_dist, w.want_sq, w.want_idx = "dist" in want, "sq" in want, "idx" in want
+        w.name += " (outputs %s)" % args.outputs
     if args.impl == "reference":
         run_reference(args, w, world, rank)
         return

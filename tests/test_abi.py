@@ -89,7 +89,9 @@ def test_host_memory_is_not_accepted_as_device_memory(L):
 def test_workspace_bytes(L):
     assert binding.tm_edt_workspace_bytes((1, 1, 0, 4)) == 0
     assert binding.tm_edt_workspace_bytes((1, 1, 64)) == 0  # a single pass needs no scratch
-    assert binding.tm_edt_workspace_bytes((2, 3, 64, 64)) >= 2 * 3 * 64 * 64
+    assert binding.tm_edt_workspace_bytes((2, 3, 64, 64)) == 0  # first two axes are fused in one kernel
+    assert binding.tm_edt_workspace_bytes((2, 3, 64, 64, 64)) >= 2 * (2 * 3 * 64 ** 3)  # 2-byte entries
+    assert binding.tm_edt_workspace_bytes((1, 1, 300, 300)) >= 2 * 300 * 300  # generic path: 16-bit offset planes
     with pytest.raises(binding.TmEdtError):
         binding.tm_edt_workspace_bytes((1, 1, binding.MAX_EXTENT + 1))
 
