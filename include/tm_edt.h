@@ -56,7 +56,8 @@ typedef enum {
     TM_EDT_ERR_BAD_POINTER = 3, /* a device buffer is not device-accessible memory of the current device
                                    (or a host buffer of tm_edt_host is device memory) */
     TM_EDT_ERR_ALLOC = 4,       /* scratch allocation failed, or the supplied workspace is too small */
-    TM_EDT_ERR_CUDA = 5         /* a CUDA runtime call or launch failed; see tm_edt_last_cuda_error() */
+    TM_EDT_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed; see tm_edt_last_cuda_error() */
+    TM_EDT_ERR_TOO_LARGE = 6    /* tm_edt_noalloc only: the problem needs more scratch than its built-in array */
 } tm_edt_status;
 
 /* The stream argument is a cudaStream_t (NULL = the legacy default stream). */
@@ -108,6 +109,40 @@ TM_EDT_API int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, c
  */
 TM_EDT_API int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
                 int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
+
+/*
+ * The transform for callers that must not allocate device memory.  (The paper has no counterpart to
+ * this entry point; it exists for deployment, not for the method.)
+ *
+ * Some hosts of this library cannot let it call cudaMalloc or the stream-ordered allocator while they
+ * run: a real-time or safety-certified loop that fixed its memory budget at start-up, a process whose
+ * device memory is entirely owned by another allocator, a driver sandbox that forbids allocation after
+ * initialisation.  tm_edt allocates its scratch, and tm_edt_ws pushes that job onto the caller; this
+ * variant does neither.  Its scratch is a fixed array of TM_EDT_NOALLOC_MAX_SCRATCH bytes that is part
+ * of the library's device image, so every GPU that loads the library holds that much memory until the
+ * process exits, whether or not this function is ever called.
+ *
+ * Arguments, outputs, stream behaviour and return codes are those of tm_edt (inputs and outputs are
+ * still the caller's device buffers).  Differences:
+ *   - A problem whose scratch need, tm_edt_workspace_bytes(ndim, shape), exceeds
+ *     TM_EDT_NOALLOC_MAX_SCRATCH is refused with TM_EDT_ERR_TOO_LARGE before anything is enqueued.
+ *   - The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with
+ *     that device current) and remembers it.  Make that first call during set-up, before any stream
+ *     capture begins.  Later calls on the device only enqueue kernels.
+ *   - No cudaMalloc, cudaFree, stream-ordered allocation or other allocating routine is called, on any
+ *     path, success or failure.
+ *   - All calls on one device share the one array.  It keeps whatever the previous call left in it;
+ *     that is harmless, because each pass writes every scratch element before a later pass reads it, so
+ *     nothing has to be cleared.  Two calls whose work overlaps on the GPU (different streams without
+ *     ordering between them, or threads racing on one device) corrupt each other's scratch: order them
+ *     on one stream or with events.  Calls on different devices do not interact.
+ */
+#define TM_EDT_NOALLOC_MAX_SCRATCH (16u * 1024u * 1024u)
+TM_EDT_API int tm_edt_noalloc(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling,
+                              float* out_dist, int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
+
+/* TM_EDT_NOALLOC_MAX_SCRATCH as the loaded library was built (bytes). */
+TM_EDT_API size_t tm_edt_noalloc_max_scratch(void);
 
 /*
  * Measurement aid: tm_edt_ws with a CUDA event recorded on `stream` before every kernel and after the

@@ -14,12 +14,12 @@ from typing import Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtm_edt.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_POINTER, ERR_ALLOC, ERR_CUDA = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_POINTER, ERR_ALLOC, ERR_CUDA, ERR_TOO_LARGE = range(7)
 MAX_DIMS = 8
 MAX_EXTENT = 8192
 
 EXPORTS = (
-    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_profile", "tm_edt_workspace_bytes", "tm_edt_strerror",
+    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count",
 )
 
@@ -50,6 +50,9 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_ws.restype = i
             L.tm_edt_host.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
             L.tm_edt_host.restype = i
+            L.tm_edt_noalloc.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
+            L.tm_edt_noalloc.restype = i
+            L.tm_edt_noalloc_max_scratch.restype = sz
             L.tm_edt_profile.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp, i, vp, vp, vp, vp]
             L.tm_edt_profile.restype = i
             L.tm_edt_workspace_bytes.argtypes = [i, vp]
@@ -170,6 +173,29 @@ def tm_edt(mask, sampling=None, return_distances=True, return_indices=False, ret
     else:
         rc = L.tm_edt_ws(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), _p(workspace),
                          ctypes.c_size_t(workspace.numel() * workspace.element_size()), st)
+    _check(rc)
+    return {"dist": d, "sq": s, "idx": x}
+
+
+def tm_edt_noalloc_max_scratch() -> int:
+    return int(lib().tm_edt_noalloc_max_scratch())
+
+
+def tm_edt_noalloc(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
+                   distances=None, indices=None, sqdist=None, stream=None):
+    """The transform through the entry point that never allocates device memory: scratch comes from a
+    fixed array inside the library, for hosts that may not call cudaMalloc once they are running (fixed
+    memory budgets, foreign allocators).  Pass pre-allocated ``distances`` / ``sqdist`` / ``indices`` if
+    the outputs, too, must not be allocated here.  Problems needing more scratch than
+    ``tm_edt_noalloc_max_scratch()`` raise ``TmEdtError`` with status ``ERR_TOO_LARGE``.  Calls that overlap
+    on the GPU share the array and would race; keep them ordered on one stream."""
+    L = lib()
+    if not mask.is_cuda:
+        raise ValueError("mask must be a CUDA tensor")
+    mask, shape, ndim, d, s, x = _prepare(
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+    rc = L.tm_edt_noalloc(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
+                          _raw_stream(stream))
     _check(rc)
     return {"dist": d, "sq": s, "idx": x}
 

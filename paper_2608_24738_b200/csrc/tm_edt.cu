@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "edt_common.cuh"
 #include "edt_generic.cuh"
 #include "edt_fast.cuh"
@@ -471,6 +473,59 @@ int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const doub
     return rc;
 }
 
+// ---- entry point that allocates nothing -------------------------------------------------------
+// Scratch for tm_edt_noalloc: one fixed array in device memory, part of the library image, so every GPU
+// that loads the library carries it until the process exits.
+#define TM_EDT_NOALLOC_SCRATCH_BYTES ((size_t)TM_EDT_NOALLOC_MAX_SCRATCH)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TM_EDT_NOALLOC_MAX_SCRATCH];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel could use:
+// the device address is asked for once per device (with that device current) and remembered.
+static void* g_noalloc_ptr[64];
+static bool g_noalloc_ready[64];
+static std::mutex g_noalloc_mutex;
+
+static int noalloc_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return TM_EDT_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ready[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            g_last_cuda_error = (int)e;
+            return TM_EDT_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+        g_noalloc_ready[dev] = true;
+    }
+    *out = g_noalloc_ptr[dev];
+    return TM_EDT_OK;
+}
+
+int tm_edt_noalloc(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                   int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl);
+    if (rc != TM_EDT_OK) return rc;
+    if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (pl.ws_bytes > TM_EDT_NOALLOC_SCRATCH_BYTES) return TM_EDT_ERR_TOO_LARGE;
+    if (!is_device_ptr(input) || (out_dist && !is_device_ptr(out_dist)) || (out_sqdist && !is_device_ptr(out_sqdist)) ||
+        (out_indices && !is_device_ptr(out_indices)))
+        return TM_EDT_ERR_BAD_POINTER;
+    void* scratch = nullptr;
+    if (pl.ws_bytes > 0) {
+        rc = noalloc_scratch_address(&scratch);
+        if (rc != TM_EDT_OK) return rc;
+    }
+    return run_device(pl, input, out_dist, out_sqdist, out_indices, scratch, (cudaStream_t)stream);
+}
+
+size_t tm_edt_noalloc_max_scratch(void) { return TM_EDT_NOALLOC_SCRATCH_BYTES; }
+
 const char* tm_edt_strerror(int status) {
     switch (status) {
         case TM_EDT_OK: return "ok";
@@ -479,6 +534,7 @@ const char* tm_edt_strerror(int status) {
         case TM_EDT_ERR_BAD_POINTER: return "buffer is not in the expected memory space";
         case TM_EDT_ERR_ALLOC: return "scratch allocation failed or workspace too small";
         case TM_EDT_ERR_CUDA: return "CUDA runtime error";
+        case TM_EDT_ERR_TOO_LARGE: return "problem needs more scratch than the built-in array of tm_edt_noalloc holds";
     }
     return "unknown status";
 }
