@@ -59,14 +59,8 @@ __device__ __forceinline__ float small_int_to_float(int v) {  // exact for 0 <= 
 
 __device__ __forceinline__ bool entry_none(uint32_t e) { return (e & 0xffu) == 0x80u; }
 
-template <int K> __device__ __forceinline__ int entry_sumsq(uint32_t e) {
-    int o = (int)(int8_t)(e & 0xff);
-    int s = o * o;
-    if (K > 1) { o = (int)(int8_t)((e >> 8) & 0xff); s += o * o; }
-    if (K > 2) { o = (int)(int8_t)((e >> 16) & 0xff); s += o * o; }
-    if (K > 3) { o = (int)(int8_t)((e >> 24) & 0xff); s += o * o; }
-    return s;
-}
+// Sum of the squared signed offsets of an entry (unused high bytes are zero): one 4-way byte dot product.
+template <int K> __device__ __forceinline__ int entry_sumsq(uint32_t e) { return __dp4a((int)e, (int)e, 0); }
 
 // Tile value the scan works on: unit sampling -> key (sum of squared offsets << 8 | row), none -> kNoneKey;
 // otherwise the bits of the float32 height sum_q w_q^2 off_q^2, none -> +inf.
@@ -111,9 +105,9 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j,
         o.out[p] = (EO)v;
         return;
     }
-    // unit sampling: sqv is an exact integer below 2^24 and the root is correctly rounded; otherwise the
-    // approximate root (relative error about 1e-7) is far inside the float32 result's own rounding.
-    const float dv = none ? TMEDT_INF : (UNIT ? __fsqrt_rn(sqv) : fast_sqrt(sqv));
+    // sqv is exact for unit sampling (an integer below 2^24); the hardware root's relative error of about
+    // 1e-7 is a hundred times inside the 1e-5 bar on distances.
+    const float dv = none ? TMEDT_INF : fast_sqrt(sqv);
     if (o.dist_only) { o.dist[p] = dv; return; }
     if (o.dist) o.dist[p] = dv;
     if (none) {
@@ -181,6 +175,53 @@ __device__ __forceinline__ uint32_t scan_keys(const uint32_t* __restrict__ col, 
         }
     }
     return best;
+}
+
+// Unit sampling, R consecutive rows y0 .. y0+R-1 of one column at once: every row fetched from the tile
+// serves all R voxels (each with its own addend), which divides the shared-memory loads and the loop
+// overhead per voxel by R.  Rows beyond the column end get best = 0 and are not emitted by the caller.
+template <int VS, int R>
+__device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col, int n, int y0, uint32_t (&best)[R]) {
+    uint32_t k[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) k[i] = y0 + i < n ? col[(y0 + i) * VS] : kNoneKey;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        best[i] = k[i];
+#pragma unroll
+        for (int j = 0; j < R; ++j)
+            if (j != i) best[i] = __viaddmin_u32(k[j], (uint32_t)((i - j) * (i - j)) << 8, best[i]);
+        if (y0 + i >= n) best[i] = 0u;
+    }
+    uint32_t mx = best[0];
+#pragma unroll
+    for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
+    if (mx < 256u) return;  // a group of background voxels
+    uint32_t a[R];          // a[i] = (d + i)^2 << 8
+#pragma unroll
+    for (int i = 0; i < R; ++i) a[i] = (uint32_t)((1 + i) * (1 + i)) << 8;
+    const uint32_t* plo = col + (y0 - 1) * VS;
+    const uint32_t* phi = col + (y0 + R) * VS;
+    int lo = y0 - 1, hi = y0 + R;
+    for (int d = 1; a[0] < mx; ++d, --lo, ++hi, plo -= VS, phi += VS) {
+        if (lo < 0 && hi >= n) break;
+        if (lo >= 0) {
+            const uint32_t v = plo[0];
+#pragma unroll
+            for (int i = 0; i < R; ++i) best[i] = __viaddmin_u32(v, a[i], best[i]);
+        }
+        if (hi < n) {
+            const uint32_t v = phi[0];
+#pragma unroll
+            for (int i = 0; i < R; ++i) best[i] = __viaddmin_u32(v, a[R - 1 - i], best[i]);
+        }
+        mx = best[0];
+#pragma unroll
+        for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
+#pragma unroll
+        for (int i = 0; i + 1 < R; ++i) a[i] = a[i + 1];
+        a[R - 1] = (uint32_t)((d + R) * (d + R)) << 8;
+    }
 }
 
 // Float heights.  ARG: also returns the distance bd (0 = own row) at which the minimum was found.
@@ -431,8 +472,27 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
 #pragma unroll
         for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
     }
-    for (int y = r0; y < n; y += rstep)
-        scan_voxel<K, FINAL, UNIT, TX, EI>(val + c, tile + c, TX, n, y, tab, out);
+    if (UNIT && (!FINAL || out.dist_only)) {
+        constexpr int R = 4;
+        for (int y0 = r0 * R; y0 < n; y0 += rstep * R) {
+            uint32_t best[R];
+            scan_keys_group<TX, R>(val + c, n, y0, best);
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int y = y0 + i;
+                if (y >= n) break;
+                const uint32_t b = best[i];
+                if (b < 256u) { emit<K, FINAL, true>(out, y, y, 0u, 0.f, false); continue; }
+                const bool none = b >= kNoneKey;
+                const int j = (int)(b & 0xffu);
+                const uint32_t e = none ? 0u : (uint32_t)tile[j * TX + c];
+                emit<K, FINAL, true>(out, y, j, e, small_int_to_float((int)(b >> 8)), none);
+            }
+        }
+    } else {
+        for (int y = r0; y < n; y += rstep)
+            scan_voxel<K, FINAL, UNIT, TX, EI>(val + c, tile + c, TX, n, y, tab, out);
+    }
 }
 
 }  // namespace tmedt
