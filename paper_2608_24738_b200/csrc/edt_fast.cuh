@@ -50,7 +50,8 @@ struct FastParams {
 // add[d] = w^2 d^2 for the axis of the pass: float32 bits (sampled) or d^2 << shift (unit sampling keys).
 struct ScanTab { uint32_t add[132]; };
 
-constexpr uint32_t kNoneKey = 0xF0000000u;
+constexpr uint32_t kNoneKey = 0xF0000000u;    // keys (value << 8 | row): values stay below 2^25
+constexpr uint32_t kNoneKey16 = 0x80000000u;  // keys (value << 16 | row << 8 | offset): values stay below 2^15
 #define TMEDT_INF (__int_as_float(0x7f800000))
 
 __device__ __forceinline__ float small_int_to_float(int v) {  // exact for 0 <= v < 2^23, two full-rate ops
@@ -180,26 +181,28 @@ __device__ __forceinline__ uint32_t scan_keys(const uint32_t* __restrict__ col, 
 // Unit sampling, R consecutive rows y0 .. y0+R-1 of one column at once: every row fetched from the tile
 // serves all R voxels (each with its own addend), which divides the shared-memory loads and the loop
 // overhead per voxel by R.  Rows beyond the column end get best = 0 and are not emitted by the caller.
-template <int VS, int R>
+template <int VS, int R, int SH = 8>
 __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col, int n, int y0, uint32_t (&best)[R]) {
+    // "no site" key: above every real key, and adding any addend to it must not wrap around
+    constexpr uint32_t NONE = SH == 16 ? kNoneKey16 : kNoneKey;
     uint32_t k[R];
 #pragma unroll
-    for (int i = 0; i < R; ++i) k[i] = y0 + i < n ? col[(y0 + i) * VS] : kNoneKey;
+    for (int i = 0; i < R; ++i) k[i] = y0 + i < n ? col[(y0 + i) * VS] : NONE;
 #pragma unroll
     for (int i = 0; i < R; ++i) {
         best[i] = k[i];
 #pragma unroll
         for (int j = 0; j < R; ++j)
-            if (j != i) best[i] = __viaddmin_u32(k[j], (uint32_t)((i - j) * (i - j)) << 8, best[i]);
+            if (j != i) best[i] = __viaddmin_u32(k[j], (uint32_t)((i - j) * (i - j)) << SH, best[i]);
         if (y0 + i >= n) best[i] = 0u;
     }
     uint32_t mx = best[0];
 #pragma unroll
     for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
-    if (mx < 256u) return;  // a group of background voxels
-    uint32_t a[R];          // a[i] = (d + i)^2 << 8
+    if (mx < (1u << SH)) return;  // a group of background voxels
+    uint32_t a[R];                // a[i] = (d + i)^2 << SH
 #pragma unroll
-    for (int i = 0; i < R; ++i) a[i] = (uint32_t)((1 + i) * (1 + i)) << 8;
+    for (int i = 0; i < R; ++i) a[i] = (uint32_t)((1 + i) * (1 + i)) << SH;
     const uint32_t* plo = col + (y0 - 1) * VS;
     const uint32_t* phi = col + (y0 + R) * VS;
     int lo = y0 - 1, hi = y0 + R;
@@ -220,7 +223,7 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
         for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
 #pragma unroll
         for (int i = 0; i + 1 < R; ++i) a[i] = a[i + 1];
-        a[R - 1] = (uint32_t)((d + R) * (d + R)) << 8;
+        a[R - 1] = (uint32_t)((d + R) * (d + R)) << SH;
     }
 }
 
@@ -395,10 +398,131 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
                 out.coord[0] = c;
                 out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
             }
-            for (int y = warp; y < n1; y += nwarps)
-                scan_voxel<1, FINAL, UNIT, 32, uint8_t>(val + lane, tile + c, tstride, n1, y, tab, out);
+            if (UNIT && (!FINAL || out.dist_only)) {
+                constexpr int R = 4;
+                for (int y0 = warp * R; y0 < n1; y0 += nwarps * R) {
+                    uint32_t best[R];
+                    scan_keys_group<32, R>(val + lane, n1, y0, best);
+#pragma unroll
+                    for (int i = 0; i < R; ++i) {
+                        const int y = y0 + i;
+                        if (y >= n1) break;
+                        const uint32_t b = best[i];
+                        if (b < 256u) { emit<1, FINAL, true>(out, y, y, 0u, 0.f, false); continue; }
+                        const bool none = b >= kNoneKey;
+                        const int j = (int)(b & 0xffu);
+                        const uint32_t e = none ? 0u : (uint32_t)tile[j * tstride + c];
+                        emit<1, FINAL, true>(out, y, j, e, small_int_to_float((int)(b >> 8)), none);
+                    }
+                }
+            } else {
+                for (int y = warp; y < n1; y += nwarps)
+                    scan_voxel<1, FINAL, UNIT, 32, uint8_t>(val + lane, tile + c, tstride, n1, y, tab, out);
+            }
         }
         __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Unit-sampling plane kernel: the first-axis pass writes scan keys straight into one tile that covers
+// the whole plane, key = (off^2 << 16) | (row << 8) | (off & 0xff), so the second-axis scan needs no
+// second tile and no gather: the chosen site's first-axis offset rides in the low byte of the key.
+// First axis, one warp per row, four voxels per lane (one 32-bit load): zero bytes are found with a
+// carry-free byte test, the nearest lanes holding a zero on either side with one ballot and clz / ffs,
+// their zero positions with two shuffles; the four voxels of the lane are then finished in registers.
+// Requires n0 % 4 == 0 (rows then start on 4-byte boundaries).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pass0_row_to_keys(const uint8_t* __restrict__ row, int n0, int y,
+                                                  uint32_t* __restrict__ vrow, int lane) {
+    const bool act = 4 * lane < n0;
+    const uint32_t v = act ? *reinterpret_cast<const uint32_t*>(row + 4 * lane) : 0x01010101u;
+    const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
+    const unsigned any = __ballot_sync(0xffffffffu, m != 0u);  // inactive lanes hold foreground: m == 0
+    // every lane of the warp stays in the shuffles below; only the final store is guarded
+    uint4 keys;
+    if (any == 0u) {  // no background in this row
+        keys = make_uint4(kNoneKey16, kNoneKey16, kNoneKey16, kNoneKey16);
+    } else {
+        const int lzin = m ? (31 - __clz(m)) >> 3 : 0;   // highest zero byte of this lane
+        const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;    // lowest zero byte of this lane
+        const unsigned ml = any & ((1u << lane) - 1u);
+        const unsigned mr = lane < 31 ? any >> (lane + 1) : 0u;
+        const int Ll = ml ? 31 - __clz(ml) : 0;
+        const int Lr = mr ? lane + __ffs(mr) : 0;
+        const int lz_l = __shfl_sync(0xffffffffu, lzin, Ll);
+        const int fz_r = __shfl_sync(0xffffffffu, fzin, Lr);
+        const int x0 = 4 * lane;
+        int cur = ml ? 4 * Ll + lz_l : -1024;   // nearest zero left of this lane's voxels
+        int dl[4], dr[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dl[b] = x0 + b - cur;
+        }
+        cur = mr ? 4 * Lr + fz_r : 2048;        // nearest zero right of this lane's voxels
+#pragma unroll
+        for (int b = 3; b >= 0; --b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dr[b] = cur - (x0 + b);
+        }
+        uint32_t kk[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = min(dl[b], dr[b]);
+            const int off = dl[b] <= dr[b] ? -a : a;
+            kk[b] = ((uint32_t)(a * a) << 16) | ((uint32_t)y << 8) | ((uint32_t)off & 0xffu);
+        }
+        keys = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+    }
+    if (act) *reinterpret_cast<uint4*>(vrow + 4 * lane) = keys;
+}
+
+template <bool FINAL, int VS>
+__global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__ FastParams P,
+                                                         const __grid_constant__ EpilogueParams ep) {
+    extern __shared__ __align__(16) uint8_t sm_plane_u[];
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_plane_u);  // [n1][VS]
+    const int n0 = P.n0, n1 = P.n;
+    const int64_t plane = blockIdx.x;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int y = warp; y < n1; y += nwarps) pass0_row_to_keys(src + y * n0, n0, y, val + y * VS, lane);
+    __syncthreads();
+    constexpr int R = 4, CG = VS / 32;
+    const int tasks = ((n1 + R - 1) / R) * CG;
+    const bool dist_only = FINAL && ep.dist && !ep.sq && !ep.idx;
+    for (int t = warp; t < tasks; t += nwarps) {
+        const int cg = t % CG, y0 = (t / CG) * R;
+        const int c = cg * 32 + lane;
+        if (c >= n0) continue;
+        uint32_t best[R];
+        scan_keys_group<VS, R, 16>(val + c, n1, y0, best);
+        const int64_t p0 = plane * (int64_t)n1 * n0 + (int64_t)y0 * n0 + c;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const int y = y0 + i;
+            if (y >= n1) break;
+            const uint32_t b = best[i];
+            const bool none = b >= kNoneKey16;
+            const int j = (int)((b >> 8) & 0xffu);
+            if (!FINAL) {
+                const uint32_t e = none ? 0x80u : ((b & 0xffu) | ((uint32_t)((j - y) & 0xff) << 8));
+                reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)e;
+            } else if (dist_only) {
+                ep.dist[p0 + (int64_t)i * n0] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b >> 16)));
+            } else {  // two processed axes: the plane is the image
+                ColumnOut<1, true> out;
+                out.stride = n0;
+                out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
+                out.sq = ep.sq ? ep.sq + plane * ep.V + c : nullptr;
+                out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+                out.V = ep.V; out.ndim = ep.ndim; out.dist_only = false;
+                out.coord[0] = c;
+                out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+                emit<1, true, true>(out, y, j, b & 0xffu, small_int_to_float((int)(b >> 16)), none);
+            }
+        }
     }
 }
 

@@ -309,7 +309,21 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
         const size_t smem = (((size_t)pl.ext[1] * tstride + 15) & ~(size_t)15) + (size_t)pl.ext[1] * 32 * 4;
         const bool fin = pl.E == 2;
         prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
-        if (fin) plane_kernel<true, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
+        const char* oldp = getenv("TM_EDT_OLD_PLANE");
+        if (UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
+            // whole-plane key tile; row stride = extent rounded up to 32, 64 or 128 columns
+            const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
+            const size_t smem_u = (size_t)pl.ext[1] * vs * 4;
+#define TM_LAUNCH_PLANE_UNIT(FIN, VSV)                                                                         \
+    do {                                                                                                       \
+        auto kern = plane_unit_kernel<FIN, VSV>;                                                               \
+        if (smem_u > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_u); \
+        kern<<<(unsigned)P.outer, threads, smem_u, st>>>(P, ep);                                               \
+    } while (0)
+            if (fin) { if (vs == 32) TM_LAUNCH_PLANE_UNIT(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(true, 64); else TM_LAUNCH_PLANE_UNIT(true, 128); }
+            else { if (vs == 32) TM_LAUNCH_PLANE_UNIT(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(false, 64); else TM_LAUNCH_PLANE_UNIT(false, 128); }
+#undef TM_LAUNCH_PLANE_UNIT
+        } else if (fin) plane_kernel<true, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
         else plane_kernel<false, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
         ++launches;
         cudaError_t e = cudaGetLastError();
