@@ -193,20 +193,111 @@ def run_reference(args, w, world, rank):
     print(json.dumps(line), flush=True)
 
 
+def load_traffic(workload_number: int, kernel_label: str):
+    """DRAM bytes per launch of a kernel from the committed ncu summary (profiles/traffic.json), or None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
+            table = json.load(fh)
+        return table.get("C%d" % workload_number, {}).get(kernel_label.split(":", 1)[1])
+    except Exception:
+        return None
+
+
+def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
+    """Device-timed throughput of one workload plus per-kernel event times (inputs resident in HBM)."""
+    import torch
+
+    from paper_2608_24738_b200 import binding
+
+    # buffers: rotate over enough independent sets that one lap exceeds twice the L2
+    io = w.io_bytes()
+    sets = max(2, min(16, -(-2 * L2_BYTES // io)))
+    host_mask = torch.from_numpy(w.mask)
+    shape = tuple(w.mask.shape)
+    calls = []
+    for _ in range(sets):
+        m = host_mask.to(dev)
+        d = torch.empty(shape, dtype=torch.float32, device=dev) if w.want_dist else None
+        s = torch.empty(shape, dtype=torch.int64, device=dev) if w.want_sq else None
+        x = torch.empty(shape[:2] + (w.ndim,) + shape[2:], dtype=torch.int64, device=dev) if w.want_idx else None
+        calls.append(binding.PreparedCall(m, w.sampling, d, s, x))
+    stream = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(stream.cuda_stream)
+    for i in range(warmup):
+        calls[i % sets](sp)
+    launches_per_step = binding.tm_edt_last_launch_count()
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.barrier()
+        torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for i in range(steps):
+        calls[i % sets](sp)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+        torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    seconds = max_over_ranks(ev0.elapsed_time(ev1) / 1e3, world, dev)
+    clocks = sampler.summary(t0, t1) if sampler is not None else None
+    value = whole_job_rate(w.voxels * steps, world, seconds) / 1e9
+
+    # per-kernel times (events between launches), same buffers, right after the timed region
+    ksum, korder = {}, []
+    for i in range(max(1, profile_steps)):
+        c = calls[i % sets]
+        _, ks = binding.tm_edt_profile(c.mask, w.sampling, distances=c.d, sqdist=c.s, indices=c.x, workspace=c.ws,
+                                       return_distances=w.want_dist, return_sqdist=w.want_sq,
+                                       return_indices=w.want_idx)
+        for j, (name, ms, nbytes) in enumerate(ks):
+            key = (j, name)
+            if key not in ksum:
+                ksum[key] = [0.0, nbytes, 0]
+                korder.append(key)
+            ksum[key][0] += ms
+            ksum[key][2] += 1
+    peak, peak_kind = measured_peak_gbs()
+    kernels = []
+    for key in korder:
+        tot, nbytes, cnt = ksum[key]
+        avg_ms = tot / cnt
+        kernels.append({"kernel": "%d:%s" % key, "avg_ms": avg_ms, "bytes": nbytes,
+                        "gbs": nbytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else None})
+    dom = max(kernels, key=lambda k: k["avg_ms"])
+    path_gbs = io * steps * 1.0 / seconds / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
+        "frac": dom["gbs"] / peak, "traffic": load_traffic(w.number, dom["kernel"]), "peak_kind": peak_kind + " copy bandwidth",
+        "path": {"io_bytes_per_step": io, "achieved": path_gbs, "frac": path_gbs / peak},
+        "kernels": kernels,
+    }
+    del calls
+    torch.cuda.empty_cache()
+    return {"io": io, "shape": shape, "host_mask": host_mask, "value": value, "seconds": seconds, "clocks": clocks,
+            "roofline": roofline, "launches_per_step": launches_per_step, "sets": sets}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-voxels", type=int, default=8 << 20, help="voxels per step of the reference arm")
     ap.add_argument("--cpu-voxels", type=int, default=64 << 20, help="sample size of the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-all-configs", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--profile-steps", type=int, default=20)
     ap.add_argument("--unit-sampling", action="store_true", help="override the workload's sampling with 1.0 per axis")
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
+    ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()
@@ -217,6 +308,11 @@ def main():
     if args.unit_sampling:
         w.sampling = None
         w.name += " (unit sampling)"
+    if args.images > 0:
+        B, C = w.mask.shape[:2]
+        flat = w.mask.reshape((B * C, 1) + w.mask.shape[2:])
+        w.mask = flat[: args.images].copy()
+        w.name += " (first %d images)" % args.images
     if args.outputs:
         want = set(args.outputs.split(","))
         w.want_dist, w.want_sq, w.want_idx = "dist" in want, "sq" in want, "idx" in want
@@ -240,76 +336,13 @@ def main():
 
         dist.init_process_group("nccl", device_id=dev)
 
-    # ---- buffers: rotate over enough independent sets that one lap exceeds twice the L2 ----
-    io = w.io_bytes()
-    sets = max(2, min(16, -(-2 * L2_BYTES // io)))
-    host_mask = torch.from_numpy(w.mask)
-    shape = tuple(w.mask.shape)
-    calls = []
-    for _ in range(sets):
-        m = host_mask.to(dev)
-        d = torch.empty(shape, dtype=torch.float32, device=dev) if w.want_dist else None
-        s = torch.empty(shape, dtype=torch.int64, device=dev) if w.want_sq else None
-        x = torch.empty(shape[:2] + (w.ndim,) + shape[2:], dtype=torch.int64, device=dev) if w.want_idx else None
-        calls.append(binding.PreparedCall(m, w.sampling, d, s, x))
     stream = torch.cuda.current_stream()
-    sp = ctypes.c_void_p(stream.cuda_stream)
-
     sampler = ClockSampler(local)
     sampler.start()
-    for i in range(args.warmup):
-        calls[i % sets](sp)
-    launches_per_step = binding.tm_edt_last_launch_count()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-        torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.perf_counter()
-    ev0.record(stream)
-    for i in range(args.steps):
-        calls[i % sets](sp)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-        torch.cuda.synchronize()
-    t1 = time.perf_counter()
-    seconds = ev0.elapsed_time(ev1) / 1e3
-    seconds = max_over_ranks(seconds, world, dev)
-    clocks = sampler.summary(t0, t1)
-    value = whole_job_rate(w.voxels * args.steps, world, seconds) / 1e9
-
-    # ---- per-kernel times (events between launches), same buffers, right after the timed region ----
-    ksum = {}
-    korder = []
-    for i in range(max(1, args.profile_steps)):
-        c = calls[i % sets]
-        _, ks = binding.tm_edt_profile(c.mask, w.sampling, distances=c.d, sqdist=c.s, indices=c.x, workspace=c.ws,
-                                       return_distances=w.want_dist, return_sqdist=w.want_sq,
-                                       return_indices=w.want_idx)
-        for j, (name, ms, nbytes) in enumerate(ks):
-            key = (j, name)
-            if key not in ksum:
-                ksum[key] = [0.0, nbytes, 0]
-                korder.append(key)
-            ksum[key][0] += ms
-            ksum[key][2] += 1
-    peak, peak_kind = measured_peak_gbs()
-    kernels = []
-    for key in korder:
-        tot, nbytes, cnt = ksum[key]
-        avg_ms = tot / cnt
-        kernels.append({"kernel": "%d:%s" % key, "avg_ms": avg_ms, "bytes": nbytes,
-                        "gbs": nbytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else None})
-    dom = max(kernels, key=lambda k: k["avg_ms"])
-    path_gbs = io * args.steps * 1.0 / seconds / 1e9
-    roofline = {
-        "bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
-        "frac": dom["gbs"] / peak, "traffic": None, "peak_kind": peak_kind,
-        "path": {"io_bytes_per_step": io, "achieved": path_gbs, "frac": path_gbs / peak},
-        "kernels": kernels,
-    }
+    m = measure_device(w, args.steps, args.warmup, args.profile_steps, dev, world, sampler)
+    io, shape, host_mask = m["io"], m["shape"], m["host_mask"]
+    value, seconds, clocks, roofline = m["value"], m["seconds"], m["clocks"], m["roofline"]
+    launches_per_step, sets = m["launches_per_step"], m["sets"]
 
     # ---- end to end: host buffers in, host buffers out, through tm_edt_host ----
     e2e = None
@@ -338,6 +371,19 @@ def main():
                "h2d_bytes_per_step": w.voxels, "d2h_bytes_per_step": io - w.voxels, "steps": e2e_steps}
     sampler.stop()
 
+    others = None
+    if world == 1 and not args.no_all_configs and not args.unit_sampling and not args.outputs and not args.images:
+        others = []
+        for num in (1, 2, 3, 4, 5):
+            if num == args.config:
+                continue
+            wo = workloads.CONFIGS[num]()
+            mo = measure_device(wo, 40, 5, 5, dev, world)
+            others.append({"workload": wo.name, "value": mo["value"], "unit": UNIT, "ms_per_step": mo["seconds"] / 40 * 1e3,
+                           "path_frac": mo["roofline"]["path"]["frac"], "dominant": mo["roofline"]["kernel"],
+                           "dominant_frac": mo["roofline"]["frac"],
+                           "kernels": [(k["kernel"], round(k["avg_ms"], 4)) for k in mo["roofline"]["kernels"]]})
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
@@ -358,7 +404,7 @@ def main():
                        "voxels_per_step": w.voxels, "l2": "rotating %d buffer sets, %d MB per set" % (sets, io >> 20),
                        "sha256": w.sha256()[:16]},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "cpu_baseline": cpu,
+            "roofline": roofline, "cpu_baseline": cpu, "other_configs": others,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

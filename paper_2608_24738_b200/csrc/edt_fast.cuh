@@ -88,6 +88,15 @@ struct ColumnOut {
     int axis[5];         // spatial axis of plane q
     int ndim;
     bool dist_only;      // final: only out_dist was requested
+    int64_t* ip[5];      // final: index plane of processed axis q (same row-0 origin as idx)
+    bool simple_idx;     // final: every spatial axis is a processed axis (no extent-1 axes to fill with 0)
+
+    // call after idx, V, ndim and axis[] are set
+    __device__ __forceinline__ void init_index_planes() {
+#pragma unroll
+        for (int q = 0; q <= K; ++q) ip[q] = idx ? idx + (int64_t)axis[q] * V : nullptr;
+        simple_idx = ndim == K + 1;
+    }
 };
 
 __device__ __forceinline__ float fast_sqrt(float v) {
@@ -118,7 +127,13 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j,
         return;
     }
     if (o.sq) o.sq[p] = (int64_t)sqv;  // unit sampling only
-    if (o.idx) {
+    if (o.idx && o.simple_idx) {
+        // one store per processed axis: own coordinate + offset (coordinates are non-negative)
+#pragma unroll
+        for (int q = 0; q < K; ++q)
+            o.ip[q][p] = (int64_t)(uint32_t)(o.coord[q] + (int)(int8_t)((e >> (8 * q)) & 0xff));
+        o.ip[K][p] = (int64_t)(uint32_t)j;
+    } else if (o.idx) {
         int off[5];
 #pragma unroll
         for (int q = 0; q < K; ++q) off[q] = (int)(int8_t)((e >> (8 * q)) & 0xff);
@@ -397,6 +412,7 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
                 out.dist_only = ep.dist && !ep.sq && !ep.idx;
                 out.coord[0] = c;
                 out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+                out.init_index_planes();
             }
             if (UNIT && (!FINAL || out.dist_only)) {
                 constexpr int R = 4;
@@ -520,6 +536,7 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
                 out.V = ep.V; out.ndim = ep.ndim; out.dist_only = false;
                 out.coord[0] = c;
                 out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+                out.init_index_planes();
                 emit<1, true, true>(out, y, j, b & 0xffu, small_int_to_float((int)(b >> 16)), none);
             }
         }
@@ -595,6 +612,7 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
         for (int q = 0; q < K; ++q) { out.coord[q] = (int)(rr % ep.ext[q]); rr /= ep.ext[q]; }
 #pragma unroll
         for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
+        out.init_index_planes();
     }
     if (UNIT && (!FINAL || out.dist_only)) {
         constexpr int R = 4;
