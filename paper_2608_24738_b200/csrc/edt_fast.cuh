@@ -449,10 +449,10 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
 // their zero positions with two shuffles; the four voxels of the lane are then finished in registers.
 // Requires n0 % 4 == 0 (rows then start on 4-byte boundaries).
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void pass0_row_to_keys(const uint8_t* __restrict__ row, int n0, int y,
-                                                  uint32_t* __restrict__ vrow, int lane) {
+__device__ __forceinline__ void pass0_row_to_keys(const uint32_t v, int n0, int y, uint32_t* __restrict__ vrow,
+                                                  int lane) {
+    // v: the lane's four mask bytes of this row (0x01010101 for lanes beyond the row)
     const bool act = 4 * lane < n0;
-    const uint32_t v = act ? *reinterpret_cast<const uint32_t*>(row + 4 * lane) : 0x01010101u;
     const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
     const unsigned any = __ballot_sync(0xffffffffu, m != 0u);  // inactive lanes hold foreground: m == 0
     // every lane of the warp stays in the shuffles below; only the final store is guarded
@@ -503,7 +503,22 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
     const int64_t plane = blockIdx.x;
     const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int y = warp; y < n1; y += nwarps) pass0_row_to_keys(src + y * n0, n0, y, val + y * VS, lane);
+    {
+        // all loads of this warp's rows are issued before the first row is processed
+        constexpr int MAXR = 16;  // rows per warp: 128 rows / 8 warps
+        uint32_t rowv[MAXR];
+        const bool act = 4 * lane < n0;
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
+        }
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            if (y < n1) pass0_row_to_keys(rowv[i], n0, y, val + y * VS, lane);
+        }
+    }
     __syncthreads();
     constexpr int R = 4, CG = VS / 32;
     const int tasks = ((n1 + R - 1) / R) * CG;
@@ -562,9 +577,10 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
     // stage entries and scan values: 16-byte chunks when rows are 16-byte aligned, single entries otherwise
     constexpr int PER16 = 16 / (int)sizeof(EI);
     if ((P.inner % PER16) == 0 && (width % PER16) == 0) {
+        constexpr int FULL = TX / PER16;
         const int chunks = width / PER16;
         for (int t = threadIdx.x; t < n * chunks; t += blockDim.x) {
-            const int y = t / chunks, ch = t - y * chunks;
+            const int y = chunks == FULL ? t / FULL : t / chunks, ch = t - y * chunks;
             const uint4 v = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + ch * PER16);
             *reinterpret_cast<uint4*>(tile + y * TX + ch * PER16) = v;
             const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
