@@ -12,6 +12,7 @@
 #include "edt_common.cuh"
 #include "edt_generic.cuh"
 #include "edt_fast.cuh"
+#include "edt_wide2d.cuh"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -56,6 +57,7 @@ struct Plan {
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
     bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    bool wide2d = false;      // two processed axes, unit sampling, extents <= 512, contiguous extent % 16 == 0
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
 };
@@ -127,6 +129,8 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
     const char* force = getenv("TM_EDT_FORCE_GENERIC");
     pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
+    pl.wide2d = !pl.fast && E == 2 && pl.unit && nmax <= 512 && pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
+    if (pl.wide2d) pl.ws_bytes = (((size_t)pl.N * 4 + 255) & ~(size_t)255) + (((size_t)pl.N * 2 + 255) & ~(size_t)255);
     if (pl.fast) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
         const size_t a = E >= 3 ? up((size_t)pl.N * (E >= 5 ? 4 : 2)) : 0;
@@ -345,6 +349,33 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     return cudaSuccess;
 }
 
+// Two-dimensional unit-sampling images with extents up to 512: key rows, then column strips.
+static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                              int& launches) {
+    WideParams P;
+    P.in = in;
+    P.keys = static_cast<uint32_t*>(ws);
+    P.offs = reinterpret_cast<int16_t*>(static_cast<char*>(ws) + (((size_t)pl.N * 4 + 255) & ~(size_t)255));
+    P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
+    P.rows = pl.N / pl.ext[0];
+    const double out_bpv = out_bytes_per_voxel(ep);
+    prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + 2.0));
+    row_keys_kernel<<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    ++launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int strips = (pl.ext[0] + 31) / 32;
+    const size_t smem = (size_t)pl.ext[1] * 32 * 4;
+    if (smem > 48 * 1024) {
+        e = cudaFuncSetAttribute(wide_column_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    prof_mark(st, "wide_column_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
+    wide_column_kernel<<<(unsigned)(pl.images * strips), 256, smem, st>>>(P, ep, strips);
+    ++launches;
+    return cudaGetLastError();
+}
+
 static bool is_device_ptr(const void* p) {
     cudaPointerAttributes at;
     if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
@@ -388,7 +419,9 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     int launches = 0;
     cudaError_t e;
-    if (pl.fast)
+    if (pl.wide2d && ((uintptr_t)input & 15u) == 0)
+        e = run_wide2d(pl, input, ep, ws, st, launches);
+    else if (pl.fast)
         e = pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
     else if (pl.use_double)
         e = pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
