@@ -558,6 +558,110 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Sampled plane kernel (general sampling, n0 % 4 == 0): like the unit-sampling one, but the tile holds
+// float32 heights w0^2 off^2 and a second, byte-sized tile keeps the first-axis offsets for the output.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pass0_row_to_heights(const uint32_t v, int n0, float w2x, uint32_t* __restrict__ vrow,
+                                                     uint8_t* __restrict__ drow, int lane) {
+    const bool act = 4 * lane < n0;
+    const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
+    const unsigned any = __ballot_sync(0xffffffffu, m != 0u);
+    uint4 hv;
+    uint32_t dpack;
+    if (any == 0u) {  // no background in this row
+        hv = make_uint4(0x7f800000u, 0x7f800000u, 0x7f800000u, 0x7f800000u);
+        dpack = 0x80808080u;
+    } else {
+        const int lzin = m ? (31 - __clz(m)) >> 3 : 0;
+        const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;
+        const unsigned ml = any & ((1u << lane) - 1u);
+        const unsigned mr = lane < 31 ? any >> (lane + 1) : 0u;
+        const int Ll = ml ? 31 - __clz(ml) : 0;
+        const int Lr = mr ? lane + __ffs(mr) : 0;
+        const int lz_l = __shfl_sync(0xffffffffu, lzin, Ll);
+        const int fz_r = __shfl_sync(0xffffffffu, fzin, Lr);
+        const int x0 = 4 * lane;
+        int cur = ml ? 4 * Ll + lz_l : -1024;
+        int dl[4], dr[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dl[b] = x0 + b - cur;
+        }
+        cur = mr ? 4 * Lr + fz_r : 2048;
+#pragma unroll
+        for (int b = 3; b >= 0; --b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dr[b] = cur - (x0 + b);
+        }
+        uint32_t hh[4];
+        dpack = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = min(dl[b], dr[b]);
+            const int off = dl[b] <= dr[b] ? -a : a;
+            hh[b] = __float_as_uint(w2x * small_int_to_float(a * a));
+            dpack |= ((uint32_t)off & 0xffu) << (8 * b);
+        }
+        hv = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+    }
+    if (act) {
+        *reinterpret_cast<uint4*>(vrow + 4 * lane) = hv;
+        *reinterpret_cast<uint32_t*>(drow + 4 * lane) = dpack;
+    }
+}
+
+template <bool FINAL, int VS>
+__global__ void __launch_bounds__(512) plane_sampled_kernel(const __grid_constant__ FastParams P,
+                                                            const __grid_constant__ EpilogueParams ep,
+                                                            const __grid_constant__ ScanTab tab) {
+    extern __shared__ __align__(16) uint8_t sm_plane_s[];
+    const int n0 = P.n0, n1 = P.n;
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_plane_s);                 // [n1][VS] float32 heights
+    uint8_t* dxt = sm_plane_s + (size_t)n1 * VS * 4;                         // [n1][VS] first-axis offsets
+    const int64_t plane = blockIdx.x;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    {
+        constexpr int MAXR = 16;
+        uint32_t rowv[MAXR];
+        const bool act = 4 * lane < n0;
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
+        }
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            if (y < n1) pass0_row_to_heights(rowv[i], n0, P.w2p[0], val + y * VS, dxt + y * VS, lane);
+        }
+    }
+    __syncthreads();
+    // a warp keeps one 32-column group and strides over the rows (nwarps is a multiple of VS / 32)
+    constexpr int CG = VS / 32;
+    const int cg = warp % CG, r0 = warp / CG, rstep = nwarps / CG;
+    const int c = cg * 32 + lane;
+    if (c >= n0) return;
+    ColumnOut<1, FINAL> out;
+    out.stride = n0;
+    if (!FINAL) {
+        out.out = reinterpret_cast<uint16_t*>(P.out) + plane * (int64_t)n1 * n0 + c;
+    } else {  // two processed axes: the plane is the image
+        out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
+        out.sq = nullptr;
+        out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+        out.V = ep.V; out.ndim = ep.ndim;
+        out.dist_only = ep.dist && !ep.idx;
+        out.coord[0] = c;
+        out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+        out.init_index_planes();
+    }
+    for (int y = r0; y < n1; y += rstep)
+        scan_voxel<1, FINAL, false, VS, uint8_t>(val + c, dxt + c, VS, n1, y, tab, out);
+}
+
 template <int K, bool FINAL, bool UNIT, int TX>
 __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ FastParams P,
                                                      const __grid_constant__ EpilogueParams ep,

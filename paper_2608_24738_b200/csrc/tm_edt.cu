@@ -327,6 +327,18 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
             if (fin) { if (vs == 32) TM_LAUNCH_PLANE_UNIT(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(true, 64); else TM_LAUNCH_PLANE_UNIT(true, 128); }
             else { if (vs == 32) TM_LAUNCH_PLANE_UNIT(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(false, 64); else TM_LAUNCH_PLANE_UNIT(false, 128); }
 #undef TM_LAUNCH_PLANE_UNIT
+        } else if (!UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
+            const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
+            const size_t smem_s = (size_t)pl.ext[1] * vs * 5;
+#define TM_LAUNCH_PLANE_SAMPLED(FIN, VSV)                                                                      \
+    do {                                                                                                       \
+        auto kern = plane_sampled_kernel<FIN, VSV>;                                                            \
+        if (smem_s > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_s); \
+        kern<<<(unsigned)P.outer, 1024, smem_s, st>>>(P, ep, tab);                                             \
+    } while (0)
+            if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SAMPLED(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_SAMPLED(true, 64); else TM_LAUNCH_PLANE_SAMPLED(true, 128); }
+            else { if (vs == 32) TM_LAUNCH_PLANE_SAMPLED(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_SAMPLED(false, 64); else TM_LAUNCH_PLANE_SAMPLED(false, 128); }
+#undef TM_LAUNCH_PLANE_SAMPLED
         } else if (fin) plane_kernel<true, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
         else plane_kernel<false, UNIT><<<(unsigned)P.outer, threads, smem, st>>>(P, ep, tab);
         ++launches;
