@@ -334,7 +334,7 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     do {                                                                                                       \
         auto kern = plane_sampled_kernel<FIN, VSV>;                                                            \
         if (smem_s > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_s); \
-        kern<<<(unsigned)P.outer, 1024, smem_s, st>>>(P, ep, tab);                                             \
+        kern<<<(unsigned)P.outer, 512, smem_s, st>>>(P, ep, tab);                                              \
     } while (0)
             if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SAMPLED(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_SAMPLED(true, 64); else TM_LAUNCH_PLANE_SAMPLED(true, 128); }
             else { if (vs == 32) TM_LAUNCH_PLANE_SAMPLED(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_SAMPLED(false, 64); else TM_LAUNCH_PLANE_SAMPLED(false, 128); }
