@@ -7,6 +7,7 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "edt_common.cuh"
@@ -425,23 +426,41 @@ static int check_call(const uint8_t* input, int ndim, const int64_t* shape, cons
     return TM_EDT_OK;
 }
 
-static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int64_t* out_sq, int64_t* out_idx,
-                      void* ws, cudaStream_t st) {
+static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_dist, int64_t* out_sq, int64_t* out_idx,
+                              void* ws, cudaStream_t st, int& launches) {
     EpilogueParams ep;
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
+    if (pl.wide2d && ((uintptr_t)input & 15u) == 0) return run_wide2d(pl, input, ep, ws, st, launches);
+    if (pl.fast)
+        return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
+    if (pl.use_double)
+        return pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
+                       : run_generic<double, int8_t>(pl, input, ep, ws, st, launches);
+    return pl.wide ? run_generic<float, int16_t>(pl, input, ep, ws, st, launches)
+                   : run_generic<float, int8_t>(pl, input, ep, ws, st, launches);
+}
+
+// Images are independent, so a batch too large for one grid (no kernel uses more than one block per
+// voxel; a grid holds 2^31 - 1 blocks) is run as consecutive image ranges on the same stream and scratch.
+static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int64_t* out_sq, int64_t* out_idx,
+                      void* ws, cudaStream_t st) {
+    int64_t max_voxels = INT32_MAX;
+    if (const char* lim = getenv("TM_EDT_CHUNK_VOXELS")) {  // test hook: smaller image ranges
+        const long long v = atoll(lim);
+        if (v > 0 && v < max_voxels) max_voxels = v;
+    }
+    const int64_t max_images = std::max<int64_t>(1, max_voxels / pl.V);
     int launches = 0;
-    cudaError_t e;
-    if (pl.wide2d && ((uintptr_t)input & 15u) == 0)
-        e = run_wide2d(pl, input, ep, ws, st, launches);
-    else if (pl.fast)
-        e = pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
-    else if (pl.use_double)
-        e = pl.wide ? run_generic<double, int16_t>(pl, input, ep, ws, st, launches)
-                    : run_generic<double, int8_t>(pl, input, ep, ws, st, launches);
-    else
-        e = pl.wide ? run_generic<float, int16_t>(pl, input, ep, ws, st, launches)
-                    : run_generic<float, int8_t>(pl, input, ep, ws, st, launches);
-    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    for (int64_t first = 0; first < pl.images; first += max_images) {
+        Plan sub = pl;
+        sub.images = std::min<int64_t>(max_images, pl.images - first);
+        sub.N = sub.images * pl.V;
+        sub.plane_bytes = (((size_t)sub.N * (pl.wide ? 2 : 1)) + 255) & ~(size_t)255;
+        const int64_t v0 = first * pl.V;
+        cudaError_t e = run_images(sub, input + v0, out_dist ? out_dist + v0 : nullptr, out_sq ? out_sq + v0 : nullptr,
+                                   out_idx ? out_idx + v0 * pl.ndim : nullptr, ws, st, launches);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    }
     g_last_launches = launches;
     return TM_EDT_OK;
 }

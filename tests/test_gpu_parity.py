@@ -148,6 +148,18 @@ def test_sparse_background_long_axis_exactness():
     full_check(mask, None)
 
 
+def test_large_batches_run_as_image_ranges(monkeypatch):
+    """A batch that does not fit one grid is cut into image ranges; a test hook makes the ranges tiny."""
+    monkeypatch.setenv("TM_EDT_CHUNK_VOXELS", str(2 * 12 * 16 * 20 + 5))  # two images per range
+    mask = workloads.random_mask(21, (5, 1, 12, 16, 20), 0.85)
+    mask[3] = 1
+    res, ref = full_check(mask, None)
+    assert binding.tm_edt_last_launch_count() == 3 * 2  # three ranges, two kernels each
+    full_check(mask, (1.5, 0.7, 1.0))
+    monkeypatch.setenv("TM_EDT_FORCE_GENERIC", "1")
+    full_check(mask, None)
+
+
 def test_workspace_variant_and_preallocated_outputs():
     import torch
 
