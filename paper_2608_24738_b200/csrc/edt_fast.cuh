@@ -45,6 +45,9 @@ struct FastParams {
     int n0;              // plane kernel: extent of the contiguous axis (== inner)
     float w2;            // squared sampling of this axis
     float w2p[4];        // squared sampling of the earlier axes (plane order)
+    int si[4];           // scaled-integer mode: scale * w^2 of the earlier axes (exact integers)
+    int sk;              // scaled-integer mode: scale * w^2 of this axis
+    float inv_scale;     // scaled-integer mode: 1 / scale
 };
 
 // add[d] = w^2 d^2 for the axis of the pass: float32 bits (sampled) or d^2 << shift (unit sampling keys).
@@ -196,10 +199,12 @@ __device__ __forceinline__ uint32_t scan_keys(const uint32_t* __restrict__ col, 
 // Unit sampling, R consecutive rows y0 .. y0+R-1 of one column at once: every row fetched from the tile
 // serves all R voxels (each with its own addend), which divides the shared-memory loads and the loop
 // overhead per voxel by R.  Rows beyond the column end get best = 0 and are not emitted by the caller.
+// wk: integer weight of the axis (1 for unit sampling); addends are wk * t^2 << SH.
 template <int VS, int R, int SH = 8>
-__device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col, int n, int y0, uint32_t (&best)[R]) {
+__device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col, int n, int y0, uint32_t (&best)[R],
+                                                const uint32_t wk = 1u) {
     // "no site" key: above every real key, and adding any addend to it must not wrap around
-    constexpr uint32_t NONE = SH == 16 ? kNoneKey16 : kNoneKey;
+    constexpr uint32_t NONE = SH == 8 ? kNoneKey : kNoneKey16;
     uint32_t k[R];
 #pragma unroll
     for (int i = 0; i < R; ++i) k[i] = y0 + i < n ? col[(y0 + i) * VS] : NONE;
@@ -208,7 +213,7 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
         best[i] = k[i];
 #pragma unroll
         for (int j = 0; j < R; ++j)
-            if (j != i) best[i] = __viaddmin_u32(k[j], (uint32_t)((i - j) * (i - j)) << SH, best[i]);
+            if (j != i) best[i] = __viaddmin_u32(k[j], (wk * (uint32_t)((i - j) * (i - j))) << SH, best[i]);
         if (y0 + i >= n) best[i] = 0u;
     }
     uint32_t mx = best[0];
@@ -217,7 +222,7 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
     if (mx < (1u << SH)) return;  // a group of background voxels
     uint32_t a[R];                // a[i] = (d + i)^2 << SH
 #pragma unroll
-    for (int i = 0; i < R; ++i) a[i] = (uint32_t)((1 + i) * (1 + i)) << SH;
+    for (int i = 0; i < R; ++i) a[i] = (wk * (uint32_t)((1 + i) * (1 + i))) << SH;
     const uint32_t* plo = col + (y0 - 1) * VS;
     const uint32_t* phi = col + (y0 + R) * VS;
     int lo = y0 - 1, hi = y0 + R;
@@ -238,7 +243,7 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
         for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
 #pragma unroll
         for (int i = 0; i + 1 < R; ++i) a[i] = a[i + 1];
-        a[R - 1] = (uint32_t)((d + R) * (d + R)) << SH;
+        a[R - 1] = (wk * (uint32_t)((d + R) * (d + R))) << SH;
     }
 }
 
@@ -754,6 +759,219 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
     } else {
         for (int y = r0; y < n; y += rstep)
             scan_voxel<K, FINAL, UNIT, TX, EI>(val + c, tile + c, TX, n, y, tab, out);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Scaled-integer mode.  When a common scale S makes every S * w_q^2 an integer (sampling given with a
+// few decimals: 0.8, 1.25, 2.5 ..) and the largest possible value S * sum_q w_q^2 (n_q - 1)^2 stays below
+// 2^24, the transform with that sampling is exact integer arithmetic again: keys are
+// (S * height) << 7 | row, candidates are combined with the fused add-min, and four rows share every
+// fetched candidate, exactly as for unit sampling.  Distances are sqrt(value / S).
+// ---------------------------------------------------------------------------------------------
+constexpr int kScaledShift = 7;
+
+template <int K>
+__device__ __forceinline__ uint32_t scaled_key(uint32_t e, int row, const int* si) {
+    if (entry_none(e)) return kNoneKey16;
+    int o = (int)(int8_t)(e & 0xff);
+    int v = si[0] * o * o;
+    if (K > 1) { o = (int)(int8_t)((e >> 8) & 0xff); v += si[1] * o * o; }
+    if (K > 2) { o = (int)(int8_t)((e >> 16) & 0xff); v += si[2] * o * o; }
+    if (K > 3) { o = (int)(int8_t)((e >> 24) & 0xff); v += si[3] * o * o; }
+    return ((uint32_t)v << kScaledShift) | (uint32_t)row;
+}
+
+// Outputs of row y from a scaled key; ent[row * ES] are the entries of the column.
+template <int K, bool FINAL, typename ET>
+__device__ __forceinline__ void emit_scaled(const ColumnOut<K, FINAL>& out, const ET* __restrict__ ent, int ES, int y,
+                                            uint32_t b, float inv_scale) {
+    if (b < (1u << kScaledShift)) { emit<K, FINAL, false>(out, y, y, 0u, 0.f, false); return; }
+    const bool none = b >= kNoneKey16;
+    const int j = (int)(b & ((1u << kScaledShift) - 1u));
+    const uint32_t e = none ? 0u : (uint32_t)ent[j * ES];
+    emit<K, FINAL, false>(out, y, j, e, __uint2float_rn(b >> kScaledShift) * inv_scale, none);  // values reach 2^24
+}
+
+__device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n0, int y, int s0,
+                                                         uint32_t* __restrict__ vrow, uint8_t* __restrict__ drow,
+                                                         int lane) {
+    const bool act = 4 * lane < n0;
+    const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
+    const unsigned any = __ballot_sync(0xffffffffu, m != 0u);
+    uint4 kv;
+    uint32_t dpack;
+    if (any == 0u) {  // no background in this row
+        kv = make_uint4(kNoneKey16, kNoneKey16, kNoneKey16, kNoneKey16);
+        dpack = 0x80808080u;
+    } else {
+        const int lzin = m ? (31 - __clz(m)) >> 3 : 0;
+        const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;
+        const unsigned ml = any & ((1u << lane) - 1u);
+        const unsigned mr = lane < 31 ? any >> (lane + 1) : 0u;
+        const int Ll = ml ? 31 - __clz(ml) : 0;
+        const int Lr = mr ? lane + __ffs(mr) : 0;
+        const int lz_l = __shfl_sync(0xffffffffu, lzin, Ll);
+        const int fz_r = __shfl_sync(0xffffffffu, fzin, Lr);
+        const int x0 = 4 * lane;
+        int cur = ml ? 4 * Ll + lz_l : -1024;
+        int dl[4], dr[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dl[b] = x0 + b - cur;
+        }
+        cur = mr ? 4 * Lr + fz_r : 2048;
+#pragma unroll
+        for (int b = 3; b >= 0; --b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dr[b] = cur - (x0 + b);
+        }
+        uint32_t kk[4];
+        dpack = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = min(dl[b], dr[b]);
+            const int off = dl[b] <= dr[b] ? -a : a;
+            kk[b] = ((uint32_t)(s0 * a * a) << kScaledShift) | (uint32_t)y;
+            dpack |= ((uint32_t)off & 0xffu) << (8 * b);
+        }
+        kv = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+    }
+    if (act) {
+        *reinterpret_cast<uint4*>(vrow + 4 * lane) = kv;
+        *reinterpret_cast<uint32_t*>(drow + 4 * lane) = dpack;
+    }
+}
+
+template <bool FINAL, int VS>
+__global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant__ FastParams P,
+                                                           const __grid_constant__ EpilogueParams ep) {
+    extern __shared__ __align__(16) uint8_t sm_plane_i[];
+    const int n0 = P.n0, n1 = P.n;
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_plane_i);   // [n1][VS] keys
+    uint8_t* dxt = sm_plane_i + (size_t)n1 * VS * 4;           // [n1][VS] first-axis offsets
+    const int64_t plane = blockIdx.x;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    {
+        constexpr int MAXR = 16;
+        uint32_t rowv[MAXR];
+        const bool act = 4 * lane < n0;
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
+        }
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * nwarps;
+            if (y < n1) pass0_row_to_scaled_keys(rowv[i], n0, y, P.si[0], val + y * VS, dxt + y * VS, lane);
+        }
+    }
+    __syncthreads();
+    constexpr int R = 4, CG = VS / 32;
+    const int cg = warp % CG, r0 = warp / CG, rstep = nwarps / CG;
+    const int c = cg * 32 + lane;
+    if (c >= n0) return;
+    ColumnOut<1, FINAL> out;
+    out.stride = n0;
+    if (!FINAL) {
+        out.out = reinterpret_cast<uint16_t*>(P.out) + plane * (int64_t)n1 * n0 + c;
+    } else {  // two processed axes: the plane is the image
+        out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
+        out.sq = nullptr;
+        out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+        out.V = ep.V; out.ndim = ep.ndim;
+        out.dist_only = ep.dist && !ep.idx;
+        out.coord[0] = c;
+        out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
+        out.init_index_planes();
+    }
+    for (int y0 = r0 * R; y0 < n1; y0 += rstep * R) {
+        uint32_t best[R];
+        scan_keys_group<VS, R, kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            if (y0 + i < n1) emit_scaled<1, FINAL, uint8_t>(out, dxt + c, VS, y0 + i, best[i], P.inv_scale);
+    }
+}
+
+template <int K, bool FINAL, int TX>
+__global__ void __launch_bounds__(256) column_scaled_kernel(const __grid_constant__ FastParams P,
+                                                            const __grid_constant__ EpilogueParams ep,
+                                                            const int tiles_per_slab) {
+    using EI = typename EntryType<entry_bytes(K)>::type;
+    extern __shared__ __align__(16) uint8_t sm_col_i[];
+    constexpr int G = TX / 32;
+    const int n = P.n;
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_col_i);               // [n][TX]
+    EI* tile = reinterpret_cast<EI*>(sm_col_i + (size_t)n * TX * 4);     // [n][TX]
+    const int64_t slab = blockIdx.x / tiles_per_slab;
+    const int64_t i0 = (int64_t)(blockIdx.x - slab * tiles_per_slab) * TX;
+    const int width = (int)min((int64_t)TX, P.inner - i0);
+    const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
+    const int si[4] = {P.si[0], P.si[1], P.si[2], P.si[3]};
+    constexpr int PER16 = 16 / (int)sizeof(EI);
+    if ((P.inner % PER16) == 0 && width == TX) {  // full tile, 16-byte aligned rows
+        constexpr int FULL = TX / PER16;
+        for (int t = threadIdx.x; t < n * FULL; t += blockDim.x) {
+            const int y = t / FULL, ch = t - y * FULL;
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + ch * PER16);
+            *reinterpret_cast<uint4*>(tile + y * TX + ch * PER16) = v;
+            const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+            uint32_t sv[PER16];
+#pragma unroll
+            for (int i = 0; i < PER16; ++i) {
+                const uint32_t word = wv[(i * (int)sizeof(EI)) >> 2];
+                const uint32_t e = sizeof(EI) == 4 ? word
+                                 : sizeof(EI) == 2 ? ((word >> (16 * (i & 1))) & 0xffffu)
+                                                   : ((word >> (8 * (i & 3))) & 0xffu);
+                sv[i] = scaled_key<K>(e, y, si);
+            }
+#pragma unroll
+            for (int i = 0; i < PER16; i += 4)
+                *reinterpret_cast<uint4*>(val + y * TX + ch * PER16 + i) = make_uint4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
+        }
+    } else {
+        for (int t = threadIdx.x; t < n * width; t += blockDim.x) {
+            const int y = t / width, x = t - y * width;
+            const EI e = src[(int64_t)y * P.inner + x];
+            tile[y * TX + x] = e;
+            val[y * TX + x] = scaled_key<K>((uint32_t)e, y, si);
+        }
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = warp % G, r0 = warp / G, rstep = nwarps / G;
+    const int c = g * 32 + lane;
+    if (c >= width) return;
+    ColumnOut<K, FINAL> out;
+    out.stride = P.inner;
+    if (!FINAL) {
+        using EO = typename EntryType<entry_bytes(K + 1)>::type;
+        out.out = reinterpret_cast<EO*>(P.out) + slab * (int64_t)n * P.inner + i0 + c;
+    } else {  // last pass: the slab is the image
+        const int64_t v0 = i0 + c;
+        out.dist = ep.dist ? ep.dist + slab * ep.V + v0 : nullptr;
+        out.sq = nullptr;
+        out.idx = ep.idx ? ep.idx + slab * ep.ndim * ep.V + v0 : nullptr;
+        out.V = ep.V; out.ndim = ep.ndim;
+        out.dist_only = ep.dist && !ep.idx;
+        int64_t rr = v0;
+#pragma unroll
+        for (int q = 0; q < K; ++q) { out.coord[q] = (int)(rr % ep.ext[q]); rr /= ep.ext[q]; }
+#pragma unroll
+        for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
+        out.init_index_planes();
+    }
+    constexpr int R = 4;
+    for (int y0 = r0 * R; y0 < n; y0 += rstep * R) {
+        uint32_t best[R];
+        scan_keys_group<TX, R, kScaledShift>(val + c, n, y0, best, (uint32_t)P.sk);
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+            if (y0 + i < n) emit_scaled<K, FINAL, EI>(out, tile + c, TX, y0 + i, best[i], P.inv_scale);
     }
 }
 

@@ -58,6 +58,9 @@ struct Plan {
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
     bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
+    int si[kMaxDims];         // those integers
+    double scale = 1.0;
     bool wide2d = false;      // two processed axes, unit sampling, extents <= 512, contiguous extent % 16 == 0
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
@@ -132,6 +135,26 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
     pl.wide2d = !pl.fast && E == 2 && pl.unit && nmax <= 512 && pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
     if (pl.wide2d) pl.ws_bytes = (((size_t)pl.N * 4 + 255) & ~(size_t)255) + (((size_t)pl.N * 2 + 255) & ~(size_t)255);
+    if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
+        // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
+        // the largest possible value below 2^24 (keys are value << 7 | row in 32 bits)
+        static const int cand[] = {1, 4, 16, 25, 64, 100, 256, 400, 625, 1024, 2500, 10000};
+        for (int S : cand) {
+            bool ok = true;
+            double total = 0.0, edge = 0.0;
+            for (int p = 0; p < E && ok; ++p) {
+                const double v = pl.w[p] * pl.w[p] * S, r = nearbyint(v);
+                if (r < 1.0 || r > 1048576.0 || fabs(v - r) > 1e-9 * v) { ok = false; break; }
+                pl.si[p] = (int)r;
+                total += r * (double)(pl.ext[p] - 1) * (double)(pl.ext[p] - 1);
+                const double e2 = r * (double)(pl.ext[p] + 4) * (double)(pl.ext[p] + 4);
+                edge = e2 > edge ? e2 : edge;
+            }
+            // total: largest true value; edge: largest addend.  Both below 2^24 keep every real key below the
+            // "no site" key 2^31 and every key + addend below 2^32.
+            if (ok && total < 16777216.0 && edge < 16777216.0) { pl.scaled = true; pl.scale = S; break; }
+        }
+    }
     if (pl.fast) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
         const size_t a = E >= 3 ? up((size_t)pl.N * (E >= 5 ? 4 : 2)) : 0;
@@ -362,6 +385,86 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     return cudaSuccess;
 }
 
+template <int K, bool FINAL>
+static cudaError_t launch_column_scaled(const FastParams& P, const EpilogueParams& ep, cudaStream_t st, double out_bpv) {
+    const size_t eb = (size_t)entry_bytes(K);
+    int G = 1;
+    while (G < 4 && P.n * 32 * G * 2 <= 4096 && 32 * G < P.inner) G <<= 1;
+    const int TX = 32 * G;
+    const size_t smem = (size_t)P.n * TX * (4 + eb);
+    const int tiles = (int)((P.inner + TX - 1) / TX);
+    const int64_t blocks = P.outer * tiles;
+    const double vox = (double)P.outer * P.n * (double)P.inner;
+    prof_mark(st, FINAL ? "column_scaled_final" : "column_scaled",
+              vox * ((double)eb + (FINAL ? out_bpv : (double)entry_bytes(K + 1))));
+#define TM_LAUNCH_COLUMN_SCALED(TXV)                                                                           \
+    do {                                                                                                       \
+        auto kern = column_scaled_kernel<K, FINAL, TXV>;                                                       \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        kern<<<(unsigned)blocks, 256, smem, st>>>(P, ep, tiles);                                               \
+    } while (0)
+    if (G == 1) TM_LAUNCH_COLUMN_SCALED(32); else if (G == 2) TM_LAUNCH_COLUMN_SCALED(64); else TM_LAUNCH_COLUMN_SCALED(128);
+#undef TM_LAUNCH_COLUMN_SCALED
+    return cudaGetLastError();
+}
+
+// Packed-entry path in scaled integers (see edt_fast.cuh): fused plane kernel, then column kernels.
+static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                              int& launches) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    char* bufA = static_cast<char*>(ws);
+    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * (pl.E >= 5 ? 4 : 2)) : 0);
+    const double out_bpv = out_bytes_per_voxel(ep);
+    auto fill = [&](FastParams& P, int k) {
+        memset(&P, 0, sizeof(P));
+        P.n = pl.ext[k]; P.inner = pl.inner[k]; P.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+        for (int p = 0; p < k && p < 4; ++p) P.si[p] = pl.si[p];
+        P.sk = pl.si[k];
+        P.inv_scale = (float)(1.0 / pl.scale);
+    };
+    FastParams P;
+    fill(P, 1);
+    P.in = in; P.out = bufA; P.n0 = pl.ext[0];
+    {
+        const bool fin = pl.E == 2;
+        const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
+        const size_t smem = (size_t)pl.ext[1] * vs * 5;
+        prof_mark(st, fin ? "plane_scaled_final" : "plane_scaled", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
+#define TM_LAUNCH_PLANE_SCALED(FIN, VSV)                                                                       \
+    do {                                                                                                       \
+        auto kern = plane_scaled_kernel<FIN, VSV>;                                                             \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        kern<<<(unsigned)P.outer, 512, smem, st>>>(P, ep);                                                     \
+    } while (0)
+        if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64); else TM_LAUNCH_PLANE_SCALED(true, 128); }
+        else { if (vs == 32) TM_LAUNCH_PLANE_SCALED(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(false, 64); else TM_LAUNCH_PLANE_SCALED(false, 128); }
+#undef TM_LAUNCH_PLANE_SCALED
+        ++launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    char* src = bufA;
+    char* dst = bufB;
+    for (int k = 2; k < pl.E; ++k) {
+        fill(P, k);
+        P.in = src; P.out = dst;
+        const bool fin = k == pl.E - 1;
+        cudaError_t e = cudaErrorInvalidValue;
+        if (fin) {
+            if (k == 2) e = launch_column_scaled<2, true>(P, ep, st, out_bpv);
+            else if (k == 3) e = launch_column_scaled<3, true>(P, ep, st, out_bpv);
+            else if (k == 4) e = launch_column_scaled<4, true>(P, ep, st, out_bpv);
+        } else {
+            if (k == 2) e = launch_column_scaled<2, false>(P, ep, st, out_bpv);
+            else if (k == 3) e = launch_column_scaled<3, false>(P, ep, st, out_bpv);
+        }
+        ++launches;
+        if (e != cudaSuccess) return e;
+        char* t = src; src = dst; dst = t;
+    }
+    return cudaSuccess;
+}
+
 // Two-dimensional unit-sampling images with extents up to 512: key rows, then column strips.
 static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
                               int& launches) {
@@ -431,6 +534,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     EpilogueParams ep;
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     if (pl.wide2d && ((uintptr_t)input & 15u) == 0) return run_wide2d(pl, input, ep, ws, st, launches);
+    if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
         return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
     if (pl.use_double)
