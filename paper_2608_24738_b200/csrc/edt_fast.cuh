@@ -429,7 +429,6 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
                         const int y = y0 + i;
                         if (y >= n1) break;
                         const uint32_t b = best[i];
-                        if (b < 256u) { emit<1, FINAL, true>(out, y, y, 0u, 0.f, false); continue; }
                         const bool none = b >= kNoneKey;
                         const int j = (int)(b & 0xffu);
                         const uint32_t e = none ? 0u : (uint32_t)tile[j * tstride + c];
@@ -748,8 +747,8 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
             for (int i = 0; i < R; ++i) {
                 const int y = y0 + i;
                 if (y >= n) break;
+                // no special case for background voxels: their key names their own row, whose entry is 0
                 const uint32_t b = best[i];
-                if (b < 256u) { emit<K, FINAL, true>(out, y, y, 0u, 0.f, false); continue; }
                 const bool none = b >= kNoneKey;
                 const int j = (int)(b & 0xffu);
                 const uint32_t e = none ? 0u : (uint32_t)tile[j * TX + c];
@@ -786,8 +785,7 @@ __device__ __forceinline__ uint32_t scaled_key(uint32_t e, int row, const int* s
 template <int K, bool FINAL, typename ET>
 __device__ __forceinline__ void emit_scaled(const ColumnOut<K, FINAL>& out, const ET* __restrict__ ent, int ES, int y,
                                             uint32_t b, float inv_scale) {
-    if (b < (1u << kScaledShift)) { emit<K, FINAL, false>(out, y, y, 0u, 0.f, false); return; }
-    const bool none = b >= kNoneKey16;
+    const bool none = b >= kNoneKey16;  // background voxels need no special case: their key names their own row
     const int j = (int)(b & ((1u << kScaledShift) - 1u));
     const uint32_t e = none ? 0u : (uint32_t)ent[j * ES];
     emit<K, FINAL, false>(out, y, j, e, __uint2float_rn(b >> kScaledShift) * inv_scale, none);  // values reach 2^24

@@ -148,6 +148,19 @@ def test_sparse_background_long_axis_exactness():
     full_check(mask, None)
 
 
+def test_sampling_without_a_common_integer_scale():
+    """Sampling whose squares share no small integer scale stays on float32 heights; decimal sampling
+    (handled in exact scaled integers) must agree with it within the distance tolerance."""
+    import math
+
+    mask = workloads.random_mask(31, (2, 1, 40, 64, 48), 0.9)
+    full_check(mask, (math.pi / 3.0, math.sqrt(2.0), 1.0))
+    full_check(mask, (2.5, 0.8, 1.0))
+    mask4 = workloads.random_mask(32, (1, 1, 6, 24, 32, 16), 0.85)
+    full_check(mask4, (math.e / 2.0, 1.0, math.sqrt(3.0), 0.9))
+    full_check(mask4, (1.25, 1.0, 0.5, 2.0))
+
+
 def test_large_batches_run_as_image_ranges(monkeypatch):
     """A batch that does not fit one grid is cut into image ranges; a test hook makes the ranges tiny."""
     monkeypatch.setenv("TM_EDT_CHUNK_VOXELS", str(2 * 12 * 16 * 20 + 5))  # two images per range
