@@ -225,8 +225,26 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
     for (int i = 0; i < R; ++i) a[i] = (wk * (uint32_t)((1 + i) * (1 + i))) << SH;
     const uint32_t* plo = col + (y0 - 1) * VS;
     const uint32_t* phi = col + (y0 + R) * VS;
-    int lo = y0 - 1, hi = y0 + R;
-    for (int d = 1; a[0] < mx; ++d, --lo, ++hi, plo -= VS, phi += VS) {
+    int d = 1;
+    // interior steps: both rows exist, no bounds tests
+    const int dsafe = min(y0, n - R - y0);
+    for (; d <= dsafe && a[0] < mx; ++d, plo -= VS, phi += VS) {
+        const uint32_t vlo = plo[0], vhi = phi[0];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            best[i] = __viaddmin_u32(vlo, a[i], best[i]);
+            best[i] = __viaddmin_u32(vhi, a[R - 1 - i], best[i]);
+        }
+        mx = best[0];
+#pragma unroll
+        for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
+#pragma unroll
+        for (int i = 0; i + 1 < R; ++i) a[i] = a[i + 1];
+        a[R - 1] = (wk * (uint32_t)((d + R) * (d + R))) << SH;
+    }
+    // steps that reach past one end of the column
+    int lo = y0 - d, hi = y0 + R - 1 + d;
+    for (; a[0] < mx; ++d, --lo, ++hi, plo -= VS, phi += VS) {
         if (lo < 0 && hi >= n) break;
         if (lo >= 0) {
             const uint32_t v = plo[0];
