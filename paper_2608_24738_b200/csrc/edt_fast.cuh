@@ -5,13 +5,17 @@
 // first); 1, 2, 4 bytes for 1, 2, 3..4 axes.  Byte 0 == 0x80 marks "no site yet".  An entry of all
 // zeros is a background voxel.  Entries make every load, gather and store of a voxel one access.
 //
-// Kernels:
-//   plane_kernel   first axis + second axis fused: one thread block per (n_1 x n_0) plane.  The rows
-//                  of the raw mask are bit-packed with warp ballots and turned into 1-byte offsets in
-//                  shared memory (first-axis pass); then the pass along axis 1 runs on that tile and
-//                  writes 2-byte entries or the final outputs.
-//   column_kernel  one further axis: a block stages an (n x TX) tile of entries in shared memory
-//                  (TX consecutive positions of the contiguous `inner` index) and runs the pass on it.
+// Kernels (one thread block per (n_1 x n_0) plane, or per (n x 32 G) tile of a later axis):
+//   plane_unit_kernel     unit sampling: the first-axis pass (four voxels per lane, ballot + shuffles)
+//                         writes scan keys straight into a plane-wide shared tile, the second-axis pass
+//                         scans it; 2-byte entries or the final outputs go to global memory.
+//   plane_scaled_kernel   the same for sampling that becomes integer under a common scale.
+//   plane_sampled_kernel  the same with float32 heights (any sampling).
+//   plane_kernel          fallback for contiguous extents that are no multiple of 4 or unaligned input:
+//                         byte loads, up to four ballot words per row, 32-column groups.
+//   column_kernel         one further axis: a block stages a tile of entries in shared memory (TX
+//                         consecutive positions of the contiguous `inner` index) and runs the pass on it.
+//   column_scaled_kernel  the same in scaled integers.
 //
 // The pass along an axis (g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (w_k (x_k - j))^2 ], paper
 // Section 2.3.2) is taken voxel by voxel as an exact bounded scan instead of a sequential envelope
@@ -22,9 +26,10 @@
 // columns of the same row (loads and stores are contiguous runs, neighbouring voxels have similar scan
 // lengths), and background voxels (height 0) leave the loop at once.
 //
-// Unit sampling: heights are integers; the tile holds keys (height << 8 | row) so that one fused
-// add-and-min instruction per candidate tracks value and site together, exactly.  Other sampling:
-// heights are float32, the site is tracked by a compare and select.
+// Integer heights (unit sampling, or scaled integers): the tile holds keys (height << s | row) so that
+// one fused add-and-min instruction per candidate tracks value and site together, exactly; four
+// consecutive rows of a column are scanned together so that every fetched candidate serves four voxels.
+// Other sampling: heights are float32, the site is tracked by a compare and select.
 #pragma once
 #include "edt_common.cuh"
 

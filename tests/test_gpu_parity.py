@@ -161,6 +161,37 @@ def test_sampling_without_a_common_integer_scale():
     full_check(mask4, (1.25, 1.0, 0.5, 2.0))
 
 
+@pytest.mark.parametrize("shape", [(1, 1, 9, 4), (2, 1, 33, 8), (1, 1, 17, 12), (1, 2, 64, 20), (1, 1, 100, 124),
+                                   (1, 1, 5, 128), (1, 1, 30, 16, 36), (1, 1, 300, 16), (1, 1, 77, 512)])
+def test_any_nonzero_byte_is_foreground(shape):
+    """Masks with arbitrary byte values (0x01, 0x7f, 0x80, 0xff ..): only 0 is background.  Exercises the
+    zero-byte tests of the 4- and 16-voxels-per-lane first-axis passes."""
+    rng = np.random.default_rng(zlib.crc32(repr(shape).encode()))
+    vals = np.array([0, 1, 2, 0x7F, 0x80, 0x81, 0xFE, 0xFF], dtype=np.uint8)
+    mask = vals[rng.integers(0, len(vals), size=shape)]
+    mask[rng.random(shape) < 0.6] = 0xFF  # keep the background sparse
+    full_check(mask, None)
+    full_check(mask, tuple(1.0 + 0.5 * k for k in range(len(shape) - 2)))
+
+
+def test_unaligned_input_pointer():
+    """An input that does not start on a 4- or 16-byte boundary must take the byte-load kernels."""
+    import torch
+
+    for shape, samp in (((1, 1, 40, 64), None), ((1, 1, 12, 32, 64), (2.5, 0.8, 1.0)), ((1, 1, 200, 256), None)):
+        mask = workloads.random_mask(41, shape, 0.85)
+        ref = oracle.sep(mask, samp, want_idx=False)
+        buf = torch.zeros(mask.size + 64, dtype=torch.uint8, device="cuda")
+        for shift in (1, 3, 8):
+            view = buf[shift: shift + mask.size].view(shape)
+            view.copy_(torch.from_numpy(mask))
+            assert view.data_ptr() % 16 != 0
+            r = binding.tm_edt(view, samp, return_distances=True, return_indices=True)
+            torch.cuda.synchronize()
+            checker.check_dist(r["dist"].cpu().numpy(), ref["dist"])
+            checker.check_indices(r["idx"].cpu().numpy(), mask, ref, samp)
+
+
 def test_large_batches_run_as_image_ranges(monkeypatch):
     """A batch that does not fit one grid is cut into image ranges; a test hook makes the ranges tiny."""
     monkeypatch.setenv("TM_EDT_CHUNK_VOXELS", str(2 * 12 * 16 * 20 + 5))  # two images per range
