@@ -231,8 +231,29 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
     const uint32_t* plo = col + (y0 - 1) * VS;
     const uint32_t* phi = col + (y0 + R) * VS;
     int d = 1;
-    // interior steps: both rows exist, no bounds tests
+    // interior steps, two at a time: both rows exist on both sides, no bounds tests, one stop test per pair
     const int dsafe = min(y0, n - R - y0);
+    for (; d + 1 <= dsafe && a[0] < mx; d += 2, plo -= 2 * VS, phi += 2 * VS) {
+        const uint32_t vlo0 = plo[0], vhi0 = phi[0], vlo1 = plo[-VS], vhi1 = phi[VS];
+        const uint32_t aR = (wk * (uint32_t)((d + R) * (d + R))) << SH;  // addend of distance d + R
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            best[i] = __viaddmin_u32(vlo0, a[i], best[i]);
+            best[i] = __viaddmin_u32(vhi0, a[R - 1 - i], best[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < R; ++i) {  // step d + 1: distances (d + 1 + i) and (d + 1 + R - 1 - i)
+            best[i] = __viaddmin_u32(vlo1, i + 1 < R ? a[i + 1] : aR, best[i]);
+            best[i] = __viaddmin_u32(vhi1, R - i < R ? a[R - i] : aR, best[i]);
+        }
+        mx = best[0];
+#pragma unroll
+        for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
+#pragma unroll
+        for (int i = 0; i + 2 < R; ++i) a[i] = a[i + 2];
+        a[R - 2] = aR;
+        a[R - 1] = (wk * (uint32_t)((d + R + 1) * (d + R + 1))) << SH;
+    }
     for (; d <= dsafe && a[0] < mx; ++d, plo -= VS, phi += VS) {
         const uint32_t vlo = plo[0], vhi = phi[0];
 #pragma unroll
