@@ -327,14 +327,18 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the transform has no CPU path")
-    buildlib.build()
-    binding.lib()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
         import torch.distributed as dist
 
         dist.init_process_group("nccl", device_id=dev)
+        if local == 0:
+            buildlib.build()  # one rank per node compiles (a no-op when the library is up to date)
+        dist.barrier()
+    else:
+        buildlib.build()
+    binding.lib()
 
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
@@ -397,7 +401,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32" if w.sampling is not None else "f32 (exact integers)", "data": "synthetic",
+            "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "shape": list(shape), "sampling": w.sampling,
                        "outputs": [n for n, f in (("dist_f32", w.want_dist), ("sqdist_i64", w.want_sq),
                                                    ("indices_i64", w.want_idx)) if f],
