@@ -24,8 +24,10 @@
  * out_indices names is unspecified; it always names one at the minimal distance, and a background
  * voxel names itself.
  *
- * All entry points are thread-safe and keep no state between calls apart from cached device
- * attributes.  Nothing is thrown and no device trap is ever raised: every problem is a return code,
+ * All entry points are thread-safe.  The only state kept between calls is, per device, a private
+ * stream-ordered memory pool from which tm_edt and tm_edt_host take their scratch (so that one call's
+ * memory is reused by the next; tm_edt_trim_memory() gives it back) and the address of the built-in
+ * scratch array of tm_edt_noalloc.  Nothing is thrown and no device trap is ever raised: every problem is a return code,
  * and every argument check happens before any work is enqueued.
  */
 #ifndef TM_EDT_H_
@@ -78,8 +80,8 @@ typedef struct CUstream_st* tm_edt_stream_t;
  *   out_indices  device int64 (B, C, ndim, n...), or NULL.  out_indices[b, c, a, x] is the coordinate
  *                along spatial axis a of the background voxel chosen for voxel x.
  *   At least one output must be non-NULL.  The caller owns every buffer; the library keeps no
- *   pointer once the enqueued work has run.  Scratch memory is taken from the stream-ordered
- *   allocator of the device (allocation and release are both ordered on `stream`).
+ *   pointer once the enqueued work has run.  Scratch memory is taken from the library's private
+ *   stream-ordered memory pool of the device (allocation and release are both ordered on `stream`).
  *
  * Returns a tm_edt_status.  On any error other than TM_EDT_ERR_CUDA nothing has been enqueued.
  */
@@ -158,6 +160,13 @@ TM_EDT_API int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* sha
                               float* out_dist, int64_t* out_sqdist, int64_t* out_indices, void* workspace,
                               size_t workspace_bytes, tm_edt_stream_t stream, int max_kernels, float* kernel_ms,
                               double* kernel_bytes, char* kernel_names, int* n_kernels);
+
+/*
+ * Returns to the driver whatever the library's private memory pool of the current device holds and no
+ * enqueued work still uses (tm_edt and tm_edt_host keep their scratch pooled between calls).  No
+ * counterpart in the paper, which leaves memory to PyTorch's caching allocator (Section 2.2, Fig. 2).
+ */
+TM_EDT_API int tm_edt_trim_memory(void);
 
 /* Static description of a status code. Never NULL. */
 TM_EDT_API const char* tm_edt_strerror(int status);

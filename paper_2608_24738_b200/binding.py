@@ -20,7 +20,7 @@ MAX_EXTENT = 8192
 
 EXPORTS = (
     "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_workspace_bytes", "tm_edt_strerror",
-    "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count",
+    "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
 )
 
 _lock = threading.Lock()
@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_last_cuda_error.restype = i
             L.tm_edt_last_launch_count.restype = i
             L.tm_edt_version.restype = ctypes.c_char_p
+            L.tm_edt_trim_memory.restype = i
             _lib = L
     return _lib
 
@@ -76,6 +77,11 @@ def tm_edt_version() -> str:
 
 def tm_edt_last_cuda_error() -> int:
     return int(lib().tm_edt_last_cuda_error())
+
+
+def tm_edt_trim_memory() -> None:
+    """Give the library's pooled scratch memory of the current device back to the driver."""
+    _check(int(lib().tm_edt_trim_memory()))
 
 
 def tm_edt_last_launch_count() -> int:

@@ -492,6 +492,37 @@ static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueP
     return cudaGetLastError();
 }
 
+// Stream-ordered scratch of tm_edt and tm_edt_host comes from a memory pool of the library's own, one per
+// device, created on first use.  Its release threshold is unlimited, so the memory of one call is reused by
+// the next instead of going back to the driver at every synchronisation; tm_edt_trim_memory() returns it.
+static cudaMemPool_t g_pool[64];
+static bool g_pool_ready[64];
+static std::mutex g_pool_mutex;
+
+static cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaMallocAsync(p, bytes, st);
+    {
+        std::lock_guard<std::mutex> lock(g_pool_mutex);
+        if (!g_pool_ready[dev]) {
+            cudaMemPoolProps props;
+            memset(&props, 0, sizeof(props));
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            e = cudaMemPoolCreate(&g_pool[dev], &props);
+            if (e != cudaSuccess) return e;
+            uint64_t keep = UINT64_MAX;
+            cudaMemPoolSetAttribute(g_pool[dev], cudaMemPoolAttrReleaseThreshold, &keep);
+            g_pool_ready[dev] = true;
+        }
+    }
+    return cudaMallocFromPoolAsync(p, bytes, g_pool[dev], st);
+}
+
 static bool is_device_ptr(const void* p) {
     cudaPointerAttributes at;
     if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
@@ -611,7 +642,7 @@ int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, const double* s
     cudaStream_t st = (cudaStream_t)stream;
     void* ws = nullptr;
     if (pl.ws_bytes > 0) {
-        cudaError_t e = cudaMallocAsync(&ws, pl.ws_bytes, st);
+        cudaError_t e = scratch_alloc(&ws, pl.ws_bytes, st);
         if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
     }
     rc = run_device(pl, input, out_dist, out_sqdist, out_indices, ws, st);
@@ -634,7 +665,7 @@ int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape, const doub
     const size_t b_in = up(N), b_d = out_dist ? up(N * 4) : 0, b_s = out_sqdist ? up(N * 8) : 0,
                  b_x = out_indices ? up(N * 8 * (size_t)ndim) : 0, b_ws = up(pl.ws_bytes);
     char* dev = nullptr;
-    cudaError_t e = cudaMallocAsync((void**)&dev, b_in + b_d + b_s + b_x + b_ws, st);
+    cudaError_t e = scratch_alloc((void**)&dev, b_in + b_d + b_s + b_x + b_ws, st);
     if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
     uint8_t* d_in = (uint8_t*)dev;
     float* d_d = out_dist ? (float*)(dev + b_in) : nullptr;
@@ -704,6 +735,18 @@ int tm_edt_noalloc(const uint8_t* input, int ndim, const int64_t* shape, const d
         if (rc != TM_EDT_OK) return rc;
     }
     return run_device(pl, input, out_dist, out_sqdist, out_indices, scratch, (cudaStream_t)stream);
+}
+
+int tm_edt_trim_memory(void) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TM_EDT_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return TM_EDT_OK;
+    std::lock_guard<std::mutex> lock(g_pool_mutex);
+    if (g_pool_ready[dev]) {
+        cudaError_t e = cudaMemPoolTrimTo(g_pool[dev], 0);
+        if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    }
+    return TM_EDT_OK;
 }
 
 size_t tm_edt_noalloc_max_scratch(void) { return TM_EDT_NOALLOC_SCRATCH_BYTES; }

@@ -224,6 +224,25 @@ def test_workspace_variant_and_preallocated_outputs():
     assert ei.value.status == binding.ERR_ALLOC
 
 
+def test_pooled_scratch_and_trim():
+    """tm_edt takes its scratch from the library's own memory pool; repeated calls reuse it and
+    tm_edt_trim_memory hands it back without disturbing later calls."""
+    import torch
+
+    mask = workloads.random_mask(51, (2, 1, 40, 48, 64), 0.85)
+    ref = oracle.sep(mask, None, want_idx=False)
+    t = torch.from_numpy(mask).cuda()
+    for _ in range(3):
+        r = binding.tm_edt(t, None, return_distances=True, return_sqdist=True)
+    torch.cuda.synchronize()
+    checker.check_sq_exact(r["sq"].cpu().numpy(), ref["sq"])
+    binding.tm_edt_trim_memory()
+    r = binding.tm_edt(t, None, return_distances=True, return_sqdist=True)
+    torch.cuda.synchronize()
+    checker.check_sq_exact(r["sq"].cpu().numpy(), ref["sq"])
+    binding.tm_edt_trim_memory()
+
+
 def test_side_stream_is_honoured():
     import torch
 
