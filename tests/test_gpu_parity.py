@@ -300,3 +300,39 @@ def test_full_size_configs(number):
     compare(w.mask, w.sampling, res, ref, w.want_dist, w.want_sq, w.want_idx)
     if number == 5:
         assert np.isinf(res["dist"][1]).all() and np.isfinite(res["dist"][0]).all()
+
+
+def _fuzz_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    extents = [1, 2, 3, 4, 5, 7, 8, 12, 16, 20, 31, 32, 33, 48, 64, 100, 128, 129, 200, 256]
+    cases = []
+    while len(cases) < count:
+        ndim = int(rng.integers(1, 9))
+        spatial = tuple(int(rng.choice(extents[: 9 if ndim > 4 else len(extents)])) for _ in range(ndim))
+        bc = (int(rng.integers(1, 4)), int(rng.integers(1, 3)))
+        if np.prod(spatial) * bc[0] * bc[1] > 250_000:
+            continue
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            samp = None
+        elif kind == 1:
+            samp = tuple(float(rng.choice([0.5, 0.8, 1.0, 1.25, 2.0, 2.5])) for _ in range(ndim))
+        else:
+            samp = tuple(float(rng.uniform(0.3, 3.0)) for _ in range(ndim))
+        p_fg = float(rng.choice([0.0, 0.3, 0.8, 0.97, 1.0]))
+        cases.append((bc + spatial, samp, p_fg, int(rng.integers(0, 2**31))))
+    return cases
+
+
+@pytest.mark.parametrize("chunk", range(8))
+def test_random_shapes_samplings_and_outputs(chunk):
+    """Seeded differential fuzzing against the oracle: ranks 1..8, odd and aligned extents, batch and channel
+    counts, unit / decimal / arbitrary sampling, empty and full masks, every output combination."""
+    for shape, samp, p_fg, seed in _fuzz_cases(25, 1000 + chunk):
+        mask = workloads.random_mask(seed, shape, p_fg)
+        if p_fg not in (0.0, 1.0) and mask.shape[0] > 1:
+            mask[-1, -1] = 1  # an image without background inside a normal batch
+        try:
+            full_check(mask, samp)
+        except AssertionError as exc:  # name the case
+            raise AssertionError("shape %r sampling %r p_fg %r seed %r: %s" % (shape, samp, p_fg, seed, exc))
