@@ -52,7 +52,8 @@ extern "C" {
 typedef enum {
     TM_EDT_OK = 0,
     TM_EDT_ERR_INVALID_ARG = 1, /* NULL input/shape, ndim outside 1..8, negative extent, sampling not finite
-                                   and > 0, no output requested, outputs overlapping each other or the input */
+                                   and > 0, no output requested, an output not aligned to its element size,
+                                   outputs overlapping each other or the input */
     TM_EDT_ERR_UNSUPPORTED = 2, /* extent > TM_EDT_MAX_EXTENT, out_sqdist with non-unit sampling, more than
                                    2^40 elements, or more than 2^31 - 1 voxels per image */
     TM_EDT_ERR_BAD_POINTER = 3, /* a device buffer is not device-accessible memory of the current device

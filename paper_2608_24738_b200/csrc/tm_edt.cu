@@ -551,6 +551,7 @@ static int check_call(const uint8_t* input, int ndim, const int64_t* shape, cons
     const int rc = make_plan(ndim, shape, sampling, pl);
     if (rc != TM_EDT_OK) return rc;
     if (!out_dist && !out_sq && !out_idx) return TM_EDT_ERR_INVALID_ARG;
+    if (((uintptr_t)out_dist & 3u) || ((uintptr_t)out_sq & 7u) || ((uintptr_t)out_idx & 7u)) return TM_EDT_ERR_INVALID_ARG;
     if (out_sq && !pl.unit) return TM_EDT_ERR_UNSUPPORTED;
     const size_t N = (size_t)pl.N;
     const size_t bi = N, bd = N * 4, bs = N * 8, bx = N * 8 * (size_t)ndim;

@@ -77,6 +77,14 @@ def test_overlapping_buffers_are_rejected(L):
     assert L.tm_edt(ctypes.c_void_p(0x20000), 2, shp, None, a, b, None, None) == binding.ERR_INVALID_ARG
 
 
+def test_misaligned_outputs_are_rejected(L):
+    shp = (ctypes.c_int64 * 4)(1, 1, 4, 4)
+    inp = ctypes.c_void_p(0x20000)
+    assert L.tm_edt(inp, 2, shp, None, ctypes.c_void_p(0x10002), None, None, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt(inp, 2, shp, None, None, ctypes.c_void_p(0x10004), None, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt(inp, 2, shp, None, None, None, ctypes.c_void_p(0x10004), None) == binding.ERR_INVALID_ARG
+
+
 def test_host_memory_is_not_accepted_as_device_memory(L):
     # Valid arguments, but the buffers are ordinary host arrays: BAD_POINTER (with or without a GPU present).
     m = np.ones((1, 1, 4, 4), dtype=np.uint8)
