@@ -61,7 +61,7 @@ struct Plan {
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
     int si[kMaxDims];         // those integers
     double scale = 1.0;
-    bool wide2d = false;      // two processed axes, unit sampling, extents <= 512, contiguous extent % 16 == 0
+    bool wide2d = false;      // two processed axes, unit sampling, extents <= 1024, contiguous extent % 16 == 0
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
 };
@@ -133,7 +133,7 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
     const char* force = getenv("TM_EDT_FORCE_GENERIC");
     pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
-    pl.wide2d = !pl.fast && E == 2 && pl.unit && nmax <= 512 && pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
+    pl.wide2d = !pl.fast && E == 2 && pl.unit && nmax <= 1024 && pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
     if (pl.wide2d) pl.ws_bytes = (((size_t)pl.N * 4 + 255) & ~(size_t)255) + (((size_t)pl.N * 2 + 255) & ~(size_t)255);
     if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
         // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
@@ -475,19 +475,25 @@ static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueP
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     const double out_bpv = out_bytes_per_voxel(ep);
+    // keys carry 9 row bits up to extent 512 and 10 up to 1024; a lane of the row kernel takes 16 or 32 voxels
+    const bool big = pl.ext[0] > 512 || pl.ext[1] > 512;
     prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + 2.0));
-    row_keys_kernel<<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
+    if (!big) row_keys_kernel<16, 9><<<row_blocks, 256, 0, st>>>(P);
+    else if (pl.ext[0] <= 512) row_keys_kernel<16, 10><<<row_blocks, 256, 0, st>>>(P);
+    else row_keys_kernel<32, 10><<<row_blocks, 256, 0, st>>>(P);
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int strips = (pl.ext[0] + 31) / 32;
     const size_t smem = (size_t)pl.ext[1] * 32 * 4;
+    auto kern = big ? wide_column_kernel<10> : wide_column_kernel<9>;
     if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(wide_column_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     prof_mark(st, "wide_column_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
-    wide_column_kernel<<<(unsigned)(pl.images * strips), 256, smem, st>>>(P, ep, strips);
+    kern<<<(unsigned)(pl.images * strips), pl.ext[1] > 512 ? 512 : 256, smem, st>>>(P, ep, strips);
     ++launches;
     return cudaGetLastError();
 }

@@ -66,6 +66,7 @@ SMALL = [
     (1, 1, 128, 128), (2, 1, 127, 128), (1, 1, 128, 100), (1, 2, 50, 128, 64), (1, 1, 128, 20, 48),
     (1, 1, 16, 40, 24, 32), (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128),
     (2, 1, 200, 256), (1, 1, 129, 144), (1, 1, 300, 16), (1, 2, 512, 48), (1, 1, 1, 40, 1, 160),
+    (1, 1, 1024, 48), (1, 1, 40, 1024), (2, 1, 600, 528), (1, 1, 513, 1008),
 ]
 
 
@@ -129,7 +130,7 @@ def test_half_space_and_far_sites(path):
     full_check(mask, (2.5, 0.8, 1.0))
 
 
-@pytest.mark.parametrize("n", [512, 513, 1100, 2048])
+@pytest.mark.parametrize("n", [512, 513, 1024, 1100, 2048])
 def test_long_lines(n):
     """Extents above 128 use 16-bit offsets; unit sampling beyond 512 switches the envelope to float64."""
     mask = workloads.random_mask(n, (1, 1, 24, n), 0.97)
