@@ -203,13 +203,17 @@ def run_reference(args, w, world, rank):
 
 
 def load_traffic(workload_number: int, kernel_label: str):
-    """DRAM bytes per launch of a kernel from the committed ncu summary (profiles/traffic.json), or None."""
+    """DRAM bytes per launch of a kernel from the committed ncu summary (profiles/traffic.txt), or None."""
     try:
-        with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
-            table = json.load(fh)
-        return table.get("C%d" % workload_number, {}).get(kernel_label.split(":", 1)[1])
+        want = ("C%d" % workload_number, kernel_label.split(":", 1)[1])
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as fh:
+            for line in fh:
+                parts = line.split()
+                if len(parts) == 3 and (parts[0], parts[1]) == want:
+                    return int(parts[2])
     except Exception:
-        return None
+        pass
+    return None
 
 
 def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
