@@ -98,7 +98,8 @@ TM_EDT_API size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape);
 /*
  * Same transform with caller-provided scratch: `workspace` is device memory of at least
  * tm_edt_workspace_bytes(ndim, shape) bytes, 256-byte aligned, private to this call until the
- * enqueued work has run.  Allocates nothing.  A too-small workspace gives TM_EDT_ERR_ALLOC.
+ * enqueued work has run.  Allocates nothing and only enqueues kernels, so the call can be captured into a
+ * CUDA graph and replayed.  A too-small workspace gives TM_EDT_ERR_ALLOC.
  */
 TM_EDT_API int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
               int64_t* out_sqdist, int64_t* out_indices, void* workspace, size_t workspace_bytes,

@@ -244,6 +244,33 @@ def test_pooled_scratch_and_trim():
     binding.tm_edt_trim_memory()
 
 
+def test_workspace_call_inside_a_cuda_graph():
+    """tm_edt_ws only enqueues kernels (no allocation, no synchronisation), so it can be captured into a
+    CUDA graph and replayed on new data in the same buffers."""
+    import torch
+
+    shape = (2, 1, 24, 40, 64)
+    first = workloads.random_mask(61, shape, 0.85)
+    second = workloads.random_mask(62, shape, 0.6)
+    t = torch.from_numpy(first).cuda()
+    ws = torch.empty(binding.tm_edt_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    d = torch.empty(shape, dtype=torch.float32, device="cuda")
+    x = torch.empty(shape[:2] + (3,) + shape[2:], dtype=torch.int64, device="cuda")
+    binding.tm_edt(t, None, distances=d, indices=x, workspace=ws)  # warm-up outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        binding.tm_edt(t, None, distances=d, indices=x, workspace=ws, stream=torch.cuda.current_stream())
+    for mask in (first, second):
+        t.copy_(torch.from_numpy(mask))
+        d.fill_(-1.0)
+        g.replay()
+        torch.cuda.synchronize()
+        ref = oracle.sep(mask, None, want_idx=False)
+        checker.check_dist(d.cpu().numpy(), ref["dist"])
+        checker.check_indices(x.cpu().numpy(), mask, ref, None)
+
+
 def test_side_stream_is_honoured():
     import torch
 
