@@ -225,14 +225,33 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
 #pragma unroll
     for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
     if (mx < (1u << SH)) return;  // a group of background voxels
-    uint32_t a[R];                // a[i] = (d + i)^2 << SH
-#pragma unroll
-    for (int i = 0; i < R; ++i) a[i] = (wk * (uint32_t)((1 + i) * (1 + i))) << SH;
-    const uint32_t* plo = col + (y0 - 1) * VS;
-    const uint32_t* phi = col + (y0 + R) * VS;
+    const int dsafe = min(y0, n - R - y0);  // steps for which both outer rows exist
     int d = 1;
+    // The first W steps as straight-line code with constant addends, no stop tests and no loop state: most
+    // groups of real masks are finished by then (trying a few rows too many does not change the minimum).
+    constexpr int W = 4;
+    if (dsafe >= W) {
+#pragma unroll
+        for (int s = 1; s <= W; ++s) {
+            const uint32_t vlo = col[(y0 - s) * VS], vhi = col[(y0 + R - 1 + s) * VS];
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                best[i] = __viaddmin_u32(vlo, (wk * (uint32_t)((s + i) * (s + i))) << SH, best[i]);
+                best[i] = __viaddmin_u32(vhi, (wk * (uint32_t)((s + R - 1 - i) * (s + R - 1 - i))) << SH, best[i]);
+            }
+        }
+        d = W + 1;
+        mx = best[0];
+#pragma unroll
+        for (int i = 1; i < R; ++i) mx = max(mx, best[i]);
+        if ((wk * (uint32_t)(d * d)) << SH >= mx) return;
+    }
+    uint32_t a[R];  // a[i] = (d + i)^2 << SH
+#pragma unroll
+    for (int i = 0; i < R; ++i) a[i] = (wk * (uint32_t)((d + i) * (d + i))) << SH;
+    const uint32_t* plo = col + (y0 - d) * VS;
+    const uint32_t* phi = col + (y0 + R - 1 + d) * VS;
     // interior steps, two at a time: both rows exist on both sides, no bounds tests, one stop test per pair
-    const int dsafe = min(y0, n - R - y0);
     for (; d + 1 <= dsafe && a[0] < mx; d += 2, plo -= 2 * VS, phi += 2 * VS) {
         const uint32_t vlo0 = plo[0], vhi0 = phi[0], vlo1 = plo[-VS], vhi1 = phi[VS];
         const uint32_t aR = (wk * (uint32_t)((d + R) * (d + R))) << SH;  // addend of distance d + R
