@@ -1,0 +1,197 @@
+// Unit sampling with extents beyond the 128 of the packed 8-bit entries: two processed axes with extents up
+// to 1024, three with extents up to 512.  Kernels:
+//   row_keys_kernel     first-axis pass, one warp per row, 16 or 32 voxels per lane (128-bit loads).
+//                       Writes, per voxel, the scan key  (off^2 << SH) | row  (32 bit; SH = 9 row bits for
+//                       extents up to 512, 10 up to 1024: 2 * 1023^2 << 10 still stays below 2^31) and the
+//                       signed 16-bit offset to the nearest zero of the row.
+//   wide_axis_kernel    every further axis: a block stages the keys of an (n x 32) strip in shared memory and
+//                       runs the grouped bounded scan on it (edt_fast.cuh).  A middle pass writes the key of
+//                       the next pass and the site's offsets (16 bits per axis); the last pass writes the
+//                       outputs and fetches the chosen site's offsets only when indices are requested.
+// Same mathematics as the fast path: g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (x_k - j)^2 ], exact in
+// integers: values stay below 3 * 511^2 < 2^20 (three axes, 9 row bits) or 2 * 1023^2 < 2^21 (two axes, 10).
+#pragma once
+#include "edt_fast.cuh"
+
+namespace tmedt {
+
+
+struct WideParams {
+    const uint8_t* in;   // (images, n1, n0)
+    uint32_t* keys;      // (images, n1, n0)
+    int16_t* offs;       // (images, n1, n0)
+    int64_t rows;        // images * n1
+    int n0, n1;
+};
+
+template <int VPL, int SH>  // voxels per lane (16 or 32), row bits of the key
+__global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ WideParams P) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= P.rows) return;  // the whole warp leaves together
+    const int n0 = P.n0;
+    const int y = (int)(row % P.n1);
+    const uint8_t* src = P.in + row * n0;
+    constexpr int CH = VPL / 16;  // 16-byte chunks per lane
+    uint32_t zb = 0u;             // bit b set: voxel b of this lane is zero
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+        uint4 v = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+        if (VPL * lane + 16 * c < n0) v = *reinterpret_cast<const uint4*>(src + VPL * lane + 16 * c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t m = ~(((w[i] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w[i]) & 0x80808080u;
+            // gather the four flag bits (bits 7, 15, 23, 31) into bits 0..3
+            zb |= ((((m >> 7) * 0x00204081u) >> 21) & 0xfu) << (16 * c + 4 * i);
+        }
+    }
+    const unsigned any = __ballot_sync(0xffffffffu, zb != 0u);
+    uint32_t keys[VPL];
+    int16_t offs[VPL];
+    if (any == 0u) {
+#pragma unroll
+        for (int b = 0; b < VPL; ++b) { keys[b] = kNoneKey16; offs[b] = (int16_t)-32768; }
+    } else {
+        const int lzin = zb ? 31 - __clz(zb) : 0;
+        const int fzin = zb ? __ffs(zb) - 1 : 0;
+        const unsigned ml = any & ((1u << lane) - 1u);
+        const unsigned mr = lane < 31 ? any >> (lane + 1) : 0u;
+        const int Ll = ml ? 31 - __clz(ml) : 0;
+        const int Lr = mr ? lane + __ffs(mr) : 0;
+        const int lz_l = __shfl_sync(0xffffffffu, lzin, Ll);
+        const int fz_r = __shfl_sync(0xffffffffu, fzin, Lr);
+        const int x0 = VPL * lane;
+        int dl[VPL];
+        int cur = ml ? VPL * Ll + lz_l : -4096;
+#pragma unroll
+        for (int b = 0; b < VPL; ++b) {
+            if ((zb >> b) & 1u) cur = x0 + b;
+            dl[b] = x0 + b - cur;
+        }
+        cur = mr ? VPL * Lr + fz_r : 8192;
+#pragma unroll
+        for (int b = VPL - 1; b >= 0; --b) {
+            if ((zb >> b) & 1u) cur = x0 + b;
+            const int dr = cur - (x0 + b);
+            const int a = min(dl[b], dr);
+            offs[b] = (int16_t)(dl[b] <= dr ? -a : a);
+            keys[b] = ((uint32_t)(a * a) << SH) | (uint32_t)y;
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+        if (VPL * lane + 16 * c < n0) {
+            uint4* kdst = reinterpret_cast<uint4*>(P.keys + row * n0 + VPL * lane + 16 * c);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                kdst[i] = make_uint4(keys[16 * c + 4 * i], keys[16 * c + 4 * i + 1], keys[16 * c + 4 * i + 2],
+                                     keys[16 * c + 4 * i + 3]);
+            uint32_t pk[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                pk[i] = (uint32_t)(uint16_t)offs[16 * c + 2 * i] | ((uint32_t)(uint16_t)offs[16 * c + 2 * i + 1] << 16);
+            uint4* odst = reinterpret_cast<uint4*>(P.offs + row * n0 + VPL * lane + 16 * c);
+            odst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            odst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        }
+    }
+}
+
+// One further axis of the wide path.  The array is viewed as (outer, n, inner); a block takes one slab and
+// a strip of 32 consecutive `inner` positions, stages the keys of its n rows in shared memory and runs the
+// grouped bounded scan.  K = number of 16-bit offsets every voxel carries so far (1 or 2).
+//   FINAL == false  writes the key of the next pass (value << SH | index of the slab along the next axis)
+//                   and K + 1 offsets per voxel (the chosen site's offsets, fetched from global memory, plus
+//                   the offset along this axis);
+//   FINAL == true   writes distances, squared distances and index planes (the slab is the image).
+struct WideAxisParams {
+    const uint32_t* keys_in;   // (outer, n, inner)
+    const int16_t* offs_in;    // (outer, n, inner, K)
+    uint32_t* keys_out;        // (outer, n, inner), unused when FINAL
+    int16_t* offs_out;         // (outer, n, inner, K + 1), unused when FINAL
+    int64_t outer, inner;
+    int n;
+    int next_n;                // extent of the next axis (non-final)
+    int n0;                    // extent of the contiguous axis (to split an inner position into coordinates)
+};
+
+template <int K, bool FINAL, int SH>
+__global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ WideAxisParams P,
+                                                        const __grid_constant__ EpilogueParams ep,
+                                                        const int strips_per_slab) {
+    extern __shared__ __align__(16) uint8_t sm_wide[];
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_wide);  // [n][32]
+    const int n = P.n;
+    const int64_t slab = blockIdx.x / strips_per_slab;
+    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
+    const int64_t slab_base = slab * (int64_t)n * P.inner;
+    const uint32_t* src = P.keys_in + slab_base + c0;
+    // stage: 8 threads copy one row of 32 keys (inner is a multiple of 16, so a strip is 16 or 32 positions wide)
+    const int width = (int)min((int64_t)32, P.inner - c0);
+    for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
+        const int y = t >> 3, ch = t & 7;
+        if (4 * ch < width)
+            *reinterpret_cast<uint4*>(val + y * 32 + 4 * ch) = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + 4 * ch);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if (lane >= width) return;
+    const int64_t c = c0 + lane;  // position along inner
+    constexpr int R = 4;
+    constexpr uint32_t kRowMask = (1u << SH) - 1u;
+    const int64_t col_base = slab_base + c;  // voxel (row 0) of this column
+    const uint32_t next_row = FINAL ? 0u : (uint32_t)(slab % P.next_n);
+    // own coordinates along the earlier axes (final pass, index output): plane 0 = contiguous axis
+    const int cx = (int)(c % P.n0), cy = (int)(c / P.n0);
+    for (int y0 = warp * R; y0 < n; y0 += nwarps * R) {
+        uint32_t best[R];
+        scan_keys_group<32, R, SH>(val + lane, n, y0, best);
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const int y = y0 + i;
+            if (y >= n) break;
+            const uint32_t b = best[i];
+            const bool none = b >= kNoneKey16;
+            const int j = (int)(b & kRowMask);
+            const int64_t p = col_base + (int64_t)y * P.inner;    // this voxel
+            const int64_t pj = col_base + (int64_t)j * P.inner;   // the chosen site's voxel of this column
+            if (!FINAL) {
+                P.keys_out[p] = none ? kNoneKey16 : ((b & ~kRowMask) | next_row);
+                if (K == 1) {
+                    const uint32_t o0 = none ? 0x8000u : (uint32_t)(uint16_t)P.offs_in[pj];
+                    reinterpret_cast<uint32_t*>(P.offs_out)[p] = o0 | ((uint32_t)(uint16_t)(int16_t)(j - y) << 16);
+                }
+            } else {
+                const int sq = (int)(b >> SH);
+                if (ep.dist) ep.dist[p] = none ? TMEDT_INF : __fsqrt_rn(small_int_to_float(sq));
+                if (ep.sq) ep.sq[p] = none ? INT64_MAX : (int64_t)sq;
+                if (ep.idx) {
+                    // processed axes in plane order: contiguous axis, (second axis,) this axis; others have extent 1
+                    int site[3] = {0, 0, 0};
+                    if (!none) {
+                        if (K == 1) {
+                            site[0] = cx + (int)P.offs_in[pj];
+                            site[1] = j;
+                        } else {
+                            const uint32_t o = reinterpret_cast<const uint32_t*>(P.offs_in)[pj];
+                            site[0] = cx + (int)(int16_t)(o & 0xffffu);
+                            site[1] = cy + (int)(int16_t)(o >> 16);
+                            site[2] = j;
+                        }
+                    }
+                    const int64_t vox = p - slab_base;  // voxel index inside the image
+                    for (int a = 0; a < ep.ndim; ++a) {
+                        int64_t v = 0;
+#pragma unroll
+                        for (int q = 0; q <= K; ++q)
+                            if (a == ep.axis[q]) v = site[q];
+                        ep.idx[(slab * ep.ndim + a) * ep.V + vox] = none ? -1 : v;
+                    }
+                }
+            }
+        }
+    }
+}
+
+}  // namespace tmedt

@@ -13,7 +13,7 @@
 #include "edt_common.cuh"
 #include "edt_generic.cuh"
 #include "edt_fast.cuh"
-#include "edt_wide2d.cuh"
+#include "edt_wide.cuh"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -61,7 +61,7 @@ struct Plan {
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
     int si[kMaxDims];         // those integers
     double scale = 1.0;
-    bool wide2d = false;      // two processed axes, unit sampling, extents <= 1024, contiguous extent % 16 == 0
+    bool wide_keys = false;      // unit sampling, contiguous extent % 16 == 0: two axes <= 1024 or three axes <= 512
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
 };
@@ -133,8 +133,13 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
     const char* force = getenv("TM_EDT_FORCE_GENERIC");
     pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
-    pl.wide2d = !pl.fast && E == 2 && pl.unit && nmax <= 1024 && pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
-    if (pl.wide2d) pl.ws_bytes = (((size_t)pl.N * 4 + 255) & ~(size_t)255) + (((size_t)pl.N * 2 + 255) & ~(size_t)255);
+    pl.wide_keys = !pl.fast && pl.unit && ((E == 2 && nmax <= 1024) || (E == 3 && nmax <= 512)) && pl.ext[0] % 16 == 0 &&
+                !(force && force[0] == '1');
+    if (pl.wide_keys) {
+        auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+        pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
+        if (E == 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
+    }
     if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
         // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
         // the largest possible value below 2^24 (keys are value << 7 | row in 32 bits)
@@ -465,13 +470,30 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
     return cudaSuccess;
 }
 
-// Two-dimensional unit-sampling images with extents up to 512: key rows, then column strips.
-static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+// Unit sampling beyond extent 128 (two axes up to 1024, three up to 512): key rows, then strip scans.
+template <int K, bool FINAL>
+static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, bool ten_bits, cudaStream_t st) {
+    const int strips = (int)((A.inner + 31) / 32);
+    const size_t smem = (size_t)A.n * 32 * 4;
+    auto kern = ten_bits ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<(unsigned)(A.outer * strips), A.n > 512 ? 512 : 256, smem, st>>>(A, ep, strips);
+    return cudaGetLastError();
+}
+
+static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
                               int& launches) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    char* w = static_cast<char*>(ws);
+    uint32_t* keysA = reinterpret_cast<uint32_t*>(w);
+    int16_t* offsA = reinterpret_cast<int16_t*>(w + up((size_t)pl.N * 4));
+    uint32_t* keysB = reinterpret_cast<uint32_t*>(w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
+    int16_t* offsB = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
     WideParams P;
-    P.in = in;
-    P.keys = static_cast<uint32_t*>(ws);
-    P.offs = reinterpret_cast<int16_t*>(static_cast<char*>(ws) + (((size_t)pl.N * 4 + 255) & ~(size_t)255));
+    P.in = in; P.keys = keysA; P.offs = offsA;
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     const double out_bpv = out_bytes_per_voxel(ep);
@@ -485,17 +507,28 @@ static cudaError_t run_wide2d(const Plan& pl, const uint8_t* in, const EpilogueP
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int strips = (pl.ext[0] + 31) / 32;
-    const size_t smem = (size_t)pl.ext[1] * 32 * 4;
-    auto kern = big ? wide_column_kernel<10> : wide_column_kernel<9>;
-    if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
+    WideAxisParams A;
+    memset(&A, 0, sizeof(A));
+    A.keys_in = keysA; A.offs_in = offsA; A.keys_out = keysB; A.offs_out = offsB;
+    A.n = pl.ext[1]; A.inner = pl.inner[1]; A.outer = pl.N / ((int64_t)pl.ext[1] * pl.inner[1]);
+    A.n0 = pl.ext[0];
+    if (pl.E == 2) {
+        prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
+        e = launch_wide_axis<1, true>(A, ep, big, st);
+        ++launches;
+        return e;
     }
-    prof_mark(st, "wide_column_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
-    kern<<<(unsigned)(pl.images * strips), pl.ext[1] > 512 ? 512 : 256, smem, st>>>(P, ep, strips);
+    A.next_n = pl.ext[2];
+    prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 2.0 + 4.0 + 4.0));
+    e = launch_wide_axis<1, false>(A, ep, false, st);
     ++launches;
-    return cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    A.keys_in = keysB; A.offs_in = offsB; A.keys_out = nullptr; A.offs_out = nullptr;
+    A.n = pl.ext[2]; A.inner = pl.inner[2]; A.outer = pl.N / ((int64_t)pl.ext[2] * pl.inner[2]);
+    prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 4.0 : 0.0)));
+    e = launch_wide_axis<2, true>(A, ep, false, st);
+    ++launches;
+    return e;
 }
 
 // Stream-ordered scratch of tm_edt and tm_edt_host comes from a memory pool of the library's own, one per
@@ -571,7 +604,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
                               void* ws, cudaStream_t st, int& launches) {
     EpilogueParams ep;
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
-    if (pl.wide2d && ((uintptr_t)input & 15u) == 0) return run_wide2d(pl, input, ep, ws, st, launches);
+    if (pl.wide_keys && ((uintptr_t)input & 15u) == 0) return run_wide(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
         return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);

@@ -100,7 +100,8 @@ def test_workspace_bytes(L):
     assert binding.tm_edt_workspace_bytes((2, 3, 64, 64)) == 0  # first two axes are fused in one kernel
     assert binding.tm_edt_workspace_bytes((2, 3, 64, 64, 64)) >= 2 * (2 * 3 * 64 ** 3)  # 2-byte entries
     assert binding.tm_edt_workspace_bytes((1, 1, 300, 300)) >= 2 * 300 * 300  # generic path: 16-bit offset planes
-    assert binding.tm_edt_workspace_bytes((1, 1, 1024, 1024)) == 6 * 1024 * 1024  # wide 2-D path: key + offset
+    assert binding.tm_edt_workspace_bytes((1, 1, 1024, 1024)) == 6 * 1024 * 1024  # wide path, two axes: key + offset
+    assert binding.tm_edt_workspace_bytes((1, 1, 256, 256, 256)) == 14 * 256 ** 3  # three axes: 2 keys + 1 + 2 offsets
     with pytest.raises(binding.TmEdtError):
         binding.tm_edt_workspace_bytes((1, 1, binding.MAX_EXTENT + 1))
 

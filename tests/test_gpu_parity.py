@@ -67,6 +67,7 @@ SMALL = [
     (1, 1, 16, 40, 24, 32), (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128),
     (2, 1, 200, 256), (1, 1, 129, 144), (1, 1, 300, 16), (1, 2, 512, 48), (1, 1, 1, 40, 1, 160),
     (1, 1, 1024, 48), (1, 1, 40, 1024), (2, 1, 600, 528), (1, 1, 513, 1008),
+    (1, 1, 130, 48, 160), (1, 2, 20, 200, 64), (2, 1, 512, 6, 16), (1, 1, 9, 16, 512), (1, 1, 140, 1, 33, 1, 48),
 ]
 
 
