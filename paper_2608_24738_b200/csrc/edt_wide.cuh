@@ -22,8 +22,10 @@ struct WideParams {
     int16_t* offs;       // (images, n1, n0)
     int64_t rows;        // images * n1
     int n0, n1;
+    float w2x;           // squared sampling of the contiguous axis (float-height variant)
 };
 
+// SH >= 0: integer keys (off^2 << SH | row).  SH < 0: float32 heights w^2 off^2 for general sampling (+inf = no site).
 template <int VPL, int SH>  // voxels per lane (16 or 32), row bits of the key
 __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ WideParams P) {
     const int lane = threadIdx.x & 31;
@@ -51,7 +53,7 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
     int16_t offs[VPL];
     if (any == 0u) {
 #pragma unroll
-        for (int b = 0; b < VPL; ++b) { keys[b] = kNoneKey16; offs[b] = (int16_t)-32768; }
+        for (int b = 0; b < VPL; ++b) { keys[b] = SH < 0 ? 0x7f800000u : kNoneKey16; offs[b] = (int16_t)-32768; }
     } else {
         const int lzin = zb ? 31 - __clz(zb) : 0;
         const int fzin = zb ? __ffs(zb) - 1 : 0;
@@ -76,7 +78,7 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
             const int dr = cur - (x0 + b);
             const int a = min(dl[b], dr);
             offs[b] = (int16_t)(dl[b] <= dr ? -a : a);
-            keys[b] = ((uint32_t)(a * a) << SH) | (uint32_t)y;
+            keys[b] = SH < 0 ? __float_as_uint(P.w2x * (float)(a * a)) : (((uint32_t)(a * a) << (SH < 0 ? 0 : SH)) | (uint32_t)y);
         }
     }
 #pragma unroll
@@ -114,7 +116,27 @@ struct WideAxisParams {
     int n;
     int next_n;                // extent of the next axis (non-final)
     int n0;                    // extent of the contiguous axis (to split an inner position into coordinates)
+    float w2;                  // squared sampling of this axis (float-height variant)
 };
+
+// Bounded scan of one voxel on float32 heights (general sampling): returns the best value and the distance bd
+// (0 = own row) at which it was found; the caller resolves the side.
+template <int VS>
+__device__ __forceinline__ float scan_heights_plain(const uint32_t* __restrict__ col, int n, int y, float w2, int& bd) {
+    float best = __uint_as_float(col[y * VS]);
+    bd = 0;
+    float fd = 1.0f;
+    for (int d = 1; d < n; ++d, fd += 1.0f) {
+        const float add = w2 * fd * fd;
+        if (add >= best) break;
+        if (y - d < 0 && y + d >= n) break;
+        const float lo = y - d >= 0 ? __uint_as_float(col[(y - d) * VS]) : TMEDT_INF;
+        const float hi = y + d < n ? __uint_as_float(col[(y + d) * VS]) : TMEDT_INF;
+        const float c = fminf(lo, hi) + add;
+        if (c < best) { best = c; bd = d; }
+    }
+    return best;
+}
 
 template <int K, bool FINAL, int SH>
 __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ WideAxisParams P,
@@ -139,33 +161,55 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     if (lane >= width) return;
     const int64_t c = c0 + lane;  // position along inner
     constexpr int R = 4;
-    constexpr uint32_t kRowMask = (1u << SH) - 1u;
+    constexpr uint32_t kRowMask = SH < 0 ? 0u : (1u << (SH < 0 ? 0 : SH)) - 1u;
     const int64_t col_base = slab_base + c;  // voxel (row 0) of this column
     const uint32_t next_row = FINAL ? 0u : (uint32_t)(slab % P.next_n);
     // own coordinates along the earlier axes (final pass, index output): plane 0 = contiguous axis
     const int cx = (int)(c % P.n0), cy = (int)(c / P.n0);
     for (int y0 = warp * R; y0 < n; y0 += nwarps * R) {
         uint32_t best[R];
-        scan_keys_group<32, R, SH>(val + lane, n, y0, best);
+        int jrow[R];
+        if (SH >= 0) {
+            scan_keys_group<32, R, (SH < 0 ? 9 : SH)>(val + lane, n, y0, best);
+#pragma unroll
+            for (int i = 0; i < R; ++i) jrow[i] = (int)(best[i] & kRowMask);
+        } else {
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int y = y0 + i;
+                best[i] = 0u; jrow[i] = y;
+                if (y >= n) continue;
+                int bd;
+                best[i] = __float_as_uint(scan_heights_plain<32>(val + lane, n, y, P.w2, bd));
+                if (bd > 0) {
+                    const float lo = y - bd >= 0 ? __uint_as_float(val[(y - bd) * 32 + lane]) : TMEDT_INF;
+                    const float hi = y + bd < n ? __uint_as_float(val[(y + bd) * 32 + lane]) : TMEDT_INF;
+                    jrow[i] = lo <= hi ? y - bd : y + bd;
+                }
+            }
+        }
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             const int y = y0 + i;
             if (y >= n) break;
             const uint32_t b = best[i];
-            const bool none = b >= kNoneKey16;
-            const int j = (int)(b & kRowMask);
+            const bool none = SH < 0 ? b == 0x7f800000u : b >= kNoneKey16;
+            const int j = jrow[i];
             const int64_t p = col_base + (int64_t)y * P.inner;    // this voxel
             const int64_t pj = col_base + (int64_t)j * P.inner;   // the chosen site's voxel of this column
             if (!FINAL) {
-                P.keys_out[p] = none ? kNoneKey16 : ((b & ~kRowMask) | next_row);
+                if (SH < 0) P.keys_out[p] = b;  // the height itself is the next pass's scan value
+                else P.keys_out[p] = none ? kNoneKey16 : ((b & ~kRowMask) | next_row);
                 if (K == 1) {
                     const uint32_t o0 = none ? 0x8000u : (uint32_t)(uint16_t)P.offs_in[pj];
                     reinterpret_cast<uint32_t*>(P.offs_out)[p] = o0 | ((uint32_t)(uint16_t)(int16_t)(j - y) << 16);
                 }
             } else {
-                const int sq = (int)(b >> SH);
-                if (ep.dist) ep.dist[p] = none ? TMEDT_INF : __fsqrt_rn(small_int_to_float(sq));
-                if (ep.sq) ep.sq[p] = none ? INT64_MAX : (int64_t)sq;
+                const int sq = SH < 0 ? 0 : (int)(b >> (SH < 0 ? 0 : SH));
+                if (ep.dist)
+                    ep.dist[p] = none ? TMEDT_INF
+                                      : (SH < 0 ? __fsqrt_rn(__uint_as_float(b)) : __fsqrt_rn(small_int_to_float(sq)));
+                if (ep.sq) ep.sq[p] = none ? INT64_MAX : (int64_t)sq;  // unit sampling only
                 if (ep.idx) {
                     // processed axes in plane order: contiguous axis, (second axis,) this axis; others have extent 1
                     int site[3] = {0, 0, 0};

@@ -133,8 +133,9 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
     const char* force = getenv("TM_EDT_FORCE_GENERIC");
     pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
-    pl.wide_keys = !pl.fast && pl.unit && ((E == 2 && nmax <= 1024) || (E == 3 && nmax <= 512)) && pl.ext[0] % 16 == 0 &&
-                !(force && force[0] == '1');
+    // unit sampling: integer keys (two axes up to extent 1024, three up to 512); other sampling: float heights
+    pl.wide_keys = !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || E == 2 || nmax <= 512) &&
+                   pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
     if (pl.wide_keys) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
         pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
@@ -471,11 +472,12 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
 }
 
 // Unit sampling beyond extent 128 (two axes up to 1024, three up to 512): key rows, then strip scans.
+// sh: row bits of the integer keys (9 or 10), or -1 for float heights
 template <int K, bool FINAL>
-static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, bool ten_bits, cudaStream_t st) {
+static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, int sh, cudaStream_t st) {
     const int strips = (int)((A.inner + 31) / 32);
     const size_t smem = (size_t)A.n * 32 * 4;
-    auto kern = ten_bits ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>;
+    auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1> : (sh == 10 ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -496,14 +498,23 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     P.in = in; P.keys = keysA; P.offs = offsA;
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
+    P.w2x = (float)(pl.w[0] * pl.w[0]);
     const double out_bpv = out_bytes_per_voxel(ep);
-    // keys carry 9 row bits up to extent 512 and 10 up to 1024; a lane of the row kernel takes 16 or 32 voxels
-    const bool big = pl.ext[0] > 512 || pl.ext[1] > 512;
+    // integer keys carry 9 row bits up to extent 512 and 10 up to 1024 (two axes only); general sampling uses float
+    // heights.  A lane of the row kernel takes 16 voxels (rows up to 512) or 32.
+    int nmax = 1;
+    for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
+    const int sh = !pl.unit ? -1 : (nmax > 512 ? 10 : 9);
     prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + 2.0));
     const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
-    if (!big) row_keys_kernel<16, 9><<<row_blocks, 256, 0, st>>>(P);
-    else if (pl.ext[0] <= 512) row_keys_kernel<16, 10><<<row_blocks, 256, 0, st>>>(P);
-    else row_keys_kernel<32, 10><<<row_blocks, 256, 0, st>>>(P);
+    if (pl.ext[0] <= 512) {
+        if (sh < 0) row_keys_kernel<16, -1><<<row_blocks, 256, 0, st>>>(P);
+        else if (sh == 9) row_keys_kernel<16, 9><<<row_blocks, 256, 0, st>>>(P);
+        else row_keys_kernel<16, 10><<<row_blocks, 256, 0, st>>>(P);
+    } else {
+        if (sh < 0) row_keys_kernel<32, -1><<<row_blocks, 256, 0, st>>>(P);
+        else row_keys_kernel<32, 10><<<row_blocks, 256, 0, st>>>(P);
+    }
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -512,21 +523,23 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     A.keys_in = keysA; A.offs_in = offsA; A.keys_out = keysB; A.offs_out = offsB;
     A.n = pl.ext[1]; A.inner = pl.inner[1]; A.outer = pl.N / ((int64_t)pl.ext[1] * pl.inner[1]);
     A.n0 = pl.ext[0];
+    A.w2 = (float)(pl.w[1] * pl.w[1]);
     if (pl.E == 2) {
         prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
-        e = launch_wide_axis<1, true>(A, ep, big, st);
+        e = launch_wide_axis<1, true>(A, ep, sh, st);
         ++launches;
         return e;
     }
     A.next_n = pl.ext[2];
     prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 2.0 + 4.0 + 4.0));
-    e = launch_wide_axis<1, false>(A, ep, false, st);
+    e = launch_wide_axis<1, false>(A, ep, sh, st);
     ++launches;
     if (e != cudaSuccess) return e;
     A.keys_in = keysB; A.offs_in = offsB; A.keys_out = nullptr; A.offs_out = nullptr;
     A.n = pl.ext[2]; A.inner = pl.inner[2]; A.outer = pl.N / ((int64_t)pl.ext[2] * pl.inner[2]);
+    A.w2 = (float)(pl.w[2] * pl.w[2]);
     prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 4.0 : 0.0)));
-    e = launch_wide_axis<2, true>(A, ep, false, st);
+    e = launch_wide_axis<2, true>(A, ep, sh, st);
     ++launches;
     return e;
 }
