@@ -14,6 +14,7 @@
 #include "edt_generic.cuh"
 #include "edt_fast.cuh"
 #include "edt_wide.cuh"
+#include "edt_small.cuh"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -58,6 +59,7 @@ struct Plan {
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
     bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    bool small = false;       // every extent <= 8: register-resident lines, value (+ site index) carry
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
     int si[kMaxDims];         // those integers
     double scale = 1.0;
@@ -132,7 +134,8 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.plane_bytes = (((size_t)pl.N * elem) + 255) & ~(size_t)255;
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
     const char* force = getenv("TM_EDT_FORCE_GENERIC");
-    pl.fast = nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
+    pl.small = nmax <= 8 && !(force && force[0] == '1');
+    pl.fast = !pl.small && nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
     // unit sampling: integer keys (two axes up to extent 1024, three up to 512); other sampling: float heights
     pl.wide_keys = !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || E == 2 || nmax <= 512) &&
                    pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
@@ -141,6 +144,7 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
         pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
         if (E == 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
     }
+    if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
     if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
         // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
         // the largest possible value below 2^24 (keys are value << 7 | row in 32 bits)
@@ -471,6 +475,71 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
     return cudaSuccess;
 }
 
+// Every extent <= 8: consecutive axes grouped while the product of their extents stays <= 256, one kernel
+// per group, squared distances (and site indices) carried between kernels as plain arrays.
+template <bool SITE>
+static cudaError_t run_small(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                             int& launches) {
+    const size_t buf = (((size_t)pl.N * 4) + 255) & ~(size_t)255;
+    char* w = static_cast<char*>(ws);
+    float* val[2] = {reinterpret_cast<float*>(w), reinterpret_cast<float*>(w + buf)};
+    int32_t* site[2] = {reinterpret_cast<int32_t*>(w + 2 * buf), reinterpret_cast<int32_t*>(w + 3 * buf)};
+    const double out_bpv = out_bytes_per_voxel(ep);
+    int g = 0;
+    for (int k = 0; k < pl.E; ++g) {
+        SmallParams P;
+        memset(&P, 0, sizeof(P));
+        P.prod = 1;
+        const int k0 = k;
+        while (k < pl.E && (k == k0 || P.prod * pl.ext[k] <= kSmallProd)) {
+            P.n[P.m] = pl.ext[k];
+            P.w2[P.m] = (float)(pl.w[k] * pl.w[k]);
+            P.prod *= pl.ext[k];
+            ++P.m; ++k;
+        }
+        const bool first = k0 == 0, fin = k == pl.E;
+        const size_t smem = (size_t)P.prod * kSmallT * (SITE ? 8 : 4);
+        P.mask = in;
+        P.in_val = val[(g + 1) & 1]; P.in_site = site[(g + 1) & 1];
+        P.out_val = val[g & 1]; P.out_site = site[g & 1];
+        P.inner = pl.inner[k0]; P.outer = pl.N / (P.inner * P.prod);
+        P.V = pl.V;
+        const double carry = SITE ? 8.0 : 4.0;
+        prof_mark(st, fin ? "small_group_final" : "small_group",
+                  (double)pl.N * ((first ? 1.0 : carry) + (fin ? out_bpv : carry)));
+        const int64_t tiles = P.inner == 1 ? (P.outer + kSmallT - 1) / kSmallT
+                                           : P.outer * ((P.inner + kSmallT - 1) / kSmallT);
+        const unsigned blocks = (unsigned)tiles;
+#define TM_SMALL_LAUNCH3(FIRST, FIN, NM)                                                                         \
+    do {                                                                                                         \
+        auto kern = small_group_kernel<SITE, FIRST, FIN, NM>;                                                    \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        kern<<<blocks, threads, smem, st>>>(P, ep);                                                        \
+    } while (0)
+#define TM_SMALL_LAUNCH(FIRST, FIN)                                                                              \
+    do {                                                                                                         \
+        if (nm <= 4) TM_SMALL_LAUNCH3(FIRST, FIN, 4);                                                            \
+        else if (nm <= 6) TM_SMALL_LAUNCH3(FIRST, FIN, 6);                                                       \
+        else TM_SMALL_LAUNCH3(FIRST, FIN, 8);                                                                    \
+    } while (0)
+        int nm = 0, nmin = 8;
+        for (int q = 0; q < P.m; ++q) { nm = std::max(nm, P.n[q]); nmin = std::min(nmin, P.n[q]); }
+        // one thread per line of the axis with the most lines, within [128, 512]
+        const int max_lines = P.prod / nmin * kSmallT;
+        const unsigned threads = (unsigned)std::min(kSmallThreads, std::max(128, (max_lines + 31) / 32 * 32));
+        if (first && fin) TM_SMALL_LAUNCH(true, true);
+        else if (first) TM_SMALL_LAUNCH(true, false);
+        else if (fin) TM_SMALL_LAUNCH(false, true);
+        else TM_SMALL_LAUNCH(false, false);
+#undef TM_SMALL_LAUNCH3
+#undef TM_SMALL_LAUNCH
+        ++launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 // Unit sampling beyond extent 128 (two axes up to 1024, three up to 512): key rows, then strip scans.
 // sh: row bits of the integer keys (9 or 10), or -1 for float heights
 template <int K, bool FINAL>
@@ -617,6 +686,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
                               void* ws, cudaStream_t st, int& launches) {
     EpilogueParams ep;
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
+    if (pl.small) return ep.idx ? run_small<true>(pl, input, ep, ws, st, launches) : run_small<false>(pl, input, ep, ws, st, launches);
     if (pl.wide_keys && ((uintptr_t)input & 15u) == 0) return run_wide(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)

@@ -86,6 +86,27 @@ def test_small_shapes_every_rank(shape, p_fg, kind, path):
     full_check(mask, _sampling(len(shape) - 2, kind))
 
 
+TINY = [(37, 1, 5), (1, 1, 8), (70, 1, 3, 3), (3, 1, 8, 8, 8, 8), (2, 2, 7, 5, 3, 8, 2), (5, 1, 4, 4, 4, 4, 4),
+        (1, 1, 2, 2, 2, 2, 2, 2, 2, 2), (1, 1, 8, 8, 8), (2, 1, 6, 1, 7, 1, 5, 6, 2), (1, 3, 5, 8, 7, 6, 5)]
+
+
+@pytest.mark.parametrize("shape", TINY, ids=["x".join(map(str, s)) for s in TINY])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_extents_up_to_eight(shape, kind):
+    """Every extent <= 8: axes are grouped (product of extents <= 256) and each group runs as one kernel over
+    shared-memory tiles; the shapes split into groups at different places, leave ragged tiles along both the batch
+    and the inner index, and cover line lengths 2..8.  Checked with the index map and, separately, distance only."""
+    sampling = _sampling(len(shape) - 2, kind)
+    for p_fg in (0.5, 0.97):
+        mask = workloads.random_mask(zlib.crc32(repr((shape, kind, p_fg)).encode()), shape, p_fg)
+        _, ref = full_check(mask, sampling)
+        res = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
+        compare(mask, sampling, res, ref, True, False, False)
+    mask = np.ones(shape, dtype=np.uint8)
+    mask[-1].flat[-1] = 0  # one background voxel in the last image, none in the others
+    full_check(mask, sampling)
+
+
 @pytest.mark.parametrize("shape", [(1, 1, 64), (2, 1, 20, 30), (1, 2, 8, 9, 10), (1, 1, 200, 40)])
 def test_degenerate_masks(shape, path):
     ndim = len(shape) - 2
