@@ -505,7 +505,7 @@ static cudaError_t run_small(const Plan& pl, const uint8_t* in, const EpiloguePa
         P.inner = pl.inner[k0]; P.outer = pl.N / (P.inner * P.prod);
         P.V = pl.V;
         const double carry = SITE ? 8.0 : 4.0;
-        prof_mark(st, fin ? "small_group_final" : "small_group",
+        prof_mark(st, fin ? "small_group_final" : first ? "small_group_first" : "small_group",
                   (double)pl.N * ((first ? 1.0 : carry) + (fin ? out_bpv : carry)));
         const int64_t tiles = P.inner == 1 ? (P.outer + kSmallT - 1) / kSmallT
                                            : P.outer * ((P.inner + kSmallT - 1) / kSmallT);
