@@ -15,6 +15,7 @@
 #include "edt_fast.cuh"
 #include "edt_wide.cuh"
 #include "edt_small.cuh"
+#include "edt_long.cuh"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -59,6 +60,7 @@ struct Plan {
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
     bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    bool long_lines = false;  // two or three axes, extents up to 8192: plain heights scanned through the cache
     bool small = false;       // every extent <= 8: register-resident lines, value (+ site index) carry
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
     int si[kMaxDims];         // those integers
@@ -139,10 +141,14 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     // unit sampling: integer keys (two axes up to extent 1024, three up to 512); other sampling: float heights
     pl.wide_keys = !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || E == 2 || nmax <= 512) &&
                    pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
-    if (pl.wide_keys) {
+    pl.long_lines = !pl.small && !pl.fast && !pl.wide_keys && (E == 2 || E == 3) && nmax <= 8192 &&
+                    pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
+    if (pl.wide_keys || pl.long_lines) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+        const size_t bm = pl.long_lines ? up((size_t)pl.N / 4 + 1024) : 0;  // block minima of the long path
         pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
         if (E == 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
+        pl.ws_bytes += bm;
     }
     if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
     if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
@@ -613,6 +619,74 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     return e;
 }
 
+// Two or three axes with extents up to 8192: heights and 16-bit offsets per voxel, scans through the cache.
+template <bool FLT>
+static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                            int& launches) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    char* w = static_cast<char*>(ws);
+    uint32_t* hA = reinterpret_cast<uint32_t*>(w);
+    int16_t* offsA = reinterpret_cast<int16_t*>(w + up((size_t)pl.N * 4));
+    uint32_t* hB = reinterpret_cast<uint32_t*>(w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
+    int16_t* offsB = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
+    uint32_t* blockmin = reinterpret_cast<uint32_t*>(
+        w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2) + (pl.E == 3 ? 2 * up((size_t)pl.N * 4) : 0));
+    WideParams P;
+    P.in = in; P.keys = hA; P.offs = offsA;
+    P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
+    P.rows = pl.N / pl.ext[0];
+    P.w2x = (float)(pl.w[0] * pl.w[0]);
+    const double out_bpv = out_bytes_per_voxel(ep);
+    prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + 2.0));
+    long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    ++launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    LongAxisParams A;
+    memset(&A, 0, sizeof(A));
+    auto set_axis = [&](int k) {
+        A.n = pl.ext[k]; A.inner = pl.inner[k]; A.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+        A.n0 = pl.ext[0];
+        A.w2 = (float)(pl.w[k] * pl.w[k]);
+        A.strips_per_slab = (int)((A.inner + 31) / 32);
+        A.row_blocks = (A.n + kLongRows - 1) / kLongRows;
+        A.blockmin = A.n > 128 ? blockmin : nullptr;  // short axes: the row-by-row phase covers the column
+        return (unsigned)(A.outer * A.strips_per_slab * A.row_blocks);
+    };
+    // block minima of the heights the next axis pass reads
+    auto block_minima = [&]() -> cudaError_t {
+        if (!A.blockmin) return cudaSuccess;
+        const int64_t items = A.outer * ((A.n + 31) / 32) * A.inner;
+        prof_mark(st, "long_blockmin", (double)pl.N * 4.0);
+        long_blockmin_kernel<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(A);
+        ++launches;
+        return cudaGetLastError();
+    };
+    A.h_in = hA; A.offs_in = offsA; A.h_out = hB; A.offs_out = offsB;
+    unsigned blocks = set_axis(1);
+    e = block_minima();
+    if (e != cudaSuccess) return e;
+    if (pl.E == 2) {
+        prof_mark(st, "long_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
+        long_axis_kernel<1, true, FLT><<<blocks, 256, 0, st>>>(A, ep);
+        ++launches;
+        return cudaGetLastError();
+    }
+    prof_mark(st, "long_axis", (double)pl.N * (4.0 + 2.0 + 4.0 + 4.0));
+    long_axis_kernel<1, false, FLT><<<blocks, 256, 0, st>>>(A, ep);
+    ++launches;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    A.h_in = hB; A.offs_in = offsB; A.h_out = nullptr; A.offs_out = nullptr;
+    blocks = set_axis(2);
+    e = block_minima();
+    if (e != cudaSuccess) return e;
+    prof_mark(st, "long_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 4.0 : 0.0)));
+    long_axis_kernel<2, true, FLT><<<blocks, 256, 0, st>>>(A, ep);
+    ++launches;
+    return cudaGetLastError();
+}
+
 // Stream-ordered scratch of tm_edt and tm_edt_host comes from a memory pool of the library's own, one per
 // device, created on first use.  Its release threshold is unlimited, so the memory of one call is reused by
 // the next instead of going back to the driver at every synchronisation; tm_edt_trim_memory() returns it.
@@ -688,6 +762,8 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     if (pl.small) return ep.idx ? run_small<true>(pl, input, ep, ws, st, launches) : run_small<false>(pl, input, ep, ws, st, launches);
     if (pl.wide_keys && ((uintptr_t)input & 15u) == 0) return run_wide(pl, input, ep, ws, st, launches);
+    if (pl.long_lines && ((uintptr_t)input & 15u) == 0)
+        return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
         return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);

@@ -162,6 +162,50 @@ def test_long_lines(n):
     full_check(mask, (1.7, 0.6))
 
 
+LONG = [(1, 1, 1100, 48), (2, 1, 48, 2064), (1, 1, 1040, 1056), (1, 1, 3000, 32), (1, 1, 16, 8192),
+        (1, 1, 1100, 16, 32), (1, 2, 6, 1040, 48), (1, 1, 20, 32, 1040)]
+
+
+@pytest.mark.parametrize("shape", LONG, ids=["x".join(map(str, s)) for s in LONG])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_long_line_path(shape, kind):
+    """Two or three axes with an extent above 1024 and a contiguous extent that is a multiple of 16: plain
+    heights scanned through the cache, rows of several 1024-voxel chunks in the first-axis pass.  Dense
+    background, sparse background (long scans, rows without any background) and an image without background."""
+    sampling = _sampling(len(shape) - 2, kind)
+    seed = zlib.crc32(repr((shape, kind)).encode())
+    full_check(workloads.random_mask(seed, shape, 0.9), sampling)
+    mask = np.ones(shape, dtype=np.uint8)
+    rng = np.random.default_rng(seed)
+    for _ in range(10):
+        mask[(0, 0) + tuple(int(rng.integers(0, n)) for n in shape[2:])] = 0
+    res, ref = full_check(mask, sampling)
+    d = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
+    compare(mask, sampling, d, ref, True, False, False)
+
+
+@pytest.mark.parametrize("pattern", ["left_edge", "top_edge", "disc", "frame", "diagonal"])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_long_line_far_sites(pattern, kind):
+    """Long-line path with background far away (hundreds of rows): the block-wise far phase with its pruning by
+    block minima, ties at the centre of a disc, sites on both sides."""
+    n1, n0 = 1200, 1056
+    yy, xx = np.mgrid[0:n1, 0:n0]
+    mask = np.ones((n1, n0), dtype=np.uint8)
+    if pattern == "left_edge":
+        mask[:, 0] = 0
+    elif pattern == "top_edge":
+        mask[0, :] = 0
+    elif pattern == "disc":
+        mask = (((yy - n1 / 2) ** 2 + (xx - n0 / 2) ** 2) <= 500.0 ** 2).astype(np.uint8)
+    elif pattern == "frame":
+        mask[0, :] = 0; mask[-1, :] = 0; mask[:, 0] = 0; mask[:, -1] = 0
+    else:
+        mask[(yy * 7 + 3) % n1 == (xx * 5) % n1] = 0
+        mask[300:900, :] = 1
+    full_check(mask[None, None], _sampling(2, kind))
+
+
 def test_sparse_background_long_axis_exactness():
     """Few background voxels and large extents: squared distances up to ~1e7 must stay exact."""
     mask = np.ones((1, 1, 2048, 300), dtype=np.uint8)
