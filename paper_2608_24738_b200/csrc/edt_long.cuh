@@ -136,6 +136,57 @@ __global__ void __launch_bounds__(256) long_row_kernel(const __grid_constant__ W
     }
 }
 
+// First-axis pass for rows of any length up to 8192 and any alignment: lanes take consecutive voxels, so every
+// load and store of the warp is contiguous.  The zero bits of the row are collected as ballot words in shared
+// memory (at most 256 of them); a voxel finds its nearest zero to the left and to the right inside its own word
+// with __clz / __ffs, and otherwise takes the last zero before / first zero after the word.
+template <bool FLT>
+__global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant__ WideParams P) {
+    constexpr int MAXW = 256;
+    __shared__ uint32_t s_word[8][MAXW];
+    __shared__ int s_next[8][MAXW];  // first zero after word b
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;
+    if (row >= P.rows) return;  // the whole warp leaves together
+    const int n0 = P.n0;
+    const int W = (n0 + 31) >> 5;
+    const uint8_t* src = P.in + row * n0;
+    for (int b = 0; b < W; ++b) {
+        const int x = 32 * b + lane;
+        const unsigned word = __ballot_sync(0xffffffffu, x < n0 && src[x] == 0);
+        if (lane == 0) s_word[warp][b] = word;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        int nxt = kLongFar;
+        for (int b = W - 1; b >= 0; --b) {
+            s_next[warp][b] = nxt;
+            const uint32_t word = s_word[warp][b];
+            if (word) nxt = 32 * b + __ffs(word) - 1;
+        }
+    }
+    __syncwarp();
+    int carry_l = -kLongFar;  // last zero before word b
+    bool row_has_zero = false;
+    for (int b = 0; b < W; ++b) row_has_zero |= s_word[warp][b] != 0u;
+    for (int b = 0; b < W; ++b) {
+        const uint32_t word = s_word[warp][b];
+        const int x = 32 * b + lane;
+        const uint32_t ml = word & (0xffffffffu >> (31 - lane));  // zeros at or before this voxel
+        const uint32_t mr = word >> lane;                          // zeros at or after it
+        const int zl = ml ? 32 * b + 31 - __clz(ml) : carry_l;
+        const int zr = mr ? x + __ffs(mr) - 1 : s_next[warp][b];
+        const int dl = x - zl, dr = zr - x;
+        const int a = min(dl, dr);
+        if (x < n0) {
+            P.offs[row * n0 + x] = row_has_zero ? (int16_t)(dl <= dr ? -a : a) : (int16_t)-32768;
+            P.keys[row * n0 + x] = !row_has_zero ? (FLT ? kLongNoneFlt : kLongNoneInt)
+                                                 : (FLT ? __float_as_uint(__fmul_rn(P.w2x, (float)(a * a))) : (uint32_t)(a * a));
+        }
+        if (word) carry_l = 32 * b + 31 - __clz(word);
+    }
+}
+
 struct LongAxisParams {
     const uint32_t* h_in;      // (outer, n, inner) heights
     const int16_t* offs_in;    // (outer, n, inner, K)

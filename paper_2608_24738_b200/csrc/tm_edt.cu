@@ -142,7 +142,7 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.wide_keys = !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || E == 2 || nmax <= 512) &&
                    pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
     pl.long_lines = !pl.small && !pl.fast && !pl.wide_keys && (E == 2 || E == 3) && nmax <= 8192 &&
-                    pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
+                    !(force && force[0] == '1');
     if (pl.wide_keys || pl.long_lines) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
         const size_t bm = pl.long_lines ? up((size_t)pl.N / 4 + 1024) : 0;  // block minima of the long path
@@ -638,7 +638,8 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
     P.w2x = (float)(pl.w[0] * pl.w[0]);
     const double out_bpv = out_bytes_per_voxel(ep);
     prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + 2.0));
-    long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    if (pl.ext[0] % 16 == 0 && ((uintptr_t)in & 15u) == 0) long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    else long_row_any_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -762,7 +763,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     if (pl.small) return ep.idx ? run_small<true>(pl, input, ep, ws, st, launches) : run_small<false>(pl, input, ep, ws, st, launches);
     if (pl.wide_keys && ((uintptr_t)input & 15u) == 0) return run_wide(pl, input, ep, ws, st, launches);
-    if (pl.long_lines && ((uintptr_t)input & 15u) == 0)
+    if (pl.long_lines)
         return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
