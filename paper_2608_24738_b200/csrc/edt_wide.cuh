@@ -117,6 +117,7 @@ struct WideAxisParams {
     int next_n;                // extent of the next axis (non-final)
     int n0;                    // extent of the contiguous axis (to split an inner position into coordinates)
     float w2;                  // squared sampling of this axis (float-height variant)
+    int row_parts;             // blocks that share one strip, each taking a contiguous range of its rows
 };
 
 // Bounded scan of one voxel on float32 heights (general sampling): returns the best value and the distance bd
@@ -145,10 +146,14 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     extern __shared__ __align__(16) uint8_t sm_wide[];
     uint32_t* val = reinterpret_cast<uint32_t*>(sm_wide);  // [n][32]
     const int n = P.n;
-    const int64_t slab = blockIdx.x / strips_per_slab;
-    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
+    const unsigned part = blockIdx.x % (unsigned)P.row_parts, sidx = blockIdx.x / (unsigned)P.row_parts;
+    const int64_t slab = sidx / (unsigned)strips_per_slab;
+    const int64_t c0 = (int64_t)(sidx - slab * strips_per_slab) * 32;
     const int64_t slab_base = slab * (int64_t)n * P.inner;
     const uint32_t* src = P.keys_in + slab_base + c0;
+    // rows of this block (a multiple of R per part); every part stages the whole strip, a scan may reach any row
+    const int rows_per_part = ((n + P.row_parts - 1) / P.row_parts + 3) & ~3;
+    const int y_begin = (int)part * rows_per_part, y_end = min(n, y_begin + rows_per_part);
     // stage: 8 threads copy one row of 32 keys (inner is a multiple of 16, so a strip is 16 or 32 positions wide)
     const int width = (int)min((int64_t)32, P.inner - c0);
     for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
@@ -166,7 +171,7 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     const uint32_t next_row = FINAL ? 0u : (uint32_t)(slab % P.next_n);
     // own coordinates along the earlier axes (final pass, index output): plane 0 = contiguous axis
     const int cx = (int)(c % P.n0), cy = (int)(c / P.n0);
-    for (int y0 = warp * R; y0 < n; y0 += nwarps * R) {
+    for (int y0 = y_begin + warp * R; y0 < y_end; y0 += nwarps * R) {
         uint32_t best[R];
         int jrow[R];
         if (SH >= 0) {

@@ -557,7 +557,15 @@ static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParam
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<(unsigned)(A.outer * strips), A.n > 512 ? 512 : 256, smem, st>>>(A, ep, strips);
+    // 16 warps per strip from 384 rows on: shared memory allows few blocks per SM there, and a strip's rows
+    // are independent work
+    // few strips (a single large image): several blocks share a strip, each taking a range of its rows, until
+    // there are about two blocks per SM
+    WideAxisParams B = A;
+    const int64_t base_blocks = A.outer * strips;
+    B.row_parts = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(8, A.n / 64), 296 / base_blocks));
+    if (const char* v = getenv("TM_EDT_WIDE_PARTS")) B.row_parts = atoi(v);
+    kern<<<(unsigned)(base_blocks * B.row_parts), A.n >= 384 ? 512 : 256, smem, st>>>(B, ep, strips);
     return cudaGetLastError();
 }
 
