@@ -140,7 +140,9 @@ __global__ void __launch_bounds__(256) long_row_kernel(const __grid_constant__ W
 // load and store of the warp is contiguous.  The zero bits of the row are collected as ballot words in shared
 // memory (at most 256 of them); a voxel finds its nearest zero to the left and to the right inside its own word
 // with __clz / __ffs, and otherwise takes the last zero before / first zero after the word.
-template <bool FLT>
+// SH >= 0: wide-path keys (off^2 << SH | row index along the second axis); SH == -1: float32 heights; SH == -2: plain
+// integer heights.
+template <int SH>
 __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant__ WideParams P) {
     constexpr int MAXW = 256;
     __shared__ uint32_t s_word[8][MAXW];
@@ -148,7 +150,9 @@ __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;
     if (row >= P.rows) return;  // the whole warp leaves together
+    constexpr bool FLT = SH == -1;
     const int n0 = P.n0;
+    const uint32_t yrow = SH >= 0 ? (uint32_t)(row % P.n1) : 0u;
     const int W = (n0 + 31) >> 5;
     const uint8_t* src = P.in + row * n0;
     for (int b = 0; b < W; ++b) {
@@ -181,7 +185,8 @@ __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant
         if (x < n0) {
             P.offs[row * n0 + x] = row_has_zero ? (int16_t)(dl <= dr ? -a : a) : (int16_t)-32768;
             P.keys[row * n0 + x] = !row_has_zero ? (FLT ? kLongNoneFlt : kLongNoneInt)
-                                                 : (FLT ? __float_as_uint(__fmul_rn(P.w2x, (float)(a * a))) : (uint32_t)(a * a));
+                                                 : (FLT ? __float_as_uint(__fmul_rn(P.w2x, (float)(a * a)))
+                                                        : (((uint32_t)(a * a) << (SH > 0 ? SH : 0)) | yrow));
         }
         if (word) carry_l = 32 * b + 31 - __clz(word);
     }

@@ -1,15 +1,17 @@
-// Unit sampling with extents beyond the 128 of the packed 8-bit entries: two processed axes with extents up
-// to 1024, three with extents up to 512.  Kernels:
-//   row_keys_kernel     first-axis pass, one warp per row, 16 or 32 voxels per lane (128-bit loads).
-//                       Writes, per voxel, the scan key  (off^2 << SH) | row  (32 bit; SH = 9 row bits for
-//                       extents up to 512, 10 up to 1024: 2 * 1023^2 << 10 still stays below 2^31) and the
-//                       signed 16-bit offset to the nearest zero of the row.
-//   wide_axis_kernel    every further axis: a block stages the keys of an (n x 32) strip in shared memory and
-//                       runs the grouped bounded scan on it (edt_fast.cuh).  A middle pass writes the key of
-//                       the next pass and the site's offsets (16 bits per axis); the last pass writes the
-//                       outputs and fetches the chosen site's offsets only when indices are requested.
-// Same mathematics as the fast path: g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (x_k - j)^2 ], exact in
-// integers: values stay below 3 * 511^2 < 2^20 (three axes, 9 row bits) or 2 * 1023^2 < 2^21 (two axes, 10).
+// Extents beyond the 128 of the packed 8-bit entries, two or three processed axes, extents up to 1024.
+// Kernels:
+//   row_keys_kernel     first-axis pass, one warp per row, 16 or 32 voxels per lane (128-bit loads; rows that
+//                       are not 16-byte aligned use long_row_any_kernel of edt_long.cuh instead).
+//                       Writes, per voxel, the scan value and the signed 16-bit offset to the nearest zero of
+//                       the row.  Unit sampling: the key (off^2 << SH) | row (32 bit; SH = 9 row bits for
+//                       extents up to 512, 10 up to 1024), as long as every key stays below 2^31 (two axes up
+//                       to 1024, three up to about 830).  Otherwise: the float32 height w^2 off^2.
+//   wide_axis_kernel    every further axis: a block stages the values of an (n x 32) strip in shared memory and
+//                       runs the bounded scan on it (grouped, edt_fast.cuh, for keys).  A middle pass writes
+//                       the value of the next pass and the site's offsets (16 bits per axis); the last pass
+//                       writes the outputs and fetches the chosen site's offsets only when indices are requested.
+// Same mathematics as the fast path: g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (w_k (x_k - j))^2 ], exact in
+// integers under unit sampling.
 #pragma once
 #include "edt_fast.cuh"
 
@@ -154,12 +156,19 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     // rows of this block (a multiple of R per part); every part stages the whole strip, a scan may reach any row
     const int rows_per_part = ((n + P.row_parts - 1) / P.row_parts + 3) & ~3;
     const int y_begin = (int)part * rows_per_part, y_end = min(n, y_begin + rows_per_part);
-    // stage: 8 threads copy one row of 32 keys (inner is a multiple of 16, so a strip is 16 or 32 positions wide)
+    // stage: 8 threads copy one row of 32 keys in 16-byte pieces when rows are 16-byte aligned, single keys otherwise
     const int width = (int)min((int64_t)32, P.inner - c0);
-    for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
-        const int y = t >> 3, ch = t & 7;
-        if (4 * ch < width)
-            *reinterpret_cast<uint4*>(val + y * 32 + 4 * ch) = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + 4 * ch);
+    if ((P.inner & 3) == 0) {
+        for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
+            const int y = t >> 3, ch = t & 7;
+            if (4 * ch < width)
+                *reinterpret_cast<uint4*>(val + y * 32 + 4 * ch) = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + 4 * ch);
+        }
+    } else {
+        for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
+            const int y = t >> 5, x = t & 31;
+            if (x < width) val[y * 32 + x] = src[(int64_t)y * P.inner + x];
+        }
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;

@@ -139,8 +139,12 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     pl.small = nmax <= 8 && !(force && force[0] == '1');
     pl.fast = !pl.small && nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
     // unit sampling: integer keys (two axes up to extent 1024, three up to 512); other sampling: float heights
-    pl.wide_keys = !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || E == 2 || nmax <= 512) &&
-                   pl.ext[0] % 16 == 0 && !(force && force[0] == '1');
+    // integer keys (value << sh | row, sh = 9 row bits up to extent 512, else 10): every real key must stay below the
+    // "no site" key 2^31 and "no site" plus the largest addend below 2^32
+    const double key_scale = nmax > 512 ? 1024.0 : 512.0;
+    const bool keys_fit = sumsq * key_scale < 2147483648.0 && (double)(nmax + 4) * (nmax + 4) * key_scale < 2147483648.0;
+    pl.wide_keys = !pl.small && !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || keys_fit) &&
+                   !(force && force[0] == '1');
     pl.long_lines = !pl.small && !pl.fast && !pl.wide_keys && (E == 2 || E == 3) && nmax <= 8192 &&
                     !(force && force[0] == '1');
     if (pl.wide_keys || pl.long_lines) {
@@ -590,7 +594,12 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     const int sh = !pl.unit ? -1 : (nmax > 512 ? 10 : 9);
     prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + 2.0));
     const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
-    if (pl.ext[0] <= 512) {
+    if (pl.ext[0] % 16 != 0 || ((uintptr_t)in & 15u) != 0) {
+        // rows that are not 16-byte aligned: one voxel per lane, ballot words
+        if (sh < 0) long_row_any_kernel<-1><<<row_blocks, 256, 0, st>>>(P);
+        else if (sh == 9) long_row_any_kernel<9><<<row_blocks, 256, 0, st>>>(P);
+        else long_row_any_kernel<10><<<row_blocks, 256, 0, st>>>(P);
+    } else if (pl.ext[0] <= 512) {
         if (sh < 0) row_keys_kernel<16, -1><<<row_blocks, 256, 0, st>>>(P);
         else if (sh == 9) row_keys_kernel<16, 9><<<row_blocks, 256, 0, st>>>(P);
         else row_keys_kernel<16, 10><<<row_blocks, 256, 0, st>>>(P);
@@ -647,7 +656,7 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
     const double out_bpv = out_bytes_per_voxel(ep);
     prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + 2.0));
     if (pl.ext[0] % 16 == 0 && ((uintptr_t)in & 15u) == 0) long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
-    else long_row_any_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
+    else long_row_any_kernel<FLT ? -1 : -2><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -770,7 +779,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     EpilogueParams ep;
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     if (pl.small) return ep.idx ? run_small<true>(pl, input, ep, ws, st, launches) : run_small<false>(pl, input, ep, ws, st, launches);
-    if (pl.wide_keys && ((uintptr_t)input & 15u) == 0) return run_wide(pl, input, ep, ws, st, launches);
+    if (pl.wide_keys) return run_wide(pl, input, ep, ws, st, launches);
     if (pl.long_lines)
         return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);

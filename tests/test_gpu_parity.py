@@ -163,15 +163,16 @@ def test_long_lines(n):
 
 
 LONG = [(1, 1, 1100, 48), (2, 1, 48, 2064), (1, 1, 1040, 1056), (1, 1, 3000, 32), (1, 1, 16, 8192),
-        (1, 1, 1100, 16, 32), (1, 2, 6, 1040, 48), (1, 1, 20, 32, 1040)]
+        (1, 1, 1100, 16, 32), (1, 2, 6, 1040, 48), (1, 1, 20, 32, 1040),
+        (1, 1, 20, 32, 640), (1, 1, 600, 18, 50), (1, 1, 7, 800, 44), (2, 1, 500, 500), (1, 1, 1000, 999), (1, 1, 150, 150, 150)]
 
 
 @pytest.mark.parametrize("shape", LONG, ids=["x".join(map(str, s)) for s in LONG])
 @pytest.mark.parametrize("kind", ["unit", "sampled"])
 def test_long_line_path(shape, kind):
-    """Two or three axes with an extent above 1024 and a contiguous extent that is a multiple of 16: plain
-    heights scanned through the cache, rows of several 1024-voxel chunks in the first-axis pass.  Dense
-    background, sparse background (long scans, rows without any background) and an image without background."""
+    """Two or three axes with an extent above 128: shared-memory strips up to extent 1024 (integer keys while they
+    fit 31 bits, float heights otherwise), cached height scans beyond, rows of any length and alignment in the
+    first-axis pass.  Dense background and sparse background (long scans, rows without any background)."""
     sampling = _sampling(len(shape) - 2, kind)
     seed = zlib.crc32(repr((shape, kind)).encode())
     full_check(workloads.random_mask(seed, shape, 0.9), sampling)
