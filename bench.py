@@ -232,8 +232,9 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
         m = host_mask.to(dev)
         d = torch.empty(shape, dtype=torch.float32, device=dev) if w.want_dist else None
         s = torch.empty(shape, dtype=torch.int64, device=dev) if w.want_sq else None
-        x = torch.empty(shape[:2] + (w.ndim,) + shape[2:], dtype=torch.int64, device=dev) if w.want_idx else None
-        calls.append(binding.PreparedCall(m, w.sampling, d, s, x))
+        xshape = shape if w.flat_index else shape[:2] + (w.ndim,) + shape[2:]
+        x = torch.empty(xshape, dtype=torch.int64, device=dev) if w.want_idx else None
+        calls.append(binding.PreparedCall(m, w.sampling, d, s, x, flags=binding.FLAG_FLAT_INDEX if w.flat_index else 0))
     stream = torch.cuda.current_stream()
     sp = ctypes.c_void_p(stream.cuda_stream)
     for i in range(warmup):
@@ -266,7 +267,7 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
         c = calls[i % sets]
         _, ks = binding.tm_edt_profile(c.mask, w.sampling, distances=c.d, sqdist=c.s, indices=c.x, workspace=c.ws,
                                        return_distances=w.want_dist, return_sqdist=w.want_sq,
-                                       return_indices=w.want_idx)
+                                       return_indices=w.want_idx, flags=c.flags)
         for j, (name, ms, nbytes) in enumerate(ks):
             key = (j, name)
             if key not in ksum:
@@ -310,6 +311,8 @@ def main():
     ap.add_argument("--profile-steps", type=int, default=20)
     ap.add_argument("--unit-sampling", action="store_true", help="override the workload's sampling with 1.0 per axis")
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
+    ap.add_argument("--flat-index", action="store_true",
+                    help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -330,6 +333,9 @@ def main():
         want = set(args.outputs.split(","))
         w.want_dist, w.want_sq, w.want_idx = "dist" in want, "sq" in want, "idx" in want
         w.name += " (outputs %s)" % args.outputs
+    if args.flat_index:
+        w.flat_index = True
+        w.name += " (flat index)"
     if args.impl == "reference":
         run_reference(args, w, world, rank)
         return
@@ -363,7 +369,7 @@ def main():
 
     # ---- end to end: host buffers in, host buffers out, through tm_edt_host ----
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not w.flat_index:  # the host entry point has the headline index layout only
         hm = host_mask.pin_memory()
         hd = torch.empty(shape, dtype=torch.float32, pin_memory=True) if w.want_dist else None
         hs = torch.empty(shape, dtype=torch.int64, pin_memory=True) if w.want_sq else None
@@ -389,7 +395,7 @@ def main():
     sampler.stop()
 
     others = None
-    if world == 1 and not args.no_all_configs and not args.unit_sampling and not args.outputs and not args.images:
+    if world == 1 and not args.no_all_configs and not args.unit_sampling and not args.outputs and not args.images and not args.flat_index:
         others = []
         for num in (1, 2, 3, 4, 5):
             if num == args.config:

@@ -90,6 +90,30 @@ TM_EDT_API int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, cons
            int64_t* out_sqdist, int64_t* out_indices, tm_edt_stream_t stream);
 
 /*
+ * Variants of the transform behind a flags word (0 = exactly tm_edt / tm_edt_ws):
+ *
+ *   TM_EDT_FLAG_VIRTUAL_BACKGROUND  An image without any background voxel gets, instead of +inf / INT64_MAX /
+ *       -1, the values of the virtual out-of-bounds convention the paper takes over from scipy.ndimage
+ *       (Section 2.3.2, "Distance-transform kernels"): as if its only background voxel sat at coordinate -1
+ *       on spatial axis 0 and 0 on every other axis, i.e.
+ *       d(x) = sqrt((w_0 (x_0 + 1))^2 + sum_{k>=1} (w_k x_k)^2), indices (-1, 0, .., 0).
+ *   TM_EDT_FLAG_FLAT_INDEX  out_indices is (B, C, n...) int64: the row-major linear index, inside its image,
+ *       of the chosen background voxel (one value per voxel instead of ndim; -1 for an image without
+ *       background, minus the stride of axis 0 under the virtual-background convention).  The paper's index
+ *       map has one coordinate per axis; this layout is an extra of this library.
+ *
+ *   workspace    device scratch of at least tm_edt_workspace_bytes(ndim, shape) bytes, 256-byte aligned, or
+ *                NULL to take scratch from the library's memory pool as tm_edt does (workspace_bytes ignored).
+ *   Every other argument, the ownership rules and the error behaviour are those of tm_edt; an unknown flag
+ *   bit gives TM_EDT_ERR_INVALID_ARG.  With a workspace the call allocates nothing and only enqueues kernels.
+ */
+#define TM_EDT_FLAG_VIRTUAL_BACKGROUND 1u
+#define TM_EDT_FLAG_FLAT_INDEX 2u
+TM_EDT_API int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+              int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace, size_t workspace_bytes,
+              tm_edt_stream_t stream);
+
+/*
  * Scratch bytes tm_edt_ws needs for a call with this geometry (0 for empty problems, and (size_t)-1
  * if ndim/shape are invalid or unsupported).  Depends only on ndim and shape.
  */
@@ -162,6 +186,13 @@ TM_EDT_API int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* sha
                               float* out_dist, int64_t* out_sqdist, int64_t* out_indices, void* workspace,
                               size_t workspace_bytes, tm_edt_stream_t stream, int max_kernels, float* kernel_ms,
                               double* kernel_bytes, char* kernel_names, int* n_kernels);
+
+/* tm_edt_profile for the variants of tm_edt_ex: the same measurement with a flags word (workspace required when the
+ * geometry needs scratch). */
+TM_EDT_API int tm_edt_profile_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling,
+                                 float* out_dist, int64_t* out_sqdist, int64_t* out_indices, unsigned flags,
+                                 void* workspace, size_t workspace_bytes, tm_edt_stream_t stream, int max_kernels,
+                                 float* kernel_ms, double* kernel_bytes, char* kernel_names, int* n_kernels);
 
 /*
  * Returns to the driver whatever the library's private memory pool of the current device holds and no

@@ -113,3 +113,33 @@ def sep(mask, sampling=None, want_idx=True):
 def sep_axes(mask, axes, sampling=None, want_idx=True):
     """Intermediate after nested minima over the listed spatial axes only, in that order."""
     return _run("sep", mask, sampling, want_idx, axes=list(axes))
+
+
+def virtual_background(mask, sampling=None, want_idx=True, kind="sep"):
+    """The transform with the virtual out-of-bounds convention for images without background (paper,
+    Section 2.3.2: the convention of scipy.ndimage): such an image is transformed as if it had exactly one
+    background voxel, at coordinate -1 on spatial axis 0 and 0 on every other axis.
+
+    Written as that definition: every image without background is extended by one slice in front of axis 0,
+    foreground except for its voxel (0, .., 0); the extended image goes through the ordinary oracle, the extra
+    slice is cut off again and the indices along axis 0 are shifted back by one.  Images with background are
+    untouched.  Pins: the closed form and scipy.ndimage itself (tests/test_oracle_pins.py)."""
+    run = brute if kind == "brute" else sep
+    mask = np.ascontiguousarray(mask)
+    res = run(mask, sampling, want_idx)
+    ndim = mask.ndim - 2
+    for b in range(mask.shape[0]):
+        for c in range(mask.shape[1]):
+            if not mask[b, c].all():
+                continue
+            ext = np.ones((1, 1, mask.shape[2] + 1) + mask.shape[3:], dtype=np.uint8)
+            ext[(0, 0) + (0,) * ndim] = 0
+            r = run(ext, sampling, want_idx)
+            for key in ("dist", "sqf", "sq"):
+                if res[key] is not None:
+                    res[key][b, c] = r[key][0, 0, 1:]
+            if want_idx:
+                ix = r["idx"][0, 0][:, 1:].copy()
+                ix[0] -= 1
+                res["idx"][b, c] = ix
+    return res

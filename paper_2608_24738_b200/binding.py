@@ -19,7 +19,7 @@ MAX_DIMS = 8
 MAX_EXTENT = 8192
 
 EXPORTS = (
-    "tm_edt", "tm_edt_ws", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_workspace_bytes", "tm_edt_strerror",
+    "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
 )
 
@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
             L.tm_edt.restype = i
             L.tm_edt_ws.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp]
             L.tm_edt_ws.restype = i
+            L.tm_edt_ex.argtypes = [vp, i, vp, vp, vp, vp, vp, ctypes.c_uint, vp, sz, vp]
+            L.tm_edt_ex.restype = i
             L.tm_edt_host.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
             L.tm_edt_host.restype = i
             L.tm_edt_noalloc.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -55,6 +57,8 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_noalloc_max_scratch.restype = sz
             L.tm_edt_profile.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp, i, vp, vp, vp, vp]
             L.tm_edt_profile.restype = i
+            L.tm_edt_profile_ex.argtypes = [vp, i, vp, vp, vp, vp, vp, ctypes.c_uint, vp, sz, vp, i, vp, vp, vp, vp]
+            L.tm_edt_profile_ex.restype = i
             L.tm_edt_workspace_bytes.argtypes = [i, vp]
             L.tm_edt_workspace_bytes.restype = sz
             L.tm_edt_strerror.argtypes = [i]
@@ -122,7 +126,12 @@ def _check(status: int) -> None:
         raise TmEdtError(status, tm_edt_strerror(status))
 
 
-def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, device):
+FLAG_VIRTUAL_BACKGROUND = 1
+FLAG_FLAT_INDEX = 2
+
+
+def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, device,
+             flat_index=False):
     import torch
 
     if mask.dim() < 3:
@@ -151,7 +160,7 @@ def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, di
         mk = lambda want, dtype, shp, buf: out(buf, want, dtype, shp)
     d = mk(return_distances, torch.float32, shape, distances)
     s = mk(return_sqdist, torch.int64, shape, sqdist)
-    x = mk(return_indices, torch.int64, shape[:2] + (ndim,) + shape[2:], indices)
+    x = mk(return_indices, torch.int64, shape if flat_index else shape[:2] + (ndim,) + shape[2:], indices)
     return mask, shape, ndim, d, s, x
 
 
@@ -160,21 +169,30 @@ def _p(t):
 
 
 def tm_edt(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
-           distances=None, indices=None, sqdist=None, workspace=None, stream=None):
+           distances=None, indices=None, sqdist=None, workspace=None, stream=None,
+           virtual_background=False, flat_index=False):
     """Distance transform of a CUDA mask tensor (B, C, spatial...), uint8 or bool.
 
     Returns a dict with the requested tensors among ``dist`` (float32), ``sq`` (int64, unit sampling
     only) and ``idx`` (int64, (B, C, ndim, spatial...)).  With ``workspace`` (a CUDA uint8 tensor of at
     least ``tm_edt_workspace_bytes(mask.shape)`` bytes) the call goes through ``tm_edt_ws`` and allocates
     nothing; otherwise through ``tm_edt``.  Work is enqueued on ``stream`` (default: current stream).
+    ``virtual_background`` / ``flat_index`` select the variants of ``tm_edt_ex``: SciPy's values for images
+    without background, and ``idx`` as one linear index per voxel, shaped like the mask.
     """
     L = lib()
     if not mask.is_cuda:
         raise ValueError("mask must be a CUDA tensor (use tm_edt_host for host buffers)")
     mask, shape, ndim, d, s, x = _prepare(
-        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device,
+        flat_index=flat_index)
     shp, smp, st = _shape_array(shape), _sampling_array(sampling, ndim), _raw_stream(stream)
-    if workspace is None:
+    flags = (FLAG_VIRTUAL_BACKGROUND if virtual_background else 0) | (FLAG_FLAT_INDEX if flat_index else 0)
+    if flags:
+        nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        rc = L.tm_edt_ex(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), ctypes.c_uint(flags), _p(workspace),
+                         ctypes.c_size_t(nbytes), st)
+    elif workspace is None:
         rc = L.tm_edt(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), st)
     else:
         rc = L.tm_edt_ws(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), _p(workspace),
@@ -222,14 +240,15 @@ def tm_edt_host(mask, sampling=None, return_distances=True, return_indices=False
 
 
 def tm_edt_profile(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
-                   distances=None, indices=None, sqdist=None, workspace=None, stream=None):
+                   distances=None, indices=None, sqdist=None, workspace=None, stream=None, flags=0):
     """tm_edt_ws with per-kernel device times: returns (outputs dict, [(kernel label, milliseconds, bytes the launch must move), ...]).
     Blocks until the work is done.  ``workspace`` is required when the shape needs scratch."""
     import torch
 
     L = lib()
     mask, shape, ndim, d, s, x = _prepare(
-        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device,
+        flat_index=bool(flags & FLAG_FLAT_INDEX))
     if workspace is None:
         workspace = torch.empty(max(1, tm_edt_workspace_bytes(shape)), dtype=torch.uint8, device=mask.device)
     kmax = 32
@@ -237,9 +256,9 @@ def tm_edt_profile(mask, sampling=None, return_distances=True, return_indices=Fa
     nbytes = (ctypes.c_double * kmax)()
     names = ctypes.create_string_buffer(48 * kmax)
     n = ctypes.c_int(0)
-    rc = L.tm_edt_profile(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
-                          _p(workspace), ctypes.c_size_t(workspace.numel()), _raw_stream(stream), kmax, ms, nbytes, names,
-                          ctypes.byref(n))
+    rc = L.tm_edt_profile_ex(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
+                             ctypes.c_uint(flags), _p(workspace), ctypes.c_size_t(workspace.numel()), _raw_stream(stream),
+                             kmax, ms, nbytes, names, ctypes.byref(n))
     _check(rc)
     out = [(names.raw[48 * k: 48 * k + 48].split(b"\0", 1)[0].decode(), float(ms[k]), float(nbytes[k]))
            for k in range(n.value)]
@@ -249,21 +268,25 @@ def tm_edt_profile(mask, sampling=None, return_distances=True, return_indices=Fa
 class PreparedCall:
     """A tm_edt_ws call with its arguments marshalled once, for callers that repeat it (benchmarks, loops)."""
 
-    def __init__(self, mask, sampling=None, distances=None, sqdist=None, indices=None, workspace=None):
+    def __init__(self, mask, sampling=None, distances=None, sqdist=None, indices=None, workspace=None, flags=0):
         import torch
 
         self._L = lib()
+        self.flags = int(flags)
         self.mask, self.shape, self.ndim, self.d, self.s, self.x = _prepare(
             mask, sampling, distances is not None, sqdist is not None, indices is not None, distances, sqdist,
-            indices, mask.device)
+            indices, mask.device, flat_index=bool(self.flags & FLAG_FLAT_INDEX))
         need = tm_edt_workspace_bytes(self.shape)
         if workspace is None:
             workspace = torch.empty(max(1, need), dtype=torch.uint8, device=mask.device)
         self.ws = workspace
-        self._args = (_p(self.mask), self.ndim, _shape_array(self.shape), _sampling_array(sampling, self.ndim),
-                      _p(self.d), _p(self.s), _p(self.x), _p(self.ws), ctypes.c_size_t(self.ws.numel()))
+        head = (_p(self.mask), self.ndim, _shape_array(self.shape), _sampling_array(sampling, self.ndim),
+                _p(self.d), _p(self.s), _p(self.x))
+        tail = (_p(self.ws), ctypes.c_size_t(self.ws.numel()))
+        self._fn = self._L.tm_edt_ex if self.flags else self._L.tm_edt_ws
+        self._args = head + ((ctypes.c_uint(self.flags),) if self.flags else ()) + tail
 
     def __call__(self, stream_ptr):
-        rc = self._L.tm_edt_ws(*self._args, stream_ptr)
+        rc = self._fn(*self._args, stream_ptr)
         if rc != OK:
             _check(rc)

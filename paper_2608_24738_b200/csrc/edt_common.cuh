@@ -23,7 +23,7 @@ template <> struct OffTraits<int16_t> { static constexpr int kNone = -32768; };
 struct EpilogueParams {
     float* dist;        // (images, V) or nullptr
     int64_t* sq;        // (images, V) or nullptr
-    int64_t* idx;       // (images, ndim, V) or nullptr
+    int64_t* idx;       // (images, ndim, V), or (images, V) when flat, or nullptr
     int64_t V;          // voxels per image
     int ndim;           // spatial rank of the call
     int E;              // number of processed axes
@@ -31,6 +31,9 @@ struct EpilogueParams {
     int plane_of_axis[kMaxDims]; // plane of spatial axis a, or -1 if its extent is 1 (never processed)
     int ext[kMaxDims];           // extent of plane p
     double w2[kMaxDims];         // squared sampling of plane p
+    int flat;                    // 1: idx holds one value per voxel, the linear index of the site inside its image
+    int idx_planes;              // index values per voxel: 1 when flat, else ndim
+    int64_t pstride[kMaxDims];   // voxel stride of plane p inside an image
 };
 
 template <typename CT> __device__ __forceinline__ CT sqrt_ct(CT v);
@@ -47,7 +50,8 @@ __device__ __forceinline__ void emit_outputs(const EpilogueParams& ep, int64_t i
     if (none) {
         if (ep.dist) ep.dist[e] = __int_as_float(0x7f800000);
         if (ep.sq) ep.sq[e] = INT64_MAX;
-        if (ep.idx)
+        if (ep.idx && ep.flat) ep.idx[e] = -1;
+        else if (ep.idx)
             for (int a = 0; a < ep.ndim; ++a) ep.idx[(img * ep.ndim + a) * ep.V + v] = -1;
         return;
     }
@@ -65,7 +69,13 @@ __device__ __forceinline__ void emit_outputs(const EpilogueParams& ep, int64_t i
             if (p < ep.E) s += (int64_t)off[p] * (int64_t)off[p];
         ep.sq[e] = s;
     }
-    if (ep.idx) {
+    if (ep.idx && ep.flat) {
+        int64_t f = 0;
+#pragma unroll
+        for (int p = 0; p < kMaxDims; ++p)
+            if (p < ep.E) f += (int64_t)(coord[p] + off[p]) * ep.pstride[p];
+        ep.idx[e] = f;
+    } else if (ep.idx) {
         for (int a = 0; a < ep.ndim; ++a) {
             const int p = ep.plane_of_axis[a];
             int64_t val = 0;

@@ -98,12 +98,17 @@ struct ColumnOut {
     bool dist_only;      // final: only out_dist was requested
     int64_t* ip[5];      // final: index plane of processed axis q (same row-0 origin as idx)
     bool simple_idx;     // final: every spatial axis is a processed axis (no extent-1 axes to fill with 0)
+    bool flat;           // final: idx holds one value per voxel, the site's linear index inside the image
+    int pst[5];          // flat: voxel stride of plane q inside the image
 
     // call after idx, V, ndim and axis[] are set
-    __device__ __forceinline__ void init_index_planes() {
+    __device__ __forceinline__ void init_index_planes(const EpilogueParams& ep) {
 #pragma unroll
         for (int q = 0; q <= K; ++q) ip[q] = idx ? idx + (int64_t)axis[q] * V : nullptr;
         simple_idx = ndim == K + 1;
+        flat = ep.flat != 0;
+#pragma unroll
+        for (int q = 0; q <= K; ++q) pst[q] = (int)ep.pstride[q];
     }
 };
 
@@ -130,12 +135,18 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j,
     if (o.dist) o.dist[p] = dv;
     if (none) {
         if (o.sq) o.sq[p] = INT64_MAX;
-        if (o.idx)
+        if (o.idx && o.flat) o.idx[p] = -1;
+        else if (o.idx)
             for (int a = 0; a < o.ndim; ++a) o.idx[(int64_t)a * o.V + p] = -1;
         return;
     }
     if (o.sq) o.sq[p] = (int64_t)sqv;  // unit sampling only
-    if (o.idx && o.simple_idx) {
+    if (o.idx && o.flat) {
+        int f = j * o.pst[K];
+#pragma unroll
+        for (int q = 0; q < K; ++q) f += (o.coord[q] + (int)(int8_t)((e >> (8 * q)) & 0xff)) * o.pst[q];
+        o.idx[p] = (int64_t)f;
+    } else if (o.idx && o.simple_idx) {
         // one store per processed axis: own coordinate + offset (coordinates are non-negative)
 #pragma unroll
         for (int q = 0; q < K; ++q)
@@ -475,12 +486,12 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
             } else {  // two processed axes: the plane is the image
                 out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
                 out.sq = ep.sq ? ep.sq + plane * ep.V + c : nullptr;
-                out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+                out.idx = ep.idx ? ep.idx + plane * ep.idx_planes * ep.V + c : nullptr;
                 out.V = ep.V; out.ndim = ep.ndim;
                 out.dist_only = ep.dist && !ep.sq && !ep.idx;
                 out.coord[0] = c;
                 out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
-                out.init_index_planes();
+                out.init_index_planes(ep);
             }
             if (UNIT && (!FINAL || out.dist_only)) {
                 constexpr int R = 4;
@@ -614,11 +625,11 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
                 out.stride = n0;
                 out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
                 out.sq = ep.sq ? ep.sq + plane * ep.V + c : nullptr;
-                out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+                out.idx = ep.idx ? ep.idx + plane * ep.idx_planes * ep.V + c : nullptr;
                 out.V = ep.V; out.ndim = ep.ndim; out.dist_only = false;
                 out.coord[0] = c;
                 out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
-                out.init_index_planes();
+                out.init_index_planes(ep);
                 emit<1, true, true>(out, y, j, b & 0xffu, small_int_to_float((int)(b >> 16)), none);
             }
         }
@@ -718,12 +729,12 @@ __global__ void __launch_bounds__(512) plane_sampled_kernel(const __grid_constan
     } else {  // two processed axes: the plane is the image
         out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
         out.sq = nullptr;
-        out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+        out.idx = ep.idx ? ep.idx + plane * ep.idx_planes * ep.V + c : nullptr;
         out.V = ep.V; out.ndim = ep.ndim;
         out.dist_only = ep.dist && !ep.idx;
         out.coord[0] = c;
         out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
-        out.init_index_planes();
+        out.init_index_planes(ep);
     }
     for (int y = r0; y < n1; y += rstep)
         scan_voxel<1, FINAL, false, VS, uint8_t>(val + c, dxt + c, VS, n1, y, tab, out);
@@ -791,17 +802,21 @@ __global__ void __launch_bounds__(256) column_kernel(const __grid_constant__ Fas
         const int64_t v0 = i0 + c;
         out.dist = ep.dist ? ep.dist + slab * ep.V + v0 : nullptr;
         out.sq = ep.sq ? ep.sq + slab * ep.V + v0 : nullptr;
-        out.idx = ep.idx ? ep.idx + slab * ep.ndim * ep.V + v0 : nullptr;
+        out.idx = ep.idx ? ep.idx + slab * ep.idx_planes * ep.V + v0 : nullptr;
         out.V = ep.V; out.ndim = ep.ndim;
         out.dist_only = ep.dist && !ep.sq && !ep.idx;
-        int64_t rr = v0;
+        uint32_t rr = (uint32_t)v0;  // a position inside one image: below 2^31
 #pragma unroll
-        for (int q = 0; q < K; ++q) { out.coord[q] = (int)(rr % ep.ext[q]); rr /= ep.ext[q]; }
+        for (int q = 0; q < K; ++q) {
+            const uint32_t nq = (uint32_t)ep.ext[q], hi = rr / nq;
+            out.coord[q] = (int)(rr - hi * nq);
+            rr = hi;
+        }
 #pragma unroll
         for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
-        out.init_index_planes();
+        out.init_index_planes(ep);
     }
-    if (UNIT && (!FINAL || out.dist_only)) {
+    if (UNIT) {
         constexpr int R = 4;
         for (int y0 = r0 * R; y0 < n; y0 += rstep * R) {
             uint32_t best[R];
@@ -942,12 +957,12 @@ __global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant
     } else {  // two processed axes: the plane is the image
         out.dist = ep.dist ? ep.dist + plane * ep.V + c : nullptr;
         out.sq = nullptr;
-        out.idx = ep.idx ? ep.idx + plane * ep.ndim * ep.V + c : nullptr;
+        out.idx = ep.idx ? ep.idx + plane * ep.idx_planes * ep.V + c : nullptr;
         out.V = ep.V; out.ndim = ep.ndim;
         out.dist_only = ep.dist && !ep.idx;
         out.coord[0] = c;
         out.axis[0] = ep.axis[0]; out.axis[1] = ep.axis[1];
-        out.init_index_planes();
+        out.init_index_planes(ep);
     }
     for (int y0 = r0 * R; y0 < n1; y0 += rstep * R) {
         uint32_t best[R];
@@ -1016,15 +1031,19 @@ __global__ void __launch_bounds__(256) column_scaled_kernel(const __grid_constan
         const int64_t v0 = i0 + c;
         out.dist = ep.dist ? ep.dist + slab * ep.V + v0 : nullptr;
         out.sq = nullptr;
-        out.idx = ep.idx ? ep.idx + slab * ep.ndim * ep.V + v0 : nullptr;
+        out.idx = ep.idx ? ep.idx + slab * ep.idx_planes * ep.V + v0 : nullptr;
         out.V = ep.V; out.ndim = ep.ndim;
         out.dist_only = ep.dist && !ep.idx;
-        int64_t rr = v0;
+        uint32_t rr = (uint32_t)v0;  // a position inside one image: below 2^31
 #pragma unroll
-        for (int q = 0; q < K; ++q) { out.coord[q] = (int)(rr % ep.ext[q]); rr /= ep.ext[q]; }
+        for (int q = 0; q < K; ++q) {
+            const uint32_t nq = (uint32_t)ep.ext[q], hi = rr / nq;
+            out.coord[q] = (int)(rr - hi * nq);
+            rr = hi;
+        }
 #pragma unroll
         for (int q = 0; q <= K; ++q) out.axis[q] = ep.axis[q];
-        out.init_index_planes();
+        out.init_index_planes(ep);
     }
     constexpr int R = 4;
     for (int y0 = r0 * R; y0 < n; y0 += rstep * R) {

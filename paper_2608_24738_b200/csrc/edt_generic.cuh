@@ -40,13 +40,15 @@ __device__ __forceinline__ void pass0_store(const Pass0Params& P, const Epilogue
         if (none) {
             if (ep.dist) ep.dist[e] = __int_as_float(0x7f800000);
             if (ep.sq) ep.sq[e] = INT64_MAX;
-            if (ep.idx)
+            if (ep.idx && ep.flat) ep.idx[e] = -1;
+            else if (ep.idx)
                 for (int a = 0; a < ep.ndim; ++a) ep.idx[(line * ep.ndim + a) * ep.V + x] = -1;
         } else {
             const int ao = off < 0 ? -off : off;
             if (ep.dist) ep.dist[e] = (float)(P.w * (double)ao);
             if (ep.sq) ep.sq[e] = (int64_t)ao * ao;
-            if (ep.idx)
+            if (ep.idx && ep.flat) ep.idx[e] = (int64_t)(x + off) * ep.pstride[0];
+            else if (ep.idx)
                 for (int a = 0; a < ep.ndim; ++a)
                     ep.idx[(line * ep.ndim + a) * ep.V + x] = (a == ep.axis[0]) ? (int64_t)(x + off) : 0;
         }

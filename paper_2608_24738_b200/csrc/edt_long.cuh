@@ -359,6 +359,12 @@ __global__ void __launch_bounds__(256) long_axis_kernel(const __grid_constant__ 
                         }
                     }
                     const int64_t vox = p - slab_base;  // voxel index inside the image
+                    if (ep.flat) {
+                        int64_t f = 0;
+#pragma unroll
+                        for (int q = 0; q <= K; ++q) f += (int64_t)site[q] * ep.pstride[q];
+                        ep.idx[slab * ep.V + vox] = none ? -1 : f;
+                    } else
                     for (int a = 0; a < ep.ndim; ++a) {
                         int64_t val = 0;
 #pragma unroll

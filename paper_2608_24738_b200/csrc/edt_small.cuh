@@ -136,7 +136,9 @@ __global__ void __launch_bounds__(kSmallThreads) small_group_kernel(const __grid
             const bool none = best == inf;
             if (ep.dist) ep.dist[g] = __fsqrt_rn(best);
             if (ep.sq) ep.sq[g] = none ? INT64_MAX : (int64_t)best;  // unit sampling: an exact small integer
-            if (SITE) {
+            if (SITE && ep.flat) {
+                ep.idx[g] = none ? -1 : (int64_t)ss[e];  // the carried site index is the linear index inside the image
+            } else if (SITE) {
                 // site = linear index inside the image; planes in processing order, plane 0 fastest
                 const int64_t img = g / P.V, vox = g - img * P.V;
                 int coord[kMaxDims];

@@ -16,6 +16,7 @@
 #include "edt_wide.cuh"
 #include "edt_small.cuh"
 #include "edt_long.cuh"
+#include "edt_compat.cuh"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -60,6 +61,9 @@ struct Plan {
     bool use_double = false;  // arithmetic type of the envelope passes
     bool wide = false;        // int16 offsets instead of int8
     bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    unsigned flags = 0;       // TM_EDT_FLAG_* of the call
+    int64_t shape_sp[kMaxDims];  // spatial extents of the call
+    double w_sp[kMaxDims];       // sampling per spatial axis
     bool long_lines = false;  // two or three axes, extents up to 8192: plain heights scanned through the cache
     bool small = false;       // every extent <= 8: register-resident lines, value (+ site index) carry
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
@@ -194,10 +198,13 @@ static void fill_epilogue(const Plan& pl, float* dist, int64_t* sq, int64_t* idx
         ep.w2[p] = p < pl.E ? pl.w[p] * pl.w[p] : 0.0;
     }
     for (int a = 0; a < kMaxDims; ++a) ep.plane_of_axis[a] = a < pl.ndim ? pl.plane_of_axis[a] : -1;
+    ep.flat = (pl.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : 0;
+    ep.idx_planes = ep.flat ? 1 : pl.ndim;
+    for (int p = 0; p < kMaxDims; ++p) ep.pstride[p] = p < pl.E ? pl.inner[p] : 0;
 }
 
 static double out_bytes_per_voxel(const EpilogueParams& ep) {
-    return (ep.dist ? 4.0 : 0.0) + (ep.sq ? 8.0 : 0.0) + (ep.idx ? 8.0 * ep.ndim : 0.0);
+    return (ep.dist ? 4.0 : 0.0) + (ep.sq ? 8.0 : 0.0) + (ep.idx ? 8.0 * ep.idx_planes : 0.0);
 }
 
 template <typename OT>
@@ -759,15 +766,18 @@ static bool overlap(const void* a, size_t na, const void* b, size_t nb) {
 
 // Argument checks common to every entry point (no CUDA work).
 static int check_call(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
-                      int64_t* out_sq, int64_t* out_idx, Plan& pl) {
+                      int64_t* out_sq, int64_t* out_idx, Plan& pl, unsigned flags = 0) {
     if (!input) return TM_EDT_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(TM_EDT_FLAG_VIRTUAL_BACKGROUND | TM_EDT_FLAG_FLAT_INDEX)) return TM_EDT_ERR_INVALID_ARG;
     const int rc = make_plan(ndim, shape, sampling, pl);
     if (rc != TM_EDT_OK) return rc;
+    pl.flags = flags;
+    for (int a = 0; a < ndim; ++a) { pl.shape_sp[a] = shape[2 + a]; pl.w_sp[a] = sampling ? sampling[a] : 1.0; }
     if (!out_dist && !out_sq && !out_idx) return TM_EDT_ERR_INVALID_ARG;
     if (((uintptr_t)out_dist & 3u) || ((uintptr_t)out_sq & 7u) || ((uintptr_t)out_idx & 7u)) return TM_EDT_ERR_INVALID_ARG;
     if (out_sq && !pl.unit) return TM_EDT_ERR_UNSUPPORTED;
     const size_t N = (size_t)pl.N;
-    const size_t bi = N, bd = N * 4, bs = N * 8, bx = N * 8 * (size_t)ndim;
+    const size_t bi = N, bd = N * 4, bs = N * 8, bx = N * 8 * (size_t)((flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : ndim);
     if (overlap(input, bi, out_dist, bd) || overlap(input, bi, out_sq, bs) || overlap(input, bi, out_idx, bx) ||
         overlap(out_dist, bd, out_sq, bs) || overlap(out_dist, bd, out_idx, bx) || overlap(out_sq, bs, out_idx, bx))
         return TM_EDT_ERR_INVALID_ARG;
@@ -810,7 +820,26 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
         sub.plane_bytes = (((size_t)sub.N * (pl.wide ? 2 : 1)) + 255) & ~(size_t)255;
         const int64_t v0 = first * pl.V;
         cudaError_t e = run_images(sub, input + v0, out_dist ? out_dist + v0 : nullptr, out_sq ? out_sq + v0 : nullptr,
-                                   out_idx ? out_idx + v0 * pl.ndim : nullptr, ws, st, launches);
+                                   out_idx ? out_idx + v0 * ((pl.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : pl.ndim) : nullptr, ws, st,
+                                   launches);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+    }
+    if (pl.flags & TM_EDT_FLAG_VIRTUAL_BACKGROUND) {
+        // images the transform marked as having no background get the virtual-background values
+        VirtualParams VP;
+        memset(&VP, 0, sizeof(VP));
+        VP.images = pl.images; VP.V = pl.V; VP.ndim = pl.ndim;
+        for (int a = 0; a < pl.ndim; ++a) { VP.shape[a] = pl.shape_sp[a]; VP.w[a] = pl.w_sp[a]; }
+        VP.stride0 = pl.V / pl.shape_sp[0];
+        EpilogueParams ep;
+        fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
+        const int64_t max_items = (int64_t)INT32_MAX * 128;  // grid limit with 256 threads per block
+        if (pl.N > max_items) return TM_EDT_ERR_UNSUPPORTED;
+        prof_mark(st, "virtual_background", 0.0);
+        virtual_background_kernel<<<(unsigned)((pl.N + 255) / 256), 256, 0, st>>>(VP, ep);
+        virtual_background_first_kernel<<<(unsigned)((pl.images + 255) / 256), 256, 0, st>>>(VP, ep);
+        launches += 2;
+        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
     }
     g_last_launches = launches;
@@ -857,6 +886,33 @@ int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, const double* s
         (out_indices && !is_device_ptr(out_indices)))
         return TM_EDT_ERR_BAD_POINTER;
     cudaStream_t st = (cudaStream_t)stream;
+    void* ws = nullptr;
+    if (pl.ws_bytes > 0) {
+        cudaError_t e = scratch_alloc(&ws, pl.ws_bytes, st);
+        if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
+    }
+    rc = run_device(pl, input, out_dist, out_sqdist, out_indices, ws, st);
+    if (ws) cudaFreeAsync(ws, st);
+    return rc;
+}
+
+int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+              int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace, size_t workspace_bytes,
+              tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl, flags);
+    if (rc != TM_EDT_OK) return rc;
+    if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (!is_device_ptr(input) || (out_dist && !is_device_ptr(out_dist)) || (out_sqdist && !is_device_ptr(out_sqdist)) ||
+        (out_indices && !is_device_ptr(out_indices)))
+        return TM_EDT_ERR_BAD_POINTER;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (workspace) {
+        if (workspace_bytes < pl.ws_bytes) return TM_EDT_ERR_ALLOC;
+        if (((uintptr_t)workspace & 255u) != 0) return TM_EDT_ERR_INVALID_ARG;
+        if (!is_device_ptr(workspace)) return TM_EDT_ERR_BAD_POINTER;
+        return run_device(pl, input, out_dist, out_sqdist, out_indices, workspace, st);
+    }
     void* ws = nullptr;
     if (pl.ws_bytes > 0) {
         cudaError_t e = scratch_alloc(&ws, pl.ws_bytes, st);
@@ -985,6 +1041,14 @@ int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* shape, const d
                    int64_t* out_sqdist, int64_t* out_indices, void* workspace, size_t workspace_bytes,
                    tm_edt_stream_t stream, int max_kernels, float* kernel_ms, double* kernel_bytes, char* kernel_names,
                    int* n_kernels) {
+    return tm_edt_profile_ex(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, 0u, workspace,
+                             workspace_bytes, stream, max_kernels, kernel_ms, kernel_bytes, kernel_names, n_kernels);
+}
+
+int tm_edt_profile_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
+                      int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace, size_t workspace_bytes,
+                      tm_edt_stream_t stream, int max_kernels, float* kernel_ms, double* kernel_bytes,
+                      char* kernel_names, int* n_kernels) {
     if (!kernel_ms || !n_kernels || max_kernels < 1) return TM_EDT_ERR_INVALID_ARG;
     *n_kernels = 0;
     cudaStream_t st = (cudaStream_t)stream;
@@ -996,8 +1060,10 @@ int tm_edt_profile(const uint8_t* input, int ndim, const int64_t* shape, const d
             return TM_EDT_ERR_CUDA;
         }
     g_prof.active = true;
-    int rc = tm_edt_ws(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, workspace, workspace_bytes,
-                       stream);
+    int rc = flags ? tm_edt_ex(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, flags, workspace,
+                               workspace_bytes, stream)
+                   : tm_edt_ws(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, workspace, workspace_bytes,
+                               stream);
     g_prof.active = false;
     const int cnt = g_prof.count;
     if (rc == TM_EDT_OK && cnt > 0) {

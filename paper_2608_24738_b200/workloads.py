@@ -29,6 +29,7 @@ class Workload:
     want_dist: bool = True
     want_sq: bool = False
     want_idx: bool = False
+    flat_index: bool = False  # index output as one linear index per voxel (a variant, not a benchmark default)
     note: str = ""
     meta: dict = field(default_factory=dict)
 
@@ -42,7 +43,8 @@ class Workload:
 
     def io_bytes(self) -> int:
         """Bytes the call must read and write: 1 per voxel in, 4 (f32) + 8 (i64) + 8*ndim out."""
-        per = 1 + (4 if self.want_dist else 0) + (8 if self.want_sq else 0) + (8 * self.ndim if self.want_idx else 0)
+        nidx = 1 if self.flat_index else self.ndim  # one linear index per voxel, or a coordinate per axis
+        per = 1 + (4 if self.want_dist else 0) + (8 if self.want_sq else 0) + (8 * nidx if self.want_idx else 0)
         return per * self.voxels
 
     def sha256(self) -> str:

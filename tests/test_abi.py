@@ -55,6 +55,19 @@ def test_invalid_arguments_return_before_any_device_work(L):
     assert _call(L, d=0, s=0, x=0) == E.ERR_INVALID_ARG
 
 
+def test_flag_word_of_tm_edt_ex(L):
+    """Unknown flag bits are an argument error; with the flat-index flag the index buffer is one int64 per voxel,
+    which changes the overlap rule between the outputs."""
+    shp = (ctypes.c_int64 * 4)(1, 1, 4, 4)
+    inp, d = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x10000)
+    assert L.tm_edt_ex(inp, 2, shp, None, d, None, None, 4, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt_ex(inp, 2, shp, None, d, None, None, 0x80000000, None, 0, None) == binding.ERR_INVALID_ARG
+    x = ctypes.c_void_p(0x30000)          # 16 voxels: 256 B of coordinate planes, 128 B of flat indices
+    after = ctypes.c_void_p(0x30000 + 128)  # inside the coordinate planes, just behind the flat indices
+    assert L.tm_edt_ex(inp, 2, shp, None, after, None, x, 0, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt_ex(inp, 2, shp, None, after, None, x, binding.FLAG_FLAT_INDEX, None, 0, None) == binding.ERR_BAD_POINTER
+
+
 def test_unsupported(L):
     E = binding
     assert _call(L, shape=(1, 1, E.MAX_EXTENT + 1, 4)) == E.ERR_UNSUPPORTED

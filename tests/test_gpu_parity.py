@@ -107,6 +107,50 @@ def test_extents_up_to_eight(shape, kind):
     full_check(mask, sampling)
 
 
+FLAG_SHAPES = [(2, 1, 7), (2, 1, 300), (2, 1, 6, 5, 4, 7), (2, 1, 40, 36), (2, 1, 12, 20, 24), (2, 2, 6, 10, 12, 8),
+               (2, 1, 140, 150), (2, 1, 1100, 40), (2, 1, 9, 9, 9, 9, 9, 9), (2, 1, 1, 30, 1, 20)]
+
+
+@pytest.mark.parametrize("shape", FLAG_SHAPES, ids=["x".join(map(str, s)) for s in FLAG_SHAPES])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_flags_flat_index_and_virtual_background(shape, kind, path):
+    """tm_edt_ex: one linear site index per voxel instead of coordinate planes, and the virtual-background
+    values for images without background, on every kernel family.  Image 0 has background, image 1 has none."""
+    sampling = _sampling(len(shape) - 2, kind)
+    unit = sampling is None
+    spatial = shape[2:]
+    ndim = len(spatial)
+    mask = workloads.random_mask(zlib.crc32(repr((shape, kind, "flags")).encode()), shape, 0.8)
+    mask[1] = 1
+    mask[0, 0].flat[3 % mask[0, 0].size] = 0
+    ref = oracle.sep(mask, sampling, want_idx=False)
+    stride0 = int(np.prod(spatial[1:]))
+
+    def coords(flat):  # (C, n...) -> (C, ndim, n...)
+        return np.stack(np.unravel_index(flat, spatial), axis=1)
+
+    # flat index only
+    res = run_gpu(mask, sampling, dist=True, sq=unit, idx=True, flat_index=True)
+    assert res["idx"].shape == tuple(shape) and res["idx"].dtype == np.int64
+    compare(mask, sampling, res, ref, True, unit, False)
+    assert (res["idx"][1] == -1).all()
+    checker.check_indices(coords(res["idx"][0])[None], mask[:1], {k: (None if v is None else v[:1]) for k, v in ref.items()},
+                          sampling)
+    # virtual background, coordinate planes
+    vref = oracle.virtual_background(mask, sampling, want_idx=False)
+    res = run_gpu(mask, sampling, dist=True, sq=unit, idx=True, virtual_background=True)
+    checker.check_dist(res["dist"], vref["dist"])
+    if unit:
+        checker.check_sq_exact(res["sq"], vref["sq"])
+    checker.check_indices(res["idx"][:1], mask[:1], {k: (None if v is None else v[:1]) for k, v in ref.items()}, sampling)
+    assert (res["idx"][1][:, 0] == -1).all() and (res["idx"][1][:, 1:] == 0).all()
+    # both flags, index output only
+    res = run_gpu(mask, sampling, dist=False, sq=False, idx=True, virtual_background=True, flat_index=True)
+    assert (res["idx"][1] == -stride0).all()
+    checker.check_indices(coords(res["idx"][0])[None], mask[:1], {k: (None if v is None else v[:1]) for k, v in ref.items()},
+                          sampling)
+
+
 @pytest.mark.parametrize("shape", [(1, 1, 64), (2, 1, 20, 30), (1, 2, 8, 9, 10), (1, 1, 200, 40)])
 def test_degenerate_masks(shape, path):
     ndim = len(shape) - 2

@@ -261,6 +261,33 @@ def test_scipy_black_box_values(shape, samp):
         np.testing.assert_allclose(r["dist"][b, 0], ref, rtol=1e-12, atol=1e-12)
 
 
+@pytest.mark.parametrize("shape,samp", [((7,), None), ((5, 6), None), ((4, 3, 5), (2.5, 0.8, 1.0)),
+                                         ((3, 2, 4, 3), (1.0, 1.5, 0.5, 2.0)), ((2, 3, 2, 2, 3, 2, 2, 3), None)])
+@pytest.mark.parametrize("kind", ["brute", "sep"])
+def test_virtual_background_convention(shape, samp, kind):
+    """Images without background under the virtual out-of-bounds convention (Section 2.3.2): pinned against the
+    closed form d = sqrt((w_0 (x_0 + 1))^2 + sum_{k>=1} (w_k x_k)^2) with indices (-1, 0, .., 0), and against
+    scipy.ndimage, whose convention it is.  Images with background in the same batch stay as they are."""
+    ndi = pytest.importorskip("scipy.ndimage")
+    ndim = len(shape)
+    mask = np.ones((2, 1) + shape, dtype=np.uint8)
+    mask[(1, 0) + tuple(n // 2 for n in shape)] = 0
+    r = oracle.virtual_background(mask, samp, want_idx=True, kind=kind)
+    w = np.ones(ndim) if samp is None else np.asarray(samp, dtype=np.float64)
+    grid = np.meshgrid(*[np.arange(n) for n in shape], indexing="ij")
+    sqf = (w[0] * (grid[0] + 1)) ** 2 + sum((w[k] * grid[k]) ** 2 for k in range(1, ndim))
+    np.testing.assert_allclose(r["dist"][0, 0], np.sqrt(sqf), rtol=1e-13)
+    if samp is None:
+        assert np.array_equal(r["sq"][0, 0], (grid[0] + 1) ** 2 + sum(grid[k] ** 2 for k in range(1, ndim)))
+    assert (r["idx"][0, 0][0] == -1).all() and (r["idx"][0, 0][1:] == 0).all()
+    d_sp, i_sp = ndi.distance_transform_edt(mask[0, 0], sampling=samp, return_indices=True)
+    np.testing.assert_allclose(r["dist"][0, 0], d_sp, rtol=1e-12)
+    assert np.array_equal(r["idx"][0, 0], i_sp)
+    plain = (oracle.brute if kind == "brute" else oracle.sep)(mask, samp)
+    np.testing.assert_array_equal(r["dist"][1, 0], plain["dist"][1, 0])
+    np.testing.assert_array_equal(r["idx"][1, 0], plain["idx"][1, 0])
+
+
 def test_bad_arguments_are_rejected():
     with pytest.raises(RuntimeError):
         oracle.sep(np.ones((1, 1, 3), dtype=np.uint8), (0.0,))
