@@ -1,4 +1,4 @@
-// Extents beyond the 128 of the packed 8-bit entries, two or three processed axes, extents up to 1024.
+// Extents beyond the 128 of the packed 8-bit entries, two to four processed axes, extents up to 1024.
 // Kernels:
 //   row_keys_kernel     first-axis pass, one warp per row, 16 or 32 voxels per lane (128-bit loads; rows that
 //                       are not 16-byte aligned use long_row_any_kernel of edt_long.cuh instead).
@@ -104,20 +104,21 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
 
 // One further axis of the wide path.  The array is viewed as (outer, n, inner); a block takes one slab and
 // a strip of 32 consecutive `inner` positions, stages the keys of its n rows in shared memory and runs the
-// grouped bounded scan.  K = number of 16-bit offsets every voxel carries so far (1 or 2).
+// grouped bounded scan.  K = number of 16-bit offsets every voxel carries so far (1, 2 or 3).
 //   FINAL == false  writes the key of the next pass (value << SH | index of the slab along the next axis)
 //                   and K + 1 offsets per voxel (the chosen site's offsets, fetched from global memory, plus
 //                   the offset along this axis);
 //   FINAL == true   writes distances, squared distances and index planes (the slab is the image).
 struct WideAxisParams {
     const uint32_t* keys_in;   // (outer, n, inner)
-    const int16_t* offs_in;    // (outer, n, inner, K)
+    const int16_t* offs_in;    // (outer, n, inner, K)  -- three offsets are stored as four (8 bytes per voxel)
     uint32_t* keys_out;        // (outer, n, inner), unused when FINAL
     int16_t* offs_out;         // (outer, n, inner, K + 1), unused when FINAL
     int64_t outer, inner;
     int n;
     int next_n;                // extent of the next axis (non-final)
     int n0;                    // extent of the contiguous axis (to split an inner position into coordinates)
+    int n1;                    // extent of the second axis (fourth-axis pass only)
     float w2;                  // squared sampling of this axis (float-height variant)
     int row_parts;             // blocks that share one strip, each taking a contiguous range of its rows
 };
@@ -179,7 +180,9 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     const int64_t col_base = slab_base + c;  // voxel (row 0) of this column
     const uint32_t next_row = FINAL ? 0u : (uint32_t)(slab % P.next_n);
     // own coordinates along the earlier axes (final pass, index output): plane 0 = contiguous axis
-    const int cx = (int)(c % P.n0), cy = (int)(c / P.n0);
+    const int cx = (int)(c % P.n0);
+    const int cyz = (int)(c / P.n0);
+    const int cy = K == 3 ? cyz % P.n1 : cyz, cz = K == 3 ? cyz / P.n1 : 0;
     for (int y0 = y_begin + warp * R; y0 < y_end; y0 += nwarps * R) {
         uint32_t best[R];
         int jrow[R];
@@ -217,6 +220,9 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
                 if (K == 1) {
                     const uint32_t o0 = none ? 0x8000u : (uint32_t)(uint16_t)P.offs_in[pj];
                     reinterpret_cast<uint32_t*>(P.offs_out)[p] = o0 | ((uint32_t)(uint16_t)(int16_t)(j - y) << 16);
+                } else if (K == 2) {
+                    const uint32_t o01 = none ? 0x8000u : reinterpret_cast<const uint32_t*>(P.offs_in)[pj];
+                    reinterpret_cast<uint2*>(P.offs_out)[p] = make_uint2(o01, (uint32_t)(uint16_t)(int16_t)(j - y));
                 }
             } else {
                 const int sq = SH < 0 ? 0 : (int)(b >> (SH < 0 ? 0 : SH));
@@ -226,16 +232,22 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
                 if (ep.sq) ep.sq[p] = none ? INT64_MAX : (int64_t)sq;  // unit sampling only
                 if (ep.idx) {
                     // processed axes in plane order: contiguous axis, (second axis,) this axis; others have extent 1
-                    int site[3] = {0, 0, 0};
+                    int site[4] = {0, 0, 0, 0};
                     if (!none) {
                         if (K == 1) {
                             site[0] = cx + (int)P.offs_in[pj];
                             site[1] = j;
-                        } else {
+                        } else if (K == 2) {
                             const uint32_t o = reinterpret_cast<const uint32_t*>(P.offs_in)[pj];
                             site[0] = cx + (int)(int16_t)(o & 0xffffu);
                             site[1] = cy + (int)(int16_t)(o >> 16);
                             site[2] = j;
+                        } else {
+                            const uint2 o = reinterpret_cast<const uint2*>(P.offs_in)[pj];
+                            site[0] = cx + (int)(int16_t)(o.x & 0xffffu);
+                            site[1] = cy + (int)(int16_t)(o.x >> 16);
+                            site[2] = cz + (int)(int16_t)(o.y & 0xffffu);
+                            site[3] = j;
                         }
                     }
                     const int64_t vox = p - slab_base;  // voxel index inside the image

@@ -147,7 +147,7 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     // "no site" key 2^31 and "no site" plus the largest addend below 2^32
     const double key_scale = nmax > 512 ? 1024.0 : 512.0;
     const bool keys_fit = sumsq * key_scale < 2147483648.0 && (double)(nmax + 4) * (nmax + 4) * key_scale < 2147483648.0;
-    pl.wide_keys = !pl.small && !pl.fast && (E == 2 || E == 3) && nmax <= 1024 && (!pl.unit || keys_fit) &&
+    pl.wide_keys = !pl.small && !pl.fast && E >= 2 && E <= 4 && nmax <= 1024 && (!pl.unit || keys_fit) &&
                    !(force && force[0] == '1');
     pl.long_lines = !pl.small && !pl.fast && !pl.wide_keys && (E == 2 || E == 3) && nmax <= 8192 &&
                     !(force && force[0] == '1');
@@ -155,7 +155,8 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
         const size_t bm = pl.long_lines ? up((size_t)pl.N / 4 + 1024) : 0;  // block minima of the long path
         pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
-        if (E == 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
+        if (E >= 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
+        if (E == 4) pl.ws_bytes += up((size_t)pl.N * 8);                                    // 3 offsets, stored as 4
         pl.ws_bytes += bm;
     }
     if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
@@ -617,30 +618,32 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    int16_t* offsC = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2) + up((size_t)pl.N * 4));
     WideAxisParams A;
     memset(&A, 0, sizeof(A));
-    A.keys_in = keysA; A.offs_in = offsA; A.keys_out = keysB; A.offs_out = offsB;
-    A.n = pl.ext[1]; A.inner = pl.inner[1]; A.outer = pl.N / ((int64_t)pl.ext[1] * pl.inner[1]);
-    A.n0 = pl.ext[0];
-    A.w2 = (float)(pl.w[1] * pl.w[1]);
-    if (pl.E == 2) {
-        prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
-        e = launch_wide_axis<1, true>(A, ep, sh, st);
+    A.n0 = pl.ext[0]; A.n1 = pl.ext[1];
+    // axis k reads what axis k - 1 wrote: keys ping-pong between the two key buffers, offsets grow by one per axis
+    const uint32_t* keys_in[4] = {nullptr, keysA, keysB, keysA};
+    uint32_t* keys_out[4] = {nullptr, keysB, keysA, nullptr};
+    const int16_t* offs_in[4] = {nullptr, offsA, offsB, offsC};
+    int16_t* offs_out[4] = {nullptr, offsB, offsC, nullptr};
+    for (int k = 1; k < pl.E; ++k) {
+        const bool fin = k == pl.E - 1;
+        A.keys_in = keys_in[k]; A.offs_in = offs_in[k];
+        A.keys_out = fin ? nullptr : keys_out[k]; A.offs_out = fin ? nullptr : offs_out[k];
+        A.n = pl.ext[k]; A.inner = pl.inner[k]; A.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+        A.next_n = fin ? 0 : pl.ext[k + 1];
+        A.w2 = (float)(pl.w[k] * pl.w[k]);
+        const double offs_b = k == 3 ? 8.0 : 2.0 * k;  // bytes of offsets per voxel read by this axis
+        if (fin) prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? offs_b : 0.0)));
+        else prof_mark(st, "wide_axis", (double)pl.N * (4.0 + offs_b + 4.0 + (k == 2 ? 8.0 : 4.0)));
+        if (k == 1) e = fin ? launch_wide_axis<1, true>(A, ep, sh, st) : launch_wide_axis<1, false>(A, ep, sh, st);
+        else if (k == 2) e = fin ? launch_wide_axis<2, true>(A, ep, sh, st) : launch_wide_axis<2, false>(A, ep, sh, st);
+        else e = launch_wide_axis<3, true>(A, ep, sh, st);
         ++launches;
-        return e;
+        if (e != cudaSuccess) return e;
     }
-    A.next_n = pl.ext[2];
-    prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 2.0 + 4.0 + 4.0));
-    e = launch_wide_axis<1, false>(A, ep, sh, st);
-    ++launches;
-    if (e != cudaSuccess) return e;
-    A.keys_in = keysB; A.offs_in = offsB; A.keys_out = nullptr; A.offs_out = nullptr;
-    A.n = pl.ext[2]; A.inner = pl.inner[2]; A.outer = pl.N / ((int64_t)pl.ext[2] * pl.inner[2]);
-    A.w2 = (float)(pl.w[2] * pl.w[2]);
-    prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 4.0 : 0.0)));
-    e = launch_wide_axis<2, true>(A, ep, sh, st);
-    ++launches;
-    return e;
+    return cudaSuccess;
 }
 
 // Two or three axes with extents up to 8192: heights and 16-bit offsets per voxel, scans through the cache.

@@ -107,7 +107,7 @@ def test_extents_up_to_eight(shape, kind):
     full_check(mask, sampling)
 
 
-FLAG_SHAPES = [(2, 1, 7), (2, 1, 300), (2, 1, 6, 5, 4, 7), (2, 1, 40, 36), (2, 1, 12, 20, 24), (2, 2, 6, 10, 12, 8),
+FLAG_SHAPES = [(2, 1, 7), (2, 1, 300), (2, 1, 5, 6, 7, 130), (2, 1, 6, 5, 4, 7), (2, 1, 40, 36), (2, 1, 12, 20, 24), (2, 2, 6, 10, 12, 8),
                (2, 1, 140, 150), (2, 1, 1100, 40), (2, 1, 9, 9, 9, 9, 9, 9), (2, 1, 1, 30, 1, 20)]
 
 
@@ -208,7 +208,8 @@ def test_long_lines(n):
 
 LONG = [(1, 1, 1100, 48), (2, 1, 48, 2064), (1, 1, 1040, 1056), (1, 1, 3000, 32), (1, 1, 16, 8192),
         (1, 1, 1100, 16, 32), (1, 2, 6, 1040, 48), (1, 1, 20, 32, 1040),
-        (1, 1, 20, 32, 640), (1, 1, 600, 18, 50), (1, 1, 7, 800, 44), (2, 1, 500, 500), (1, 1, 1000, 999), (1, 1, 150, 150, 150)]
+        (1, 1, 20, 32, 640), (1, 1, 600, 18, 50), (1, 1, 7, 800, 44), (2, 1, 500, 500), (1, 1, 1000, 999), (1, 1, 150, 150, 150),
+        (1, 1, 6, 140, 20, 24), (1, 1, 130, 9, 10, 16), (2, 1, 4, 6, 8, 300), (1, 1, 5, 7, 520, 12)]
 
 
 @pytest.mark.parametrize("shape", LONG, ids=["x".join(map(str, s)) for s in LONG])
