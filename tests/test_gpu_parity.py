@@ -476,3 +476,38 @@ def test_random_shapes_samplings_and_outputs(chunk):
             full_check(mask, samp)
         except AssertionError as exc:  # name the case
             raise AssertionError("shape %r sampling %r p_fg %r seed %r: %s" % (shape, samp, p_fg, seed, exc))
+
+
+def _large_extent_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    big = [130, 131, 150, 257, 300, 500, 513, 1000, 1025, 1100, 2049]
+    small = [1, 2, 3, 5, 8, 12, 16, 17, 33, 40]
+    cases = []
+    while len(cases) < count:
+        ndim = int(rng.integers(2, 5))
+        spatial = [int(rng.choice(small)) for _ in range(ndim)]
+        for pos in rng.choice(ndim, size=int(rng.integers(1, 3)), replace=False):
+            spatial[int(pos)] = int(rng.choice(big))
+        bc = (int(rng.integers(1, 3)), 1)
+        if np.prod(spatial) * bc[0] > 1_500_000:
+            continue
+        kind = int(rng.integers(0, 3))
+        samp = None if kind == 0 else tuple(
+            float(rng.choice([0.5, 0.8, 1.0, 2.5])) if kind == 1 else float(rng.uniform(0.4, 2.5)) for _ in range(ndim))
+        p_fg = float(rng.choice([0.5, 0.9, 0.999]))
+        cases.append((bc + tuple(spatial), samp, p_fg, int(rng.integers(0, 2**31))))
+    return cases
+
+
+@pytest.mark.parametrize("chunk", range(6))
+def test_random_large_extents(chunk):
+    """Seeded fuzzing of the paths beyond extent 128: two to four axes, one or two long axes with odd and aligned
+    lengths in any position, dense to very sparse background."""
+    for shape, samp, p_fg, seed in _large_extent_cases(8, 2000 + chunk):
+        mask = workloads.random_mask(seed, shape, p_fg)
+        if p_fg > 0.99:
+            mask[0, 0].flat[seed % mask[0, 0].size] = 0  # at least one background voxel in the first image
+        try:
+            full_check(mask, samp)
+        except AssertionError as exc:  # name the case
+            raise AssertionError("shape %r sampling %r p_fg %r seed %r: %s" % (shape, samp, p_fg, seed, exc))
