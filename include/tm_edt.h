@@ -102,16 +102,33 @@ TM_EDT_API int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, cons
  *       background, minus the stride of axis 0 under the virtual-background convention).  The paper's index
  *       map has one coordinate per axis; this layout is an extra of this library.
  *
- *   workspace    device scratch of at least tm_edt_workspace_bytes(ndim, shape) bytes, 256-byte aligned, or
- *                NULL to take scratch from the library's memory pool as tm_edt does (workspace_bytes ignored).
+ *   TM_EDT_FLAG_DIST_F64  out_dist is float64 (B, C, n...): the distance to the chosen background voxel,
+ *       recomputed in double precision from its coordinates (exactly rounded under unit sampling).  The transform
+ *       then always produces the site of every voxel (in out_indices if given, else as one linear index per voxel
+ *       in scratch) and a second kernel turns sites into distances: a compatibility path, slower than float32.
+ *
+ *   in_strides   host, ndim + 2 entries, BYTE strides of the mask per array dimension (B, C, n_0 ..), each >= 0,
+ *                or NULL for the contiguous layout.  A non-contiguous mask is first gathered into scratch
+ *                (1 byte per voxel), then transformed: also a compatibility path.
+ *   out_dist     float32, or float64 with TM_EDT_FLAG_DIST_F64 (8-byte aligned).
+ *   workspace    device scratch of at least tm_edt_ex_workspace_bytes(...) bytes for the same arguments, 256-byte
+ *                aligned, or NULL to take scratch from the library's memory pool as tm_edt does (workspace_bytes
+ *                ignored).
  *   Every other argument, the ownership rules and the error behaviour are those of tm_edt; an unknown flag
- *   bit gives TM_EDT_ERR_INVALID_ARG.  With a workspace the call allocates nothing and only enqueues kernels.
+ *   bit or a negative stride gives TM_EDT_ERR_INVALID_ARG.  With a workspace the call allocates nothing and only
+ *   enqueues kernels.
  */
 #define TM_EDT_FLAG_VIRTUAL_BACKGROUND 1u
 #define TM_EDT_FLAG_FLAT_INDEX 2u
-TM_EDT_API int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
-              int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace, size_t workspace_bytes,
-              tm_edt_stream_t stream);
+#define TM_EDT_FLAG_DIST_F64 4u
+TM_EDT_API int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const int64_t* in_strides,
+                         const double* sampling, void* out_dist, int64_t* out_sqdist, int64_t* out_indices,
+                         unsigned flags, void* workspace, size_t workspace_bytes, tm_edt_stream_t stream);
+
+/* Scratch bytes tm_edt_ex needs: those of tm_edt_workspace_bytes, plus the gathered mask for a non-contiguous
+ * input, plus one int64 per voxel for float64 distances without an index output ((size_t)-1 on invalid arguments). */
+TM_EDT_API size_t tm_edt_ex_workspace_bytes(int ndim, const int64_t* shape, const int64_t* in_strides, unsigned flags,
+                                            int with_distances, int with_indices);
 
 /*
  * Scratch bytes tm_edt_ws needs for a call with this geometry (0 for empty problems, and (size_t)-1

@@ -19,7 +19,7 @@ MAX_DIMS = 8
 MAX_EXTENT = 8192
 
 EXPORTS = (
-    "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
+    "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_ex_workspace_bytes", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
 )
 
@@ -48,8 +48,10 @@ def lib() -> ctypes.CDLL:
             L.tm_edt.restype = i
             L.tm_edt_ws.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, sz, vp]
             L.tm_edt_ws.restype = i
-            L.tm_edt_ex.argtypes = [vp, i, vp, vp, vp, vp, vp, ctypes.c_uint, vp, sz, vp]
+            L.tm_edt_ex.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, ctypes.c_uint, vp, sz, vp]
             L.tm_edt_ex.restype = i
+            L.tm_edt_ex_workspace_bytes.argtypes = [i, vp, vp, ctypes.c_uint, i, i]
+            L.tm_edt_ex_workspace_bytes.restype = sz
             L.tm_edt_host.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
             L.tm_edt_host.restype = i
             L.tm_edt_noalloc.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
@@ -128,10 +130,11 @@ def _check(status: int) -> None:
 
 FLAG_VIRTUAL_BACKGROUND = 1
 FLAG_FLAT_INDEX = 2
+FLAG_DIST_F64 = 4
 
 
 def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, device,
-             flat_index=False):
+             flat_index=False, dist_f64=False, keep_strides=False):
     import torch
 
     if mask.dim() < 3:
@@ -140,7 +143,7 @@ def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, di
         mask = mask.view(torch.uint8)
     if mask.dtype != torch.uint8:
         raise TypeError("mask must be uint8 or bool")
-    if not mask.is_contiguous():
+    if not mask.is_contiguous() and not keep_strides:
         mask = mask.contiguous()
     shape = tuple(mask.shape)
     ndim = len(shape) - 2
@@ -158,7 +161,7 @@ def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, di
             torch.empty(shp, dtype=dtype, pin_memory=True) if want else None)
     else:
         mk = lambda want, dtype, shp, buf: out(buf, want, dtype, shp)
-    d = mk(return_distances, torch.float32, shape, distances)
+    d = mk(return_distances, torch.float64 if dist_f64 else torch.float32, shape, distances)
     s = mk(return_sqdist, torch.int64, shape, sqdist)
     x = mk(return_indices, torch.int64, shape if flat_index else shape[:2] + (ndim,) + shape[2:], indices)
     return mask, shape, ndim, d, s, x
@@ -168,29 +171,45 @@ def _p(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
+def tm_edt_ex_workspace_bytes(shape, strides=None, flags=0, with_distances=True, with_indices=False) -> int:
+    """Scratch bytes of a ``tm_edt_ex`` call; ``strides`` are BYTE strides of the (B, C, spatial...) mask or None."""
+    L = lib()
+    st = None if strides is None else (ctypes.c_int64 * len(strides))(*[int(v) for v in strides])
+    n = L.tm_edt_ex_workspace_bytes(len(shape) - 2, _shape_array(shape), st, ctypes.c_uint(flags), int(with_distances),
+                                    int(with_indices))
+    if n == ctypes.c_size_t(-1).value:
+        raise TmEdtError(ERR_INVALID_ARG, "invalid or unsupported shape / strides")
+    return int(n)
+
+
 def tm_edt(mask, sampling=None, return_distances=True, return_indices=False, return_sqdist=False,
            distances=None, indices=None, sqdist=None, workspace=None, stream=None,
-           virtual_background=False, flat_index=False):
+           virtual_background=False, flat_index=False, dist_f64=False, keep_strides=False):
     """Distance transform of a CUDA mask tensor (B, C, spatial...), uint8 or bool.
 
     Returns a dict with the requested tensors among ``dist`` (float32), ``sq`` (int64, unit sampling
     only) and ``idx`` (int64, (B, C, ndim, spatial...)).  With ``workspace`` (a CUDA uint8 tensor of at
     least ``tm_edt_workspace_bytes(mask.shape)`` bytes) the call goes through ``tm_edt_ws`` and allocates
     nothing; otherwise through ``tm_edt``.  Work is enqueued on ``stream`` (default: current stream).
-    ``virtual_background`` / ``flat_index`` select the variants of ``tm_edt_ex``: SciPy's values for images
-    without background, and ``idx`` as one linear index per voxel, shaped like the mask.
+    The remaining keywords select the variants of ``tm_edt_ex``: ``virtual_background`` (SciPy's values for images
+    without background), ``flat_index`` (``idx`` as one linear index per voxel, shaped like the mask), ``dist_f64``
+    (``dist`` as float64) and ``keep_strides`` (a non-contiguous mask is passed with its strides and gathered by
+    the library instead of being made contiguous here).
     """
     L = lib()
     if not mask.is_cuda:
         raise ValueError("mask must be a CUDA tensor (use tm_edt_host for host buffers)")
     mask, shape, ndim, d, s, x = _prepare(
         mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device,
-        flat_index=flat_index)
+        flat_index=flat_index, dist_f64=dist_f64, keep_strides=keep_strides)
     shp, smp, st = _shape_array(shape), _sampling_array(sampling, ndim), _raw_stream(stream)
-    flags = (FLAG_VIRTUAL_BACKGROUND if virtual_background else 0) | (FLAG_FLAT_INDEX if flat_index else 0)
-    if flags:
+    flags = ((FLAG_VIRTUAL_BACKGROUND if virtual_background else 0) | (FLAG_FLAT_INDEX if flat_index else 0)
+             | (FLAG_DIST_F64 if dist_f64 else 0))
+    strided = keep_strides and not mask.is_contiguous()
+    if flags or strided:
         nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-        rc = L.tm_edt_ex(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), ctypes.c_uint(flags), _p(workspace),
+        strides = (ctypes.c_int64 * len(shape))(*[int(v) for v in mask.stride()]) if strided else None
+        rc = L.tm_edt_ex(_p(mask), ndim, shp, strides, smp, _p(d), _p(s), _p(x), ctypes.c_uint(flags), _p(workspace),
                          ctypes.c_size_t(nbytes), st)
     elif workspace is None:
         rc = L.tm_edt(_p(mask), ndim, shp, smp, _p(d), _p(s), _p(x), st)
@@ -280,11 +299,15 @@ class PreparedCall:
         if workspace is None:
             workspace = torch.empty(max(1, need), dtype=torch.uint8, device=mask.device)
         self.ws = workspace
-        head = (_p(self.mask), self.ndim, _shape_array(self.shape), _sampling_array(sampling, self.ndim),
-                _p(self.d), _p(self.s), _p(self.x))
+        shp, smp = _shape_array(self.shape), _sampling_array(sampling, self.ndim)
+        outs = (_p(self.d), _p(self.s), _p(self.x))
         tail = (_p(self.ws), ctypes.c_size_t(self.ws.numel()))
-        self._fn = self._L.tm_edt_ex if self.flags else self._L.tm_edt_ws
-        self._args = head + ((ctypes.c_uint(self.flags),) if self.flags else ()) + tail
+        if self.flags:
+            self._fn = self._L.tm_edt_ex
+            self._args = (_p(self.mask), self.ndim, shp, None, smp) + outs + (ctypes.c_uint(self.flags),) + tail
+        else:
+            self._fn = self._L.tm_edt_ws
+            self._args = (_p(self.mask), self.ndim, shp, smp) + outs + tail
 
     def __call__(self, stream_ptr):
         rc = self._fn(*self._args, stream_ptr)

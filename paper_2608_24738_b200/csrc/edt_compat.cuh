@@ -62,4 +62,78 @@ __global__ void __launch_bounds__(256) virtual_background_first_kernel(const __g
     virtual_fill(P, ep, img, 0);
 }
 
+// Gathers a strided mask (byte strides per array dimension, batch and channel included) into the contiguous
+// row-major layout the transform reads.  dims = ndim + 2.
+struct GatherParams {
+    const uint8_t* in;
+    uint8_t* out;
+    int64_t total;
+    int dims;
+    int64_t shape[kMaxDims + 2];
+    int64_t stride[kMaxDims + 2];
+};
+
+// PER voxels of one row per thread (PER = 4 needs a last extent that is a multiple of 4): one index split, PER
+// loads, one PER-byte store.
+template <int PER>
+__global__ void __launch_bounds__(256) gather_strided_kernel(const __grid_constant__ GatherParams P) {
+    const int64_t e = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * PER;
+    if (e >= P.total) return;
+    int64_t off = 0;
+    if (P.total <= 0xffffffffll) {  // 32-bit index arithmetic whenever the element count allows it
+        uint32_t rr = (uint32_t)e;
+        for (int a = P.dims - 1; a >= 0; --a) {
+            const uint32_t n = (uint32_t)P.shape[a], q = rr / n;
+            off += (int64_t)(rr - q * n) * P.stride[a];
+            rr = q;
+        }
+    } else {
+        int64_t rr = e;
+        for (int a = P.dims - 1; a >= 0; --a) {
+            const int64_t q = rr / P.shape[a];
+            off += (rr - q * P.shape[a]) * P.stride[a];
+            rr = q;
+        }
+    }
+    if (PER == 1) {
+        P.out[e] = P.in[off];
+    } else {
+        const int64_t sl = P.stride[P.dims - 1];
+        uint32_t v = 0;
+#pragma unroll
+        for (int k = 0; k < PER; ++k) v |= (uint32_t)P.in[off + k * sl] << (8 * k);
+        *reinterpret_cast<uint32_t*>(P.out + e) = v;
+    }
+}
+
+// float64 distances, recomputed from the chosen site of every voxel:
+//     d(x) = sqrt( sum_k (w_k (x_k - s_k))^2 )   in double precision
+// (exactly rounded under unit sampling, where the sum is an integer).  The site comes from the index output of
+// the transform: coordinate planes (images, ndim, V) or one linear index per voxel (flat).  A negative linear
+// index, or -1 in the last coordinate plane, marks an image without background (+inf) unless the virtual-background
+// convention is on, where it names the virtual voxel (-1, 0, .., 0).
+__global__ void __launch_bounds__(256) dist_f64_kernel(const __grid_constant__ VirtualParams P, const int64_t* idx,
+                                                       const int flat, const int virtual_bg, double* out) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= P.images * P.V) return;
+    const int64_t img = e / P.V, vox = e - img * P.V;
+    int64_t rr = vox;
+    int64_t fs = flat ? idx[e] : 0;
+    const bool neg = flat ? fs < 0 : idx[(img * P.ndim + (P.ndim - 1)) * P.V + vox] == -1 && !virtual_bg;
+    if (neg && !virtual_bg) { out[e] = __longlong_as_double(0x7ff0000000000000ll); return; }
+    double h = 0.0;
+    for (int a = P.ndim - 1; a >= 0; --a) {
+        const int64_t q = rr / P.shape[a];
+        const int64_t x = rr - q * P.shape[a];
+        rr = q;
+        int64_t sa;
+        if (!flat) sa = idx[(img * P.ndim + a) * P.V + vox];
+        else if (neg) sa = a == 0 ? -1 : 0;
+        else { const int64_t qs = fs / P.shape[a]; sa = fs - qs * P.shape[a]; fs = qs; }
+        const double t = P.w[a] * (double)(x - sa);
+        h += t * t;
+    }
+    out[e] = sqrt(h);
+}
+
 }  // namespace tmedt

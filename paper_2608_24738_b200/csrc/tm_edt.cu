@@ -771,16 +771,18 @@ static bool overlap(const void* a, size_t na, const void* b, size_t nb) {
 static int check_call(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
                       int64_t* out_sq, int64_t* out_idx, Plan& pl, unsigned flags = 0) {
     if (!input) return TM_EDT_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(TM_EDT_FLAG_VIRTUAL_BACKGROUND | TM_EDT_FLAG_FLAT_INDEX)) return TM_EDT_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(TM_EDT_FLAG_VIRTUAL_BACKGROUND | TM_EDT_FLAG_FLAT_INDEX | TM_EDT_FLAG_DIST_F64))
+        return TM_EDT_ERR_INVALID_ARG;
     const int rc = make_plan(ndim, shape, sampling, pl);
     if (rc != TM_EDT_OK) return rc;
     pl.flags = flags;
     for (int a = 0; a < ndim; ++a) { pl.shape_sp[a] = shape[2 + a]; pl.w_sp[a] = sampling ? sampling[a] : 1.0; }
     if (!out_dist && !out_sq && !out_idx) return TM_EDT_ERR_INVALID_ARG;
-    if (((uintptr_t)out_dist & 3u) || ((uintptr_t)out_sq & 7u) || ((uintptr_t)out_idx & 7u)) return TM_EDT_ERR_INVALID_ARG;
+    const bool f64 = (flags & TM_EDT_FLAG_DIST_F64) != 0;
+    if (((uintptr_t)out_dist & (f64 ? 7u : 3u)) || ((uintptr_t)out_sq & 7u) || ((uintptr_t)out_idx & 7u)) return TM_EDT_ERR_INVALID_ARG;
     if (out_sq && !pl.unit) return TM_EDT_ERR_UNSUPPORTED;
     const size_t N = (size_t)pl.N;
-    const size_t bi = N, bd = N * 4, bs = N * 8, bx = N * 8 * (size_t)((flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : ndim);
+    const size_t bi = N, bd = N * (f64 ? 8 : 4), bs = N * 8, bx = N * 8 * (size_t)((flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : ndim);
     if (overlap(input, bi, out_dist, bd) || overlap(input, bi, out_sq, bs) || overlap(input, bi, out_idx, bx) ||
         overlap(out_dist, bd, out_sq, bs) || overlap(out_dist, bd, out_idx, bx) || overlap(out_sq, bs, out_idx, bx))
         return TM_EDT_ERR_INVALID_ARG;
@@ -899,30 +901,127 @@ int tm_edt(const uint8_t* input, int ndim, const int64_t* shape, const double* s
     return rc;
 }
 
-int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
-              int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace, size_t workspace_bytes,
-              tm_edt_stream_t stream) {
+// Contiguous byte strides of (B, C, n...), or the caller's; returns false if a stride is negative.
+static bool resolve_strides(int ndim, const int64_t* shape, const int64_t* in_strides, int64_t* st, bool& strided,
+                            size_t& span) {
+    const int dims = ndim + 2;
+    int64_t c = 1;
+    strided = false;
+    span = 1;
+    for (int a = dims - 1; a >= 0; --a) {
+        st[a] = in_strides ? in_strides[a] : c;
+        if (st[a] < 0) return false;
+        if (shape[a] > 1 && st[a] != c) strided = true;
+        if (shape[a] > 0) span += (size_t)(shape[a] - 1) * (size_t)st[a];
+        c *= shape[a];
+    }
+    return true;
+}
+
+struct ExLayout { size_t core, mask, fidx, total; };
+
+static ExLayout ex_layout(const Plan& pl, bool strided, unsigned flags, bool with_indices, bool with_dist) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    ExLayout L;
+    L.core = up(pl.ws_bytes);
+    L.mask = strided ? up((size_t)pl.N) : 0;
+    L.fidx = ((flags & TM_EDT_FLAG_DIST_F64) && with_dist && !with_indices) ? up((size_t)pl.N * 8) : 0;
+    L.total = L.core + L.mask + L.fidx;
+    if (L.mask == 0 && L.fidx == 0) L.total = pl.ws_bytes;
+    return L;
+}
+
+size_t tm_edt_ex_workspace_bytes(int ndim, const int64_t* shape, const int64_t* in_strides, unsigned flags,
+                                 int with_distances, int with_indices) {
     Plan pl;
-    int rc = check_call(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, pl, flags);
+    if (make_plan(ndim, shape, nullptr, pl) != TM_EDT_OK) return (size_t)-1;
+    int64_t st[kMaxDims + 2];
+    bool strided = false;
+    size_t span = 0;
+    if (!resolve_strides(ndim, shape, in_strides, st, strided, span)) return (size_t)-1;
+    return ex_layout(pl, strided, flags, with_indices != 0, with_distances != 0).total;
+}
+
+int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const int64_t* in_strides, const double* sampling,
+              void* out_dist, int64_t* out_sqdist, int64_t* out_indices, unsigned flags, void* workspace,
+              size_t workspace_bytes, tm_edt_stream_t stream) {
+    Plan pl;
+    int rc = check_call(input, ndim, shape, sampling, static_cast<float*>(out_dist), out_sqdist, out_indices, pl, flags);
     if (rc != TM_EDT_OK) return rc;
+    int64_t strides[kMaxDims + 2];
+    bool strided = false;
+    size_t span = 0;
+    if (!resolve_strides(ndim, shape, in_strides, strides, strided, span)) return TM_EDT_ERR_INVALID_ARG;
     if (pl.N == 0) { g_last_launches = 0; return TM_EDT_OK; }
+    if (strided) {  // the outputs must not overlap the bytes the strided mask spans
+        const size_t N = (size_t)pl.N;
+        if (overlap(input, span, out_dist, N * ((flags & TM_EDT_FLAG_DIST_F64) ? 8 : 4)) || overlap(input, span, out_sqdist, N * 8) ||
+            overlap(input, span, out_indices, N * 8 * (size_t)((flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : ndim)))
+            return TM_EDT_ERR_INVALID_ARG;
+    }
     if (!is_device_ptr(input) || (out_dist && !is_device_ptr(out_dist)) || (out_sqdist && !is_device_ptr(out_sqdist)) ||
         (out_indices && !is_device_ptr(out_indices)))
         return TM_EDT_ERR_BAD_POINTER;
+    const bool f64 = (flags & TM_EDT_FLAG_DIST_F64) && out_dist;
+    const ExLayout L = ex_layout(pl, strided, flags, out_indices != nullptr, out_dist != nullptr);
     cudaStream_t st = (cudaStream_t)stream;
+    char* ws = static_cast<char*>(workspace);
+    bool pooled = false;
     if (workspace) {
-        if (workspace_bytes < pl.ws_bytes) return TM_EDT_ERR_ALLOC;
+        if (workspace_bytes < L.total) return TM_EDT_ERR_ALLOC;
         if (((uintptr_t)workspace & 255u) != 0) return TM_EDT_ERR_INVALID_ARG;
         if (!is_device_ptr(workspace)) return TM_EDT_ERR_BAD_POINTER;
-        return run_device(pl, input, out_dist, out_sqdist, out_indices, workspace, st);
-    }
-    void* ws = nullptr;
-    if (pl.ws_bytes > 0) {
-        cudaError_t e = scratch_alloc(&ws, pl.ws_bytes, st);
+    } else if (L.total > 0) {
+        cudaError_t e = scratch_alloc((void**)&ws, L.total, st);
         if (e != cudaSuccess) { cudaGetLastError(); g_last_cuda_error = (int)e; return TM_EDT_ERR_ALLOC; }
+        pooled = true;
     }
-    rc = run_device(pl, input, out_dist, out_sqdist, out_indices, ws, st);
-    if (ws) cudaFreeAsync(ws, st);
+    int extra_launches = 0;
+    const uint8_t* mask = input;
+    if (strided) {
+        GatherParams G;
+        memset(&G, 0, sizeof(G));
+        G.in = input; G.out = reinterpret_cast<uint8_t*>(ws + L.core); G.total = pl.N; G.dims = ndim + 2;
+        for (int a = 0; a < ndim + 2; ++a) { G.shape[a] = shape[a]; G.stride[a] = strides[a]; }
+        if (pl.N > (int64_t)INT32_MAX * 128) rc = TM_EDT_ERR_UNSUPPORTED;
+        else {
+            prof_mark(st, "gather_strided", (double)pl.N * 2.0);
+            if (shape[ndim + 1] % 4 == 0) gather_strided_kernel<4><<<(unsigned)((pl.N / 4 + 255) / 256), 256, 0, st>>>(G);
+            else gather_strided_kernel<1><<<(unsigned)((pl.N + 255) / 256), 256, 0, st>>>(G);
+            ++extra_launches;
+            mask = G.out;
+        }
+    }
+    if (rc == TM_EDT_OK) {
+        if (!f64) {
+            rc = run_device(pl, mask, static_cast<float*>(out_dist), out_sqdist, out_indices, ws, st);
+        } else {
+            // float64 distances: the transform delivers the site of every voxel (the caller's index output, or one
+            // linear index per voxel in scratch), a second kernel turns sites into distances
+            Plan p2 = pl;
+            int64_t* site = out_indices;
+            if (!site) { site = reinterpret_cast<int64_t*>(ws + L.core + L.mask); p2.flags |= TM_EDT_FLAG_FLAT_INDEX; }
+            rc = run_device(p2, mask, nullptr, out_sqdist, site, ws, st);
+            if (rc == TM_EDT_OK) {
+                if (pl.N > (int64_t)INT32_MAX * 128) rc = TM_EDT_ERR_UNSUPPORTED;
+                else {
+                    VirtualParams VP;
+                    memset(&VP, 0, sizeof(VP));
+                    VP.images = pl.images; VP.V = pl.V; VP.ndim = pl.ndim;
+                    for (int a = 0; a < pl.ndim; ++a) { VP.shape[a] = pl.shape_sp[a]; VP.w[a] = pl.w_sp[a]; }
+                    prof_mark(st, "dist_f64", (double)pl.N * (8.0 + 8.0 * ((p2.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : pl.ndim)));
+                    dist_f64_kernel<<<(unsigned)((pl.N + 255) / 256), 256, 0, st>>>(
+                        VP, site, (p2.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : 0, (flags & TM_EDT_FLAG_VIRTUAL_BACKGROUND) ? 1 : 0,
+                        static_cast<double*>(out_dist));
+                    ++extra_launches;
+                    cudaError_t e = cudaGetLastError();
+                    if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = TM_EDT_ERR_CUDA; }
+                }
+            }
+        }
+    }
+    if (rc == TM_EDT_OK) g_last_launches += extra_launches;
+    if (pooled) cudaFreeAsync(ws, st);
     return rc;
 }
 
@@ -1063,7 +1162,7 @@ int tm_edt_profile_ex(const uint8_t* input, int ndim, const int64_t* shape, cons
             return TM_EDT_ERR_CUDA;
         }
     g_prof.active = true;
-    int rc = flags ? tm_edt_ex(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, flags, workspace,
+    int rc = flags ? tm_edt_ex(input, ndim, shape, nullptr, sampling, out_dist, out_sqdist, out_indices, flags, workspace,
                                workspace_bytes, stream)
                    : tm_edt_ws(input, ndim, shape, sampling, out_dist, out_sqdist, out_indices, workspace, workspace_bytes,
                                stream);

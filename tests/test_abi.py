@@ -60,12 +60,36 @@ def test_flag_word_of_tm_edt_ex(L):
     which changes the overlap rule between the outputs."""
     shp = (ctypes.c_int64 * 4)(1, 1, 4, 4)
     inp, d = ctypes.c_void_p(0x20000), ctypes.c_void_p(0x10000)
-    assert L.tm_edt_ex(inp, 2, shp, None, d, None, None, 4, None, 0, None) == binding.ERR_INVALID_ARG
-    assert L.tm_edt_ex(inp, 2, shp, None, d, None, None, 0x80000000, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt_ex(inp, 2, shp, None, None, d, None, None, 8, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt_ex(inp, 2, shp, None, None, d, None, None, 0x80000000, None, 0, None) == binding.ERR_INVALID_ARG
     x = ctypes.c_void_p(0x30000)          # 16 voxels: 256 B of coordinate planes, 128 B of flat indices
     after = ctypes.c_void_p(0x30000 + 128)  # inside the coordinate planes, just behind the flat indices
-    assert L.tm_edt_ex(inp, 2, shp, None, after, None, x, 0, None, 0, None) == binding.ERR_INVALID_ARG
-    assert L.tm_edt_ex(inp, 2, shp, None, after, None, x, binding.FLAG_FLAT_INDEX, None, 0, None) == binding.ERR_BAD_POINTER
+    assert L.tm_edt_ex(inp, 2, shp, None, None, after, None, x, 0, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tm_edt_ex(inp, 2, shp, None, None, after, None, x, binding.FLAG_FLAT_INDEX, None, 0, None) == binding.ERR_BAD_POINTER
+    # float64 distances: 8-byte alignment and 8 bytes per voxel in the overlap rule
+    assert L.tm_edt_ex(inp, 2, shp, None, None, ctypes.c_void_p(0x10004), None, None, binding.FLAG_DIST_F64, None, 0,
+                       None) == binding.ERR_INVALID_ARG
+    sq = ctypes.c_void_p(0x10000 + 64)   # behind 16 float32 distances, inside 16 float64 ones
+    assert L.tm_edt_ex(inp, 2, shp, None, None, d, sq, None, 0, None, 0, None) == binding.ERR_BAD_POINTER
+    assert L.tm_edt_ex(inp, 2, shp, None, None, d, sq, None, binding.FLAG_DIST_F64, None, 0, None) == binding.ERR_INVALID_ARG
+    # strides: negative ones are rejected; a strided mask must not reach into an output
+    bad = (ctypes.c_int64 * 4)(16, 16, -4, 1)
+    assert L.tm_edt_ex(inp, 2, shp, bad, None, d, None, None, 0, None, 0, None) == binding.ERR_INVALID_ARG
+    wide = (ctypes.c_int64 * 4)(0, 0, 0x4000, 1)  # rows 16 KiB apart: the mask spans 48 KiB + 4 bytes
+    assert L.tm_edt_ex(ctypes.c_void_p(0x8000), 2, shp, wide, None, d, None, None, 0, None, 0, None) == binding.ERR_INVALID_ARG
+
+
+def test_workspace_bytes_of_tm_edt_ex(L):
+    base = binding.tm_edt_workspace_bytes((2, 1, 64, 64, 64))
+    n = 2 * 64 ** 3
+    assert binding.tm_edt_ex_workspace_bytes((2, 1, 64, 64, 64)) == base
+    strides = (64 ** 3 * 2, 64 ** 3 * 2, 64 * 64 * 2, 64 * 2, 2)  # every second byte of a larger buffer
+    assert binding.tm_edt_ex_workspace_bytes((2, 1, 64, 64, 64), strides) >= base + n
+    f64 = binding.tm_edt_ex_workspace_bytes((2, 1, 64, 64, 64), None, binding.FLAG_DIST_F64)
+    assert f64 >= base + 8 * n
+    assert binding.tm_edt_ex_workspace_bytes((2, 1, 64, 64, 64), None, binding.FLAG_DIST_F64, with_indices=True) == base
+    with pytest.raises(binding.TmEdtError):
+        binding.tm_edt_ex_workspace_bytes((1, 1, 4, 4), (16, 16, -4, 1))
 
 
 def test_unsupported(L):

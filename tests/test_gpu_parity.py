@@ -511,3 +511,67 @@ def test_random_large_extents(chunk):
             full_check(mask, samp)
         except AssertionError as exc:  # name the case
             raise AssertionError("shape %r sampling %r p_fg %r seed %r: %s" % (shape, samp, p_fg, seed, exc))
+
+
+F64_SHAPES = [(2, 1, 7), (2, 1, 40, 36), (2, 1, 12, 20, 24), (2, 1, 140, 150), (2, 1, 6, 5, 4, 7), (2, 1, 9, 9, 9, 9, 9, 9)]
+
+
+@pytest.mark.parametrize("shape", F64_SHAPES, ids=["x".join(map(str, s)) for s in F64_SHAPES])
+@pytest.mark.parametrize("kind", ["unit", "sampled"])
+def test_float64_distances(shape, kind):
+    """tm_edt_ex with float64 distances: recomputed in double precision from the chosen site, with the site taken
+    from coordinate planes, from a flat index, or from scratch when no index output is requested.  Unit sampling:
+    the correctly rounded root of the exact squared distance.  Image 1 has no background."""
+    sampling = _sampling(len(shape) - 2, kind)
+    unit = sampling is None
+    mask = workloads.random_mask(zlib.crc32(repr((shape, kind, "f64")).encode()), shape, 0.85)
+    mask[1] = 1
+    mask[0, 0].flat[5 % mask[0, 0].size] = 0
+    ref = oracle.sep(mask, sampling, want_idx=False)
+    vref = oracle.virtual_background(mask, sampling, want_idx=False)
+
+    def check(d, r):
+        assert d.dtype == np.float64 and d.shape == tuple(shape)
+        assert np.array_equal(np.isinf(d), np.isinf(r["dist"]))
+        fin = np.isfinite(d)
+        if unit:
+            assert np.array_equal(d[fin], np.sqrt(r["sq"][fin].astype(np.float64)))
+        else:
+            np.testing.assert_allclose(d[fin], r["dist"][fin], rtol=2e-6, atol=0)
+
+    for idx, flat in ((False, False), (True, False), (True, True)):
+        res = run_gpu(mask, sampling, dist=True, sq=False, idx=idx, dist_f64=True, flat_index=flat)
+        check(res["dist"], ref)
+        res = run_gpu(mask, sampling, dist=True, sq=False, idx=idx, dist_f64=True, flat_index=flat, virtual_background=True)
+        check(res["dist"], vref)
+
+
+def test_strided_masks_are_gathered_by_the_library():
+    """tm_edt_ex with byte strides: permuted, sliced and broadcast views give exactly what their contiguous copies
+    give, and the oracle's values."""
+    import torch
+
+    base = torch.from_numpy(workloads.random_mask(77, (2, 3, 20, 24, 28), 0.9)).cuda()
+    views = [
+        base.permute(0, 1, 4, 2, 3),            # spatial axes permuted
+        base[:, 1:3, ::2, :, 3:19],             # channel range, every second slice, a column range
+        base[:, :1, 5:6].expand(2, 1, 7, 24, 28),  # a broadcast axis (stride 0)
+        base.view(torch.bool)[:, :, :, ::3],    # bool mask, strided
+    ]
+    for v in views:
+        assert not v.is_contiguous()
+        got = binding.tm_edt(v, (1.5, 1.0, 0.5), return_indices=True, keep_strides=True)
+        want = binding.tm_edt(v.contiguous(), (1.5, 1.0, 0.5), return_indices=True)
+        torch.cuda.synchronize()
+        assert torch.equal(got["dist"], want["dist"]) and torch.equal(got["idx"], want["idx"])
+        m = v.contiguous().view(torch.uint8).cpu().numpy()
+        ref = oracle.sep(m, (1.5, 1.0, 0.5), want_idx=False)
+        checker.check_dist(got["dist"].cpu().numpy(), ref["dist"])
+    # with a caller-provided workspace of the size the library reports
+    v = views[0]
+    nbytes = binding.tm_edt_ex_workspace_bytes(tuple(v.shape), tuple(v.stride()))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    got = binding.tm_edt(v, None, return_sqdist=True, keep_strides=True, workspace=ws)
+    want = binding.tm_edt(v.contiguous(), None, return_sqdist=True)
+    torch.cuda.synchronize()
+    assert torch.equal(got["sq"], want["sq"])
