@@ -21,6 +21,7 @@ MAX_EXTENT = 8192
 EXPORTS = (
     "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_ex_workspace_bytes", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
+    "tm_grey_morph", "tm_binary_morph",
 )
 
 _lock = threading.Lock()
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_last_launch_count.restype = i
             L.tm_edt_version.restype = ctypes.c_char_p
             L.tm_edt_trim_memory.restype = i
+            L.tm_grey_morph.argtypes = [vp, i, vp, vp, vp, vp, vp, i, i, ctypes.c_float, vp, vp]
+            L.tm_grey_morph.restype = i
+            L.tm_binary_morph.argtypes = [vp, i, vp, vp, vp, vp, i, i, vp, vp]
+            L.tm_binary_morph.restype = i
             _lib = L
     return _lib
 
@@ -313,3 +318,71 @@ class PreparedCall:
         rc = self._fn(*self._args, stream_ptr)
         if rc != OK:
             _check(rc)
+
+
+MORPH_MODES = {"constant": 0, "reflect": 1, "nearest": 2, "mirror": 3, "wrap": 4}
+
+
+def _element(footprint, ndim):
+    import numpy as np
+
+    fp = np.ascontiguousarray(np.asarray(footprint) != 0, dtype=np.uint8)
+    if fp.ndim != ndim:
+        raise ValueError("the structuring element needs one axis per spatial axis")
+    return fp, (ctypes.c_int64 * ndim)(*fp.shape)
+
+
+def _origin(origin, ndim):
+    return None if origin is None else (ctypes.c_int64 * ndim)(*[int(o) for o in origin])
+
+
+def tm_grey_morph(image, footprint, structure=None, op="erosion", mode="reflect", cval=0.0, origin=None, out=None,
+                  stream=None):
+    """Greyscale erosion or dilation of a CUDA float32 tensor (B, C, spatial...) with scipy.ndimage conventions:
+    ``footprint`` (array-like, one axis per spatial axis) marks the active positions, ``structure`` (same shape,
+    optional) is the additive structuring function, ``mode`` one of constant / reflect / nearest / mirror / wrap."""
+    import numpy as np
+    import torch
+
+    L = lib()
+    if not image.is_cuda or image.dtype != torch.float32 or image.dim() < 3:
+        raise ValueError("image must be a CUDA float32 tensor shaped (B, C, spatial...)")
+    image = image.contiguous()
+    ndim = image.dim() - 2
+    fp, fps = _element(footprint, ndim)
+    st = None
+    if structure is not None:
+        st = np.ascontiguousarray(structure, dtype=np.float32)
+        if st.shape != fp.shape:
+            raise ValueError("structure and footprint differ in shape")
+    if out is None:
+        out = torch.empty_like(image)
+    rc = L.tm_grey_morph(_p(image), ndim, _shape_array(tuple(image.shape)), fp.ctypes.data_as(ctypes.c_void_p),
+                         None if st is None else st.ctypes.data_as(ctypes.c_void_p), fps, _origin(origin, ndim),
+                         {"erosion": 0, "dilation": 1}[op], MORPH_MODES[mode], ctypes.c_float(cval), _p(out),
+                         _raw_stream(stream))
+    _check(rc)
+    return out
+
+
+def tm_binary_morph(mask, structure, op="erosion", border_value=0, origin=None, out=None, stream=None):
+    """Binary erosion or dilation of a CUDA uint8 / bool tensor (B, C, spatial...); returns uint8 holding 0 or 1."""
+    import torch
+
+    L = lib()
+    if not mask.is_cuda or mask.dim() < 3:
+        raise ValueError("mask must be a CUDA tensor shaped (B, C, spatial...)")
+    if mask.dtype == torch.bool:
+        mask = mask.view(torch.uint8)
+    if mask.dtype != torch.uint8:
+        raise TypeError("mask must be uint8 or bool")
+    mask = mask.contiguous()
+    ndim = mask.dim() - 2
+    fp, fps = _element(structure, ndim)
+    if out is None:
+        out = torch.empty_like(mask)
+    rc = L.tm_binary_morph(_p(mask), ndim, _shape_array(tuple(mask.shape)), fp.ctypes.data_as(ctypes.c_void_p), fps,
+                           _origin(origin, ndim), {"erosion": 0, "dilation": 1}[op], int(bool(border_value)), _p(out),
+                           _raw_stream(stream))
+    _check(rc)
+    return out

@@ -17,6 +17,7 @@
 #include "edt_small.cuh"
 #include "edt_long.cuh"
 #include "edt_compat.cuh"
+#include "host_shared.h"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -765,6 +766,14 @@ static bool overlap(const void* a, size_t na, const void* b, size_t nb) {
     if (!a || !b || na == 0 || nb == 0) return false;
     const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
     return a0 < b0 + nb && b0 < a0 + na;
+}
+
+cudaError_t shared_scratch_alloc(void** p, size_t bytes, cudaStream_t st) { return scratch_alloc(p, bytes, st); }
+bool shared_is_device_ptr(const void* p) { return is_device_ptr(p); }
+bool shared_overlap(const void* a, size_t na, const void* b, size_t nb) { return overlap(a, na, b, nb); }
+void shared_record(int cuda_error, int launches) {
+    if (cuda_error >= 0) g_last_cuda_error = cuda_error;
+    g_last_launches = launches;
 }
 
 // Argument checks common to every entry point (no CUDA work).

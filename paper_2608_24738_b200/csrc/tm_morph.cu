@@ -1,0 +1,151 @@
+// tm_morph: host side of the fused erosion / dilation kernel (see include/tm_morph.h and morph.cuh).
+// Flattens the structuring element into its active entries, reflects it for a dilation (with the origin rule of
+// scipy.ndimage for even sizes), computes the per-axis offset extrema for the interior test, copies the entry
+// list to the device and launches one kernel.
+#include <math.h>
+#include <string.h>
+
+#include <vector>
+
+#include "../../include/tm_morph.h"
+#include "host_shared.h"
+#include "morph.cuh"
+
+using namespace tmmorph;
+
+namespace {
+
+struct Geometry {
+    int ndim;
+    int64_t images, V, total;
+    int ext[kMaxDims], stride[kMaxDims];
+};
+
+int check_geometry(int ndim, const int64_t* shape, Geometry& g) {
+    if (ndim < 1 || ndim > kMaxDims || !shape) return TM_EDT_ERR_INVALID_ARG;
+    g.ndim = ndim;
+    if (shape[0] < 0 || shape[1] < 0) return TM_EDT_ERR_INVALID_ARG;
+    g.images = shape[0] * shape[1];
+    g.V = 1;
+    for (int a = 0; a < ndim; ++a) {
+        if (shape[2 + a] < 0) return TM_EDT_ERR_INVALID_ARG;
+        if (shape[2 + a] > 0 && g.V > (int64_t)INT32_MAX / shape[2 + a]) return TM_EDT_ERR_UNSUPPORTED;  // int offsets
+        g.V *= shape[2 + a];
+    }
+    if (g.images > 0 && g.V > 0 && g.images > ((int64_t)1 << 40) / g.V) return TM_EDT_ERR_UNSUPPORTED;
+    g.total = g.images * g.V;
+    int64_t st = 1;
+    for (int a = ndim - 1; a >= 0; --a) {
+        g.ext[a] = (int)shape[2 + a];
+        g.stride[a] = (int)st;
+        st *= shape[2 + a];
+    }
+    return TM_EDT_OK;
+}
+
+// Active entries of the element, for an erosion-style combine out(x) = op_k f(x + k - c).  A dilation is the same
+// combine with the element reflected through its centre and the origin negated (minus one on even sizes).
+int flatten(const Geometry& g, const uint8_t* fp, const float* st, const int64_t* fp_shape, const int64_t* origin,
+            bool reflect, std::vector<Entry>& out, int* lo, int* hi) {
+    if (!fp || !fp_shape) return TM_EDT_ERR_INVALID_ARG;
+    int m[kMaxDims], c[kMaxDims];
+    int64_t count = 1;
+    for (int a = 0; a < g.ndim; ++a) {
+        if (fp_shape[a] < 1 || fp_shape[a] > 255) return TM_EDT_ERR_INVALID_ARG;
+        m[a] = (int)fp_shape[a];
+        int64_t o = origin ? origin[a] : 0;
+        if (reflect) o = -o - (m[a] % 2 == 0 ? 1 : 0);
+        const int64_t centre = m[a] / 2 + o;
+        if (centre < 0 || centre >= m[a]) return TM_EDT_ERR_INVALID_ARG;
+        c[a] = (int)centre;
+        count *= m[a];
+        if (count > (int64_t)1 << 24) return TM_EDT_ERR_UNSUPPORTED;
+        lo[a] = INT32_MAX; hi[a] = INT32_MIN;
+    }
+    int k[kMaxDims] = {0};
+    for (int64_t i = 0; i < count; ++i) {
+        // position k of the (possibly reflected) element <- position m - 1 - k of the caller's array
+        int64_t src = 0;
+        for (int a = 0; a < g.ndim; ++a) src = src * m[a] + (reflect ? m[a] - 1 - k[a] : k[a]);
+        if (fp[src] != 0) {
+            if ((int)out.size() >= TM_MORPH_MAX_ENTRIES) return TM_EDT_ERR_UNSUPPORTED;
+            Entry en;
+            memset(&en, 0, sizeof(en));
+            for (int a = 0; a < g.ndim; ++a) {
+                const int off = k[a] - c[a];
+                en.off[a] = (int16_t)off;
+                en.flat += off * g.stride[a];
+                lo[a] = off < lo[a] ? off : lo[a];
+                hi[a] = off > hi[a] ? off : hi[a];
+            }
+            en.s = st ? st[src] : 0.0f;
+            out.push_back(en);
+        }
+        for (int a = g.ndim - 1; a >= 0; --a) {
+            if (++k[a] < m[a]) break;
+            k[a] = 0;
+        }
+    }
+    return out.empty() ? TM_EDT_ERR_INVALID_ARG : TM_EDT_OK;
+}
+
+template <typename T, bool BINARY>
+int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const float* st, const int64_t* fp_shape,
+        const int64_t* origin, int op, int mode, float cval, int border_value, void* output, tm_edt_stream_t stream) {
+    if (!input || !output) return TM_EDT_ERR_INVALID_ARG;
+    if (op != TM_MORPH_EROSION && op != TM_MORPH_DILATION) return TM_EDT_ERR_INVALID_ARG;
+    if (mode < TM_MORPH_CONSTANT || mode > TM_MORPH_WRAP) return TM_EDT_ERR_INVALID_ARG;
+    Geometry g;
+    int rc = check_geometry(ndim, shape, g);
+    if (rc != TM_EDT_OK) return rc;
+    std::vector<Entry> entries;
+    Params P;
+    memset(&P, 0, sizeof(P));
+    rc = flatten(g, fp, st, fp_shape, origin, op == TM_MORPH_DILATION, entries, P.lo, P.hi);
+    if (rc != TM_EDT_OK) return rc;
+    if (g.total == 0) { tmedt::shared_record(-1, 0); return TM_EDT_OK; }
+    const size_t out_bytes = (size_t)g.total * (BINARY ? 1 : 4);
+    if (tmedt::shared_overlap(input, (size_t)g.total * sizeof(T), output, out_bytes)) return TM_EDT_ERR_INVALID_ARG;
+    if (((uintptr_t)input % sizeof(T)) || ((uintptr_t)output % (BINARY ? 1 : 4))) return TM_EDT_ERR_INVALID_ARG;
+    if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(output)) return TM_EDT_ERR_BAD_POINTER;
+    if (g.total > (int64_t)INT32_MAX * 128) return TM_EDT_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    void* dev = nullptr;
+    const size_t bytes = entries.size() * sizeof(Entry);
+    cudaError_t e = tmedt::shared_scratch_alloc(&dev, bytes, s);
+    if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    e = cudaMemcpyAsync(dev, entries.data(), bytes, cudaMemcpyHostToDevice, s);  // pageable source: consumed on return
+    if (e == cudaSuccess) {
+        P.in = input; P.out = output; P.entries = static_cast<const Entry*>(dev); P.n_entries = (int)entries.size();
+        P.ndim = g.ndim; P.total = g.total; P.V = (int)g.V;
+        for (int a = 0; a < g.ndim; ++a) { P.ext[a] = g.ext[a]; P.stride[a] = g.stride[a]; }
+        P.mode = BINARY ? kConstant : mode;
+        P.cval = cval; P.border_value = border_value ? 1 : 0;
+        const unsigned blocks = (unsigned)((g.total + 255) / 256);
+        if (op == TM_MORPH_EROSION) morph_kernel<T, true, BINARY><<<blocks, 256, 0, s>>>(P);
+        else morph_kernel<T, false, BINARY><<<blocks, 256, 0, s>>>(P);
+        e = cudaGetLastError();
+    }
+    cudaFreeAsync(dev, s);
+    if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
+    tmedt::shared_record(-1, 1);
+    return TM_EDT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tm_grey_morph(const float* input, int ndim, const int64_t* shape, const uint8_t* footprint, const float* structure,
+                  const int64_t* fp_shape, const int64_t* origin, int op, int mode, float cval, float* output,
+                  tm_edt_stream_t stream) {
+    return run<float, false>(input, ndim, shape, footprint, structure, fp_shape, origin, op, mode, cval, 0, output, stream);
+}
+
+int tm_binary_morph(const uint8_t* input, int ndim, const int64_t* shape, const uint8_t* structure, const int64_t* fp_shape,
+                    const int64_t* origin, int op, int border_value, uint8_t* output, tm_edt_stream_t stream) {
+    return run<uint8_t, true>(input, ndim, shape, structure, nullptr, fp_shape, origin, op, TM_MORPH_CONSTANT, 0.0f,
+                              border_value, output, stream);
+}
+
+}  // extern "C"

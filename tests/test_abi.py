@@ -19,8 +19,8 @@ def L():
 
 
 def test_header_symbols_are_exported(L):
-    header = open(os.path.join(ROOT, "include", "tm_edt.h")).read()
-    declared = set(re.findall(r"TM_EDT_API[^;(]*?\b(tm_edt\w*)\s*\(", header))
+    header = open(os.path.join(ROOT, "include", "tm_edt.h")).read() + open(os.path.join(ROOT, "include", "tm_morph.h")).read()
+    declared = set(re.findall(r"TM_EDT_API[^;(]*?\b(tm_\w+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     for name in declared:
         assert hasattr(L, name), name
@@ -148,3 +148,29 @@ def test_binding_refuses_host_tensor():
 
     with pytest.raises(ValueError):
         binding.tm_edt(torch.ones((1, 1, 4, 4), dtype=torch.uint8))
+
+
+def test_morphology_argument_errors(L):
+    """tm_grey_morph / tm_binary_morph reject bad arguments before any device work."""
+    E = binding
+    shp = (ctypes.c_int64 * 4)(1, 1, 8, 8)
+    fps = (ctypes.c_int64 * 2)(3, 3)
+    fp = (ctypes.c_uint8 * 9)(*([1] * 9))
+    a, b = ctypes.c_void_p(0x10000), ctypes.c_void_p(0x20000)
+    ok_args = lambda **kw: dict(dict(inp=a, ndim=2, shape=shp, fp=fp, st=None, fps=fps, org=None, op=0, mode=1, out=b), **kw)
+
+    def grey(**kw):
+        k = ok_args(**kw)
+        return L.tm_grey_morph(k["inp"], k["ndim"], k["shape"], k["fp"], k["st"], k["fps"], k["org"], k["op"], k["mode"],
+                               ctypes.c_float(0.0), k["out"], None)
+
+    assert grey(inp=None) == E.ERR_INVALID_ARG and grey(out=None) == E.ERR_INVALID_ARG
+    assert grey(op=2) == E.ERR_INVALID_ARG and grey(mode=5) == E.ERR_INVALID_ARG and grey(ndim=9) == E.ERR_INVALID_ARG
+    assert grey(fp=(ctypes.c_uint8 * 9)()) == E.ERR_INVALID_ARG                      # no active position
+    assert grey(org=(ctypes.c_int64 * 2)(2, 0)) == E.ERR_INVALID_ARG                 # centre outside the element
+    assert grey(fps=(ctypes.c_int64 * 2)(0, 3)) == E.ERR_INVALID_ARG
+    assert grey(out=ctypes.c_void_p(0x10010)) == E.ERR_INVALID_ARG                   # overlaps the input
+    assert grey(shape=(ctypes.c_int64 * 4)(0, 1, 8, 8)) == E.OK                      # empty: nothing to do
+    assert grey() == E.ERR_BAD_POINTER                                               # all fine but not device memory
+    assert L.tm_binary_morph(a, 2, shp, fp, fps, None, 1, 0, b, None) == E.ERR_BAD_POINTER
+    assert L.tm_binary_morph(a, 2, shp, fp, fps, None, 3, 0, b, None) == E.ERR_INVALID_ARG

@@ -1,0 +1,83 @@
+"""Parity of the fused erosion / dilation kernel (through the C ABI) against the numpy oracle: bit-exact, since
+both sides do one float32 subtraction or addition per active position and exact minima / maxima."""
+import zlib
+
+import numpy as np
+import pytest
+
+from oracle import morph_oracle as mo
+from paper_2608_24738_b200 import binding, buildlib
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    buildlib.build()
+    binding.lib()
+
+
+CASES = [
+    ((2, 2, 37), (3,), None), ((1, 1, 37), (4,), (1,)), ((2, 1, 19, 23), (3, 3), None), ((1, 2, 19, 23), (2, 5), (0, -2)),
+    ((1, 1, 40, 300), (7, 7), None), ((2, 1, 11, 12, 13), (3, 3, 3), None), ((1, 1, 11, 12, 13), (2, 3, 4), (0, -1, 1)),
+    ((1, 1, 5, 6, 4, 7), (3, 2, 3, 3), (0, 0, 1, -1)), ((1, 1, 3, 4), (3, 3), None), ((1, 1, 2, 2, 2), (3, 3, 3), None),
+    ((1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 3, 1, 2, 1, 3, 1, 2), None), ((1, 1, 6, 1, 9), (3, 1, 5), (1, 0, -2)),
+]
+
+
+def _element(fp_shape, seed, density=0.7):
+    rng = np.random.default_rng(seed)
+    fp = rng.random(fp_shape) < density
+    fp.flat[rng.integers(0, fp.size)] = True
+    return fp, rng.normal(size=fp_shape).astype(np.float32)
+
+
+@pytest.mark.parametrize("shape,fp_shape,origin", CASES, ids=["x".join(map(str, c[0])) + "_" + "x".join(map(str, c[1])) for c in CASES])
+@pytest.mark.parametrize("mode", mo.MODES)
+def test_grey_erosion_and_dilation(shape, fp_shape, origin, mode):
+    import torch
+
+    seed = zlib.crc32(repr((shape, fp_shape, mode)).encode())
+    img = np.random.default_rng(seed).normal(size=shape).astype(np.float32)
+    fp, st = _element(fp_shape, seed + 1)
+    t = torch.from_numpy(img).cuda()
+    for structure in (None, st):
+        for op, ref_fn in (("erosion", mo.grey_erosion), ("dilation", mo.grey_dilation)):
+            got = binding.tm_grey_morph(t, fp, structure, op=op, mode=mode, cval=0.25, origin=origin)
+            torch.cuda.synchronize()
+            want = ref_fn(img, fp, structure, mode, 0.25, origin)
+            assert np.array_equal(got.cpu().numpy(), want), (op, structure is not None)
+
+
+@pytest.mark.parametrize("shape,fp_shape,origin", CASES, ids=["x".join(map(str, c[0])) + "_" + "x".join(map(str, c[1])) for c in CASES])
+@pytest.mark.parametrize("border_value", [0, 1])
+def test_binary_erosion_and_dilation(shape, fp_shape, origin, border_value):
+    import torch
+
+    seed = zlib.crc32(repr((shape, fp_shape, border_value)).encode())
+    rng = np.random.default_rng(seed)
+    fp, _ = _element(fp_shape, seed + 1)
+    for density in (0.5, 0.95, 0.05):
+        mask = (rng.random(shape) < density).astype(np.uint8) * rng.integers(1, 255, size=shape).astype(np.uint8)
+        t = torch.from_numpy(mask).cuda()
+        for op, ref_fn in (("erosion", mo.binary_erosion), ("dilation", mo.binary_dilation)):
+            got = binding.tm_binary_morph(t, fp, op=op, border_value=border_value, origin=origin)
+            torch.cuda.synchronize()
+            assert np.array_equal(got.cpu().numpy(), ref_fn(mask, fp, border_value, origin)), op
+
+
+def test_large_volume_against_the_oracle_and_scipy():
+    """A volume of several tiles with a ragged tail (the benchmark's kind of input, smaller): 3^3 ball, all modes."""
+    import torch
+
+    ndi = pytest.importorskip("scipy.ndimage")
+    img = np.random.default_rng(7).normal(size=(2, 1, 70, 81, 93)).astype(np.float32)
+    fp = ndi.generate_binary_structure(3, 1)
+    t = torch.from_numpy(img).cuda()
+    for mode in mo.MODES:
+        got = binding.tm_grey_morph(t, fp, None, op="erosion", mode=mode).cpu().numpy()
+        assert np.array_equal(got, mo.grey_erosion(img, fp, None, mode))
+        assert np.array_equal(got[1, 0], ndi.grey_erosion(img[1, 0], footprint=fp, mode=mode))
+    b = torch.from_numpy((img > 0.5).astype(np.uint8)).cuda()
+    got = binding.tm_binary_morph(b, fp, op="dilation").cpu().numpy()
+    assert np.array_equal(got[0, 0].astype(bool), ndi.binary_dilation(img[0, 0] > 0.5, fp))
