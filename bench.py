@@ -20,6 +20,7 @@ import statistics
 import sys
 import threading
 import time
+import zlib
 
 import numpy as np
 
@@ -296,6 +297,86 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
             "roofline": roofline, "launches_per_step": launches_per_step, "sets": sets}
 
 
+MORPH_CASES = {
+    # name: (image shape (B, C, spatial...), element shape, kind); sizes follow the paper's morphology table (2-D 256^2
+    # and 1024^2 images, batched) plus one 3-D volume; inputs are larger than L2 or rotated over several buffer sets
+    "grey_erosion_2d_1024": ((64, 1, 1024, 1024), (3, 3), "grey"),
+    "grey_dilation_2d_1024": ((64, 1, 1024, 1024), (3, 3), "grey_dilation"),
+    "grey_erosion_2d_256": ((512, 1, 256, 256), (3, 3), "grey"),
+    "grey_erosion_3d_256": ((4, 1, 256, 256, 256), (3, 3, 3), "grey"),
+    "binary_erosion_2d_1024": ((64, 1, 1024, 1024), (3, 3), "binary"),
+    "binary_dilation_2d_1024": ((64, 1, 1024, 1024), (3, 3), "binary_dilation"),
+}
+
+
+def run_morph(args):
+    """Measurement of the fused erosion / dilation kernel (a later row of the scope, not the headline metric):
+    one JSON line with throughput in Gvoxel/s per case, the fraction of the HBM roofline (unavoidable bytes: input +
+    output once) and the numpy oracle timed on a bounded sample."""
+    import numpy as np
+    import torch
+
+    from oracle import morph_oracle as mo
+    from paper_2608_24738_b200 import binding, buildlib
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak_gbs()
+    peak_kind += " copy bandwidth"
+    stream = torch.cuda.current_stream()
+    cases = []
+    for name, (shape, fps, kind) in MORPH_CASES.items():
+        rng = np.random.default_rng(zlib.crc32(name.encode()))
+        binary = kind.startswith("binary")
+        fp = np.ones(fps, dtype=bool)
+        per_voxel = 2 if binary else 8
+        nvox = int(np.prod(shape))
+        sets = max(2, -(-2 * L2_BYTES // (nvox * per_voxel)))
+        if binary:
+            ins = [torch.from_numpy((rng.random(shape) < 0.8).astype(np.uint8)).to(dev) for _ in range(sets)]
+        else:
+            ins = [torch.from_numpy(rng.normal(size=shape).astype(np.float32)).to(dev) for _ in range(sets)]
+        outs = [torch.empty_like(t) for t in ins]
+        op = "dilation" if kind.endswith("dilation") else "erosion"
+        call = (lambda i: binding.tm_binary_morph(ins[i], fp, op=op, out=outs[i])) if binary else (
+            lambda i: binding.tm_grey_morph(ins[i], fp, None, op=op, mode="reflect", out=outs[i]))
+        for i in range(max(3, args.warmup)):
+            call(i % sets)
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        steps = max(10, args.steps // 4)
+        ev0.record(stream)
+        for i in range(steps):
+            call(i % sets)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1) / steps
+        gbs = nvox * per_voxel / (ms * 1e-3) / 1e9
+        # the oracle on one image of the same workload
+        one = ins[0][:1].cpu().numpy()
+        t0 = time.perf_counter()
+        (mo.binary_erosion(one, fp) if binary else mo.grey_erosion(one, fp, None, "reflect")) if op == "erosion" else (
+            mo.binary_dilation(one, fp) if binary else mo.grey_dilation(one, fp, None, "reflect"))
+        cpu_s = time.perf_counter() - t0
+        cases.append({"case": name, "shape": list(shape), "element": list(fps), "ms_per_step": ms,
+                      "value": nvox / (ms * 1e-3) / 1e9, "unit": "Gvoxel/s", "inputs_per_ms": shape[0] * shape[1] / ms,
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                   "peak_kind": peak_kind, "bytes_per_voxel": per_voxel},
+                      "cpu_baseline": {"value": one.size / cpu_s / 1e9, "unit": "Gvoxel/s", "cores": 1, "kind": "oracle",
+                                       "sample": "1 image"},
+                      "l2": "rotating %d buffer sets" % sets})
+    head = cases[0]
+    print(json.dumps({"metric": "morph_gvoxels_per_s", "value": head["value"], "unit": "Gvoxel/s", "n_gpus": 1,
+                      "steps": max(10, args.steps // 4), "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_step"],
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": head["case"], "shape": head["shape"], "element": head["element"]},
+                      "gpu_launches": max(10, args.steps // 4), "roofline": head["roofline"],
+                      "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -313,8 +394,13 @@ def main():
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
     ap.add_argument("--flat-index", action="store_true",
                     help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
+    ap.add_argument("--workload", default="edt", choices=["edt", "morph"],
+                    help="edt: the headline benchmark; morph: the fused erosion / dilation kernel (its own metric)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
+    if args.workload == "morph":
+        run_morph(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()
 

@@ -5,6 +5,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "../../include/tm_morph.h"
@@ -110,6 +111,7 @@ int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const
     if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(output)) return TM_EDT_ERR_BAD_POINTER;
     if (g.total > (int64_t)INT32_MAX * 128) return TM_EDT_ERR_UNSUPPORTED;
     cudaStream_t s = (cudaStream_t)stream;
+    int launches = 0;
     void* dev = nullptr;
     const size_t bytes = entries.size() * sizeof(Entry);
     cudaError_t e = tmedt::shared_scratch_alloc(&dev, bytes, s);
@@ -121,14 +123,54 @@ int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const
         for (int a = 0; a < g.ndim; ++a) { P.ext[a] = g.ext[a]; P.stride[a] = g.stride[a]; }
         P.mode = BINARY ? kConstant : mode;
         P.cval = cval; P.border_value = border_value ? 1 : 0;
-        const unsigned blocks = (unsigned)((g.total + 255) / 256);
-        if (op == TM_MORPH_EROSION) morph_kernel<T, true, BINARY><<<blocks, 256, 0, s>>>(P);
-        else morph_kernel<T, false, BINARY><<<blocks, 256, 0, s>>>(P);
-        e = cudaGetLastError();
+        // four voxels per lane (128 consecutive voxels of a row per warp) when rows are a multiple of that
+        const bool vec = g.ext[g.ndim - 1] % 128 == 0;
+        const int vpt = vec ? 4 : 1;
+        const int64_t threads = (g.total + vpt - 1) / vpt;
+        const unsigned blocks = (unsigned)((threads + 255) / 256);
+        const size_t smem = entries.size() * 8;
+        const bool ero = op == TM_MORPH_EROSION;
+        if (vec) {
+            if (ero) morph_interior_kernel<T, true, BINARY, 4><<<blocks, 256, smem, s>>>(P);
+            else morph_interior_kernel<T, false, BINARY, 4><<<blocks, 256, smem, s>>>(P);
+        } else {
+            if (ero) morph_interior_kernel<T, true, BINARY, 1><<<blocks, 256, smem, s>>>(P);
+            else morph_interior_kernel<T, false, BINARY, 1><<<blocks, 256, smem, s>>>(P);
+        }
+        launches = 1;
+        // border slabs: per axis the voxels that fail the interior test
+        Slabs S;
+        memset(&S, 0, sizeof(S));
+        for (int a = 0; a < g.ndim; ++a) {
+            const int n = g.ext[a], grp = 1;  // the interior kernel tests every voxel by itself
+            const int low_w = std::min(n, ((std::max(0, -P.lo[a]) + grp - 1) / grp) * grp);       // [0, low_w)
+            // first failing group start: the smallest multiple of grp with x0 + grp - 1 + hi >= n
+            const int need = n - std::max(0, P.hi[a]) - (grp - 1);
+            const int high_s = std::max(0, std::min(n, ((std::max(0, need) + grp - 1) / grp) * grp));  // [high_s, n)
+            auto add = [&](int start, int width) {
+                if (width <= 0) return;
+                S.axis[S.count] = a; S.start[S.count] = start; S.width[S.count] = width;
+                S.first[S.count + 1] = S.first[S.count] + g.V / n * width;
+                ++S.count;
+            };
+            if (low_w >= high_s) add(0, n);  // the two slabs meet: the whole axis is border
+            else { add(0, low_w); add(high_s, n - high_s); }
+        }
+        const int64_t items = g.images * S.first[S.count];
+        if (items > 0) {
+            if (items > (int64_t)INT32_MAX * 128) e = cudaErrorInvalidValue;
+            else {
+                const unsigned bb = (unsigned)((items + 255) / 256);
+                if (ero) morph_border_kernel<T, true, BINARY><<<bb, 256, 0, s>>>(P, S, items);
+                else morph_border_kernel<T, false, BINARY><<<bb, 256, 0, s>>>(P, S, items);
+                launches = 2;
+            }
+        }
+        if (e == cudaSuccess) e = cudaGetLastError();
     }
     cudaFreeAsync(dev, s);
     if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
-    tmedt::shared_record(-1, 1);
+    tmedt::shared_record(-1, launches);
     return TM_EDT_OK;
 }
 

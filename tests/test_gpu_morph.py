@@ -22,6 +22,9 @@ CASES = [
     ((1, 1, 40, 300), (7, 7), None), ((2, 1, 11, 12, 13), (3, 3, 3), None), ((1, 1, 11, 12, 13), (2, 3, 4), (0, -1, 1)),
     ((1, 1, 5, 6, 4, 7), (3, 2, 3, 3), (0, 0, 1, -1)), ((1, 1, 3, 4), (3, 3), None), ((1, 1, 2, 2, 2), (3, 3, 3), None),
     ((1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 3, 1, 2, 1, 3, 1, 2), None), ((1, 1, 6, 1, 9), (3, 1, 5), (1, 0, -2)),
+    # last extent a multiple of 128: four voxels per lane in the interior kernel
+    ((2, 1, 5, 128), (3, 3), None), ((1, 2, 3, 4, 256), (3, 3, 3), None), ((1, 1, 130, 384), (5, 4), (-1, 1)),
+    ((3, 1, 128), (7,), (2,)), ((1, 1, 2, 3, 128), (3, 3, 5), (0, 0, -2)),
 ]
 
 
