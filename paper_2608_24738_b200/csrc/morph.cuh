@@ -31,6 +31,7 @@ struct Params {
     int stride[kMaxDims];  // voxel strides inside an image
     int lo[kMaxDims];      // smallest offset per axis over all entries
     int hi[kMaxDims];      // largest offset per axis
+    int64_t flat_lo, flat_hi;  // bounds of the flat offsets: sum_a lo[a] * stride[a], sum_a hi[a] * stride[a]
     int mode;
     float cval;            // greyscale CONSTANT value
     int border_value;      // binary: value outside the image
@@ -62,12 +63,12 @@ __device__ __forceinline__ bool map_coord(int& c, int n, int mode) {
 }
 
 // Interior kernel.  A warp takes 32 * VPT consecutive voxels of a row; lane l owns voxels l, l + 32, .. of them, so
-// that every load and store of the warp is one contiguous 128-byte (float) request.  VPT = 4 needs a last extent
-// that is a multiple of 128; the host falls back to VPT = 1 otherwise.  A voxel whose whole neighbourhood lies
+// that every load and store of the warp is one contiguous 128-byte (float) request.  VPT = 8 or 4 needs a last extent
+// that is a multiple of 256 or 128; the host falls back to VPT = 1 otherwise.  FLAT: every structuring value is 0.  A voxel whose whole neighbourhood lies
 // inside the image adds flat offsets to its linear index and nothing else; the other voxels are left out here:
 // they belong to the border slabs of morph_border_kernel.  The flat offsets and structuring values of the
 // entries are staged in shared memory once per block.
-template <typename T, bool MIN, bool BINARY, int VPT>
+template <typename T, bool MIN, bool BINARY, int VPT, bool FLAT>
 __global__ void __launch_bounds__(256) morph_interior_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(16) unsigned char sm_morph[];
     int* s_flat = reinterpret_cast<int*>(sm_morph);
@@ -129,13 +130,30 @@ __global__ void __launch_bounds__(256) morph_interior_kernel(const __grid_consta
         float acc[VPT];
 #pragma unroll
         for (int j = 0; j < VPT; ++j) acc[j] = MIN ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
+        // Voxels at the ends of a row are not live, but as long as the warp's whole span plus the element's reach
+        // stays inside the tensor their loads are harmless (they read neighbouring rows): the whole warp then
+        // runs one loop without per-voxel tests and only the stores are guarded.
+        const int64_t span0 = warp * (32 * VPT);
+        const bool safe = span0 + P.flat_lo >= 0 && span0 + 32 * VPT - 1 + P.flat_hi < P.total;
+        if (safe) {
 #pragma unroll 4
-        for (int k = 0; k < P.n_entries; ++k) {
-            const T* __restrict__ p = p0 + s_flat[k];
-            const float sv = s_val[k];
+            for (int k = 0; k < P.n_entries; ++k) {
+                const T* __restrict__ p = p0 + s_flat[k];
+                const float sv = FLAT ? 0.f : s_val[k];
 #pragma unroll
-            for (int j = 0; j < VPT; ++j)
-                if (live[j]) acc[j] = MIN ? fminf(acc[j], __fsub_rn((float)p[32 * j], sv)) : fmaxf(acc[j], __fadd_rn((float)p[32 * j], sv));
+                for (int j = 0; j < VPT; ++j) {
+                    const float v = FLAT ? (float)p[32 * j] : (MIN ? __fsub_rn((float)p[32 * j], sv) : __fadd_rn((float)p[32 * j], sv));
+                    acc[j] = MIN ? fminf(acc[j], v) : fmaxf(acc[j], v);
+                }
+            }
+        } else {
+            for (int k = 0; k < P.n_entries; ++k) {
+                const T* __restrict__ p = p0 + s_flat[k];
+                const float sv = FLAT ? 0.f : s_val[k];
+#pragma unroll
+                for (int j = 0; j < VPT; ++j)
+                    if (live[j]) acc[j] = MIN ? fminf(acc[j], __fsub_rn((float)p[32 * j], sv)) : fmaxf(acc[j], __fadd_rn((float)p[32 * j], sv));
+            }
         }
         float* o = static_cast<float*>(P.out) + e;
 #pragma unroll

@@ -121,22 +121,25 @@ int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const
         P.in = input; P.out = output; P.entries = static_cast<const Entry*>(dev); P.n_entries = (int)entries.size();
         P.ndim = g.ndim; P.total = g.total; P.V = (int)g.V;
         for (int a = 0; a < g.ndim; ++a) { P.ext[a] = g.ext[a]; P.stride[a] = g.stride[a]; }
+        for (int a = 0; a < g.ndim; ++a) { P.flat_lo += (int64_t)P.lo[a] * g.stride[a]; P.flat_hi += (int64_t)P.hi[a] * g.stride[a]; }
         P.mode = BINARY ? kConstant : mode;
         P.cval = cval; P.border_value = border_value ? 1 : 0;
-        // four voxels per lane (128 consecutive voxels of a row per warp) when rows are a multiple of that
-        const bool vec = g.ext[g.ndim - 1] % 128 == 0;
-        const int vpt = vec ? 4 : 1;
+        // eight or four voxels per lane (256 or 128 consecutive voxels of a row per warp) when rows are a multiple of that
+        const int vpt = g.ext[g.ndim - 1] % 256 == 0 ? 8 : (g.ext[g.ndim - 1] % 128 == 0 ? 4 : 1);
         const int64_t threads = (g.total + vpt - 1) / vpt;
         const unsigned blocks = (unsigned)((threads + 255) / 256);
         const size_t smem = entries.size() * 8;
         const bool ero = op == TM_MORPH_EROSION;
-        if (vec) {
-            if (ero) morph_interior_kernel<T, true, BINARY, 4><<<blocks, 256, smem, s>>>(P);
-            else morph_interior_kernel<T, false, BINARY, 4><<<blocks, 256, smem, s>>>(P);
-        } else {
-            if (ero) morph_interior_kernel<T, true, BINARY, 1><<<blocks, 256, smem, s>>>(P);
-            else morph_interior_kernel<T, false, BINARY, 1><<<blocks, 256, smem, s>>>(P);
-        }
+        bool flat = true;
+        for (const Entry& en : entries) flat = flat && en.s == 0.0f;
+#define TM_MORPH_LAUNCH(V, F)                                                                                    \
+    do {                                                                                                         \
+        if (ero) morph_interior_kernel<T, true, BINARY, V, F><<<blocks, 256, smem, s>>>(P);                       \
+        else morph_interior_kernel<T, false, BINARY, V, F><<<blocks, 256, smem, s>>>(P);                          \
+    } while (0)
+        if (BINARY || flat) { if (vpt == 8) TM_MORPH_LAUNCH(8, true); else if (vpt == 4) TM_MORPH_LAUNCH(4, true); else TM_MORPH_LAUNCH(1, true); }
+        else { if (vpt == 8) TM_MORPH_LAUNCH(8, false); else if (vpt == 4) TM_MORPH_LAUNCH(4, false); else TM_MORPH_LAUNCH(1, false); }
+#undef TM_MORPH_LAUNCH
         launches = 1;
         // border slabs: per axis the voxels that fail the interior test
         Slabs S;
