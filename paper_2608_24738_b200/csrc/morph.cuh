@@ -108,31 +108,44 @@ __global__ void __launch_bounds__(256) morph_interior_kernel(const __grid_consta
         if (!any) return;
     }
     const T* __restrict__ p0 = static_cast<const T*>(P.in) + e;
+    // Voxels at the ends of a row are not live, but as long as the warp's whole span plus the element's reach stays
+    // inside the tensor their loads are harmless (they read neighbouring rows): the whole warp then runs one loop
+    // without per-voxel tests and only the stores are guarded ("safe" below).
     if (BINARY) {
-        int bacc[VPT];
-        int open = 0;  // voxels whose result is not decided yet
+        const int64_t span0 = warp * (32 * VPT);
+        const bool safe = span0 + P.flat_lo >= 0 && span0 + 32 * VPT - 1 + P.flat_hi < P.total;
+        // bit j of `acc`: running AND (erosion) or OR (dilation) of voxel j; a lane stops once all its voxels are decided
+        unsigned acc = MIN ? (1u << VPT) - 1u : 0u;
+        unsigned lv = 0;
 #pragma unroll
-        for (int j = 0; j < VPT; ++j) { bacc[j] = MIN ? 1 : 0; open |= live[j] ? 1 << j : 0; }
-        for (int k = 0; k < P.n_entries && open; ++k) {
-            const T* __restrict__ p = p0 + s_flat[k];
+        for (int j = 0; j < VPT; ++j) lv |= live[j] ? 1u << j : 0u;
+        if (safe) {
+            for (int k = 0; k < P.n_entries; ++k) {
+                const T* __restrict__ p = p0 + s_flat[k];
+                unsigned v = 0;
 #pragma unroll
-            for (int j = 0; j < VPT; ++j) {
-                if (!((open >> j) & 1)) continue;
-                const int v = p[32 * j] != 0;
-                if (MIN ? !v : v) { bacc[j] = v; open &= ~(1 << j); }
+                for (int j = 0; j < VPT; ++j) v |= (p[32 * j] != 0 ? 1u : 0u) << j;
+                acc = MIN ? acc & v : acc | v;
+                if (acc == (MIN ? 0u : (1u << VPT) - 1u)) break;
+            }
+        } else {
+            for (int k = 0; k < P.n_entries; ++k) {
+                const T* __restrict__ p = p0 + s_flat[k];
+                unsigned v = MIN ? (1u << VPT) - 1u : 0u;
+#pragma unroll
+                for (int j = 0; j < VPT; ++j)
+                    if (live[j]) v = (v & ~(1u << j)) | ((p[32 * j] != 0 ? 1u : 0u) << j);
+                acc = MIN ? acc & v : acc | v;
             }
         }
         uint8_t* o = static_cast<uint8_t*>(P.out) + e;
 #pragma unroll
         for (int j = 0; j < VPT; ++j)
-            if (live[j]) o[32 * j] = (uint8_t)bacc[j];
+            if ((lv >> j) & 1u) o[32 * j] = (uint8_t)((acc >> j) & 1u);
     } else {
         float acc[VPT];
 #pragma unroll
         for (int j = 0; j < VPT; ++j) acc[j] = MIN ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
-        // Voxels at the ends of a row are not live, but as long as the warp's whole span plus the element's reach
-        // stays inside the tensor their loads are harmless (they read neighbouring rows): the whole warp then
-        // runs one loop without per-voxel tests and only the stores are guarded.
         const int64_t span0 = warp * (32 * VPT);
         const bool safe = span0 + P.flat_lo >= 0 && span0 + 32 * VPT - 1 + P.flat_hi < P.total;
         if (safe) {
