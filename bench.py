@@ -329,6 +329,8 @@ def run_morph(args):
     stream = torch.cuda.current_stream()
     cases = []
     for name, (shape, fps, kind) in MORPH_CASES.items():
+        if args.morph_case and name != args.morph_case:
+            continue
         rng = np.random.default_rng(zlib.crc32(name.encode()))
         binary = kind.startswith("binary")
         fp = np.ones(fps, dtype=bool)
@@ -396,6 +398,7 @@ def main():
                     help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
     ap.add_argument("--workload", default="edt", choices=["edt", "morph"],
                     help="edt: the headline benchmark; morph: the fused erosion / dilation kernel (its own metric)")
+    ap.add_argument("--morph-case", default=None, help="with --workload morph: run only this case (profiling aid)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
     if args.workload == "morph":
