@@ -21,7 +21,7 @@ MAX_EXTENT = 8192
 EXPORTS = (
     "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_ex_workspace_bytes", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
-    "tm_grey_morph", "tm_binary_morph",
+    "tm_grey_morph", "tm_binary_morph", "tm_cdt", "tm_bfdt",
 )
 
 _lock = threading.Lock()
@@ -74,6 +74,10 @@ def lib() -> ctypes.CDLL:
             L.tm_grey_morph.restype = i
             L.tm_binary_morph.argtypes = [vp, i, vp, vp, vp, vp, i, i, vp, vp]
             L.tm_binary_morph.restype = i
+            L.tm_cdt.argtypes = [vp, i, vp, i, vp, vp]
+            L.tm_cdt.restype = i
+            L.tm_bfdt.argtypes = [vp, i, vp, vp, i, vp, vp]
+            L.tm_bfdt.restype = i
             _lib = L
     return _lib
 
@@ -385,4 +389,46 @@ def tm_binary_morph(mask, structure, op="erosion", border_value=0, origin=None, 
                            _origin(origin, ndim), {"erosion": 0, "dilation": 1}[op], int(bool(border_value)), _p(out),
                            _raw_stream(stream))
     _check(rc)
+    return out
+
+
+METRICS = {"euclidean": 0, "taxicab": 1, "chessboard": 2}
+
+
+def _mask_u8(mask):
+    import torch
+
+    if not mask.is_cuda or mask.dim() < 3:
+        raise ValueError("mask must be a CUDA tensor shaped (B, C, spatial...)")
+    if mask.dtype == torch.bool:
+        mask = mask.view(torch.uint8)
+    if mask.dtype != torch.uint8:
+        raise TypeError("mask must be uint8 or bool")
+    return mask.contiguous()
+
+
+def tm_cdt(mask, metric="chessboard", out=None, stream=None):
+    """Taxicab or chessboard distance transform (int32, -1 for an image without background), the values of
+    scipy.ndimage.distance_transform_cdt."""
+    import torch
+
+    L = lib()
+    mask = _mask_u8(mask)
+    if out is None:
+        out = torch.empty(mask.shape, dtype=torch.int32, device=mask.device)
+    _check(L.tm_cdt(_p(mask), mask.dim() - 2, _shape_array(tuple(mask.shape)), METRICS[metric], _p(out), _raw_stream(stream)))
+    return out
+
+
+def tm_bfdt(mask, sampling=None, metric="euclidean", out=None, stream=None):
+    """Brute-force distance transform (float32): every voxel against every background voxel; ranks 1..4."""
+    import torch
+
+    L = lib()
+    mask = _mask_u8(mask)
+    ndim = mask.dim() - 2
+    if out is None:
+        out = torch.empty(mask.shape, dtype=torch.float32, device=mask.device)
+    _check(L.tm_bfdt(_p(mask), ndim, _shape_array(tuple(mask.shape)), _sampling_array(sampling, ndim), METRICS[metric],
+                     _p(out), _raw_stream(stream)))
     return out

@@ -1,0 +1,131 @@
+// tm_cdt / tm_bfdt: host side (see include/tm_cdt.h and cdt.cuh).
+#include <math.h>
+#include <string.h>
+
+#include "../../include/tm_cdt.h"
+#include "cdt.cuh"
+#include "host_shared.h"
+
+using namespace tmcdt;
+
+namespace {
+
+struct Geo { int ndim; int64_t images, V, total; int64_t ext[8]; };
+
+int geometry(int ndim, const int64_t* shape, int max_ndim, Geo& g) {
+    if (ndim < 1 || ndim > max_ndim || !shape) return TM_EDT_ERR_INVALID_ARG;
+    if (shape[0] < 0 || shape[1] < 0) return TM_EDT_ERR_INVALID_ARG;
+    g.ndim = ndim; g.images = shape[0] * shape[1]; g.V = 1;
+    for (int a = 0; a < ndim; ++a) {
+        if (shape[2 + a] < 0) return TM_EDT_ERR_INVALID_ARG;
+        if (shape[2 + a] > 0 && g.V > (int64_t)INT32_MAX / shape[2 + a]) return TM_EDT_ERR_UNSUPPORTED;
+        g.V *= shape[2 + a];
+        g.ext[a] = shape[2 + a];
+    }
+    if (g.images > 0 && g.V > 0 && g.images > ((int64_t)1 << 40) / g.V) return TM_EDT_ERR_UNSUPPORTED;
+    g.total = g.images * g.V;
+    return TM_EDT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int32_t* out_dist, tm_edt_stream_t stream) {
+    if (!input || !out_dist) return TM_EDT_ERR_INVALID_ARG;
+    if (metric != TM_METRIC_TAXICAB && metric != TM_METRIC_CHESSBOARD) return TM_EDT_ERR_INVALID_ARG;
+    Geo g;
+    int rc = geometry(ndim, shape, 8, g);
+    if (rc != TM_EDT_OK) return rc;
+    if (g.total == 0) { tmedt::shared_record(-1, 0); return TM_EDT_OK; }
+    if ((uintptr_t)out_dist & 3u) return TM_EDT_ERR_INVALID_ARG;
+    if (tmedt::shared_overlap(input, (size_t)g.total, out_dist, (size_t)g.total * 4)) return TM_EDT_ERR_INVALID_ARG;
+    if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(out_dist)) return TM_EDT_ERR_BAD_POINTER;
+    if (g.total > (int64_t)INT32_MAX * 128) return TM_EDT_ERR_UNSUPPORTED;
+    // axes with more than one voxel, contiguous axis first; an image of one voxel keeps its last axis
+    int axes[8], E = 0;
+    for (int a = ndim - 1; a >= 0; --a)
+        if (g.ext[a] > 1) axes[E++] = a;
+    if (E == 0) axes[E++] = ndim - 1;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t buf = (((size_t)g.total * 4) + 255) & ~(size_t)255;
+    char* ws = nullptr;
+    if (E > 1) {
+        cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, (E > 2 ? 2 : 1) * buf, st);
+        if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    }
+    int32_t* tmp[2] = {reinterpret_cast<int32_t*>(ws), reinterpret_cast<int32_t*>(ws + buf)};
+    const int32_t* prev = nullptr;
+    cudaError_t e = cudaSuccess;
+    for (int k = 0; k < E && e == cudaSuccess; ++k) {
+        PassParams P;
+        memset(&P, 0, sizeof(P));
+        P.mask = input; P.in = prev; P.total = g.total;
+        P.first = k == 0; P.last = k == E - 1;
+        P.out = P.last ? out_dist : tmp[k & 1];
+        P.n = (int)g.ext[axes[k]];
+        P.inner = 1;
+        for (int a = axes[k] + 1; a < ndim; ++a) P.inner *= g.ext[a];
+        const unsigned blocks = (unsigned)((g.total + 255) / 256);
+        if (metric == TM_METRIC_CHESSBOARD) cdt_axis_kernel<true><<<blocks, 256, 0, st>>>(P);
+        else cdt_axis_kernel<false><<<blocks, 256, 0, st>>>(P);
+        e = cudaGetLastError();
+        prev = P.out;
+    }
+    if (ws) cudaFreeAsync(ws, st);
+    if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
+    tmedt::shared_record(-1, E);
+    return TM_EDT_OK;
+}
+
+int tm_bfdt(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, int metric, float* out_dist,
+            tm_edt_stream_t stream) {
+    if (!input || !out_dist) return TM_EDT_ERR_INVALID_ARG;
+    if (metric < TM_METRIC_EUCLIDEAN || metric > TM_METRIC_CHESSBOARD) return TM_EDT_ERR_INVALID_ARG;
+    Geo g;
+    int rc = geometry(ndim, shape, 4, g);
+    if (rc != TM_EDT_OK) return rc == TM_EDT_ERR_INVALID_ARG && ndim > 4 && ndim <= 8 ? TM_EDT_ERR_UNSUPPORTED : rc;
+    BruteParams P;
+    memset(&P, 0, sizeof(P));
+    for (int a = 0; a < ndim; ++a) {
+        const double w = sampling ? sampling[a] : 1.0;
+        if (!(w > 0.0) || !isfinite(w)) return TM_EDT_ERR_INVALID_ARG;
+        P.w[a] = (float)w;
+        P.ext[a] = (int)g.ext[a];
+    }
+    if (g.total == 0) { tmedt::shared_record(-1, 0); return TM_EDT_OK; }
+    if (g.V > (1 << 24) || g.images > 65535) return TM_EDT_ERR_UNSUPPORTED;
+    if ((uintptr_t)out_dist & 3u) return TM_EDT_ERR_INVALID_ARG;
+    if (tmedt::shared_overlap(input, (size_t)g.total, out_dist, (size_t)g.total * 4)) return TM_EDT_ERR_INVALID_ARG;
+    if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(out_dist)) return TM_EDT_ERR_BAD_POINTER;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t b_sites = (((size_t)g.total * 4) + 255) & ~(size_t)255, b_counts = (((size_t)g.images * 4) + 255) & ~(size_t)255;
+    char* ws = nullptr;
+    cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, b_sites + b_counts, st);
+    if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    int32_t* sites = reinterpret_cast<int32_t*>(ws);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + b_sites);
+    e = cudaMemsetAsync(counts, 0, (size_t)g.images * 4, st);
+    if (e == cudaSuccess) {
+        collect_background_kernel<<<(unsigned)((g.total + 255) / 256), 256, 0, st>>>(input, sites, counts, g.total, (int)g.V);
+        P.mask = input; P.sites = sites; P.counts = counts; P.out = out_dist; P.V = (int)g.V;
+        const dim3 grid((unsigned)((g.V + 255) / 256), (unsigned)g.images);
+#define TM_BRUTE(M, R) brute_kernel<M, R><<<grid, 256, 0, st>>>(P)
+#define TM_BRUTE_RANK(M)                                                                              \
+    do {                                                                                              \
+        if (ndim == 1) TM_BRUTE(M, 1); else if (ndim == 2) TM_BRUTE(M, 2); else if (ndim == 3) TM_BRUTE(M, 3); else TM_BRUTE(M, 4); \
+    } while (0)
+        if (metric == TM_METRIC_EUCLIDEAN) TM_BRUTE_RANK(0);
+        else if (metric == TM_METRIC_TAXICAB) TM_BRUTE_RANK(1);
+        else TM_BRUTE_RANK(2);
+#undef TM_BRUTE_RANK
+#undef TM_BRUTE
+        e = cudaGetLastError();
+    }
+    cudaFreeAsync(ws, st);
+    if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
+    tmedt::shared_record(-1, 2);
+    return TM_EDT_OK;
+}
+
+}  // extern "C"

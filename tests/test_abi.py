@@ -19,7 +19,7 @@ def L():
 
 
 def test_header_symbols_are_exported(L):
-    header = open(os.path.join(ROOT, "include", "tm_edt.h")).read() + open(os.path.join(ROOT, "include", "tm_morph.h")).read()
+    header = open(os.path.join(ROOT, "include", "tm_edt.h")).read() + open(os.path.join(ROOT, "include", "tm_morph.h")).read() + open(os.path.join(ROOT, "include", "tm_cdt.h")).read()
     declared = set(re.findall(r"TM_EDT_API[^;(]*?\b(tm_\w+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     for name in declared:
@@ -174,3 +174,20 @@ def test_morphology_argument_errors(L):
     assert grey() == E.ERR_BAD_POINTER                                               # all fine but not device memory
     assert L.tm_binary_morph(a, 2, shp, fp, fps, None, 1, 0, b, None) == E.ERR_BAD_POINTER
     assert L.tm_binary_morph(a, 2, shp, fp, fps, None, 3, 0, b, None) == E.ERR_INVALID_ARG
+
+
+def test_cdt_and_brute_force_argument_errors(L):
+    E = binding
+    shp = (ctypes.c_int64 * 4)(1, 1, 8, 8)
+    a, b = ctypes.c_void_p(0x10000), ctypes.c_void_p(0x20000)
+    assert L.tm_cdt(a, 2, shp, 0, b, None) == E.ERR_INVALID_ARG          # the Euclidean metric is tm_edt's
+    assert L.tm_cdt(a, 2, shp, 3, b, None) == E.ERR_INVALID_ARG
+    assert L.tm_cdt(None, 2, shp, 1, b, None) == E.ERR_INVALID_ARG
+    assert L.tm_cdt(a, 2, shp, 1, ctypes.c_void_p(0x10020), None) == E.ERR_INVALID_ARG   # overlaps the mask
+    assert L.tm_cdt(a, 2, (ctypes.c_int64 * 4)(1, 0, 8, 8), 1, b, None) == E.OK
+    assert L.tm_cdt(a, 2, shp, 1, b, None) == E.ERR_BAD_POINTER
+    assert L.tm_bfdt(a, 2, shp, None, 3, b, None) == E.ERR_INVALID_ARG
+    assert L.tm_bfdt(a, 2, shp, (ctypes.c_double * 2)(1.0, -1.0), 0, b, None) == E.ERR_INVALID_ARG
+    assert L.tm_bfdt(a, 5, (ctypes.c_int64 * 7)(1, 1, 2, 2, 2, 2, 2), None, 0, b, None) == E.ERR_UNSUPPORTED
+    assert L.tm_bfdt(a, 2, (ctypes.c_int64 * 4)(1, 1, 8192, 4096), None, 0, b, None) == E.ERR_UNSUPPORTED  # > 2^24 voxels
+    assert L.tm_bfdt(a, 2, shp, None, 2, b, None) == E.ERR_BAD_POINTER

@@ -1,0 +1,86 @@
+"""Parity of tm_cdt (bit-exact int32) and tm_bfdt (float32, relative 1e-5) against their oracles."""
+import zlib
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import cdt_oracle as co
+from paper_2608_24738_b200 import binding, buildlib, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    buildlib.build()
+    binding.lib()
+
+
+SHAPES = [(2, 2, 1), (3, 1, 37), (2, 1, 19, 23), (1, 2, 40, 300), (1, 1, 1, 50, 1), (2, 1, 11, 12, 13), (1, 1, 5, 6, 4, 7),
+          (1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 1, 260, 130), (1, 1, 6, 200, 33)]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=["x".join(map(str, s)) for s in SHAPES])
+@pytest.mark.parametrize("metric", ["taxicab", "chessboard"])
+def test_cdt_matches_the_oracle(shape, metric):
+    import torch
+
+    for p_fg in (0.3, 0.9, 0.999):
+        mask = workloads.random_mask(zlib.crc32(repr((shape, metric, p_fg)).encode()), shape, p_fg)
+        if shape[0] > 1:
+            mask[-1, -1] = 1  # an image without background
+        if p_fg > 0.99:
+            mask[0, 0].flat[7 % mask[0, 0].size] = 0
+        got = binding.tm_cdt(torch.from_numpy(mask).cuda(), metric)
+        torch.cuda.synchronize()
+        assert got.dtype == torch.int32
+        assert np.array_equal(got.cpu().numpy(), co.separable(mask, metric)), p_fg
+
+
+def test_cdt_matches_scipy_on_a_larger_image():
+    import torch
+
+    ndi = pytest.importorskip("scipy.ndimage")
+    w = workloads.config2()
+    mask = w.mask[:2]
+    t = torch.from_numpy(mask).cuda()
+    for metric in ("taxicab", "chessboard"):
+        got = binding.tm_cdt(t, metric).cpu().numpy()
+        for b in range(2):
+            assert np.array_equal(got[b, 0], ndi.distance_transform_cdt(mask[b, 0], metric=metric))
+
+
+BF_SHAPES = [(2, 1, 40), (2, 2, 17, 23), (1, 1, 9, 10, 11), (1, 1, 4, 5, 3, 6), (1, 1, 30, 40)]
+
+
+@pytest.mark.parametrize("shape", BF_SHAPES, ids=["x".join(map(str, s)) for s in BF_SHAPES])
+@pytest.mark.parametrize("metric", ["euclidean", "taxicab", "chessboard"])
+@pytest.mark.parametrize("sampled", [False, True])
+def test_brute_force_transform(shape, metric, sampled):
+    import torch
+
+    ndim = len(shape) - 2
+    sampling = tuple(0.5 + 0.75 * k for k in range(ndim)) if sampled else None
+    mask = workloads.random_mask(zlib.crc32(repr((shape, metric)).encode()), shape, 0.9)
+    if shape[0] > 1:
+        mask[-1, -1] = 1
+    got = binding.tm_bfdt(torch.from_numpy(mask).cuda(), sampling, metric).cpu().numpy()
+    if metric == "euclidean":
+        ref = oracle.brute(mask, sampling, want_idx=False)["dist"]
+    else:
+        ref = co.brute(mask, metric, sampling if sampled else (1.0,) * ndim)
+    assert np.array_equal(np.isinf(got), np.isinf(ref))
+    fin = np.isfinite(ref)
+    assert (np.abs(got[fin] - ref[fin]) <= 1e-5 * np.maximum(1.0, ref[fin])).all()
+
+
+def test_brute_force_validates_the_separable_transforms_on_the_device():
+    """The use the paper names for the brute-force transform: the separable results, recomputed on the GPU."""
+    import torch
+
+    mask = torch.from_numpy(workloads.random_mask(5, (2, 1, 24, 40, 32), 0.95)).cuda()
+    edt = binding.tm_edt(mask, (2.0, 1.0, 0.5))["dist"]
+    assert torch.allclose(edt, binding.tm_bfdt(mask, (2.0, 1.0, 0.5), "euclidean"), rtol=1e-5, atol=1e-5)
+    for metric in ("taxicab", "chessboard"):
+        assert torch.equal(binding.tm_cdt(mask, metric).float(), binding.tm_bfdt(mask, None, metric))
