@@ -379,6 +379,78 @@ def run_morph(args):
                       "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
 
 
+def run_cdt(args):
+    """Measurement of tm_cdt and tm_bfdt (later rows of the scope, their own metric): disks as in workload C2 at the
+    paper's 2-D sizes; HBM roofline = mask in + int32 out once (5 B/voxel); the brute-force transform is quadratic and
+    reported in voxel-site pairs per second."""
+    import numpy as np
+    import torch
+
+    from oracle import cdt_oracle as co
+    from paper_2608_24738_b200 import binding, buildlib, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak_gbs()
+    peak_kind += " copy bandwidth"
+    stream = torch.cuda.current_stream()
+    steps = max(10, args.steps // 4)
+
+    def timed(call, sets):
+        for i in range(max(3, args.warmup)):
+            call(i % sets)
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(steps):
+            call(i % sets)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / steps
+
+    cases = []
+    for size, batch in ((1024, 64), (256, 512)):
+        base = workloads.config2(batch=8, size=size, disks=20 * (size // 512) ** 2 if size >= 512 else 5).mask
+        mask = np.concatenate([base] * (batch // 8), axis=0)
+        nvox = mask.size
+        sets = max(2, -(-2 * L2_BYTES // (nvox * 5)))
+        ins = [torch.from_numpy(mask).to(dev) for _ in range(sets)]
+        outs = [torch.empty(mask.shape, dtype=torch.int32, device=dev) for _ in range(sets)]
+        for metric in ("chessboard", "taxicab"):
+            ms = timed(lambda i: binding.tm_cdt(ins[i], metric, out=outs[i]), sets)
+            t0 = time.perf_counter()
+            co.separable(mask[:1], metric)
+            cpu_s = time.perf_counter() - t0
+            gbs = nvox * 5 / (ms * 1e-3) / 1e9
+            cases.append({"case": "cdt_%s_2d_%d" % (metric, size), "shape": list(mask.shape), "ms_per_step": ms,
+                          "value": nvox / (ms * 1e-3) / 1e9, "unit": "Gvoxel/s", "inputs_per_ms": batch / ms,
+                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                       "peak_kind": peak_kind, "bytes_per_voxel": 5},
+                          "cpu_baseline": {"value": mask[:1].size / cpu_s / 1e9, "unit": "Gvoxel/s", "cores": 1,
+                                           "kind": "oracle", "sample": "1 image"},
+                          "l2": "rotating %d buffer sets" % sets})
+    # brute force: 64 images of 128^2 (about 6000 background voxels each)
+    bmask = workloads.config2(batch=64, size=128, disks=6).mask
+    t = torch.from_numpy(bmask).to(dev)
+    o = torch.empty(bmask.shape, dtype=torch.float32, device=dev)
+    sites = int((bmask == 0).sum()) // bmask.shape[0]
+    for metric in ("euclidean", "chessboard"):
+        ms = timed(lambda i: binding.tm_bfdt(t, None, metric, out=o), 1)
+        pairs = bmask.size * sites
+        cases.append({"case": "bfdt_%s_2d_128" % metric, "shape": list(bmask.shape), "ms_per_step": ms,
+                      "value": bmask.size / (ms * 1e-3) / 1e9, "unit": "Gvoxel/s", "inputs_per_ms": bmask.shape[0] / ms,
+                      "pairs_per_s": pairs / (ms * 1e-3), "background_voxels_per_image": sites})
+    head = cases[0]
+    print(json.dumps({"metric": "cdt_gvoxels_per_s", "value": head["value"], "unit": "Gvoxel/s", "n_gpus": 1, "steps": steps,
+                      "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+                      "config": {"workload": head["case"], "shape": head["shape"]}, "gpu_launches": 2 * steps,
+                      "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -396,13 +468,16 @@ def main():
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
     ap.add_argument("--flat-index", action="store_true",
                     help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
-    ap.add_argument("--workload", default="edt", choices=["edt", "morph"],
-                    help="edt: the headline benchmark; morph: the fused erosion / dilation kernel (its own metric)")
+    ap.add_argument("--workload", default="edt", choices=["edt", "morph", "cdt"],
+                    help="edt: the headline benchmark; morph / cdt: the erosion-dilation kernels and the taxicab / chessboard / brute-force transforms (their own metrics)")
     ap.add_argument("--morph-case", default=None, help="with --workload morph: run only this case (profiling aid)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
     if args.workload == "morph":
         run_morph(args)
+        return
+    if args.workload == "cdt":
+        run_cdt(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()

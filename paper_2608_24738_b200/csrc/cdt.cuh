@@ -35,6 +35,103 @@ __global__ void __launch_bounds__(256) cdt_axis_kernel(const __grid_constant__ P
     P.out[e] = (P.last && best >= kBig) ? -1 : best;
 }
 
+// First axis (contiguous lines of up to 8192 voxels): one warp per line, lanes take consecutive voxels.  The zero
+// bits of the line are collected as ballot words in shared memory; a voxel finds its nearest zero to the left and
+// to the right inside its own word with __clz / __ffs and otherwise takes the last zero before / first zero
+// after the word.  The 1-D distance is the same for both metrics.
+struct RowParams {
+    const uint8_t* mask;
+    int32_t* out;
+    int64_t rows;
+    int n0;
+    int last;
+};
+
+__global__ void __launch_bounds__(256) cdt_row_kernel(const __grid_constant__ RowParams P) {
+    constexpr int MAXW = 256;
+    __shared__ uint32_t s_word[8][MAXW];
+    __shared__ int s_next[8][MAXW];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;
+    if (row >= P.rows) return;  // the whole warp leaves together
+    const int n0 = P.n0, W = (n0 + 31) >> 5;
+    const uint8_t* src = P.mask + row * n0;
+    bool any = false;
+    for (int b = 0; b < W; ++b) {
+        const int x = 32 * b + lane;
+        const unsigned word = __ballot_sync(0xffffffffu, x < n0 && src[x] == 0);
+        if (lane == 0) s_word[warp][b] = word;
+        any = any || word != 0u;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        int nxt = 1 << 20;
+        for (int b = W - 1; b >= 0; --b) {
+            s_next[warp][b] = nxt;
+            const uint32_t word = s_word[warp][b];
+            if (word) nxt = 32 * b + __ffs(word) - 1;
+        }
+    }
+    __syncwarp();
+    int carry = -(1 << 20);  // last zero before word b
+    for (int b = 0; b < W; ++b) {
+        const uint32_t word = s_word[warp][b];
+        const int x = 32 * b + lane;
+        const uint32_t ml = word & (0xffffffffu >> (31 - lane)), mr = word >> lane;
+        const int zl = ml ? 32 * b + 31 - __clz(ml) : carry;
+        const int zr = mr ? x + __ffs(mr) - 1 : s_next[warp][b];
+        if (x < n0) P.out[row * n0 + x] = any ? min(x - zl, zr - x) : (P.last ? -1 : kBig);
+        if (word) carry = 32 * b + 31 - __clz(word);
+    }
+}
+
+// A further axis of up to 1024 rows: a block stages an (n x 32) strip of values in shared memory (rows of 128
+// contiguous bytes) and a warp scans four consecutive rows of its 32 columns at a time, so that every row fetched
+// from the tile serves four voxels.  The nearest candidate of a step is d rows away, which ends the scan once d
+// reaches the largest of the four minima.
+template <bool CHESS>
+__global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ PassParams P, const int strips_per_slab) {
+    extern __shared__ __align__(16) int sm_cdt[];  // [n][32]
+    const int n = P.n;
+    const int64_t slab = blockIdx.x / strips_per_slab;
+    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
+    const int64_t base = slab * (int64_t)n * P.inner + c0;
+    const int width = (int)min((int64_t)32, P.inner - c0);
+    for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
+        const int y = t >> 5, x = t & 31;
+        if (x < width) sm_cdt[t] = P.in[base + (int64_t)y * P.inner + x];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if (lane >= width) return;
+    auto op = [](int v, int d) { return CHESS ? max(v, d) : v + d; };
+    for (int y0 = warp * 4; y0 < n; y0 += nwarps * 4) {
+        int k[4], best[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) k[i] = y0 + i < n ? sm_cdt[(y0 + i) * 32 + lane] : kBig;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            best[i] = k[i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j != i) best[i] = min(best[i], op(k[j], i > j ? i - j : j - i));
+            if (y0 + i >= n) best[i] = 0;
+        }
+        int mx = max(max(best[0], best[1]), max(best[2], best[3]));
+        int lo = y0 - 1, hi = y0 + 4;
+        for (int d = 1; d < mx && (lo >= 0 || hi < n); ++d, --lo, ++hi) {
+            const int vlo = lo >= 0 ? sm_cdt[lo * 32 + lane] : kBig;
+            const int vhi = hi < n ? sm_cdt[hi * 32 + lane] : kBig;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) best[i] = min(best[i], min(op(vlo, d + i), op(vhi, d + 3 - i)));
+            mx = max(max(best[0], best[1]), max(best[2], best[3]));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (y0 + i < n) P.out[base + (int64_t)(y0 + i) * P.inner + lane] = (P.last && best[i] >= kBig) ? -1 : best[i];
+    }
+}
+
 // ---- brute force ----
 struct BruteParams {
     const uint8_t* mask;

@@ -66,9 +66,24 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
         P.n = (int)g.ext[axes[k]];
         P.inner = 1;
         for (int a = axes[k] + 1; a < ndim; ++a) P.inner *= g.ext[a];
-        const unsigned blocks = (unsigned)((g.total + 255) / 256);
-        if (metric == TM_METRIC_CHESSBOARD) cdt_axis_kernel<true><<<blocks, 256, 0, st>>>(P);
-        else cdt_axis_kernel<false><<<blocks, 256, 0, st>>>(P);
+        const bool chess = metric == TM_METRIC_CHESSBOARD;
+        if (k == 0 && P.inner == 1 && P.n <= 8192) {
+            // contiguous lines: ballot words, same distance for both metrics
+            RowParams R;
+            R.mask = input; R.out = P.out; R.rows = g.total / P.n; R.n0 = P.n; R.last = P.last;
+            cdt_row_kernel<<<(unsigned)((R.rows + 7) / 8), 256, 0, st>>>(R);
+        } else if (k > 0 && P.n <= 1024) {
+            // strided axis: (n x 32) strips in shared memory
+            const int strips = (int)((P.inner + 31) / 32);
+            const size_t smem = (size_t)P.n * 32 * 4;
+            auto kern = chess ? cdt_strip_kernel<true> : cdt_strip_kernel<false>;
+            if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            kern<<<(unsigned)(g.total / ((int64_t)P.n * P.inner) * strips), P.n >= 384 ? 512 : 256, smem, st>>>(P, strips);
+        } else {
+            const unsigned blocks = (unsigned)((g.total + 255) / 256);
+            if (chess) cdt_axis_kernel<true><<<blocks, 256, 0, st>>>(P);
+            else cdt_axis_kernel<false><<<blocks, 256, 0, st>>>(P);
+        }
         e = cudaGetLastError();
         prev = P.out;
     }

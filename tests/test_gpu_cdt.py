@@ -18,7 +18,8 @@ def _built():
 
 
 SHAPES = [(2, 2, 1), (3, 1, 37), (2, 1, 19, 23), (1, 2, 40, 300), (1, 1, 1, 50, 1), (2, 1, 11, 12, 13), (1, 1, 5, 6, 4, 7),
-          (1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 1, 260, 130), (1, 1, 6, 200, 33)]
+          (1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 1, 260, 130), (1, 1, 6, 200, 33),
+          (1, 1, 1100, 40), (1, 1, 3, 9000)]  # beyond the shared-memory strip / the ballot-word row kernel
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=["x".join(map(str, s)) for s in SHAPES])
