@@ -97,9 +97,18 @@ __global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ 
     const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
     const int64_t base = slab * (int64_t)n * P.inner + c0;
     const int width = (int)min((int64_t)32, P.inner - c0);
-    for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
-        const int y = t >> 5, x = t & 31;
-        if (x < width) sm_cdt[t] = P.in[base + (int64_t)y * P.inner + x];
+    if ((P.inner & 3) == 0) {  // rows are 16-byte aligned: eight threads copy one row of 32 values
+#pragma unroll 4
+        for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
+            const int y = t >> 3, ch = t & 7;
+            if (4 * ch < width)
+                *reinterpret_cast<int4*>(sm_cdt + y * 32 + 4 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 4 * ch);
+        }
+    } else {
+        for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
+            const int y = t >> 5, x = t & 31;
+            if (x < width) sm_cdt[t] = P.in[base + (int64_t)y * P.inner + x];
+        }
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
