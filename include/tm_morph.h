@@ -1,7 +1,7 @@
 /*
  * tm_morph -- greyscale and binary erosion / dilation on the GPU, C ABI (sm_100a).
  *
- * Operators (paper, Section 2.1 "Morphological operators"; kernel design: Section 2.3.2 "Fused morphology
+ * Operators (paper, Section 2.1 "Covered transforms"; kernel design: Section 2.3.1 "Fused morphology
  * kernel"), with the conventions of scipy.ndimage that the paper mirrors:
  *
  *   grey erosion    out(x) = min over active k of [ f(x + k - c) - s(k) ]

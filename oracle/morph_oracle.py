@@ -1,6 +1,6 @@
 """CPU oracle for greyscale and binary erosion / dilation -- TEST INFRASTRUCTURE ONLY.
 
-Plain numpy, written from the definition (paper, Section 2.1 "Morphological operators" and Section 2.3.2
+Plain numpy, written from the definition (paper, Section 2.1 "Covered transforms" and Section 2.3.1
 "Fused morphology kernel"): the output at x combines the input at x + k - c over the active positions k of the
 structuring element, c being its centre; values outside the image come from one of the five border rules of
 scipy.ndimage (greyscale) or from a single border value (binary).  The image is padded once with the border
@@ -10,8 +10,8 @@ rule and the active positions are visited one by one: no blocking, no separable 
   grey dilation   out(x) = max_k [ f(x - k + c') + s(k) ]      (the reflected element, as SciPy defines it)
   binary erosion  out(x) = AND_k f(x + k - c),   binary dilation  out(x) = OR_k f(x - k + c')
 
-with c = size // 2 + origin and, for the reflected element of a dilation, c' = (size - 1) // 2 - origin... which
-is written below as "reflect the element, then erode with the opposite combine" so that the centre rule is
+with c = size // 2 + origin.  A dilation is written below as "reflect the element (origin negated, minus one on
+even sizes, as SciPy does), then combine with max and + at the same kind of centre", so that the centre rule is
 stated only once.  Arithmetic is float32 like the CUDA path (one subtraction or addition per tap; minima and
 maxima are exact), so parity is bit-exact.
 

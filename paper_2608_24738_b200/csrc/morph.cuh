@@ -1,4 +1,4 @@
-// Fused erosion / dilation kernels (paper, Section 2.3.2 "Fused morphology kernel").  The host flattens the
+// Fused erosion / dilation kernels (paper, Section 2.3.1 "Fused morphology kernel").  The host flattens the
 // structuring element into its active entries; each entry carries the per-axis offsets and the flat offset
 // against the image's strides.  Interior voxels (whole neighbourhood inside the image, tested with the per-axis
 // offset extrema) add flat offsets to their linear index and nothing else; voxels within reach of a face map every
