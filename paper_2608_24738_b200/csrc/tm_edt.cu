@@ -577,7 +577,6 @@ static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParam
     WideAxisParams B = A;
     const int64_t base_blocks = A.outer * strips;
     B.row_parts = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(8, A.n / 64), 296 / base_blocks));
-    if (const char* v = getenv("TM_EDT_WIDE_PARTS")) B.row_parts = atoi(v);
     kern<<<(unsigned)(base_blocks * B.row_parts), A.n >= 384 ? 512 : 256, smem, st>>>(B, ep, strips);
     return cudaGetLastError();
 }
