@@ -123,13 +123,15 @@ __global__ void __launch_bounds__(256) long_row_kernel(const __grid_constant__ W
                 for (int i = 0; i < 4; ++i)
                     kdst[i] = make_uint4(hts[16 * h + 4 * i], hts[16 * h + 4 * i + 1], hts[16 * h + 4 * i + 2],
                                          hts[16 * h + 4 * i + 3]);
-                uint32_t pk[8];
+                if (P.offs) {
+                    uint32_t pk[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    pk[i] = (uint32_t)(uint16_t)offs[16 * h + 2 * i] | ((uint32_t)(uint16_t)offs[16 * h + 2 * i + 1] << 16);
-                uint4* odst = reinterpret_cast<uint4*>(P.offs + row * n0 + x);
-                odst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                odst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    for (int i = 0; i < 8; ++i)
+                        pk[i] = (uint32_t)(uint16_t)offs[16 * h + 2 * i] | ((uint32_t)(uint16_t)offs[16 * h + 2 * i + 1] << 16);
+                    uint4* odst = reinterpret_cast<uint4*>(P.offs + row * n0 + x);
+                    odst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    odst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
             }
         }
         carry_l = max(carry_l, s_last[warp][c]);
@@ -183,7 +185,7 @@ __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant
         const int dl = x - zl, dr = zr - x;
         const int a = min(dl, dr);
         if (x < n0) {
-            P.offs[row * n0 + x] = row_has_zero ? (int16_t)(dl <= dr ? -a : a) : (int16_t)-32768;
+            if (P.offs) P.offs[row * n0 + x] = row_has_zero ? (int16_t)(dl <= dr ? -a : a) : (int16_t)-32768;
             P.keys[row * n0 + x] = !row_has_zero ? (FLT ? kLongNoneFlt : kLongNoneInt)
                                                  : (FLT ? __float_as_uint(__fmul_rn(P.w2x, (float)(a * a)))
                                                         : (((uint32_t)(a * a) << (SH > 0 ? SH : 0)) | yrow));
@@ -311,7 +313,7 @@ __global__ void __launch_bounds__(256) long_axis_kernel(const __grid_constant__ 
                 }
             }
         }
-        const bool need_site = !FINAL || ep.idx != nullptr;
+        const bool need_site = FINAL ? ep.idx != nullptr : P.offs_out != nullptr;
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             const int y = y0 + i;
@@ -337,7 +339,7 @@ __global__ void __launch_bounds__(256) long_axis_kernel(const __grid_constant__ 
             const int64_t pj = col_base + (int64_t)j * st;   // the chosen site's voxel of this column
             if (!FINAL) {
                 P.h_out[p] = none ? NONE : b;
-                if (K == 1) {
+                if (K == 1 && P.offs_out) {
                     const uint32_t o0 = none ? 0x8000u : (uint32_t)(uint16_t)P.offs_in[pj];
                     reinterpret_cast<uint32_t*>(P.offs_out)[p] = o0 | ((uint32_t)(uint16_t)(int16_t)(j - y) << 16);
                 }

@@ -21,7 +21,7 @@ namespace tmedt {
 struct WideParams {
     const uint8_t* in;   // (images, n1, n0)
     uint32_t* keys;      // (images, n1, n0)
-    int16_t* offs;       // (images, n1, n0)
+    int16_t* offs;       // (images, n1, n0), or nullptr when no index output is requested
     int64_t rows;        // images * n1
     int n0, n1;
     float w2x;           // squared sampling of the contiguous axis (float-height variant)
@@ -91,13 +91,15 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
             for (int i = 0; i < 4; ++i)
                 kdst[i] = make_uint4(keys[16 * c + 4 * i], keys[16 * c + 4 * i + 1], keys[16 * c + 4 * i + 2],
                                      keys[16 * c + 4 * i + 3]);
-            uint32_t pk[8];
+            if (P.offs) {  // offsets are carried only when the index output is requested
+                uint32_t pk[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                pk[i] = (uint32_t)(uint16_t)offs[16 * c + 2 * i] | ((uint32_t)(uint16_t)offs[16 * c + 2 * i + 1] << 16);
-            uint4* odst = reinterpret_cast<uint4*>(P.offs + row * n0 + VPL * lane + 16 * c);
-            odst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            odst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                for (int i = 0; i < 8; ++i)
+                    pk[i] = (uint32_t)(uint16_t)offs[16 * c + 2 * i] | ((uint32_t)(uint16_t)offs[16 * c + 2 * i + 1] << 16);
+                uint4* odst = reinterpret_cast<uint4*>(P.offs + row * n0 + VPL * lane + 16 * c);
+                odst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                odst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
         }
     }
 }
@@ -217,7 +219,9 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
             if (!FINAL) {
                 if (SH < 0) P.keys_out[p] = b;  // the height itself is the next pass's scan value
                 else P.keys_out[p] = none ? kNoneKey16 : ((b & ~kRowMask) | next_row);
-                if (K == 1) {
+                if (!P.offs_out) {
+                    // distances only: no offsets are carried
+                } else if (K == 1) {
                     const uint32_t o0 = none ? 0x8000u : (uint32_t)(uint16_t)P.offs_in[pj];
                     reinterpret_cast<uint32_t*>(P.offs_out)[p] = o0 | ((uint32_t)(uint16_t)(int16_t)(j - y) << 16);
                 } else if (K == 2) {

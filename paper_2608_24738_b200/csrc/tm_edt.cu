@@ -589,8 +589,9 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     int16_t* offsA = reinterpret_cast<int16_t*>(w + up((size_t)pl.N * 4));
     uint32_t* keysB = reinterpret_cast<uint32_t*>(w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
     int16_t* offsB = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
+    const bool carry = ep.idx != nullptr;  // offsets are carried only for the index output
     WideParams P;
-    P.in = in; P.keys = keysA; P.offs = offsA;
+    P.in = in; P.keys = keysA; P.offs = carry ? offsA : nullptr;
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     P.w2x = (float)(pl.w[0] * pl.w[0]);
@@ -600,7 +601,7 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     int nmax = 1;
     for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
     const int sh = !pl.unit ? -1 : (nmax > 512 ? 10 : 9);
-    prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + 2.0));
+    prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + (carry ? 2.0 : 0.0)));
     const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
     if (pl.ext[0] % 16 != 0 || ((uintptr_t)in & 15u) != 0) {
         // rows that are not 16-byte aligned: one voxel per lane, ballot words
@@ -630,13 +631,13 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     for (int k = 1; k < pl.E; ++k) {
         const bool fin = k == pl.E - 1;
         A.keys_in = keys_in[k]; A.offs_in = offs_in[k];
-        A.keys_out = fin ? nullptr : keys_out[k]; A.offs_out = fin ? nullptr : offs_out[k];
+        A.keys_out = fin ? nullptr : keys_out[k]; A.offs_out = (fin || !carry) ? nullptr : offs_out[k];
         A.n = pl.ext[k]; A.inner = pl.inner[k]; A.outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
         A.next_n = fin ? 0 : pl.ext[k + 1];
         A.w2 = (float)(pl.w[k] * pl.w[k]);
         const double offs_b = k == 3 ? 8.0 : 2.0 * k;  // bytes of offsets per voxel read by this axis
         if (fin) prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? offs_b : 0.0)));
-        else prof_mark(st, "wide_axis", (double)pl.N * (4.0 + offs_b + 4.0 + (k == 2 ? 8.0 : 4.0)));
+        else prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 4.0 + (carry ? offs_b + (k == 2 ? 8.0 : 4.0) : 0.0)));
         if (k == 1) e = fin ? launch_wide_axis<1, true>(A, ep, sh, st) : launch_wide_axis<1, false>(A, ep, sh, st);
         else if (k == 2) e = fin ? launch_wide_axis<2, true>(A, ep, sh, st) : launch_wide_axis<2, false>(A, ep, sh, st);
         else e = launch_wide_axis<3, true>(A, ep, sh, st);
@@ -659,12 +660,13 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
     uint32_t* blockmin = reinterpret_cast<uint32_t*>(
         w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2) + (pl.E == 3 ? 2 * up((size_t)pl.N * 4) : 0));
     WideParams P;
-    P.in = in; P.keys = hA; P.offs = offsA;
+    const bool carry = ep.idx != nullptr;  // offsets are carried only for the index output
+    P.in = in; P.keys = hA; P.offs = carry ? offsA : nullptr;
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     P.w2x = (float)(pl.w[0] * pl.w[0]);
     const double out_bpv = out_bytes_per_voxel(ep);
-    prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + 2.0));
+    prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + (carry ? 2.0 : 0.0)));
     if (pl.ext[0] % 16 == 0 && ((uintptr_t)in & 15u) == 0) long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
     else long_row_any_kernel<FLT ? -1 : -2><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
     ++launches;
@@ -690,7 +692,7 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
         ++launches;
         return cudaGetLastError();
     };
-    A.h_in = hA; A.offs_in = offsA; A.h_out = hB; A.offs_out = offsB;
+    A.h_in = hA; A.offs_in = offsA; A.h_out = hB; A.offs_out = carry ? offsB : nullptr;
     unsigned blocks = set_axis(1);
     e = block_minima();
     if (e != cudaSuccess) return e;
@@ -700,7 +702,7 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
         ++launches;
         return cudaGetLastError();
     }
-    prof_mark(st, "long_axis", (double)pl.N * (4.0 + 2.0 + 4.0 + 4.0));
+    prof_mark(st, "long_axis", (double)pl.N * (4.0 + 4.0 + (carry ? 2.0 + 4.0 : 0.0)));
     long_axis_kernel<1, false, FLT><<<blocks, 256, 0, st>>>(A, ep);
     ++launches;
     e = cudaGetLastError();
