@@ -92,7 +92,49 @@ int flatten(const Geometry& g, const uint8_t* fp, const float* st, const int64_t
 
 template <typename T, bool BINARY>
 int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const float* st, const int64_t* fp_shape,
-        const int64_t* origin, int op, int mode, float cval, int border_value, void* output, tm_edt_stream_t stream) {
+        const int64_t* origin, int op, int mode, float cval, int border_value, void* output, tm_edt_stream_t stream,
+        bool allow_separable = true);
+
+// A flat element whose footprint is a full box is the composition of one line element per axis: the minimum (or
+// maximum) over a box is the minimum over its rows of the minima along the rows, and every border rule acts on one
+// axis at a time.  From 20 positions on, the box is therefore run as one pass per axis with ndim line elements
+// (m_0 + .. + m_{d-1} taps instead of their product), through the same kernels, with one or two scratch images.
+template <typename T, bool BINARY>
+int run_box(const T* input, int ndim, const int64_t* shape, const int64_t* fp_shape, const int64_t* origin, int op,
+            int mode, float cval, int border_value, void* output, tm_edt_stream_t stream, size_t total) {
+    cudaStream_t s = (cudaStream_t)stream;
+    int axes[kMaxDims], na = 0;
+    for (int a = 0; a < ndim; ++a)
+        if (fp_shape[a] > 1 || (origin && origin[a] != 0)) axes[na++] = a;
+    if (na == 0) axes[na++] = ndim - 1;
+    const size_t buf = ((total * sizeof(T)) + 255) & ~(size_t)255;
+    char* ws = nullptr;
+    if (na > 1) {
+        cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, (na > 2 ? 2 : 1) * buf, s);
+        if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    }
+    uint8_t line[256];
+    memset(line, 1, sizeof(line));
+    const T* src = input;
+    int rc = TM_EDT_OK, launches = 0;
+    for (int i = 0; i < na && rc == TM_EDT_OK; ++i) {
+        const int a = axes[i];
+        int64_t ls[kMaxDims], lo[kMaxDims];
+        for (int b = 0; b < ndim; ++b) { ls[b] = b == a ? fp_shape[b] : 1; lo[b] = (b == a && origin) ? origin[b] : 0; }
+        void* dst = i == na - 1 ? output : (void*)(ws + (size_t)(i & 1) * buf);
+        rc = run<T, BINARY>(src, ndim, shape, line, nullptr, ls, lo, op, mode, cval, border_value, dst, stream, false);
+        launches += 2;
+        src = static_cast<const T*>(dst);
+    }
+    if (ws) cudaFreeAsync(ws, s);
+    if (rc == TM_EDT_OK) tmedt::shared_record(-1, launches);
+    return rc;
+}
+
+template <typename T, bool BINARY>
+int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const float* st, const int64_t* fp_shape,
+        const int64_t* origin, int op, int mode, float cval, int border_value, void* output, tm_edt_stream_t stream,
+        bool allow_separable) {
     if (!input || !output) return TM_EDT_ERR_INVALID_ARG;
     if (op != TM_MORPH_EROSION && op != TM_MORPH_DILATION) return TM_EDT_ERR_INVALID_ARG;
     if (mode < TM_MORPH_CONSTANT || mode > TM_MORPH_WRAP) return TM_EDT_ERR_INVALID_ARG;
@@ -110,6 +152,15 @@ int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const
     if (((uintptr_t)input % sizeof(T)) || ((uintptr_t)output % (BINARY ? 1 : 4))) return TM_EDT_ERR_INVALID_ARG;
     if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(output)) return TM_EDT_ERR_BAD_POINTER;
     if (g.total > (int64_t)INT32_MAX * 128) return TM_EDT_ERR_UNSUPPORTED;
+    if (allow_separable && ndim >= 2 && entries.size() >= 20) {
+        int64_t box = 1;
+        bool flat = true;
+        for (int a = 0; a < ndim; ++a) box *= fp_shape[a];
+        for (const Entry& en : entries) flat = flat && en.s == 0.0f;
+        if (flat && (int64_t)entries.size() == box)
+            return run_box<T, BINARY>(input, ndim, shape, fp_shape, origin, op, mode, cval, border_value, output, stream,
+                                      (size_t)g.total);
+    }
     cudaStream_t s = (cudaStream_t)stream;
     int launches = 0;
     void* dev = nullptr;

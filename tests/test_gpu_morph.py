@@ -84,3 +84,32 @@ def test_large_volume_against_the_oracle_and_scipy():
     b = torch.from_numpy((img > 0.5).astype(np.uint8)).cuda()
     got = binding.tm_binary_morph(b, fp, op="dilation").cpu().numpy()
     assert np.array_equal(got[0, 0].astype(bool), ndi.binary_dilation(img[0, 0] > 0.5, fp))
+
+
+BOXES = [((2, 1, 19, 23), (5, 5), None), ((1, 2, 11, 12, 13), (3, 3, 3), None), ((1, 1, 20, 256), (4, 6), (-1, 2)),
+         ((1, 1, 5, 6, 4, 7), (3, 2, 2, 2), (0, 0, -1, 0)), ((1, 1, 3, 4, 128), (3, 3, 3), (1, 0, -1)), ((1, 1, 4, 4), (5, 5), None)]
+
+
+@pytest.mark.parametrize("shape,fp_shape,origin", BOXES, ids=["x".join(map(str, c[0])) + "_" + "x".join(map(str, c[1])) for c in BOXES])
+@pytest.mark.parametrize("mode", mo.MODES)
+def test_full_box_elements_run_one_pass_per_axis(shape, fp_shape, origin, mode):
+    """Flat full-box elements of 20 or more positions are decomposed into one line element per axis; the result
+    must stay bit-identical to the oracle's single N-D minimum / maximum, for every border rule, origin and op."""
+    import torch
+
+    seed = zlib.crc32(repr((shape, fp_shape, mode, "box")).encode())
+    rng = np.random.default_rng(seed)
+    img = rng.normal(size=shape).astype(np.float32)
+    fp = np.ones(fp_shape, dtype=bool)
+    t = torch.from_numpy(img).cuda()
+    for op, ref_fn in (("erosion", mo.grey_erosion), ("dilation", mo.grey_dilation)):
+        got = binding.tm_grey_morph(t, fp, None, op=op, mode=mode, cval=-0.5, origin=origin)
+        assert binding.tm_edt_last_launch_count() > 2  # several passes
+        assert np.array_equal(got.cpu().numpy(), ref_fn(img, fp, None, mode, -0.5, origin)), op
+    if mode == "constant":
+        mask = (rng.random(shape) < 0.8).astype(np.uint8)
+        b = torch.from_numpy(mask).cuda()
+        for border_value in (0, 1):
+            for op, ref_fn in (("erosion", mo.binary_erosion), ("dilation", mo.binary_dilation)):
+                got = binding.tm_binary_morph(b, fp, op=op, border_value=border_value, origin=origin)
+                assert np.array_equal(got.cpu().numpy(), ref_fn(mask, fp, border_value, origin)), (op, border_value)
