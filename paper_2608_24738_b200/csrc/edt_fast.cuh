@@ -132,7 +132,7 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j,
     // 1e-7 is a hundred times inside the 1e-5 bar on distances.
     const float dv = none ? TMEDT_INF : fast_sqrt(sqv);
     if (o.dist_only) { o.dist[p] = dv; return; }
-    if (o.dist) o.dist[p] = dv;
+    if (o.dist) __stcs(o.dist + p, dv);
     if (none) {
         if (o.sq) o.sq[p] = INT64_MAX;
         if (o.idx && o.flat) o.idx[p] = -1;
@@ -150,8 +150,8 @@ __device__ __forceinline__ void emit(const ColumnOut<K, FINAL>& o, int y, int j,
         // one store per processed axis: own coordinate + offset (coordinates are non-negative)
 #pragma unroll
         for (int q = 0; q < K; ++q)
-            o.ip[q][p] = (int64_t)(uint32_t)(o.coord[q] + (int)(int8_t)((e >> (8 * q)) & 0xff));
-        o.ip[K][p] = (int64_t)(uint32_t)j;
+            __stcs(reinterpret_cast<long long*>(o.ip[q] + p), (long long)(uint32_t)(o.coord[q] + (int)(int8_t)((e >> (8 * q)) & 0xff)));
+        __stcs(reinterpret_cast<long long*>(o.ip[K] + p), (long long)(uint32_t)j);
     } else if (o.idx) {
         int off[5];
 #pragma unroll
