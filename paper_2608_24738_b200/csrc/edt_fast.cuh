@@ -53,6 +53,8 @@ struct FastParams {
     int si[4];           // scaled-integer mode: scale * w^2 of the earlier axes (exact integers)
     int sk;              // scaled-integer mode: scale * w^2 of this axis
     float inv_scale;     // scaled-integer mode: 1 / scale
+    int value_carry;     // plane kernels, non-final: 0 = write entries; 2 / 4 = write the squared distance so far as
+                         // uint16 / uint32 (all ones = no site), for the passes of edt_value.cuh
 };
 
 // add[d] = w^2 d^2 for the axis of the pass: float32 bits (sampled) or d^2 << shift (unit sampling keys).
@@ -572,7 +574,8 @@ __device__ __forceinline__ void pass0_row_to_keys(const uint32_t v, int n0, int 
     if (act) *reinterpret_cast<uint4*>(vrow + 4 * lane) = keys;
 }
 
-template <bool FINAL, int VS>
+// VC: what a non-final pass writes: 0 = 2-byte entries, 2 / 4 = the squared distance so far as uint16 / uint32.
+template <bool FINAL, int VS, int VC = 0>
 __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__ FastParams P,
                                                          const __grid_constant__ EpilogueParams ep) {
     extern __shared__ __align__(16) uint8_t sm_plane_u[];
@@ -616,8 +619,14 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
             const bool none = b >= kNoneKey16;
             const int j = (int)((b >> 8) & 0xffu);
             if (!FINAL) {
-                const uint32_t e = none ? 0x80u : ((b & 0xffu) | ((uint32_t)((j - y) & 0xff) << 8));
-                reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)e;
+                if (VC == 2) {
+                    reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)(none ? 0xffffu : (b >> 16));
+                } else if (VC == 4) {
+                    reinterpret_cast<uint32_t*>(P.out)[p0 + (int64_t)i * n0] = none ? 0xffffffffu : (b >> 16);
+                } else {
+                    const uint32_t e = none ? 0x80u : ((b & 0xffu) | ((uint32_t)((j - y) & 0xff) << 8));
+                    reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)e;
+                }
             } else if (dist_only) {
                 ep.dist[p0 + (int64_t)i * n0] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b >> 16)));
             } else {  // two processed axes: the plane is the image
@@ -968,8 +977,16 @@ __global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant
         uint32_t best[R];
         scan_keys_group<VS, R, kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
 #pragma unroll
-        for (int i = 0; i < R; ++i)
-            if (y0 + i < n1) emit_scaled<1, FINAL, uint8_t>(out, dxt + c, VS, y0 + i, best[i], P.inv_scale);
+        for (int i = 0; i < R; ++i) {
+            if (y0 + i >= n1) break;
+            if (!FINAL && P.value_carry == 4) {
+                const uint32_t b = best[i];
+                reinterpret_cast<uint32_t*>(P.out)[plane * (int64_t)n1 * n0 + (int64_t)(y0 + i) * n0 + c] =
+                    b >= kNoneKey16 ? 0xffffffffu : (b >> kScaledShift);
+            } else {
+                emit_scaled<1, FINAL, uint8_t>(out, dxt + c, VS, y0 + i, best[i], P.inv_scale);
+            }
+        }
     }
 }
 

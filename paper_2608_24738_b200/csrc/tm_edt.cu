@@ -17,6 +17,7 @@
 #include "edt_small.cuh"
 #include "edt_long.cuh"
 #include "edt_compat.cuh"
+#include "edt_value.cuh"
 #include "host_shared.h"
 #include <stdlib.h>
 
@@ -183,7 +184,7 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     }
     if (pl.fast) {
         auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
-        const size_t a = E >= 3 ? up((size_t)pl.N * (E >= 5 ? 4 : 2)) : 0;
+        const size_t a = E >= 3 ? up((size_t)pl.N * 4) : 0;  // entries (2 or 4 B) or carried values (up to 4 B)
         const size_t b = E >= 4 ? up((size_t)pl.N * 4) : 0;
         pl.ws_bytes = a + b;
     }
@@ -341,13 +342,35 @@ static cudaError_t launch_column_any(int K, const FastParams& P, const EpilogueP
     return cudaErrorInvalidValue;
 }
 
+// A further axis on carried values (no index output requested): see edt_value.cuh.
+template <bool FINAL, typename VT, bool SCALED>
+static cudaError_t launch_column_value(const FastParams& P, const EpilogueParams& ep, cudaStream_t st, double out_bpv) {
+    int G = 1;
+    while (G < 4 && P.n * 32 * G * 2 <= 4096 && 32 * G < P.inner) G <<= 1;
+    const int TX = 32 * G;
+    const size_t smem = (size_t)P.n * TX * 4;
+    const int tiles = (int)((P.inner + TX - 1) / TX);
+    const int64_t blocks = P.outer * tiles;
+    const double vox = (double)P.outer * P.n * (double)P.inner;
+    prof_mark(st, FINAL ? "column_value_final" : "column_value", vox * ((double)sizeof(VT) + (FINAL ? out_bpv : (double)sizeof(VT))));
+#define TM_LAUNCH_COLUMN_VALUE(TXV)                                                                            \
+    do {                                                                                                       \
+        auto kern = column_value_kernel<FINAL, VT, SCALED, TXV>;                                               \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        kern<<<(unsigned)blocks, 256, smem, st>>>(P, ep, tiles);                                               \
+    } while (0)
+    if (G == 1) TM_LAUNCH_COLUMN_VALUE(32); else if (G == 2) TM_LAUNCH_COLUMN_VALUE(64); else TM_LAUNCH_COLUMN_VALUE(128);
+#undef TM_LAUNCH_COLUMN_VALUE
+    return cudaGetLastError();
+}
+
 // Packed-entry path: fused first + second axis, then one column kernel per further axis.
 template <bool UNIT>
 static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
                             int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* bufA = static_cast<char*>(ws);
-    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * (pl.E >= 5 ? 4 : 2)) : 0);
+    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * 4) : 0);
     const double out_bpv = out_bytes_per_voxel(ep);
     auto fill = [&](FastParams& P, int k) {
         memset(&P, 0, sizeof(P));
@@ -360,25 +383,40 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     fill(P, 1);
     fill_scan_tab<UNIT>(tab, pl.w[1], 8);
     P.in = in; P.out = bufA; P.n0 = pl.ext[0];
+    // without an index output the passes carry squared distances instead of offsets (unit sampling, tile plane kernel)
+    double sumsq = 0.0;
+    for (int p = 0; p < pl.E; ++p) sumsq += (double)(pl.ext[p] - 1) * (pl.ext[p] - 1);
+    const char* oldp0 = getenv("TM_EDT_OLD_PLANE");
+    const bool vc = UNIT && !ep.idx && pl.E >= 3 && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 &&
+                    !(oldp0 && oldp0[0] == '1') && !getenv("TM_EDT_NO_VALUE_CARRY");
+    const bool vc16 = vc && sumsq < 65535.0;
+    P.value_carry = vc ? (vc16 ? 2 : 4) : 0;
     {
         const int threads = 256;
         const int tstride = (pl.ext[0] + 15) & ~15;
         const size_t smem = (((size_t)pl.ext[1] * tstride + 15) & ~(size_t)15) + (size_t)pl.ext[1] * 32 * 4;
         const bool fin = pl.E == 2;
-        prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
+        prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : (P.value_carry == 4 ? 4.0 : 2.0))));
         const char* oldp = getenv("TM_EDT_OLD_PLANE");
         if (UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
             // whole-plane key tile; row stride = extent rounded up to 32, 64 or 128 columns
             const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
             const size_t smem_u = (size_t)pl.ext[1] * vs * 4;
-#define TM_LAUNCH_PLANE_UNIT(FIN, VSV)                                                                         \
+#define TM_LAUNCH_PLANE_UNIT(FIN, VSV, VCV)                                                                    \
     do {                                                                                                       \
-        auto kern = plane_unit_kernel<FIN, VSV>;                                                               \
+        auto kern = plane_unit_kernel<FIN, VSV, VCV>;                                                          \
         if (smem_u > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_u); \
         kern<<<(unsigned)P.outer, threads, smem_u, st>>>(P, ep);                                               \
     } while (0)
-            if (fin) { if (vs == 32) TM_LAUNCH_PLANE_UNIT(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(true, 64); else TM_LAUNCH_PLANE_UNIT(true, 128); }
-            else { if (vs == 32) TM_LAUNCH_PLANE_UNIT(false, 32); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(false, 64); else TM_LAUNCH_PLANE_UNIT(false, 128); }
+#define TM_LAUNCH_PLANE_UNIT_VS(FIN, VCV)                                                                      \
+    do {                                                                                                       \
+        if (vs == 32) TM_LAUNCH_PLANE_UNIT(FIN, 32, VCV); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(FIN, 64, VCV); else TM_LAUNCH_PLANE_UNIT(FIN, 128, VCV); \
+    } while (0)
+            if (fin) TM_LAUNCH_PLANE_UNIT_VS(true, 0);
+            else if (P.value_carry == 2) TM_LAUNCH_PLANE_UNIT_VS(false, 2);
+            else if (P.value_carry == 4) TM_LAUNCH_PLANE_UNIT_VS(false, 4);
+            else TM_LAUNCH_PLANE_UNIT_VS(false, 0);
+#undef TM_LAUNCH_PLANE_UNIT_VS
 #undef TM_LAUNCH_PLANE_UNIT
         } else if (!UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
             const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
@@ -405,8 +443,11 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
         fill_scan_tab<UNIT>(tab, pl.w[k], 8);
         P.in = src; P.out = dst;
         const bool fin = k == pl.E - 1;
-        cudaError_t e = fin ? launch_column_any<true, UNIT>(k, P, ep, tab, st, out_bpv)
-                            : launch_column_any<false, UNIT>(k, P, ep, tab, st, out_bpv);
+        cudaError_t e;
+        if (vc16) e = fin ? launch_column_value<true, uint16_t, false>(P, ep, st, out_bpv) : launch_column_value<false, uint16_t, false>(P, ep, st, out_bpv);
+        else if (vc) e = fin ? launch_column_value<true, uint32_t, false>(P, ep, st, out_bpv) : launch_column_value<false, uint32_t, false>(P, ep, st, out_bpv);
+        else e = fin ? launch_column_any<true, UNIT>(k, P, ep, tab, st, out_bpv)
+                     : launch_column_any<false, UNIT>(k, P, ep, tab, st, out_bpv);
         ++launches;
         if (e != cudaSuccess) return e;
         char* t = src; src = dst; dst = t;
@@ -442,7 +483,7 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
                               int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* bufA = static_cast<char*>(ws);
-    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * (pl.E >= 5 ? 4 : 2)) : 0);
+    char* bufB = bufA + (pl.E >= 3 ? up((size_t)pl.N * 4) : 0);
     const double out_bpv = out_bytes_per_voxel(ep);
     auto fill = [&](FastParams& P, int k) {
         memset(&P, 0, sizeof(P));
@@ -454,11 +495,14 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
     FastParams P;
     fill(P, 1);
     P.in = in; P.out = bufA; P.n0 = pl.ext[0];
+    // without an index output the passes carry the scaled squared distance (32 bits) instead of offsets
+    const bool vc = !ep.idx && pl.E >= 3 && !getenv("TM_EDT_NO_VALUE_CARRY");
+    P.value_carry = vc ? 4 : 0;
     {
         const bool fin = pl.E == 2;
         const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
         const size_t smem = (size_t)pl.ext[1] * vs * 5;
-        prof_mark(st, fin ? "plane_scaled_final" : "plane_scaled", (double)pl.N * (1.0 + (fin ? out_bpv : 2.0)));
+        prof_mark(st, fin ? "plane_scaled_final" : "plane_scaled", (double)pl.N * (1.0 + (fin ? out_bpv : (vc ? 4.0 : 2.0))));
 #define TM_LAUNCH_PLANE_SCALED(FIN, VSV)                                                                       \
     do {                                                                                                       \
         auto kern = plane_scaled_kernel<FIN, VSV>;                                                             \
@@ -479,7 +523,10 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
         P.in = src; P.out = dst;
         const bool fin = k == pl.E - 1;
         cudaError_t e = cudaErrorInvalidValue;
-        if (fin) {
+        if (vc) {
+            e = fin ? launch_column_value<true, uint32_t, true>(P, ep, st, out_bpv)
+                    : launch_column_value<false, uint32_t, true>(P, ep, st, out_bpv);
+        } else if (fin) {
             if (k == 2) e = launch_column_scaled<2, true>(P, ep, st, out_bpv);
             else if (k == 3) e = launch_column_scaled<3, true>(P, ep, st, out_bpv);
             else if (k == 4) e = launch_column_scaled<4, true>(P, ep, st, out_bpv);

@@ -575,3 +575,33 @@ def test_strided_masks_are_gathered_by_the_library():
     want = binding.tm_edt(v.contiguous(), None, return_sqdist=True)
     torch.cuda.synchronize()
     assert torch.equal(got["sq"], want["sq"])
+
+
+VALUE_SHAPES = [(2, 1, 12, 20, 24), (1, 2, 33, 17, 40), (1, 1, 128, 20, 48), (2, 1, 6, 10, 12, 8), (1, 1, 16, 40, 24, 32),
+                (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128), (1, 1, 128, 128, 128), (1, 1, 9, 10, 11)]
+
+
+@pytest.mark.parametrize("shape", VALUE_SHAPES, ids=["x".join(map(str, s)) for s in VALUE_SHAPES])
+@pytest.mark.parametrize("kind", ["unit", "decimal", "sampled"])
+def test_outputs_without_indices(shape, kind, monkeypatch):
+    """Without an index output the packed-entry path carries squared distances instead of offsets (16-bit values up to
+    four axes, 32-bit beyond and in scaled-integer mode).  Distances and exact squared distances against the oracle,
+    and bit-identical to what the offset-carrying kernels give."""
+    ndim = len(shape) - 2
+    sampling = None if kind == "unit" else (tuple([2.5, 0.8, 1.0, 1.25, 0.5][:ndim]) if kind == "decimal" else _sampling(ndim, "sampled"))
+    unit = sampling is None
+    for p_fg in (0.6, 0.98):
+        mask = workloads.random_mask(zlib.crc32(repr((shape, kind, p_fg, "val")).encode()), shape, p_fg)
+        if shape[0] > 1:
+            mask[-1] = 1  # an image without background
+        ref = oracle.sep(mask, sampling, want_idx=False)
+        res = run_gpu(mask, sampling, dist=True, sq=unit, idx=False)
+        compare(mask, sampling, res, ref, True, unit, False)
+        if unit:
+            only_sq = run_gpu(mask, sampling, dist=False, sq=True, idx=False)
+            checker.check_sq_exact(only_sq["sq"], ref["sq"])
+        monkeypatch.setenv("TM_EDT_NO_VALUE_CARRY", "1")
+        old = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
+        monkeypatch.delenv("TM_EDT_NO_VALUE_CARRY")
+        if kind != "sampled":  # integer paths: the same values either way
+            assert np.array_equal(res["dist"], old["dist"])
