@@ -878,6 +878,8 @@ __device__ __forceinline__ void emit_scaled(const ColumnOut<K, FINAL>& out, cons
     emit<K, FINAL, false>(out, y, j, e, __uint2float_rn(b >> kScaledShift) * inv_scale, none);  // values reach 2^24
 }
 
+// WITH_OFF: also write the signed first-axis offsets as bytes (needed only when offsets are carried or indexed)
+template <bool WITH_OFF = true>
 __device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n0, int y, int s0,
                                                          uint32_t* __restrict__ vrow, uint8_t* __restrict__ drow,
                                                          int lane) {
@@ -919,17 +921,18 @@ __device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n
             const int a = min(dl[b], dr[b]);
             const int off = dl[b] <= dr[b] ? -a : a;
             kk[b] = ((uint32_t)(s0 * a * a) << kScaledShift) | (uint32_t)y;
-            dpack |= ((uint32_t)off & 0xffu) << (8 * b);
+            if (WITH_OFF) dpack |= ((uint32_t)off & 0xffu) << (8 * b);
         }
         kv = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
     if (act) {
         *reinterpret_cast<uint4*>(vrow + 4 * lane) = kv;
-        *reinterpret_cast<uint32_t*>(drow + 4 * lane) = dpack;
+        if (WITH_OFF) *reinterpret_cast<uint32_t*>(drow + 4 * lane) = dpack;
     }
 }
 
-template <bool FINAL, int VS>
+// VC: a non-final pass writes the scaled squared distance so far (uint32) instead of entries; no offsets are kept.
+template <bool FINAL, int VS, bool VC = false>
 __global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant__ FastParams P,
                                                            const __grid_constant__ EpilogueParams ep) {
     extern __shared__ __align__(16) uint8_t sm_plane_i[];
@@ -951,7 +954,7 @@ __global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant
 #pragma unroll
         for (int i = 0; i < MAXR; ++i) {
             const int y = warp + i * nwarps;
-            if (y < n1) pass0_row_to_scaled_keys(rowv[i], n0, y, P.si[0], val + y * VS, dxt + y * VS, lane);
+            if (y < n1) pass0_row_to_scaled_keys<!VC>(rowv[i], n0, y, P.si[0], val + y * VS, dxt + y * VS, lane);
         }
     }
     __syncthreads();
@@ -979,7 +982,7 @@ __global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (y0 + i >= n1) break;
-            if (!FINAL && P.value_carry == 4) {
+            if (!FINAL && VC) {
                 const uint32_t b = best[i];
                 reinterpret_cast<uint32_t*>(P.out)[plane * (int64_t)n1 * n0 + (int64_t)(y0 + i) * n0 + c] =
                     b >= kNoneKey16 ? 0xffffffffu : (b >> kScaledShift);
