@@ -933,7 +933,7 @@ __device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n
 
 // VC: a non-final pass writes the scaled squared distance so far (uint32) instead of entries; no offsets are kept.
 template <bool FINAL, int VS, bool VC = false>
-__global__ void __launch_bounds__(512) plane_scaled_kernel(const __grid_constant__ FastParams P,
+__global__ void __launch_bounds__(512, VC ? 3 : 2) plane_scaled_kernel(const __grid_constant__ FastParams P,
                                                            const __grid_constant__ EpilogueParams ep) {
     extern __shared__ __align__(16) uint8_t sm_plane_i[];
     const int n0 = P.n0, n1 = P.n;
