@@ -1,6 +1,6 @@
 // Packed-entry path without an index output: between passes a voxel carries its squared distance so far (an
 // exact integer: squared voxel units under unit sampling, scale * sum_q w_q^2 off_q^2 in scaled-integer mode)
-// instead of the offsets of its site.  The key of a pass is then value << SH | row with no arithmetic on offsets,
+// instead of the offsets of its site.  The key of a pass is then the value itself, with no arithmetic on offsets,
 // no tile of entries is kept in shared memory, and nothing is fetched for the output:
 //     g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (w_k (x_k - j))^2 ]      (paper, Section 2.3.2)
 // is carried as g itself.  VT = uint16_t when every value fits 16 bits (unit sampling, up to four axes of extent
@@ -14,7 +14,7 @@ template <typename VT> struct ValueNone;
 template <> struct ValueNone<uint16_t> { static constexpr uint32_t v = 0xffffu; };
 template <> struct ValueNone<uint32_t> { static constexpr uint32_t v = 0xffffffffu; };
 
-// One further axis on carried values.  SCALED: keys value << 7 | row with weighted addends (P.sk), else value << 8 | row.
+// One further axis on carried values.  SCALED: weighted addends (P.sk * d^2), else d^2.
 //   FINAL == false  writes the new value (VT);  FINAL == true  writes float32 distances and / or int64 squared distances.
 template <bool FINAL, typename VT, bool SCALED, int TX>
 __global__ void __launch_bounds__(256) column_value_kernel(const __grid_constant__ FastParams P,
@@ -22,8 +22,8 @@ __global__ void __launch_bounds__(256) column_value_kernel(const __grid_constant
                                                            const int tiles_per_slab) {
     extern __shared__ __align__(16) uint8_t sm_val[];
     constexpr int G = TX / 32;
-    constexpr int SH = SCALED ? kScaledShift : 8;
-    constexpr uint32_t NONE = SCALED ? kNoneKey16 : kNoneKey;
+    constexpr int SH = 0;  // no site is needed afterwards: the key is the value itself, without row bits
+    constexpr uint32_t NONE = kNoneKey16;
     constexpr uint32_t VNONE = ValueNone<VT>::v;
     const int n = P.n;
     uint32_t* val = reinterpret_cast<uint32_t*>(sm_val);  // [n][TX]
@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(256) column_value_kernel(const __grid_constant
             for (int i = 0; i < PER16; ++i) {
                 const uint32_t word = wv[(i * (int)sizeof(VT)) >> 2];
                 const uint32_t x = sizeof(VT) == 4 ? word : ((word >> (16 * (i & 1))) & 0xffffu);
-                kv[i] = x == VNONE ? NONE : ((x << SH) | (uint32_t)y);
+                kv[i] = x == VNONE ? NONE : x;
             }
 #pragma unroll
             for (int i = 0; i < PER16; i += 4)
@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(256) column_value_kernel(const __grid_constant
         for (int t = threadIdx.x; t < n * width; t += blockDim.x) {
             const int y = t / width, x = t - y * width;
             const uint32_t v = (uint32_t)src[(int64_t)y * P.inner + x];
-            val[y * TX + x] = v == VNONE ? NONE : ((v << SH) | (uint32_t)y);
+            val[y * TX + x] = v == VNONE ? NONE : v;
         }
     }
     __syncthreads();
