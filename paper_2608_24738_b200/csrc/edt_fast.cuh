@@ -529,6 +529,8 @@ __global__ void __launch_bounds__(256) plane_kernel(const __grid_constant__ Fast
 // their zero positions with two shuffles; the four voxels of the lane are then finished in registers.
 // Requires n0 % 4 == 0 (rows then start on 4-byte boundaries).
 // ---------------------------------------------------------------------------------------------
+// PLAIN: the key is off^2 alone (no row, no offset): for passes that carry values and need no site afterwards
+template <bool PLAIN = false>
 __device__ __forceinline__ void pass0_row_to_keys(const uint32_t v, int n0, int y, uint32_t* __restrict__ vrow,
                                                   int lane) {
     // v: the lane's four mask bytes of this row (0x01010101 for lanes beyond the row)
@@ -567,7 +569,7 @@ __device__ __forceinline__ void pass0_row_to_keys(const uint32_t v, int n0, int 
         for (int b = 0; b < 4; ++b) {
             const int a = min(dl[b], dr[b]);
             const int off = dl[b] <= dr[b] ? -a : a;
-            kk[b] = ((uint32_t)(a * a) << 16) | ((uint32_t)y << 8) | ((uint32_t)off & 0xffu);
+            kk[b] = PLAIN ? (uint32_t)(a * a) : (((uint32_t)(a * a) << 16) | ((uint32_t)y << 8) | ((uint32_t)off & 0xffu));
         }
         keys = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
@@ -597,7 +599,7 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
 #pragma unroll
         for (int i = 0; i < MAXR; ++i) {
             const int y = warp + i * nwarps;
-            if (y < n1) pass0_row_to_keys(rowv[i], n0, y, val + y * VS, lane);
+            if (y < n1) pass0_row_to_keys<(VC != 0)>(rowv[i], n0, y, val + y * VS, lane);
         }
     }
     __syncthreads();
@@ -609,7 +611,7 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
         const int c = cg * 32 + lane;
         if (c >= n0) continue;
         uint32_t best[R];
-        scan_keys_group<VS, R, 16>(val + c, n1, y0, best);
+        scan_keys_group<VS, R, VC != 0 ? 0 : 16>(val + c, n1, y0, best);
         const int64_t p0 = plane * (int64_t)n1 * n0 + (int64_t)y0 * n0 + c;
 #pragma unroll
         for (int i = 0; i < R; ++i) {
@@ -620,9 +622,9 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
             const int j = (int)((b >> 8) & 0xffu);
             if (!FINAL) {
                 if (VC == 2) {
-                    reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)(none ? 0xffffu : (b >> 16));
+                    reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)(none ? 0xffffu : b);
                 } else if (VC == 4) {
-                    reinterpret_cast<uint32_t*>(P.out)[p0 + (int64_t)i * n0] = none ? 0xffffffffu : (b >> 16);
+                    reinterpret_cast<uint32_t*>(P.out)[p0 + (int64_t)i * n0] = none ? 0xffffffffu : b;
                 } else {
                     const uint32_t e = none ? 0x80u : ((b & 0xffu) | ((uint32_t)((j - y) & 0xff) << 8));
                     reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)e;
@@ -920,7 +922,8 @@ __device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n
         for (int b = 0; b < 4; ++b) {
             const int a = min(dl[b], dr[b]);
             const int off = dl[b] <= dr[b] ? -a : a;
-            kk[b] = ((uint32_t)(s0 * a * a) << kScaledShift) | (uint32_t)y;
+            // without offsets no site is needed afterwards: the key is the plain value, without row bits
+            kk[b] = WITH_OFF ? (((uint32_t)(s0 * a * a) << kScaledShift) | (uint32_t)y) : (uint32_t)(s0 * a * a);
             if (WITH_OFF) dpack |= ((uint32_t)off & 0xffu) << (8 * b);
         }
         kv = make_uint4(kk[0], kk[1], kk[2], kk[3]);
@@ -978,14 +981,14 @@ __global__ void __launch_bounds__(512, VC ? 3 : 2) plane_scaled_kernel(const __g
     }
     for (int y0 = r0 * R; y0 < n1; y0 += rstep * R) {
         uint32_t best[R];
-        scan_keys_group<VS, R, kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
+        scan_keys_group<VS, R, (VC && !FINAL) ? 0 : kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (y0 + i >= n1) break;
             if (!FINAL && VC) {
                 const uint32_t b = best[i];
                 reinterpret_cast<uint32_t*>(P.out)[plane * (int64_t)n1 * n0 + (int64_t)(y0 + i) * n0 + c] =
-                    b >= kNoneKey16 ? 0xffffffffu : (b >> kScaledShift);
+                    b >= kNoneKey16 ? 0xffffffffu : b;
             } else {
                 emit_scaled<1, FINAL, uint8_t>(out, dxt + c, VS, y0 + i, best[i], P.inv_scale);
             }
