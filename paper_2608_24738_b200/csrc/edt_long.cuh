@@ -142,7 +142,8 @@ __global__ void __launch_bounds__(256) long_row_kernel(const __grid_constant__ W
 // load and store of the warp is contiguous.  The zero bits of the row are collected as ballot words in shared
 // memory (at most 256 of them); a voxel finds its nearest zero to the left and to the right inside its own word
 // with __clz / __ffs, and otherwise takes the last zero before / first zero after the word.
-// SH >= 0: wide-path keys (off^2 << SH | row index along the second axis); SH == -1: float32 heights; SH == -2: plain
+// SH > 0: wide-path keys (off^2 << SH | row index along the second axis); SH == 0: plain off^2 with the wide path's
+// "no site" value; SH == -1: float32 heights; SH == -2: plain
 // integer heights.
 template <int SH>
 __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant__ WideParams P) {
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant
     if (row >= P.rows) return;  // the whole warp leaves together
     constexpr bool FLT = SH == -1;
     const int n0 = P.n0;
-    const uint32_t yrow = SH >= 0 ? (uint32_t)(row % P.n1) : 0u;
+    const uint32_t yrow = SH > 0 ? (uint32_t)(row % P.n1) : 0u;
     const int W = (n0 + 31) >> 5;
     const uint8_t* src = P.in + row * n0;
     for (int b = 0; b < W; ++b) {

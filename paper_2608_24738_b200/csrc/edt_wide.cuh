@@ -27,7 +27,8 @@ struct WideParams {
     float w2x;           // squared sampling of the contiguous axis (float-height variant)
 };
 
-// SH >= 0: integer keys (off^2 << SH | row).  SH < 0: float32 heights w^2 off^2 for general sampling (+inf = no site).
+// SH > 0: integer keys (off^2 << SH | row).  SH == 0: the plain integer off^2 (no site is needed afterwards: no index
+// output).  SH < 0: float32 heights w^2 off^2 for general sampling (+inf = no site).
 template <int VPL, int SH>  // voxels per lane (16 or 32), row bits of the key
 __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ WideParams P) {
     const int lane = threadIdx.x & 31;
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
             const int dr = cur - (x0 + b);
             const int a = min(dl[b], dr);
             offs[b] = (int16_t)(dl[b] <= dr ? -a : a);
-            keys[b] = SH < 0 ? __float_as_uint(P.w2x * (float)(a * a)) : (((uint32_t)(a * a) << (SH < 0 ? 0 : SH)) | (uint32_t)y);
+            keys[b] = SH < 0 ? __float_as_uint(P.w2x * (float)(a * a)) : (SH == 0 ? (uint32_t)(a * a) : (((uint32_t)(a * a) << (SH < 0 ? 0 : SH)) | (uint32_t)y));
         }
     }
 #pragma unroll
@@ -180,7 +181,7 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     constexpr int R = 4;
     constexpr uint32_t kRowMask = SH < 0 ? 0u : (1u << (SH < 0 ? 0 : SH)) - 1u;
     const int64_t col_base = slab_base + c;  // voxel (row 0) of this column
-    const uint32_t next_row = FINAL ? 0u : (uint32_t)(slab % P.next_n);
+    const uint32_t next_row = (FINAL || SH == 0) ? 0u : (uint32_t)(slab % P.next_n);  // SH == 0: plain values, no row bits
     // own coordinates along the earlier axes (final pass, index output): plane 0 = contiguous axis
     const int cx = (int)(c % P.n0);
     const int cyz = (int)(c / P.n0);

@@ -613,7 +613,8 @@ template <int K, bool FINAL>
 static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, int sh, cudaStream_t st) {
     const int strips = (int)((A.inner + 31) / 32);
     const size_t smem = (size_t)A.n * 32 * 4;
-    auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1> : (sh == 10 ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>);
+    auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1>
+                       : (sh == 0 ? wide_axis_kernel<K, FINAL, 0> : (sh == 10 ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>));
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -648,20 +649,24 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     // heights.  A lane of the row kernel takes 16 voxels (rows up to 512) or 32.
     int nmax = 1;
     for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
-    const int sh = !pl.unit ? -1 : (nmax > 512 ? 10 : 9);
+    // without an index output no site is needed afterwards: plain values as keys (sh = 0)
+    const int sh = !pl.unit ? -1 : (!carry ? 0 : (nmax > 512 ? 10 : 9));
     prof_mark(st, "row_keys", (double)pl.N * (1.0 + 4.0 + (carry ? 2.0 : 0.0)));
     const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
     if (pl.ext[0] % 16 != 0 || ((uintptr_t)in & 15u) != 0) {
         // rows that are not 16-byte aligned: one voxel per lane, ballot words
         if (sh < 0) long_row_any_kernel<-1><<<row_blocks, 256, 0, st>>>(P);
+        else if (sh == 0) long_row_any_kernel<0><<<row_blocks, 256, 0, st>>>(P);
         else if (sh == 9) long_row_any_kernel<9><<<row_blocks, 256, 0, st>>>(P);
         else long_row_any_kernel<10><<<row_blocks, 256, 0, st>>>(P);
     } else if (pl.ext[0] <= 512) {
         if (sh < 0) row_keys_kernel<16, -1><<<row_blocks, 256, 0, st>>>(P);
+        else if (sh == 0) row_keys_kernel<16, 0><<<row_blocks, 256, 0, st>>>(P);
         else if (sh == 9) row_keys_kernel<16, 9><<<row_blocks, 256, 0, st>>>(P);
         else row_keys_kernel<16, 10><<<row_blocks, 256, 0, st>>>(P);
     } else {
         if (sh < 0) row_keys_kernel<32, -1><<<row_blocks, 256, 0, st>>>(P);
+        else if (sh == 0) row_keys_kernel<32, 0><<<row_blocks, 256, 0, st>>>(P);
         else row_keys_kernel<32, 10><<<row_blocks, 256, 0, st>>>(P);
     }
     ++launches;
