@@ -226,6 +226,16 @@ __device__ __forceinline__ void scan_keys_group(const uint32_t* __restrict__ col
     uint32_t k[R];
 #pragma unroll
     for (int i = 0; i < R; ++i) k[i] = y0 + i < n ? col[(y0 + i) * VS] : NONE;
+    if (SH == 0) {  // plain values: a group of background voxels is all zeros
+        uint32_t any = k[0];
+#pragma unroll
+        for (int i = 1; i < R; ++i) any |= k[i];
+        if (any == 0u) {
+#pragma unroll
+            for (int i = 0; i < R; ++i) best[i] = 0u;
+            return;
+        }
+    }
 #pragma unroll
     for (int i = 0; i < R; ++i) {
         best[i] = k[i];
@@ -893,6 +903,10 @@ __device__ __forceinline__ void pass0_row_to_scaled_keys(const uint32_t v, int n
     if (any == 0u) {  // no background in this row
         kv = make_uint4(kNoneKey16, kNoneKey16, kNoneKey16, kNoneKey16);
         dpack = 0x80808080u;
+    } else if (__all_sync(0xffffffffu, m == 0x80808080u || !act)) {  // nothing but background: every distance is 0
+        const uint32_t k0 = WITH_OFF ? (uint32_t)y : 0u;
+        kv = make_uint4(k0, k0, k0, k0);
+        dpack = 0u;
     } else {
         const int lzin = m ? (31 - __clz(m)) >> 3 : 0;
         const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;
