@@ -551,6 +551,8 @@ __device__ __forceinline__ void pass0_row_to_keys(const uint32_t v, int n0, int 
     uint4 keys;
     if (any == 0u) {  // no background in this row
         keys = make_uint4(kNoneKey16, kNoneKey16, kNoneKey16, kNoneKey16);
+    } else if (PLAIN && __all_sync(0xffffffffu, m == 0x80808080u || !act)) {  // nothing but background: all zero
+        keys = make_uint4(0u, 0u, 0u, 0u);
     } else {
         const int lzin = m ? (31 - __clz(m)) >> 3 : 0;   // highest zero byte of this lane
         const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;    // lowest zero byte of this lane
