@@ -145,37 +145,41 @@ __device__ __forceinline__ float scan_heights_plain(const uint32_t* __restrict__
     return best;
 }
 
-template <int K, bool FINAL, int SH>
+// CW: columns of a strip (32, or 16 for long axes: smaller tiles, more blocks per SM, two row groups per warp)
+template <int K, bool FINAL, int SH, int CW = 32>
 __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ WideAxisParams P,
                                                         const __grid_constant__ EpilogueParams ep,
                                                         const int strips_per_slab) {
     extern __shared__ __align__(16) uint8_t sm_wide[];
-    uint32_t* val = reinterpret_cast<uint32_t*>(sm_wide);  // [n][32]
+    uint32_t* val = reinterpret_cast<uint32_t*>(sm_wide);  // [n][CW]
     const int n = P.n;
     const unsigned part = blockIdx.x % (unsigned)P.row_parts, sidx = blockIdx.x / (unsigned)P.row_parts;
     const int64_t slab = sidx / (unsigned)strips_per_slab;
-    const int64_t c0 = (int64_t)(sidx - slab * strips_per_slab) * 32;
+    const int64_t c0 = (int64_t)(sidx - slab * strips_per_slab) * CW;
     const int64_t slab_base = slab * (int64_t)n * P.inner;
     const uint32_t* src = P.keys_in + slab_base + c0;
     // rows of this block (a multiple of R per part); every part stages the whole strip, a scan may reach any row
     const int rows_per_part = ((n + P.row_parts - 1) / P.row_parts + 3) & ~3;
     const int y_begin = (int)part * rows_per_part, y_end = min(n, y_begin + rows_per_part);
-    // stage: 8 threads copy one row of 32 keys in 16-byte pieces when rows are 16-byte aligned, single keys otherwise
-    const int width = (int)min((int64_t)32, P.inner - c0);
+    // stage: CW / 4 threads copy one row of keys in 16-byte pieces when rows are 16-byte aligned, single keys otherwise
+    const int width = (int)min((int64_t)CW, P.inner - c0);
+    constexpr int TPR = CW / 4;
     if ((P.inner & 3) == 0) {
-        for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
-            const int y = t >> 3, ch = t & 7;
+        for (int t = threadIdx.x; t < n * TPR; t += blockDim.x) {
+            const int y = t / TPR, ch = t % TPR;
             if (4 * ch < width)
-                *reinterpret_cast<uint4*>(val + y * 32 + 4 * ch) = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + 4 * ch);
+                *reinterpret_cast<uint4*>(val + y * CW + 4 * ch) = *reinterpret_cast<const uint4*>(src + (int64_t)y * P.inner + 4 * ch);
         }
     } else {
-        for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
-            const int y = t >> 5, x = t & 31;
-            if (x < width) val[y * 32 + x] = src[(int64_t)y * P.inner + x];
+        for (int t = threadIdx.x; t < n * CW; t += blockDim.x) {
+            const int y = t / CW, x = t % CW;
+            if (x < width) val[y * CW + x] = src[(int64_t)y * P.inner + x];
         }
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    constexpr int GPW = 32 / CW;  // row groups a warp works on at a time
+    const int lane = threadIdx.x & (CW - 1), sub = (threadIdx.x & 31) / CW;
     if (lane >= width) return;
     const int64_t c = c0 + lane;  // position along inner
     constexpr int R = 4;
@@ -186,11 +190,11 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
     const int cx = (int)(c % P.n0);
     const int cyz = (int)(c / P.n0);
     const int cy = K == 3 ? cyz % P.n1 : cyz, cz = K == 3 ? cyz / P.n1 : 0;
-    for (int y0 = y_begin + warp * R; y0 < y_end; y0 += nwarps * R) {
+    for (int y0 = y_begin + (warp * GPW + sub) * R; y0 < y_end; y0 += nwarps * GPW * R) {
         uint32_t best[R];
         int jrow[R];
         if (SH >= 0) {
-            scan_keys_group<32, R, (SH < 0 ? 9 : SH)>(val + lane, n, y0, best);
+            scan_keys_group<CW, R, (SH < 0 ? 9 : SH)>(val + lane, n, y0, best);
 #pragma unroll
             for (int i = 0; i < R; ++i) jrow[i] = (int)(best[i] & kRowMask);
         } else {
@@ -200,10 +204,10 @@ __global__ void __launch_bounds__(512) wide_axis_kernel(const __grid_constant__ 
                 best[i] = 0u; jrow[i] = y;
                 if (y >= n) continue;
                 int bd;
-                best[i] = __float_as_uint(scan_heights_plain<32>(val + lane, n, y, P.w2, bd));
+                best[i] = __float_as_uint(scan_heights_plain<CW>(val + lane, n, y, P.w2, bd));
                 if (bd > 0) {
-                    const float lo = y - bd >= 0 ? __uint_as_float(val[(y - bd) * 32 + lane]) : TMEDT_INF;
-                    const float hi = y + bd < n ? __uint_as_float(val[(y + bd) * 32 + lane]) : TMEDT_INF;
+                    const float lo = y - bd >= 0 ? __uint_as_float(val[(y - bd) * CW + lane]) : TMEDT_INF;
+                    const float hi = y + bd < n ? __uint_as_float(val[(y + bd) * CW + lane]) : TMEDT_INF;
                     jrow[i] = lo <= hi ? y - bd : y + bd;
                 }
             }

@@ -609,25 +609,35 @@ static cudaError_t run_small(const Plan& pl, const uint8_t* in, const EpiloguePa
 
 // Unit sampling beyond extent 128 (two axes up to 1024, three up to 512): key rows, then strip scans.
 // sh: row bits of the integer keys (9 or 10), or -1 for float heights
-template <int K, bool FINAL>
-static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, int sh, cudaStream_t st) {
-    const int strips = (int)((A.inner + 31) / 32);
-    const size_t smem = (size_t)A.n * 32 * 4;
-    auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1>
-                       : (sh == 0 ? wide_axis_kernel<K, FINAL, 0> : (sh == 10 ? wide_axis_kernel<K, FINAL, 10> : wide_axis_kernel<K, FINAL, 9>));
+template <int K, bool FINAL, int CW>
+static cudaError_t launch_wide_axis_cw(const WideAxisParams& A, const EpilogueParams& ep, int sh, cudaStream_t st) {
+    const int strips = (int)((A.inner + CW - 1) / CW);
+    const size_t smem = (size_t)A.n * CW * 4;
+    auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1, CW>
+                       : (sh == 0 ? wide_axis_kernel<K, FINAL, 0, CW>
+                                  : (sh == 10 ? wide_axis_kernel<K, FINAL, 10, CW> : wide_axis_kernel<K, FINAL, 9, CW>));
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    // 16 warps per strip from 384 rows on: shared memory allows few blocks per SM there, and a strip's rows
-    // are independent work
     // few strips (a single large image): several blocks share a strip, each taking a range of its rows, until
     // there are about two blocks per SM
     WideAxisParams B = A;
     const int64_t base_blocks = A.outer * strips;
     B.row_parts = (int)std::max<int64_t>(1, std::min<int64_t>(std::min(8, A.n / 64), 296 / base_blocks));
-    kern<<<(unsigned)(base_blocks * B.row_parts), A.n >= 384 ? 512 : 256, smem, st>>>(B, ep, strips);
+    // 16 warps per strip from 384 rows on (8 for the narrow strips): a strip's rows are independent work
+    const int threads = A.n >= 384 ? (CW == 32 ? 512 : 256) : 256;
+    kern<<<(unsigned)(base_blocks * B.row_parts), threads, smem, st>>>(B, ep, strips);
     return cudaGetLastError();
+}
+
+// sh: row bits of the integer keys (9 or 10), 0 for plain values, or -1 for float heights
+template <int K, bool FINAL>
+static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParams& ep, int sh, cudaStream_t st) {
+    // long axes: strips of 16 columns (half the shared memory per block, so more blocks are resident and the
+    // grid divides more evenly over the SMs)
+    const int cw = A.n > 256 && A.inner >= 32 ? 16 : 32;
+    return cw == 16 ? launch_wide_axis_cw<K, FINAL, 16>(A, ep, sh, st) : launch_wide_axis_cw<K, FINAL, 32>(A, ep, sh, st);
 }
 
 static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
