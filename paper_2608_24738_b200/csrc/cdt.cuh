@@ -85,39 +85,43 @@ __global__ void __launch_bounds__(256) cdt_row_kernel(const __grid_constant__ Ro
     }
 }
 
-// A further axis of up to 1024 rows: a block stages an (n x 32) strip of values in shared memory (rows of 128
-// contiguous bytes) and a warp scans four consecutive rows of its 32 columns at a time, so that every row fetched
+// A further axis of up to 1024 rows: a block stages an (n x CW) strip of values in shared memory (rows of 128 or
+// 64 contiguous bytes) and a warp scans four consecutive rows of its 32 columns at a time, so that every row fetched
 // from the tile serves four voxels.  The nearest candidate of a step is d rows away, which ends the scan once d
 // reaches the largest of the four minima.
-template <bool CHESS>
+// CW: columns of a strip (32, or 16 for long axes: half the shared memory per block, two row groups per warp).
+template <bool CHESS, int CW>
 __global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ PassParams P, const int strips_per_slab) {
-    extern __shared__ __align__(16) int sm_cdt[];  // [n][32]
+    extern __shared__ __align__(16) int sm_cdt[];  // [n][CW]
     const int n = P.n;
     const int64_t slab = blockIdx.x / strips_per_slab;
-    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
+    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * CW;
     const int64_t base = slab * (int64_t)n * P.inner + c0;
-    const int width = (int)min((int64_t)32, P.inner - c0);
-    if ((P.inner & 3) == 0) {  // rows are 16-byte aligned: eight threads copy one row of 32 values
+    const int width = (int)min((int64_t)CW, P.inner - c0);
+    constexpr int TPR = CW / 4;
+    if ((P.inner & 3) == 0) {  // rows are 16-byte aligned: CW / 4 threads copy one row
 #pragma unroll 4
-        for (int t = threadIdx.x; t < n * 8; t += blockDim.x) {
-            const int y = t >> 3, ch = t & 7;
+        for (int t = threadIdx.x; t < n * TPR; t += blockDim.x) {
+            const int y = t / TPR, ch = t % TPR;
             if (4 * ch < width)
-                *reinterpret_cast<int4*>(sm_cdt + y * 32 + 4 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 4 * ch);
+                *reinterpret_cast<int4*>(sm_cdt + y * CW + 4 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 4 * ch);
         }
     } else {
-        for (int t = threadIdx.x; t < n * 32; t += blockDim.x) {
-            const int y = t >> 5, x = t & 31;
-            if (x < width) sm_cdt[t] = P.in[base + (int64_t)y * P.inner + x];
+        for (int t = threadIdx.x; t < n * CW; t += blockDim.x) {
+            const int y = t / CW, x = t % CW;
+            if (x < width) sm_cdt[y * CW + x] = P.in[base + (int64_t)y * P.inner + x];
         }
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    constexpr int GPW = 32 / CW;  // row groups a warp works on at a time
+    const int lane = threadIdx.x & (CW - 1), sub = (threadIdx.x & 31) / CW;
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     if (lane >= width) return;
     auto op = [](int v, int d) { return CHESS ? max(v, d) : v + d; };
-    for (int y0 = warp * 4; y0 < n; y0 += nwarps * 4) {
+    for (int y0 = (warp * GPW + sub) * 4; y0 < n; y0 += nwarps * GPW * 4) {
         int k[4], best[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) k[i] = y0 + i < n ? sm_cdt[(y0 + i) * 32 + lane] : kBig;
+        for (int i = 0; i < 4; ++i) k[i] = y0 + i < n ? sm_cdt[(y0 + i) * CW + lane] : kBig;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             best[i] = k[i];
@@ -129,8 +133,8 @@ __global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ 
         int mx = max(max(best[0], best[1]), max(best[2], best[3]));
         int lo = y0 - 1, hi = y0 + 4;
         for (int d = 1; d < mx && (lo >= 0 || hi < n); ++d, --lo, ++hi) {
-            const int vlo = lo >= 0 ? sm_cdt[lo * 32 + lane] : kBig;
-            const int vhi = hi < n ? sm_cdt[hi * 32 + lane] : kBig;
+            const int vlo = lo >= 0 ? sm_cdt[lo * CW + lane] : kBig;
+            const int vhi = hi < n ? sm_cdt[hi * CW + lane] : kBig;
 #pragma unroll
             for (int i = 0; i < 4; ++i) best[i] = min(best[i], min(op(vlo, d + i), op(vhi, d + 3 - i)));
             mx = max(max(best[0], best[1]), max(best[2], best[3]));

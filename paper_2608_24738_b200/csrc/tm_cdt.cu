@@ -73,12 +73,15 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
             R.mask = input; R.out = P.out; R.rows = g.total / P.n; R.n0 = P.n; R.last = P.last;
             cdt_row_kernel<<<(unsigned)((R.rows + 7) / 8), 256, 0, st>>>(R);
         } else if (k > 0 && P.n <= 1024) {
-            // strided axis: (n x 32) strips in shared memory
-            const int strips = (int)((P.inner + 31) / 32);
-            const size_t smem = (size_t)P.n * 32 * 4;
-            auto kern = chess ? cdt_strip_kernel<true> : cdt_strip_kernel<false>;
+            // strided axis: (n x 32) strips in shared memory, (n x 16) for axes longer than 256 rows
+            const int cw = P.n > 256 && P.inner >= 32 ? 16 : 32;
+            const int strips = (int)((P.inner + cw - 1) / cw);
+            const size_t smem = (size_t)P.n * cw * 4;
+            auto kern = cw == 16 ? (chess ? cdt_strip_kernel<true, 16> : cdt_strip_kernel<false, 16>)
+                                 : (chess ? cdt_strip_kernel<true, 32> : cdt_strip_kernel<false, 32>);
             if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            kern<<<(unsigned)(g.total / ((int64_t)P.n * P.inner) * strips), P.n >= 384 ? 512 : 256, smem, st>>>(P, strips);
+            const int threads = P.n >= 384 ? (cw == 32 ? 512 : 256) : 256;
+            kern<<<(unsigned)(g.total / ((int64_t)P.n * P.inner) * strips), threads, smem, st>>>(P, strips);
         } else {
             const unsigned blocks = (unsigned)((g.total + 255) / 256);
             if (chess) cdt_axis_kernel<true><<<blocks, 256, 0, st>>>(P);
