@@ -641,6 +641,9 @@ __global__ void __launch_bounds__(256) plane_unit_kernel(const __grid_constant__
                     const uint32_t e = none ? 0x80u : ((b & 0xffu) | ((uint32_t)((j - y) & 0xff) << 8));
                     reinterpret_cast<uint16_t*>(P.out)[p0 + (int64_t)i * n0] = (uint16_t)e;
                 }
+            } else if (VC != 0) {  // last pass without index output: plain values
+                if (ep.dist) __stcs(ep.dist + p0 + (int64_t)i * n0, none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)b)));
+                if (ep.sq) __stcs(reinterpret_cast<long long*>(ep.sq + p0 + (int64_t)i * n0), none ? (long long)INT64_MAX : (long long)b);
             } else if (dist_only) {
                 ep.dist[p0 + (int64_t)i * n0] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b >> 16)));
             } else {  // two processed axes: the plane is the image

@@ -412,7 +412,8 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     do {                                                                                                       \
         if (vs == 32) TM_LAUNCH_PLANE_UNIT(FIN, 32, VCV); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(FIN, 64, VCV); else TM_LAUNCH_PLANE_UNIT(FIN, 128, VCV); \
     } while (0)
-            if (fin) TM_LAUNCH_PLANE_UNIT_VS(true, 0);
+            if (fin && !ep.idx && !getenv("TM_EDT_NO_VALUE_CARRY")) TM_LAUNCH_PLANE_UNIT_VS(true, 4);  // plain values: no site needed
+            else if (fin) TM_LAUNCH_PLANE_UNIT_VS(true, 0);
             else if (P.value_carry == 2) TM_LAUNCH_PLANE_UNIT_VS(false, 2);
             else if (P.value_carry == 4) TM_LAUNCH_PLANE_UNIT_VS(false, 4);
             else TM_LAUNCH_PLANE_UNIT_VS(false, 0);

@@ -578,7 +578,8 @@ def test_strided_masks_are_gathered_by_the_library():
 
 
 VALUE_SHAPES = [(2, 1, 12, 20, 24), (1, 2, 33, 17, 40), (1, 1, 128, 20, 48), (2, 1, 6, 10, 12, 8), (1, 1, 16, 40, 24, 32),
-                (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128), (1, 1, 128, 128, 128), (1, 1, 9, 10, 11)]
+                (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128), (1, 1, 128, 128, 128), (1, 1, 9, 10, 11),
+                (3, 1, 40, 36), (1, 2, 128, 128), (2, 1, 7, 12), (2, 1, 1, 64, 1, 100)]  # two processed axes: the plane kernel is the last
 
 
 @pytest.mark.parametrize("shape", VALUE_SHAPES, ids=["x".join(map(str, s)) for s in VALUE_SHAPES])
