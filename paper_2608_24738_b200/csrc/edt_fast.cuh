@@ -1000,7 +1000,7 @@ __global__ void __launch_bounds__(512, VC ? 3 : 2) plane_scaled_kernel(const __g
     }
     for (int y0 = r0 * R; y0 < n1; y0 += rstep * R) {
         uint32_t best[R];
-        scan_keys_group<VS, R, (VC && !FINAL) ? 0 : kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
+        scan_keys_group<VS, R, VC ? 0 : kScaledShift>(val + c, n1, y0, best, (uint32_t)P.sk);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             if (y0 + i >= n1) break;
@@ -1008,6 +1008,10 @@ __global__ void __launch_bounds__(512, VC ? 3 : 2) plane_scaled_kernel(const __g
                 const uint32_t b = best[i];
                 reinterpret_cast<uint32_t*>(P.out)[plane * (int64_t)n1 * n0 + (int64_t)(y0 + i) * n0 + c] =
                     b >= kNoneKey16 ? 0xffffffffu : b;
+            } else if (FINAL && VC) {  // last pass, distances only: plain values
+                const uint32_t b = best[i];
+                __stcs(ep.dist + plane * ep.V + (int64_t)(y0 + i) * n0 + c,
+                       b >= kNoneKey16 ? TMEDT_INF : fast_sqrt(__uint2float_rn(b) * P.inv_scale));
             } else {
                 emit_scaled<1, FINAL, uint8_t>(out, dxt + c, VS, y0 + i, best[i], P.inv_scale);
             }

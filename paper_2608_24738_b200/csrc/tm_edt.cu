@@ -502,7 +502,8 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
     {
         const bool fin = pl.E == 2;
         const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
-        const size_t smem = (size_t)pl.ext[1] * vs * ((vc && !fin) ? 4 : 5);  // keys, plus a byte tile of first-axis offsets
+        const bool plain_fin = fin && !ep.idx && ep.dist && !getenv("TM_EDT_NO_VALUE_CARRY");
+        const size_t smem = (size_t)pl.ext[1] * vs * (((vc && !fin) || plain_fin) ? 4 : 5);  // keys, plus a byte tile of first-axis offsets
         prof_mark(st, fin ? "plane_scaled_final" : "plane_scaled", (double)pl.N * (1.0 + (fin ? out_bpv : (vc ? 4.0 : 2.0))));
 #define TM_LAUNCH_PLANE_SCALED(FIN, VSV, VCV)                                                                  \
     do {                                                                                                       \
@@ -510,7 +511,8 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
         kern<<<(unsigned)P.outer, 512, smem, st>>>(P, ep);                                                     \
     } while (0)
-        if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, false); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, false); else TM_LAUNCH_PLANE_SCALED(true, 128, false); }
+        if (fin && !ep.idx && ep.dist && !getenv("TM_EDT_NO_VALUE_CARRY")) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, true); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, true); else TM_LAUNCH_PLANE_SCALED(true, 128, true); }
+        else if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, false); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, false); else TM_LAUNCH_PLANE_SCALED(true, 128, false); }
         else if (vc) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(false, 32, true); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(false, 64, true); else TM_LAUNCH_PLANE_SCALED(false, 128, true); }
         else { if (vs == 32) TM_LAUNCH_PLANE_SCALED(false, 32, false); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(false, 64, false); else TM_LAUNCH_PLANE_SCALED(false, 128, false); }
 #undef TM_LAUNCH_PLANE_SCALED
