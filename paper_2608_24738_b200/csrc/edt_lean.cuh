@@ -1,0 +1,383 @@
+// Quad-per-lane kernels of the packed-entry path (extents up to 128, three or four processed axes, contiguous
+// extent a multiple of 4, 16-byte aligned outputs): the same passes as edt_fast.cuh and edt_value.cuh,
+//     g_k(x) = min_j [ g_{k-1}(x with x_k := j) + (w_k (x_k - j))^2 ]        (paper, Section 2.3.2)
+// taken as exact bounded scans on integer keys, with a thread mapping chosen for instruction count:
+//
+//   * a lane owns four neighbouring voxels of ONE row of the axis (a "quad": four consecutive positions of the
+//     contiguous index), so a candidate row is fetched with one 16-byte shared-memory load and serves four
+//     voxels with the same addend (an immediate in the unrolled steps), and a quad's results leave in one or
+//     two 16-byte stores;
+//   * the key tile carries kLeanPad rows of "no site" keys above and below, so the first steps of every scan
+//     run without bounds tests;
+//   * nothing is decided per voxel that can be decided per block or per template instance.
+//
+// Keys: entries mode   (sum of squared offsets << 8) | row     (plane kernel: off^2 << 16 | row << 8 | off)
+//       value mode     the squared distance so far, times the common scale in scaled-integer mode
+// "No site" is 2^31 in both; every real key and every addend stays below it (checked by the planner).
+#pragma once
+#include "edt_fast.cuh"
+
+namespace tmedt {
+
+constexpr uint32_t kLeanNone = 0x80000000u;
+constexpr int kLeanPad = 4;
+
+struct LeanParams {
+    const void* in;      // mask (plane kernel), entries or values of the earlier axes (column kernels)
+    void* out;           // entries or values including this axis (unused by final kernels)
+    int64_t inner;       // voxels between consecutive rows of the axis
+    int n;               // extent of the axis
+    int n0;              // plane kernel: extent of the contiguous axis
+    int tiles_per_slab;  // column kernels: tiles of TX columns per (n x inner) slab
+    uint32_t wk;         // integer weight of the axis: a row at distance d adds wk * d^2 (1 under unit sampling)
+    uint32_t w0;         // plane kernel: integer weight of the contiguous axis
+    float inv_scale;     // final value kernels: 1 / common scale (1 under unit sampling)
+    int shift[4];        // final entry kernels: log2 of the extent of plane q, or -1 if it is no power of two
+};
+
+// Bounded scan of one quad.  own: the quad's keys inside the padded tile (row pitch PITCH words).
+// Row distance d adds (wk d^2) << SH; the scan of a voxel may stop once that addend reaches its best key.
+template <int PITCH, int SH>
+__device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, const int y, const int n,
+                                          const uint32_t wk, uint32_t (&b)[4]) {
+    {
+        const uint4 v = *reinterpret_cast<const uint4*>(own);
+        b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
+    }
+    uint32_t mx = max(max(b[0], b[1]), max(b[2], b[3]));
+    if (mx < (1u << SH)) return;  // four background voxels
+#pragma unroll
+    for (int s = 1; s <= kLeanPad; ++s) {
+        if (s == 3 && ((wk * 9u) << SH) >= mx) return;
+        const uint32_t a = (wk * (uint32_t)(s * s)) << SH;
+        const uint4 lo = *reinterpret_cast<const uint4*>(own - s * PITCH);
+        const uint4 hi = *reinterpret_cast<const uint4*>(own + s * PITCH);
+        b[0] = __viaddmin_u32(lo.x, a, b[0]); b[1] = __viaddmin_u32(lo.y, a, b[1]);
+        b[2] = __viaddmin_u32(lo.z, a, b[2]); b[3] = __viaddmin_u32(lo.w, a, b[3]);
+        b[0] = __viaddmin_u32(hi.x, a, b[0]); b[1] = __viaddmin_u32(hi.y, a, b[1]);
+        b[2] = __viaddmin_u32(hi.z, a, b[2]); b[3] = __viaddmin_u32(hi.w, a, b[3]);
+        if (s == 2) mx = max(max(b[0], b[1]), max(b[2], b[3]));
+    }
+    mx = max(max(b[0], b[1]), max(b[2], b[3]));
+    int d = kLeanPad + 1;
+    uint32_t a = (wk * (uint32_t)(d * d)) << SH;
+    if (a >= mx) return;
+    const int up = y, dn = n - 1 - y;
+    const uint32_t* plo = own - d * PITCH;
+    const uint32_t* phi = own + d * PITCH;
+    for (; a < mx && (d <= up || d <= dn); ++d, plo -= PITCH, phi += PITCH) {
+        if (d <= up) {
+            const uint4 lo = *reinterpret_cast<const uint4*>(plo);
+            b[0] = __viaddmin_u32(lo.x, a, b[0]); b[1] = __viaddmin_u32(lo.y, a, b[1]);
+            b[2] = __viaddmin_u32(lo.z, a, b[2]); b[3] = __viaddmin_u32(lo.w, a, b[3]);
+        }
+        if (d <= dn) {
+            const uint4 hi = *reinterpret_cast<const uint4*>(phi);
+            b[0] = __viaddmin_u32(hi.x, a, b[0]); b[1] = __viaddmin_u32(hi.y, a, b[1]);
+            b[2] = __viaddmin_u32(hi.z, a, b[2]); b[3] = __viaddmin_u32(hi.w, a, b[3]);
+        }
+        mx = max(max(b[0], b[1]), max(b[2], b[3]));
+        a = (wk * (uint32_t)((d + 1) * (d + 1))) << SH;
+    }
+}
+
+// "No site" rows above and below the tile.
+template <int PITCH>
+__device__ __forceinline__ void lean_fill_pad(uint32_t* __restrict__ kt, const int n) {
+    constexpr int QPR = PITCH / 4;
+    for (int t = threadIdx.x; t < 2 * kLeanPad * QPR; t += blockDim.x) {
+        const int r = t / QPR, q = t - r * QPR;
+        const int row = r < kLeanPad ? r : n + r;
+        *reinterpret_cast<uint4*>(kt + row * PITCH + 4 * q) = make_uint4(kLeanNone, kLeanNone, kLeanNone, kLeanNone);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// First and second axis of one (n1 x n0) plane per block.
+//   VT == void      entries: writes 2-byte entries (first-axis offset, second-axis offset)
+//   VT == uint16_t  values:  writes the squared distance so far (all ones = no site)
+//   VT == uint32_t  values:  writes the (scaled) squared distance so far (2^31 = no site)
+// ---------------------------------------------------------------------------------------------
+template <int VS, typename VT>
+__global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constant__ LeanParams P) {
+    constexpr bool ENT = sizeof(VT) == 1;  // VT = uint8_t stands for "entries"
+    constexpr int SH = ENT ? 16 : 0;
+    extern __shared__ __align__(16) uint8_t sm_lean_p[];
+    uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_p);  // [n1 + 2 kLeanPad][VS]
+    const int n0 = P.n0, n1 = P.n;
+    const int64_t plane = blockIdx.x;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NW = 8;
+    lean_fill_pad<VS>(kt, n1);
+    {
+        constexpr int MAXR = 16;  // rows per warp: 128 rows / 8 warps
+        uint32_t rowv[MAXR];
+        const bool act = 4 * lane < n0;
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * NW;
+            rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
+        }
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int y = warp + i * NW;
+            if (y < n1) {
+                if (ENT) pass0_row_to_keys<false>(rowv[i], n0, y, kt + (y + kLeanPad) * VS, lane);
+                else pass0_row_to_scaled_keys<false>(rowv[i], n0, y, (int)P.w0, kt + (y + kLeanPad) * VS, nullptr, lane);
+            }
+        }
+    }
+    __syncthreads();
+    // a warp takes patches of 4 rows x 32 columns (8 quads per row): neighbouring voxels have similar scan lengths
+    constexpr int CG = VS / 32;
+    const int r = lane >> 3, q4 = 4 * (lane & 7);
+    const int64_t base0 = plane * (int64_t)n1 * n0;
+    const int patches = ((n1 + 3) >> 2) * CG;
+    for (int t = warp; t < patches; t += NW) {
+        const int y = 4 * (t / CG) + r, c4 = 32 * (t % CG) + q4;
+        if (y >= n1 || c4 >= n0) continue;
+        const int64_t base = base0 + c4;
+        uint32_t b[4];
+        lean_scan<VS, SH>(kt + (y + kLeanPad) * VS + c4, y, n1, ENT ? 1u : P.wk, b);
+        const int64_t p = base + (int64_t)y * n0;
+        if (ENT) {
+            uint32_t e[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const uint32_t j = (b[v] >> 8) & 0xffu;
+                e[v] = b[v] >= kLeanNone ? 0x80u : ((b[v] & 0xffu) | (((j - (uint32_t)y) & 0xffu) << 8));
+            }
+            *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.out) + p) = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+        } else if (sizeof(VT) == 2) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) b[v] = min(b[v], 0xffffu);
+            *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.out) + p) = make_uint2(b[0] | (b[1] << 16), b[2] | (b[3] << 16));
+        } else {
+            *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(P.out) + p) = make_uint4(b[0], b[1], b[2], b[3]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// One further axis on entries (unit sampling, index output requested).  K earlier axes, K = 2 or 3.
+//   FINAL == false  (K == 2)  writes 4-byte entries
+//   FINAL == true             writes float32 distances and / or int64 squared distances, and the index planes
+//                             (every spatial axis is a processed axis, coordinate layout)
+// ---------------------------------------------------------------------------------------------
+// Four zero-extended 32-bit values as four int64: one 256-bit streaming store (p 32-byte aligned).
+__device__ __forceinline__ void lean_store_4xi64(int64_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    const uint32_t z = 0u;
+    asm volatile("st.global.cs.v8.b32 [%0], {%1, %5, %2, %5, %3, %5, %4, %5};"
+                 :: "l"(p), "r"(a), "r"(b), "r"(c), "r"(d), "r"(z) : "memory");
+}
+
+__device__ __forceinline__ int lean_sext_byte(uint32_t e, int q) {
+    // byte q of e, sign-extended: one byte-permute (bit 3 of a selector nibble replicates the sign of the byte)
+    const uint32_t sel = (uint32_t)q | ((8u | (uint32_t)q) << 4) | ((8u | (uint32_t)q) << 8) | ((8u | (uint32_t)q) << 12);
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(e), "r"(0u), "r"(sel));
+    return (int)r;
+}
+
+template <int K, bool FINAL, int TX>
+__global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const __grid_constant__ LeanParams P,
+                                                                         const __grid_constant__ EpilogueParams ep) {
+    using EI = typename EntryType<entry_bytes(K)>::type;
+    constexpr int LPR = TX / 4, CG = TX / 32, NW = 8;
+    extern __shared__ __align__(16) uint8_t sm_lean_c[];
+    const int n = P.n;
+    uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_c);                                  // [n + 2 kLeanPad][TX]
+    EI* et = reinterpret_cast<EI*>(sm_lean_c + (size_t)(n + 2 * kLeanPad) * TX * 4);        // [n][TX]
+    const int64_t slab = blockIdx.x / P.tiles_per_slab;
+    const int64_t i0 = (int64_t)(blockIdx.x - slab * P.tiles_per_slab) * TX;
+    const int width = (int)min((int64_t)TX, P.inner - i0);
+    const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
+    lean_fill_pad<TX>(kt, n);
+    for (int t = threadIdx.x; t < n * LPR; t += 256) {
+        const int y = t / LPR, q4 = 4 * (t % LPR);
+        if (q4 >= width) continue;
+        const EI* g = src + (int64_t)y * P.inner + q4;
+        uint32_t e[4];
+        if (sizeof(EI) == 2) {
+            const uint2 w = *reinterpret_cast<const uint2*>(g);
+            *reinterpret_cast<uint2*>(et + y * TX + q4) = w;
+            e[0] = w.x & 0xffffu; e[1] = w.x >> 16; e[2] = w.y & 0xffffu; e[3] = w.y >> 16;
+        } else {
+            const uint4 w = *reinterpret_cast<const uint4*>(g);
+            *reinterpret_cast<uint4*>(et + y * TX + q4) = w;
+            e[0] = w.x; e[1] = w.y; e[2] = w.z; e[3] = w.w;
+        }
+        uint32_t k[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+            k[v] = e[v] == 0x80u ? kLeanNone : (((uint32_t)__dp4a((int)e[v], (int)e[v], 0) << 8) | (uint32_t)y);
+        *reinterpret_cast<uint4*>(kt + (y + kLeanPad) * TX + q4) = make_uint4(k[0], k[1], k[2], k[3]);
+    }
+    __syncthreads();
+    // a warp takes patches of 4 rows x 32 columns (8 quads per row), always in the same 32 columns
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c4 = 32 * (warp % CG) + 4 * (lane & 7);
+    const int yfirst = 4 * (warp / CG) + (lane >> 3);
+    constexpr int YSTEP = 4 * (NW / CG);
+    if (c4 >= width) return;
+    const uint32_t v0 = (uint32_t)(i0 + c4);  // the quad's position among the earlier planes (plane 0 fastest)
+    if (!FINAL) {
+        uint32_t* out = reinterpret_cast<uint32_t*>(P.out) + slab * (int64_t)n * P.inner + v0;
+        for (int y = yfirst; y < n; y += YSTEP) {
+            uint32_t b[4], o[4];
+            lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const uint32_t j = b[v] & 0xffu;
+                const uint32_t e = (uint32_t)et[j * TX + c4 + v];
+                o[v] = b[v] >= kLeanNone ? 0x80u : (e | (((j - (uint32_t)y) & 0xffu) << (8 * K)));
+            }
+            *reinterpret_cast<uint4*>(out + (int64_t)y * P.inner) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        return;
+    }
+    // own coordinates along the earlier planes
+    int cq[K];
+    {
+        uint32_t rr = v0;
+#pragma unroll
+        for (int q = 0; q < K; ++q) {
+            if (P.shift[q] >= 0) {
+                cq[q] = (int)(rr & (((uint32_t)1 << P.shift[q]) - 1u));
+                rr >>= P.shift[q];
+            } else {
+                const uint32_t nq = (uint32_t)ep.ext[q], hi = rr / nq;
+                cq[q] = (int)(rr - hi * nq);
+                rr = hi;
+            }
+        }
+    }
+    float* const dist = ep.dist ? ep.dist + slab * ep.V : nullptr;
+    int64_t* const sq = ep.sq ? ep.sq + slab * ep.V : nullptr;
+    int64_t* ip[K + 1];
+#pragma unroll
+    for (int q = 0; q <= K; ++q) ip[q] = ep.idx + (slab * ep.ndim + ep.axis[q]) * ep.V;
+    for (int y = yfirst; y < n; y += YSTEP) {
+        uint32_t b[4];
+        lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+        const uint32_t p = (uint32_t)y * (uint32_t)P.inner + v0;  // inside one image: below 2^31
+        uint32_t e[4], j[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            j[v] = b[v] & 0xffu;
+            e[v] = (uint32_t)et[j[v] * TX + c4 + v];
+        }
+        if (((b[0] | b[1] | b[2] | b[3]) & kLeanNone) == 0u) {
+            if (dist) {
+                float4 d;
+                d.x = fast_sqrt(small_int_to_float((int)(b[0] >> 8))); d.y = fast_sqrt(small_int_to_float((int)(b[1] >> 8)));
+                d.z = fast_sqrt(small_int_to_float((int)(b[2] >> 8))); d.w = fast_sqrt(small_int_to_float((int)(b[3] >> 8)));
+                __stcs(reinterpret_cast<float4*>(dist + p), d);
+            }
+            if (sq) lean_store_4xi64(sq + p, b[0] >> 8, b[1] >> 8, b[2] >> 8, b[3] >> 8);
+#pragma unroll
+            for (int q = 0; q < K; ++q) {
+                uint32_t s[4];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) s[v] = (uint32_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
+                lean_store_4xi64(ip[q] + p, s[0], s[1], s[2], s[3]);
+            }
+            lean_store_4xi64(ip[K] + p, j[0], j[1], j[2], j[3]);
+        } else {  // an image without background: +inf, INT64_MAX, -1 (checked voxel by voxel)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const bool none = b[v] >= kLeanNone;
+                if (dist) dist[p + v] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b[v] >> 8)));
+                if (sq) sq[p + v] = none ? INT64_MAX : (int64_t)(b[v] >> 8);
+#pragma unroll
+                for (int q = 0; q < K; ++q)
+                    ip[q][p + v] = none ? (int64_t)-1 : (int64_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
+                ip[K][p + v] = none ? (int64_t)-1 : (int64_t)j[v];
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// One further axis on carried values (no index output): the key is the value itself.
+//   VT  uint16_t (all ones = no site) or uint32_t (2^31 = no site)
+//   FINAL == false  writes the new value;  FINAL == true  writes float32 distances and / or int64 squared distances
+// ---------------------------------------------------------------------------------------------
+template <bool FINAL, typename VT, int TX>
+__global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__ LeanParams P,
+                                                         const __grid_constant__ EpilogueParams ep) {
+    constexpr int LPR = TX / 4, CG = TX / 32, NW = 8;
+    extern __shared__ __align__(16) uint8_t sm_lean_v[];
+    const int n = P.n;
+    uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_v);  // [n + 2 kLeanPad][TX]
+    const int64_t slab = blockIdx.x / P.tiles_per_slab;
+    const int64_t i0 = (int64_t)(blockIdx.x - slab * P.tiles_per_slab) * TX;
+    const int width = (int)min((int64_t)TX, P.inner - i0);
+    const VT* src = reinterpret_cast<const VT*>(P.in) + slab * (int64_t)n * P.inner + i0;
+    lean_fill_pad<TX>(kt, n);
+    for (int t = threadIdx.x; t < n * LPR; t += 256) {
+        const int y = t / LPR, q4 = 4 * (t % LPR);
+        if (q4 >= width) continue;
+        const VT* g = src + (int64_t)y * P.inner + q4;
+        uint4 k;
+        if (sizeof(VT) == 2) {
+            const uint2 w = *reinterpret_cast<const uint2*>(g);
+            k = make_uint4(w.x & 0xffffu, w.x >> 16, w.y & 0xffffu, w.y >> 16);
+            if (k.x == 0xffffu) k.x = kLeanNone;
+            if (k.y == 0xffffu) k.y = kLeanNone;
+            if (k.z == 0xffffu) k.z = kLeanNone;
+            if (k.w == 0xffffu) k.w = kLeanNone;
+        } else {
+            k = *reinterpret_cast<const uint4*>(g);
+        }
+        *reinterpret_cast<uint4*>(kt + (y + kLeanPad) * TX + q4) = k;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c4 = 32 * (warp % CG) + 4 * (lane & 7);
+    const int yfirst = 4 * (warp / CG) + (lane >> 3);
+    constexpr int YSTEP = 4 * (NW / CG);
+    if (c4 >= width) return;
+    const int64_t col = slab * (int64_t)n * P.inner + i0 + c4;  // FINAL: the slab is the image
+    for (int y = yfirst; y < n; y += YSTEP) {
+        uint32_t b[4];
+        lean_scan<TX, 0>(kt + (y + kLeanPad) * TX + c4, y, n, P.wk, b);
+        const int64_t p = col + (int64_t)y * P.inner;
+        if (!FINAL) {
+            if (sizeof(VT) == 2) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v) b[v] = min(b[v], 0xffffu);
+                *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.out) + p) = make_uint2(b[0] | (b[1] << 16), b[2] | (b[3] << 16));
+            } else {
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(P.out) + p) = make_uint4(b[0], b[1], b[2], b[3]);
+            }
+            continue;
+        }
+        const uint32_t all = b[0] | b[1] | b[2] | b[3];
+        if (ep.dist) {
+            float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (all != 0u) {
+                float f[4];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    // exact integer below 2^24 -> float32: two full-rate operations below 2^23, a conversion otherwise
+                    const float x = all < (1u << 23) ? small_int_to_float((int)b[v]) : __uint2float_rn(b[v]);
+                    f[v] = b[v] >= kLeanNone ? TMEDT_INF : fast_sqrt(x * P.inv_scale);
+                }
+                d = make_float4(f[0], f[1], f[2], f[3]);
+            }
+            __stcs(reinterpret_cast<float4*>(ep.dist + p), d);
+        }
+        if (ep.sq) {  // unit sampling only
+            if ((all & kLeanNone) == 0u) {
+                lean_store_4xi64(ep.sq + p, b[0], b[1], b[2], b[3]);
+            } else {
+#pragma unroll
+                for (int v = 0; v < 4; ++v) ep.sq[p + v] = b[v] >= kLeanNone ? INT64_MAX : (int64_t)b[v];
+            }
+        }
+    }
+}
+
+}  // namespace tmedt

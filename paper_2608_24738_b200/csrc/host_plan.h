@@ -1,0 +1,54 @@
+// Host-side plan of one call and the helpers shared by the translation units that launch the distance-transform
+// kernels.  Not exported.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "edt_common.cuh"
+
+namespace tmedt {
+
+// The contiguous (B, C, n_0 .. n_{d-1}) array is, for the pass along spatial axis a, a
+// (outer, n_a, inner) array.  Axes of extent 1 are never processed (their pass is the identity).
+// Processing order: last spatial axis first ("plane" p = p-th processed axis).
+struct Plan {
+    int ndim = 0;
+    int64_t images = 0, V = 0, N = 0;
+    int E = 0;
+    int axis[kMaxDims];
+    int plane_of_axis[kMaxDims];
+    int ext[kMaxDims];
+    int64_t inner[kMaxDims];
+    double w[kMaxDims];
+    bool unit = true;
+    bool use_double = false;  // arithmetic type of the envelope passes
+    bool wide = false;        // int16 offsets instead of int8
+    bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
+    unsigned flags = 0;       // TM_EDT_FLAG_* of the call
+    int64_t shape_sp[kMaxDims];  // spatial extents of the call
+    double w_sp[kMaxDims];       // sampling per spatial axis
+    bool long_lines = false;  // two or three axes, extents up to 8192: plain heights scanned through the cache
+    bool small = false;       // every extent <= 8: register-resident lines, value (+ site index) carry
+    bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
+    int si[kMaxDims];         // those integers
+    double scale = 1.0;
+    bool wide_keys = false;      // unit sampling, contiguous extent % 16 == 0: two axes <= 1024 or three axes <= 512
+    size_t ws_bytes = 0;
+    size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
+};
+
+// Per-kernel timing of tm_edt_profile: records an event before the launch that follows.
+// `bytes`: what that launch has to read and write once (its inputs plus its outputs).
+void prof_mark(cudaStream_t st, const char* name, double bytes);
+double out_bytes_per_voxel(const EpilogueParams& ep);
+
+// Raises a kernel's dynamic shared-memory limit when `smem` needs it; remembered per (kernel, device), so the
+// attribute is set once and not at every call.
+cudaError_t ensure_smem(const void* kernel, size_t smem);
+
+// Quad-per-lane kernels (edt_lean.cuh, launched from tm_edt_lean.cu): whether they cover a call, and the call itself.
+bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep);
+cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches);
+
+}  // namespace tmedt

@@ -19,6 +19,7 @@
 #include "edt_compat.cuh"
 #include "edt_value.cuh"
 #include "host_shared.h"
+#include "host_plan.h"
 #include <stdlib.h>
 
 namespace tmedt {
@@ -39,42 +40,13 @@ struct Profiler {
 static thread_local Profiler g_prof;
 
 // `bytes`: what this launch has to read and write once (its inputs plus its outputs).
-static void prof_mark(cudaStream_t st, const char* name, double bytes) {
+void prof_mark(cudaStream_t st, const char* name, double bytes) {
     if (!g_prof.active || g_prof.count >= kProfMax) return;
     cudaEventRecord(g_prof.ev[g_prof.count], st);
     g_prof.name[g_prof.count] = name;
     g_prof.bytes[g_prof.count] = bytes;
     ++g_prof.count;
 }
-
-// The contiguous (B, C, n_0 .. n_{d-1}) array is, for the pass along spatial axis a, a
-// (outer, n_a, inner) array.  Axes of extent 1 are never processed (their pass is the identity).
-// Processing order: last spatial axis first ("plane" p = p-th processed axis).
-struct Plan {
-    int ndim = 0;
-    int64_t images = 0, V = 0, N = 0;
-    int E = 0;
-    int axis[kMaxDims];
-    int plane_of_axis[kMaxDims];
-    int ext[kMaxDims];
-    int64_t inner[kMaxDims];
-    double w[kMaxDims];
-    bool unit = true;
-    bool use_double = false;  // arithmetic type of the envelope passes
-    bool wide = false;        // int16 offsets instead of int8
-    bool fast = false;        // packed-entry kernels (extents <= 128, 2..5 processed axes)
-    unsigned flags = 0;       // TM_EDT_FLAG_* of the call
-    int64_t shape_sp[kMaxDims];  // spatial extents of the call
-    double w_sp[kMaxDims];       // sampling per spatial axis
-    bool long_lines = false;  // two or three axes, extents up to 8192: plain heights scanned through the cache
-    bool small = false;       // every extent <= 8: register-resident lines, value (+ site index) carry
-    bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
-    int si[kMaxDims];         // those integers
-    double scale = 1.0;
-    bool wide_keys = false;      // unit sampling, contiguous extent % 16 == 0: two axes <= 1024 or three axes <= 512
-    size_t ws_bytes = 0;
-    size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
-};
 
 static int make_plan(int ndim, const int64_t* shape, const double* sampling, Plan& pl) {
     if (!shape || ndim < 1 || ndim > kMaxDims) return TM_EDT_ERR_INVALID_ARG;
@@ -206,7 +178,7 @@ static void fill_epilogue(const Plan& pl, float* dist, int64_t* sq, int64_t* idx
     for (int p = 0; p < kMaxDims; ++p) ep.pstride[p] = p < pl.E ? pl.inner[p] : 0;
 }
 
-static double out_bytes_per_voxel(const EpilogueParams& ep) {
+double out_bytes_per_voxel(const EpilogueParams& ep) {
     return (ep.dist ? 4.0 : 0.0) + (ep.sq ? 8.0 : 0.0) + (ep.idx ? 8.0 * ep.idx_planes : 0.0);
 }
 
@@ -873,6 +845,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     if (pl.wide_keys) return run_wide(pl, input, ep, ws, st, launches);
     if (pl.long_lines)
         return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
+    if (!getenv("TM_EDT_NO_LEAN") && lean_ok(pl, input, ep)) return run_lean(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
         return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);

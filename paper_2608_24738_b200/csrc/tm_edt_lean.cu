@@ -1,0 +1,192 @@
+// Launch code of the quad-per-lane kernels (edt_lean.cuh): a translation unit of its own.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "edt_lean.cuh"
+#include "host_plan.h"
+
+namespace tmedt {
+
+// Largest dynamic shared-memory size configured so far per (kernel, device): the attribute is set once, not per call.
+struct SmemAttr { const void* fn; int dev; size_t bytes; };
+static SmemAttr g_smem_attr[256];
+static int g_smem_attr_count = 0;
+static std::mutex g_smem_attr_mutex;
+
+cudaError_t ensure_smem(const void* fn, size_t smem) {
+    if (smem <= 48 * 1024) return cudaSuccess;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(g_smem_attr_mutex);
+    SmemAttr* slot = nullptr;
+    for (int i = 0; i < g_smem_attr_count; ++i)
+        if (g_smem_attr[i].fn == fn && g_smem_attr[i].dev == dev) { slot = &g_smem_attr[i]; break; }
+    if (slot && slot->bytes >= smem) return cudaSuccess;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (!slot && g_smem_attr_count < 256) slot = &g_smem_attr[g_smem_attr_count++];
+    if (slot) { slot->fn = fn; slot->dev = dev; slot->bytes = smem; }
+    return cudaSuccess;
+}
+
+// Quad-per-lane kernels (edt_lean.cuh) for the shapes they cover: three or four processed axes, contiguous extent a
+// multiple of 4, outputs aligned for 16-byte (float32) and 32-byte (int64) stores, exact integer keys (unit sampling, or scaled integers without index output),
+// coordinate index layout with every spatial axis processed.
+bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep) {
+    if (!pl.fast || pl.E < 3 || pl.E > 4 || pl.ext[0] % 4 != 0 || ((uintptr_t)in & 3u) != 0) return false;
+    if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u) || ((uintptr_t)ep.idx & 31u)) return false;
+    if (ep.idx) return pl.unit && pl.ndim == pl.E && !ep.flat;
+    return pl.unit || pl.scaled;
+}
+
+template <int VS, typename VT>
+static cudaError_t launch_lean_plane(const LeanParams& P, int64_t planes, cudaStream_t st) {
+    const size_t smem = (size_t)(P.n + 2 * kLeanPad) * VS * 4;
+    auto kern = lean_plane_kernel<VS, VT>;
+    cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)planes, 256, smem, st>>>(P);
+    return cudaGetLastError();
+}
+
+template <typename VT>
+static cudaError_t launch_lean_plane_vs(const LeanParams& P, int64_t planes, cudaStream_t st) {
+    if (P.n0 <= 32) return launch_lean_plane<32, VT>(P, planes, st);
+    if (P.n0 <= 64) return launch_lean_plane<64, VT>(P, planes, st);
+    return launch_lean_plane<128, VT>(P, planes, st);
+}
+
+// Columns per tile of a later axis: about 2048 to 4096 voxels per block.
+static int lean_tile_columns(int n, int64_t inner) {
+    if (const char* v = getenv("TM_EDT_LEAN_TX")) {  // experiment knob
+        const int f = atoi(v);
+        if (n <= 32 && (f == 32 || f == 64 || f == 128 || f == 256)) return f;
+    }
+    int tx = n <= 32 ? 128 : (n <= 64 ? 64 : 32);
+    while (tx > 32 && tx / 2 >= inner) tx >>= 1;
+    return tx;
+}
+
+template <int K, bool FINAL, int TX>
+static cudaError_t launch_lean_column_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
+    const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4 + (size_t)P.n * TX * entry_bytes(K);
+    P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    auto kern = lean_column_kernel<K, FINAL, TX>;
+    cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)(outer * P.tiles_per_slab), 256, smem, st>>>(P, ep);
+    return cudaGetLastError();
+}
+
+template <int K, bool FINAL>
+static cudaError_t launch_lean_column(const LeanParams& P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
+    const int tx = lean_tile_columns(P.n, P.inner);
+    if (tx == 256) return launch_lean_column_tx<K, FINAL, 256>(P, ep, outer, st);
+    if (tx == 128) return launch_lean_column_tx<K, FINAL, 128>(P, ep, outer, st);
+    if (tx == 64) return launch_lean_column_tx<K, FINAL, 64>(P, ep, outer, st);
+    return launch_lean_column_tx<K, FINAL, 32>(P, ep, outer, st);
+}
+
+template <bool FINAL, typename VT, int TX>
+static cudaError_t launch_lean_value_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
+    const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4;
+    P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    auto kern = lean_value_kernel<FINAL, VT, TX>;
+    cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)(outer * P.tiles_per_slab), 256, smem, st>>>(P, ep);
+    return cudaGetLastError();
+}
+
+template <bool FINAL, typename VT>
+static cudaError_t launch_lean_value(const LeanParams& P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
+    const int tx = lean_tile_columns(P.n, P.inner);
+    if (tx == 256) return launch_lean_value_tx<FINAL, VT, 256>(P, ep, outer, st);
+    if (tx == 128) return launch_lean_value_tx<FINAL, VT, 128>(P, ep, outer, st);
+    if (tx == 64) return launch_lean_value_tx<FINAL, VT, 64>(P, ep, outer, st);
+    return launch_lean_value_tx<FINAL, VT, 32>(P, ep, outer, st);
+}
+
+static cudaError_t run_lean_images(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                                   int& launches);
+
+cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                     int& launches) {
+    // Large images one after the other: what one kernel wrote is still in L2 when the next kernel reads it.
+    const char* knob = getenv("TM_EDT_LEAN_PER_IMAGE");  // experiment knob
+    const bool per_image = knob ? knob[0] == '1' : false;
+    if (!per_image || pl.images == 1) return run_lean_images(pl, in, ep, ws, st, launches);
+    for (int64_t i = 0; i < pl.images; ++i) {
+        Plan one = pl;
+        one.images = 1; one.N = pl.V;
+        EpilogueParams e1 = ep;
+        if (ep.dist) e1.dist = ep.dist + i * pl.V;
+        if (ep.sq) e1.sq = ep.sq + i * pl.V;
+        if (ep.idx) e1.idx = ep.idx + i * pl.V * ep.idx_planes;
+        cudaError_t e = run_lean_images(one, in + i * pl.V, e1, ws, st, launches);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+static cudaError_t run_lean_images(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
+                                   int& launches) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    char* bufA = static_cast<char*>(ws);
+    char* bufB = bufA + up((size_t)pl.N * 4);
+    const double out_bpv = out_bytes_per_voxel(ep);
+    const bool entries = ep.idx != nullptr;
+    double sumsq = 0.0;
+    for (int p = 0; p < pl.E; ++p) sumsq += (double)(pl.ext[p] - 1) * (pl.ext[p] - 1);
+    const bool v16 = !entries && pl.unit && sumsq < 65535.0;
+    const double carry = entries ? 2.0 : (v16 ? 2.0 : 4.0);  // bytes per voxel the plane kernel writes
+    auto weight = [&](int p) { return pl.unit ? 1u : (uint32_t)pl.si[p]; };
+    LeanParams P;
+    memset(&P, 0, sizeof(P));
+    P.in = in; P.out = bufA;
+    P.n0 = pl.ext[0]; P.n = pl.ext[1]; P.inner = pl.inner[1];
+    P.w0 = weight(0); P.wk = weight(1);
+    P.inv_scale = (float)(1.0 / pl.scale);
+    for (int q = 0; q < 4; ++q) {
+        P.shift[q] = -1;
+        if (q < pl.E)
+            for (int s = 0; s < 8; ++s)
+                if (pl.ext[q] == (1 << s)) P.shift[q] = s;
+    }
+    const int64_t planes = pl.N / ((int64_t)pl.ext[0] * pl.ext[1]);
+    prof_mark(st, "plane", (double)pl.N * (1.0 + carry));
+    cudaError_t e = entries ? launch_lean_plane_vs<uint8_t>(P, planes, st)
+                            : (v16 ? launch_lean_plane_vs<uint16_t>(P, planes, st) : launch_lean_plane_vs<uint32_t>(P, planes, st));
+    ++launches;
+    if (e != cudaSuccess) return e;
+    char* src = bufA;
+    char* dst = bufB;
+    for (int k = 2; k < pl.E; ++k) {
+        const bool fin = k == pl.E - 1;
+        P.in = src; P.out = dst;
+        P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = weight(k);
+        const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+        if (entries) {
+            const double eb = (double)entry_bytes(k);
+            prof_mark(st, fin ? "column_final" : "column", (double)pl.N * (eb + (fin ? out_bpv : (double)entry_bytes(k + 1))));
+            if (k == 2) e = fin ? launch_lean_column<2, true>(P, ep, outer, st) : launch_lean_column<2, false>(P, ep, outer, st);
+            else e = launch_lean_column<3, true>(P, ep, outer, st);
+        } else {
+            prof_mark(st, fin ? "column_value_final" : "column_value", (double)pl.N * (carry + (fin ? out_bpv : carry)));
+            if (v16) e = fin ? launch_lean_value<true, uint16_t>(P, ep, outer, st) : launch_lean_value<false, uint16_t>(P, ep, outer, st);
+            else e = fin ? launch_lean_value<true, uint32_t>(P, ep, outer, st) : launch_lean_value<false, uint32_t>(P, ep, outer, st);
+        }
+        ++launches;
+        if (e != cudaSuccess) return e;
+        char* t = src; src = dst; dst = t;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace tmedt
