@@ -35,30 +35,35 @@ struct LeanParams {
     int shift[4];        // final entry kernels: log2 of the extent of plane q, or -1 if it is no power of two
 };
 
+__device__ __forceinline__ uint32_t lean_max4(const uint32_t (&b)[4]) { return max(max(b[0], b[1]), max(b[2], b[3])); }
+
+__device__ __forceinline__ void lean_try_row(const uint32_t* __restrict__ row, const uint32_t a, uint32_t (&b)[4]) {
+    const uint4 c = *reinterpret_cast<const uint4*>(row);
+    b[0] = __viaddmin_u32(c.x, a, b[0]); b[1] = __viaddmin_u32(c.y, a, b[1]);
+    b[2] = __viaddmin_u32(c.z, a, b[2]); b[3] = __viaddmin_u32(c.w, a, b[3]);
+}
+
 // Bounded scan of one quad.  own: the quad's keys inside the padded tile (row pitch PITCH words).
-// Row distance d adds (wk d^2) << SH; the scan of a voxel may stop once that addend reaches its best key.
+// Row distance d adds (wk d^2) << SH; a voxel is finished once that addend reaches its best key, so the work of a
+// voxel grows with its distance to the background along the axis and never exceeds the extent.
 template <int PITCH, int SH>
-__device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, const int y, const int n,
-                                          const uint32_t wk, uint32_t (&b)[4]) {
+__device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, const int y, const int n, const uint32_t wk,
+                                          uint32_t (&b)[4]) {
     {
         const uint4 v = *reinterpret_cast<const uint4*>(own);
         b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
     }
-    uint32_t mx = max(max(b[0], b[1]), max(b[2], b[3]));
+    uint32_t mx = lean_max4(b);
     if (mx < (1u << SH)) return;  // four background voxels
 #pragma unroll
-    for (int s = 1; s <= kLeanPad; ++s) {
+    for (int s = 1; s <= kLeanPad; ++s) {  // no bounds tests: the tile is padded
         if (s == 3 && ((wk * 9u) << SH) >= mx) return;
         const uint32_t a = (wk * (uint32_t)(s * s)) << SH;
-        const uint4 lo = *reinterpret_cast<const uint4*>(own - s * PITCH);
-        const uint4 hi = *reinterpret_cast<const uint4*>(own + s * PITCH);
-        b[0] = __viaddmin_u32(lo.x, a, b[0]); b[1] = __viaddmin_u32(lo.y, a, b[1]);
-        b[2] = __viaddmin_u32(lo.z, a, b[2]); b[3] = __viaddmin_u32(lo.w, a, b[3]);
-        b[0] = __viaddmin_u32(hi.x, a, b[0]); b[1] = __viaddmin_u32(hi.y, a, b[1]);
-        b[2] = __viaddmin_u32(hi.z, a, b[2]); b[3] = __viaddmin_u32(hi.w, a, b[3]);
-        if (s == 2) mx = max(max(b[0], b[1]), max(b[2], b[3]));
+        lean_try_row(own - s * PITCH, a, b);
+        lean_try_row(own + s * PITCH, a, b);
+        if (s == 2) mx = lean_max4(b);
     }
-    mx = max(max(b[0], b[1]), max(b[2], b[3]));
+    mx = lean_max4(b);
     int d = kLeanPad + 1;
     uint32_t a = (wk * (uint32_t)(d * d)) << SH;
     if (a >= mx) return;
@@ -66,17 +71,9 @@ __device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, cons
     const uint32_t* plo = own - d * PITCH;
     const uint32_t* phi = own + d * PITCH;
     for (; a < mx && (d <= up || d <= dn); ++d, plo -= PITCH, phi += PITCH) {
-        if (d <= up) {
-            const uint4 lo = *reinterpret_cast<const uint4*>(plo);
-            b[0] = __viaddmin_u32(lo.x, a, b[0]); b[1] = __viaddmin_u32(lo.y, a, b[1]);
-            b[2] = __viaddmin_u32(lo.z, a, b[2]); b[3] = __viaddmin_u32(lo.w, a, b[3]);
-        }
-        if (d <= dn) {
-            const uint4 hi = *reinterpret_cast<const uint4*>(phi);
-            b[0] = __viaddmin_u32(hi.x, a, b[0]); b[1] = __viaddmin_u32(hi.y, a, b[1]);
-            b[2] = __viaddmin_u32(hi.z, a, b[2]); b[3] = __viaddmin_u32(hi.w, a, b[3]);
-        }
-        mx = max(max(b[0], b[1]), max(b[2], b[3]));
+        if (d <= up) lean_try_row(plo, a, b);
+        if (d <= dn) lean_try_row(phi, a, b);
+        mx = lean_max4(b);
         a = (wk * (uint32_t)((d + 1) * (d + 1))) << SH;
     }
 }
@@ -93,42 +90,99 @@ __device__ __forceinline__ void lean_fill_pad(uint32_t* __restrict__ kt, const i
 }
 
 // ---------------------------------------------------------------------------------------------
+// First-axis pass of one row into the key tile: one warp per row, four voxels per lane (one 32-bit load of the mask).
+// Zero bytes are found with a carry-free byte test, the nearest lanes holding a zero on either side with one ballot
+// and clz / ffs, their zero positions with two shuffles; the lane's four voxels are finished in registers.
+//   ENT   key = off^2 << 16 | row << 8 | (off & 0xff)   (off = signed offset to the nearest zero of the row)
+//   !ENT  key = w0 * off^2
+// Returns the AND of the lane's four keys (all ones for lanes beyond the row): bit 31 stays set only if all are "no site".
+// ---------------------------------------------------------------------------------------------
+template <bool ENT>
+__device__ __forceinline__ uint32_t lean_first_axis(const uint32_t v, const int n0, const int y, const uint32_t w0,
+                                                uint32_t* __restrict__ krow, const int lane) {
+    const bool act = 4 * lane < n0;
+    const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
+    const unsigned any = __ballot_sync(0xffffffffu, m != 0u);  // lanes beyond the row hold foreground: m == 0
+    uint4 keys;
+    if (any == 0u) {  // no background in this row
+        keys = make_uint4(kLeanNone, kLeanNone, kLeanNone, kLeanNone);
+    } else if (__all_sync(0xffffffffu, m == 0x80808080u || !act)) {  // nothing but background
+        const uint32_t k0 = ENT ? (uint32_t)y << 8 : 0u;
+        keys = make_uint4(k0, k0, k0, k0);
+    } else {
+        // every lane of the warp stays in the shuffles; only the store is guarded
+        const int lzin = m ? (31 - __clz(m)) >> 3 : 0;   // highest zero byte of this lane
+        const int fzin = m ? (__ffs(m) - 1) >> 3 : 0;    // lowest zero byte of this lane
+        const unsigned ml = any & ((1u << lane) - 1u);
+        const unsigned mr = lane < 31 ? any >> (lane + 1) : 0u;
+        const int Ll = ml ? 31 - __clz(ml) : 0;
+        const int Lr = mr ? lane + __ffs(mr) : 0;
+        const int lz_l = __shfl_sync(0xffffffffu, lzin, Ll);
+        const int fz_r = __shfl_sync(0xffffffffu, fzin, Lr);
+        const int x0 = 4 * lane;
+        int cur = ml ? 4 * Ll + lz_l : -1024;   // nearest zero left of this lane's voxels
+        int dl[4], dr[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dl[b] = x0 + b - cur;
+        }
+        cur = mr ? 4 * Lr + fz_r : 2048;        // nearest zero right of this lane's voxels
+#pragma unroll
+        for (int b = 3; b >= 0; --b) {
+            if ((m >> (8 * b + 7)) & 1u) cur = x0 + b;
+            dr[b] = cur - (x0 + b);
+        }
+        uint32_t kk[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int a = min(dl[b], dr[b]);
+            const int off = dl[b] <= dr[b] ? -a : a;
+            kk[b] = ENT ? (((uint32_t)(a * a) << 16) | ((uint32_t)y << 8) | ((uint32_t)off & 0xffu)) : w0 * (uint32_t)(a * a);
+        }
+        keys = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+    }
+    if (act) *reinterpret_cast<uint4*>(krow + 4 * lane) = keys;
+    return act ? (keys.x & keys.y & keys.z & keys.w) : 0xffffffffu;
+}
+
+// ---------------------------------------------------------------------------------------------
 // First and second axis of one (n1 x n0) plane per block.
-//   VT == void      entries: writes 2-byte entries (first-axis offset, second-axis offset)
+//   VT == uint8_t   entries: writes 2-byte entries (first-axis offset, second-axis offset)
 //   VT == uint16_t  values:  writes the squared distance so far (all ones = no site)
 //   VT == uint32_t  values:  writes the (scaled) squared distance so far (2^31 = no site)
 // ---------------------------------------------------------------------------------------------
 template <int VS, typename VT>
 __global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constant__ LeanParams P) {
-    constexpr bool ENT = sizeof(VT) == 1;  // VT = uint8_t stands for "entries"
+    constexpr bool ENT = sizeof(VT) == 1;
     constexpr int SH = ENT ? 16 : 0;
     extern __shared__ __align__(16) uint8_t sm_lean_p[];
-    uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_p);  // [n1 + 2 kLeanPad][VS]
     const int n0 = P.n0, n1 = P.n;
+    uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_p);      // [n1 + 2 kLeanPad][VS]
     const int64_t plane = blockIdx.x;
     const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int NW = 8;
+    const uint32_t wk = ENT ? 1u : P.wk;
     lean_fill_pad<VS>(kt, n1);
+    uint32_t all = 0xffffffffu;  // AND of this thread's keys
     {
         constexpr int MAXR = 16;  // rows per warp: 128 rows / 8 warps
         uint32_t rowv[MAXR];
         const bool act = 4 * lane < n0;
 #pragma unroll
-        for (int i = 0; i < MAXR; ++i) {
+        for (int i = 0; i < MAXR; ++i) {  // all loads of this warp's rows are issued before the first row is processed
             const int y = warp + i * NW;
             rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
         }
 #pragma unroll
         for (int i = 0; i < MAXR; ++i) {
             const int y = warp + i * NW;
-            if (y < n1) {
-                if (ENT) pass0_row_to_keys<false>(rowv[i], n0, y, kt + (y + kLeanPad) * VS, lane);
-                else pass0_row_to_scaled_keys<false>(rowv[i], n0, y, (int)P.w0, kt + (y + kLeanPad) * VS, nullptr, lane);
-            }
+            if (y < n1) all &= lean_first_axis<ENT>(rowv[i], n0, y, P.w0, kt + (y + kLeanPad) * VS, lane);
         }
     }
-    __syncthreads();
+    // barrier; a plane without any background voxel needs no scan (every result is "no site")
+    const int any_site = __syncthreads_or((all & kLeanNone) == 0u);
     // a warp takes patches of 4 rows x 32 columns (8 quads per row): neighbouring voxels have similar scan lengths
     constexpr int CG = VS / 32;
     const int r = lane >> 3, q4 = 4 * (lane & 7);
@@ -137,10 +191,10 @@ __global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constan
     for (int t = warp; t < patches; t += NW) {
         const int y = 4 * (t / CG) + r, c4 = 32 * (t % CG) + q4;
         if (y >= n1 || c4 >= n0) continue;
-        const int64_t base = base0 + c4;
         uint32_t b[4];
-        lean_scan<VS, SH>(kt + (y + kLeanPad) * VS + c4, y, n1, ENT ? 1u : P.wk, b);
-        const int64_t p = base + (int64_t)y * n0;
+        if (any_site) lean_scan<VS, SH>(kt + (y + kLeanPad) * VS + c4, y, n1, wk, b);
+        else b[0] = b[1] = b[2] = b[3] = kLeanNone;
+        const int64_t p = base0 + (int64_t)y * n0 + c4;
         if (ENT) {
             uint32_t e[4];
 #pragma unroll
@@ -194,6 +248,7 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     const int width = (int)min((int64_t)TX, P.inner - i0);
     const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);
+    uint32_t all = 0xffffffffu;  // AND of this thread's keys
     for (int t = threadIdx.x; t < n * LPR; t += 256) {
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
@@ -213,8 +268,10 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
         for (int v = 0; v < 4; ++v)
             k[v] = e[v] == 0x80u ? kLeanNone : (((uint32_t)__dp4a((int)e[v], (int)e[v], 0) << 8) | (uint32_t)y);
         *reinterpret_cast<uint4*>(kt + (y + kLeanPad) * TX + q4) = make_uint4(k[0], k[1], k[2], k[3]);
+        all &= k[0] & k[1] & k[2] & k[3];
     }
-    __syncthreads();
+    // barrier; a tile without any site (an image without background) needs no scan
+    const int any_site = __syncthreads_or((all & kLeanNone) == 0u);
     // a warp takes patches of 4 rows x 32 columns (8 quads per row), always in the same 32 columns
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c4 = 32 * (warp % CG) + 4 * (lane & 7);
@@ -226,7 +283,8 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
         uint32_t* out = reinterpret_cast<uint32_t*>(P.out) + slab * (int64_t)n * P.inner + v0;
         for (int y = yfirst; y < n; y += YSTEP) {
             uint32_t b[4], o[4];
-            lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+            if (any_site) lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+            else b[0] = b[1] = b[2] = b[3] = kLeanNone;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 const uint32_t j = b[v] & 0xffu;
@@ -260,7 +318,8 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     for (int q = 0; q <= K; ++q) ip[q] = ep.idx + (slab * ep.ndim + ep.axis[q]) * ep.V;
     for (int y = yfirst; y < n; y += YSTEP) {
         uint32_t b[4];
-        lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+        if (any_site) lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+        else b[0] = b[1] = b[2] = b[3] = kLeanNone;
         const uint32_t p = (uint32_t)y * (uint32_t)P.inner + v0;  // inside one image: below 2^31
         uint32_t e[4], j[4];
 #pragma unroll
@@ -316,6 +375,7 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
     const int width = (int)min((int64_t)TX, P.inner - i0);
     const VT* src = reinterpret_cast<const VT*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);
+    uint32_t all = 0xffffffffu;  // AND of this thread's keys
     for (int t = threadIdx.x; t < n * LPR; t += 256) {
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
@@ -332,8 +392,9 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
             k = *reinterpret_cast<const uint4*>(g);
         }
         *reinterpret_cast<uint4*>(kt + (y + kLeanPad) * TX + q4) = k;
+        all &= k.x & k.y & k.z & k.w;
     }
-    __syncthreads();
+    const int any_site = __syncthreads_or((all & kLeanNone) == 0u);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c4 = 32 * (warp % CG) + 4 * (lane & 7);
     const int yfirst = 4 * (warp / CG) + (lane >> 3);
@@ -342,7 +403,8 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
     const int64_t col = slab * (int64_t)n * P.inner + i0 + c4;  // FINAL: the slab is the image
     for (int y = yfirst; y < n; y += YSTEP) {
         uint32_t b[4];
-        lean_scan<TX, 0>(kt + (y + kLeanPad) * TX + c4, y, n, P.wk, b);
+        if (any_site) lean_scan<TX, 0>(kt + (y + kLeanPad) * TX + c4, y, n, P.wk, b);
+        else b[0] = b[1] = b[2] = b[3] = kLeanNone;
         const int64_t p = col + (int64_t)y * P.inner;
         if (!FINAL) {
             if (sizeof(VT) == 2) {

@@ -1,7 +1,6 @@
 // Launch code of the quad-per-lane kernels (edt_lean.cuh): a translation unit of its own.
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -64,10 +63,6 @@ static cudaError_t launch_lean_plane_vs(const LeanParams& P, int64_t planes, cud
 
 // Columns per tile of a later axis: about 2048 to 4096 voxels per block.
 static int lean_tile_columns(int n, int64_t inner) {
-    if (const char* v = getenv("TM_EDT_LEAN_TX")) {  // experiment knob
-        const int f = atoi(v);
-        if (n <= 32 && (f == 32 || f == 64 || f == 128 || f == 256)) return f;
-    }
     int tx = n <= 32 ? 128 : (n <= 64 ? 64 : 32);
     while (tx > 32 && tx / 2 >= inner) tx >>= 1;
     return tx;
@@ -87,7 +82,6 @@ static cudaError_t launch_lean_column_tx(LeanParams P, const EpilogueParams& ep,
 template <int K, bool FINAL>
 static cudaError_t launch_lean_column(const LeanParams& P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const int tx = lean_tile_columns(P.n, P.inner);
-    if (tx == 256) return launch_lean_column_tx<K, FINAL, 256>(P, ep, outer, st);
     if (tx == 128) return launch_lean_column_tx<K, FINAL, 128>(P, ep, outer, st);
     if (tx == 64) return launch_lean_column_tx<K, FINAL, 64>(P, ep, outer, st);
     return launch_lean_column_tx<K, FINAL, 32>(P, ep, outer, st);
@@ -107,36 +101,12 @@ static cudaError_t launch_lean_value_tx(LeanParams P, const EpilogueParams& ep, 
 template <bool FINAL, typename VT>
 static cudaError_t launch_lean_value(const LeanParams& P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const int tx = lean_tile_columns(P.n, P.inner);
-    if (tx == 256) return launch_lean_value_tx<FINAL, VT, 256>(P, ep, outer, st);
     if (tx == 128) return launch_lean_value_tx<FINAL, VT, 128>(P, ep, outer, st);
     if (tx == 64) return launch_lean_value_tx<FINAL, VT, 64>(P, ep, outer, st);
     return launch_lean_value_tx<FINAL, VT, 32>(P, ep, outer, st);
 }
 
-static cudaError_t run_lean_images(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
-                                   int& launches);
-
-cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
-                     int& launches) {
-    // Large images one after the other: what one kernel wrote is still in L2 when the next kernel reads it.
-    const char* knob = getenv("TM_EDT_LEAN_PER_IMAGE");  // experiment knob
-    const bool per_image = knob ? knob[0] == '1' : false;
-    if (!per_image || pl.images == 1) return run_lean_images(pl, in, ep, ws, st, launches);
-    for (int64_t i = 0; i < pl.images; ++i) {
-        Plan one = pl;
-        one.images = 1; one.N = pl.V;
-        EpilogueParams e1 = ep;
-        if (ep.dist) e1.dist = ep.dist + i * pl.V;
-        if (ep.sq) e1.sq = ep.sq + i * pl.V;
-        if (ep.idx) e1.idx = ep.idx + i * pl.V * ep.idx_planes;
-        cudaError_t e = run_lean_images(one, in + i * pl.V, e1, ws, st, launches);
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
-}
-
-static cudaError_t run_lean_images(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
-                                   int& launches) {
+cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* bufA = static_cast<char*>(ws);
     char* bufB = bufA + up((size_t)pl.N * 4);
