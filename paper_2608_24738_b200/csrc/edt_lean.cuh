@@ -67,9 +67,20 @@ __device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, cons
     int d = kLeanPad + 1;
     uint32_t a = (wk * (uint32_t)(d * d)) << SH;
     if (a >= mx) return;
-    const int up = y, dn = n - 1 - y;
+    const int up = y, dn = n - 1 - y, both = min(up, dn);
     const uint32_t* plo = own - d * PITCH;
     const uint32_t* phi = own + d * PITCH;
+    // rows that exist on both sides, two distances per stop test
+    for (; d + 1 <= both && a < mx; d += 2, plo -= 2 * PITCH, phi += 2 * PITCH) {
+        const uint32_t a1 = (wk * (uint32_t)((d + 1) * (d + 1))) << SH;
+        lean_try_row(plo, a, b);
+        lean_try_row(phi, a, b);
+        lean_try_row(plo - PITCH, a1, b);
+        lean_try_row(phi + PITCH, a1, b);
+        mx = lean_max4(b);
+        a = (wk * (uint32_t)((d + 2) * (d + 2))) << SH;
+    }
+    // the rest: one distance at a time, the tile's ends tested
     for (; a < mx && (d <= up || d <= dn); ++d, plo -= PITCH, phi += PITCH) {
         if (d <= up) lean_try_row(plo, a, b);
         if (d <= dn) lean_try_row(phi, a, b);
@@ -234,6 +245,63 @@ __device__ __forceinline__ int lean_sext_byte(uint32_t e, int q) {
     return (int)r;
 }
 
+// Final outputs of one quad (index output requested, every spatial axis processed): b = the quad's final keys
+// (squared distance << 8 | site row), e = the entries of the four sites along the K earlier axes, cq = the quad's own
+// coordinates along those axes (plane 0 is the contiguous one: voxel v sits at cq[0] + v), p = its position inside
+// the image, ip[q] = index plane of processed axis q.
+template <int K>
+__device__ __forceinline__ void lean_emit_final(const uint32_t (&b)[4], const uint32_t (&e)[4], const int (&cq)[K],
+                                                float* __restrict__ dist, int64_t* __restrict__ sq,
+                                                int64_t* const (&ip)[K + 1], const uint32_t p) {
+    uint32_t j[4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v) j[v] = b[v] & 0xffu;
+    if (((b[0] | b[1] | b[2] | b[3]) & kLeanNone) == 0u) {
+        if (dist) {
+            float4 d;
+            d.x = fast_sqrt(small_int_to_float((int)(b[0] >> 8))); d.y = fast_sqrt(small_int_to_float((int)(b[1] >> 8)));
+            d.z = fast_sqrt(small_int_to_float((int)(b[2] >> 8))); d.w = fast_sqrt(small_int_to_float((int)(b[3] >> 8)));
+            __stcs(reinterpret_cast<float4*>(dist + p), d);
+        }
+        if (sq) lean_store_4xi64(sq + p, b[0] >> 8, b[1] >> 8, b[2] >> 8, b[3] >> 8);
+#pragma unroll
+        for (int q = 0; q < K; ++q) {
+            uint32_t s[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) s[v] = (uint32_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
+            lean_store_4xi64(ip[q] + p, s[0], s[1], s[2], s[3]);
+        }
+        lean_store_4xi64(ip[K] + p, j[0], j[1], j[2], j[3]);
+    } else {  // an image without background: +inf, INT64_MAX, -1 (checked voxel by voxel)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const bool none = b[v] >= kLeanNone;
+            if (dist) dist[p + v] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b[v] >> 8)));
+            if (sq) sq[p + v] = none ? INT64_MAX : (int64_t)(b[v] >> 8);
+#pragma unroll
+            for (int q = 0; q < K; ++q)
+                ip[q][p + v] = none ? (int64_t)-1 : (int64_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
+            ip[K][p + v] = none ? (int64_t)-1 : (int64_t)j[v];
+        }
+    }
+}
+
+// Own coordinates along the K earlier planes of position v0 (plane 0 fastest).
+template <int K>
+__device__ __forceinline__ void lean_decode(uint32_t v0, const LeanParams& P, const EpilogueParams& ep, int (&cq)[K]) {
+#pragma unroll
+    for (int q = 0; q < K; ++q) {
+        if (P.shift[q] >= 0) {
+            cq[q] = (int)(v0 & (((uint32_t)1 << P.shift[q]) - 1u));
+            v0 >>= P.shift[q];
+        } else {
+            const uint32_t nq = (uint32_t)ep.ext[q], hi = v0 / nq;
+            cq[q] = (int)(v0 - hi * nq);
+            v0 = hi;
+        }
+    }
+}
+
 template <int K, bool FINAL, int TX>
 __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const __grid_constant__ LeanParams P,
                                                                          const __grid_constant__ EpilogueParams ep) {
@@ -295,66 +363,20 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
         }
         return;
     }
-    // own coordinates along the earlier planes
     int cq[K];
-    {
-        uint32_t rr = v0;
-#pragma unroll
-        for (int q = 0; q < K; ++q) {
-            if (P.shift[q] >= 0) {
-                cq[q] = (int)(rr & (((uint32_t)1 << P.shift[q]) - 1u));
-                rr >>= P.shift[q];
-            } else {
-                const uint32_t nq = (uint32_t)ep.ext[q], hi = rr / nq;
-                cq[q] = (int)(rr - hi * nq);
-                rr = hi;
-            }
-        }
-    }
+    lean_decode<K>(v0, P, ep, cq);
     float* const dist = ep.dist ? ep.dist + slab * ep.V : nullptr;
     int64_t* const sq = ep.sq ? ep.sq + slab * ep.V : nullptr;
     int64_t* ip[K + 1];
 #pragma unroll
     for (int q = 0; q <= K; ++q) ip[q] = ep.idx + (slab * ep.ndim + ep.axis[q]) * ep.V;
     for (int y = yfirst; y < n; y += YSTEP) {
-        uint32_t b[4];
+        uint32_t b[4], e[4];
         if (any_site) lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
         else b[0] = b[1] = b[2] = b[3] = kLeanNone;
-        const uint32_t p = (uint32_t)y * (uint32_t)P.inner + v0;  // inside one image: below 2^31
-        uint32_t e[4], j[4];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            j[v] = b[v] & 0xffu;
-            e[v] = (uint32_t)et[j[v] * TX + c4 + v];
-        }
-        if (((b[0] | b[1] | b[2] | b[3]) & kLeanNone) == 0u) {
-            if (dist) {
-                float4 d;
-                d.x = fast_sqrt(small_int_to_float((int)(b[0] >> 8))); d.y = fast_sqrt(small_int_to_float((int)(b[1] >> 8)));
-                d.z = fast_sqrt(small_int_to_float((int)(b[2] >> 8))); d.w = fast_sqrt(small_int_to_float((int)(b[3] >> 8)));
-                __stcs(reinterpret_cast<float4*>(dist + p), d);
-            }
-            if (sq) lean_store_4xi64(sq + p, b[0] >> 8, b[1] >> 8, b[2] >> 8, b[3] >> 8);
-#pragma unroll
-            for (int q = 0; q < K; ++q) {
-                uint32_t s[4];
-#pragma unroll
-                for (int v = 0; v < 4; ++v) s[v] = (uint32_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
-                lean_store_4xi64(ip[q] + p, s[0], s[1], s[2], s[3]);
-            }
-            lean_store_4xi64(ip[K] + p, j[0], j[1], j[2], j[3]);
-        } else {  // an image without background: +inf, INT64_MAX, -1 (checked voxel by voxel)
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const bool none = b[v] >= kLeanNone;
-                if (dist) dist[p + v] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b[v] >> 8)));
-                if (sq) sq[p + v] = none ? INT64_MAX : (int64_t)(b[v] >> 8);
-#pragma unroll
-                for (int q = 0; q < K; ++q)
-                    ip[q][p + v] = none ? (int64_t)-1 : (int64_t)(cq[q] + (q == 0 ? v : 0) + lean_sext_byte(e[v], q));
-                ip[K][p + v] = none ? (int64_t)-1 : (int64_t)j[v];
-            }
-        }
+        for (int v = 0; v < 4; ++v) e[v] = (uint32_t)et[(b[v] & 0xffu) * TX + c4 + v];
+        lean_emit_final<K>(b, e, cq, dist, sq, ip, (uint32_t)y * (uint32_t)P.inner + v0);  // inside one image: below 2^31
     }
 }
 
