@@ -1,7 +1,7 @@
 /*
  * tm_cdt / tm_bfdt -- taxicab and chessboard distance transforms, and a brute-force distance transform, C ABI
- * (sm_100a).  Paper: Section 2.1 (operators) and Section 2.3.2 ("The chamfer transform ..", "The brute-force
- * transform ..").  Status codes, stream type and error helpers are those of tm_edt.h; every call enqueues on
+ * (sm_100a).  Paper: Section 2.1 (operators) and Section 2.3.2 (its paragraphs on the chamfer transform and on
+ * the brute-force transform).  Status codes, stream type and error helpers are those of tm_edt.h; every call enqueues on
  * `stream` of the current device and returns without synchronising; scratch comes from the library's memory pool.
  */
 #ifndef TM_CDT_H

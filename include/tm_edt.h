@@ -5,8 +5,8 @@
  * Section 2.3.2 "Distance-transform kernels"): every nonzero (foreground) element of a batched
  * mask is labelled with its Euclidean distance to the nearest zero (background) element of the
  * same image, with scipy.ndimage.distance_transform_edt semantics: per-axis sampling, optional
- * nearest-background index map (Section 2.3.2, "indices are propagated through the passes on
- * request"), inputs shaped (B, C, Spatial...) with 1 <= spatial rank <= 8 (Section 2.2.1
+ * nearest-background index map (Section 2.3.2, closing paragraph: the index output is optional and
+ * carried through the passes), inputs shaped (B, C, Spatial...) with 1 <= spatial rank <= 8 (Section 2.2.1
  * "API surface"), pre-allocated outputs, work issued on the caller's stream (Section 2.2.4,
  * runtime tests).
  *
@@ -131,14 +131,32 @@ TM_EDT_API size_t tm_edt_ex_workspace_bytes(int ndim, const int64_t* shape, cons
                                             int with_distances, int with_indices);
 
 /*
- * Scratch bytes tm_edt_ws needs for a call with this geometry (0 for empty problems, and (size_t)-1
- * if ndim/shape are invalid or unsupported).  Depends only on ndim and shape.
+ * Scratch bytes that suffice for any tm_edt_ws call with this geometry, whatever its sampling and outputs
+ * (0 for empty problems, and (size_t)-1 if ndim/shape are invalid or unsupported).  Depends only on ndim and
+ * shape: it is the largest need over unit and other sampling, with the index output requested.
  */
 TM_EDT_API size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape);
 
 /*
+ * Scratch bytes of one particular call (paper, Section 2.2.1: outputs are optional and may be pre-allocated):
+ * the geometry, its sampling (NULL = unit) and which outputs it requests (non-zero = requested).  Never more than
+ * tm_edt_workspace_bytes(ndim, shape); less when no index output is requested on extents above 128 (the offsets
+ * to the site are then not carried between the passes).  tm_edt_ws accepts a workspace of this size for that call.
+ */
+TM_EDT_API size_t tm_edt_workspace_bytes_for(int ndim, const int64_t* shape, const double* sampling, int want_dist,
+                                             int want_sqdist, int want_indices);
+
+/*
+ * Debug and test switches (environment variables TM_EDT_FORCE_GENERIC, TM_EDT_NO_SCALED, TM_EDT_OLD_PLANE,
+ * TM_EDT_NO_VALUE_CARRY, TM_EDT_NO_LEAN, TM_EDT_CHUNK_VOXELS; none changes any result) are read from the
+ * environment once, at the first call that plans a transform.  This call reads them again.
+ */
+TM_EDT_API void tm_edt_reload_switches(void);
+
+/*
  * Same transform with caller-provided scratch: `workspace` is device memory of at least
- * tm_edt_workspace_bytes(ndim, shape) bytes, 256-byte aligned, private to this call until the
+ * tm_edt_workspace_bytes_for(...) bytes for this call (tm_edt_workspace_bytes(ndim, shape) always suffices),
+ * 256-byte aligned, private to this call until the
  * enqueued work has run.  Allocates nothing and only enqueues kernels, so the call can be captured into a
  * CUDA graph and replayed.  A too-small workspace gives TM_EDT_ERR_ALLOC.
  */
@@ -169,7 +187,7 @@ TM_EDT_API int tm_edt_host(const uint8_t* input, int ndim, const int64_t* shape,
  *
  * Arguments, outputs, stream behaviour and return codes are those of tm_edt (inputs and outputs are
  * still the caller's device buffers).  Differences:
- *   - A problem whose scratch need, tm_edt_workspace_bytes(ndim, shape), exceeds
+ *   - A problem whose scratch need, tm_edt_workspace_bytes_for(...) of the call, exceeds
  *     TM_EDT_NOALLOC_MAX_SCRATCH is refused with TM_EDT_ERR_TOO_LARGE before anything is enqueued.
  *   - The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with
  *     that device current) and remembers it.  Make that first call during set-up, before any stream

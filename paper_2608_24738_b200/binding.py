@@ -21,6 +21,7 @@ MAX_EXTENT = 8192
 EXPORTS = (
     "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_ex_workspace_bytes", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
+    "tm_edt_workspace_bytes_for", "tm_edt_reload_switches",
     "tm_grey_morph", "tm_binary_morph", "tm_cdt", "tm_bfdt",
 )
 
@@ -64,6 +65,9 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_profile_ex.restype = i
             L.tm_edt_workspace_bytes.argtypes = [i, vp]
             L.tm_edt_workspace_bytes.restype = sz
+            L.tm_edt_workspace_bytes_for.argtypes = [i, vp, vp, i, i, i]
+            L.tm_edt_workspace_bytes_for.restype = sz
+            L.tm_edt_reload_switches.restype = None
             L.tm_edt_strerror.argtypes = [i]
             L.tm_edt_strerror.restype = ctypes.c_char_p
             L.tm_edt_last_cuda_error.restype = i
@@ -124,6 +128,22 @@ def tm_edt_workspace_bytes(shape: Sequence[int]) -> int:
     return n
 
 
+def tm_edt_workspace_bytes_for(shape: Sequence[int], sampling=None, want_dist=True, want_sqdist=False,
+                               want_indices=False) -> int:
+    """Scratch bytes of one particular call: shape = (B, C, n_0 .. n_{d-1}), its sampling and requested outputs."""
+    ndim = len(shape) - 2
+    n = int(lib().tm_edt_workspace_bytes_for(ndim, _shape_array(shape), _sampling_array(sampling, ndim), int(want_dist),
+                                             int(want_sqdist), int(want_indices)))
+    if n == ctypes.c_size_t(-1).value:
+        raise TmEdtError(ERR_INVALID_ARG, "invalid or unsupported shape")
+    return n
+
+
+def tm_edt_reload_switches() -> None:
+    """Read the library's debug switches from the environment again (they are otherwise read once)."""
+    lib().tm_edt_reload_switches()
+
+
 def _raw_stream(stream) -> Optional[int]:
     import torch
 
@@ -142,8 +162,27 @@ FLAG_FLAT_INDEX = 2
 FLAG_DIST_F64 = 4
 
 
+def _contiguous_on(t, stream):
+    """A contiguous copy of a CUDA tensor for kernels that will run on ``stream``.
+
+    The copy is made on that stream (after what the current stream has queued, which may still be producing ``t``),
+    so it is complete before the kernels read it and its memory is not handed out again before they have run."""
+    import torch
+
+    if t.is_contiguous():
+        return t
+    if not t.is_cuda or stream is None:
+        return t.contiguous()
+    cur = torch.cuda.current_stream(t.device)
+    if stream == cur:
+        return t.contiguous()
+    stream.wait_stream(cur)
+    with torch.cuda.stream(stream):
+        return t.contiguous()
+
+
 def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, device,
-             flat_index=False, dist_f64=False, keep_strides=False):
+             flat_index=False, dist_f64=False, keep_strides=False, stream=None):
     import torch
 
     if mask.dim() < 3:
@@ -153,7 +192,7 @@ def _prepare(mask, sampling, return_distances, return_sqdist, return_indices, di
     if mask.dtype != torch.uint8:
         raise TypeError("mask must be uint8 or bool")
     if not mask.is_contiguous() and not keep_strides:
-        mask = mask.contiguous()
+        mask = _contiguous_on(mask, stream)
     shape = tuple(mask.shape)
     ndim = len(shape) - 2
 
@@ -210,7 +249,7 @@ def tm_edt(mask, sampling=None, return_distances=True, return_indices=False, ret
         raise ValueError("mask must be a CUDA tensor (use tm_edt_host for host buffers)")
     mask, shape, ndim, d, s, x = _prepare(
         mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device,
-        flat_index=flat_index, dist_f64=dist_f64, keep_strides=keep_strides)
+        flat_index=flat_index, dist_f64=dist_f64, keep_strides=keep_strides, stream=stream)
     shp, smp, st = _shape_array(shape), _sampling_array(sampling, ndim), _raw_stream(stream)
     flags = ((FLAG_VIRTUAL_BACKGROUND if virtual_background else 0) | (FLAG_FLAT_INDEX if flat_index else 0)
              | (FLAG_DIST_F64 if dist_f64 else 0))
@@ -245,7 +284,7 @@ def tm_edt_noalloc(mask, sampling=None, return_distances=True, return_indices=Fa
     if not mask.is_cuda:
         raise ValueError("mask must be a CUDA tensor")
     mask, shape, ndim, d, s, x = _prepare(
-        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device)
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device, stream=stream)
     rc = L.tm_edt_noalloc(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
                           _raw_stream(stream))
     _check(rc)
@@ -260,7 +299,7 @@ def tm_edt_host(mask, sampling=None, return_distances=True, return_indices=False
     if mask.is_cuda:
         raise ValueError("tm_edt_host takes host tensors")
     mask, shape, ndim, d, s, x = _prepare(
-        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, "cpu_pinned")
+        mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, "cpu_pinned", stream=stream)
     rc = L.tm_edt_host(_p(mask), ndim, _shape_array(shape), _sampling_array(sampling, ndim), _p(d), _p(s), _p(x),
                        _raw_stream(stream))
     _check(rc)
@@ -276,7 +315,7 @@ def tm_edt_profile(mask, sampling=None, return_distances=True, return_indices=Fa
     L = lib()
     mask, shape, ndim, d, s, x = _prepare(
         mask, sampling, return_distances, return_sqdist, return_indices, distances, sqdist, indices, mask.device,
-        flat_index=bool(flags & FLAG_FLAT_INDEX))
+        flat_index=bool(flags & FLAG_FLAT_INDEX), stream=stream)
     if workspace is None:
         workspace = torch.empty(max(1, tm_edt_workspace_bytes(shape)), dtype=torch.uint8, device=mask.device)
     kmax = 32
@@ -351,7 +390,7 @@ def tm_grey_morph(image, footprint, structure=None, op="erosion", mode="reflect"
     L = lib()
     if not image.is_cuda or image.dtype != torch.float32 or image.dim() < 3:
         raise ValueError("image must be a CUDA float32 tensor shaped (B, C, spatial...)")
-    image = image.contiguous()
+    image = _contiguous_on(image, stream)
     ndim = image.dim() - 2
     fp, fps = _element(footprint, ndim)
     st = None
@@ -380,7 +419,7 @@ def tm_binary_morph(mask, structure, op="erosion", border_value=0, origin=None, 
         mask = mask.view(torch.uint8)
     if mask.dtype != torch.uint8:
         raise TypeError("mask must be uint8 or bool")
-    mask = mask.contiguous()
+    mask = _contiguous_on(mask, stream)
     ndim = mask.dim() - 2
     fp, fps = _element(structure, ndim)
     if out is None:
@@ -395,7 +434,7 @@ def tm_binary_morph(mask, structure, op="erosion", border_value=0, origin=None, 
 METRICS = {"euclidean": 0, "taxicab": 1, "chessboard": 2}
 
 
-def _mask_u8(mask):
+def _mask_u8(mask, stream=None):
     import torch
 
     if not mask.is_cuda or mask.dim() < 3:
@@ -404,7 +443,7 @@ def _mask_u8(mask):
         mask = mask.view(torch.uint8)
     if mask.dtype != torch.uint8:
         raise TypeError("mask must be uint8 or bool")
-    return mask.contiguous()
+    return _contiguous_on(mask, stream)
 
 
 def tm_cdt(mask, metric="chessboard", out=None, stream=None):
@@ -413,7 +452,7 @@ def tm_cdt(mask, metric="chessboard", out=None, stream=None):
     import torch
 
     L = lib()
-    mask = _mask_u8(mask)
+    mask = _mask_u8(mask, stream)
     if out is None:
         out = torch.empty(mask.shape, dtype=torch.int32, device=mask.device)
     _check(L.tm_cdt(_p(mask), mask.dim() - 2, _shape_array(tuple(mask.shape)), METRICS[metric], _p(out), _raw_stream(stream)))
@@ -425,7 +464,7 @@ def tm_bfdt(mask, sampling=None, metric="euclidean", out=None, stream=None):
     import torch
 
     L = lib()
-    mask = _mask_u8(mask)
+    mask = _mask_u8(mask, stream)
     ndim = mask.dim() - 2
     if out is None:
         out = torch.empty(mask.shape, dtype=torch.float32, device=mask.device)

@@ -38,6 +38,17 @@ struct Plan {
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
 };
 
+// Debug and test switches, read from the environment once (and again by tm_edt_reload_switches()).
+struct Switches {
+    bool force_generic = false;   // TM_EDT_FORCE_GENERIC=1: rank- and extent-generic kernels for every shape
+    bool no_scaled = false;       // TM_EDT_NO_SCALED: no scaled-integer mode
+    bool old_plane = false;       // TM_EDT_OLD_PLANE=1: byte-load plane kernel
+    bool no_value_carry = false;  // TM_EDT_NO_VALUE_CARRY: offsets are carried even without an index output
+    bool no_lean = false;         // TM_EDT_NO_LEAN: one-voxel-per-lane kernels instead of the quad kernels
+    long long chunk_voxels = 0;   // TM_EDT_CHUNK_VOXELS=n: image ranges of at most n voxels (0 = grid limit)
+};
+const Switches& switches();
+
 // Per-kernel timing of tm_edt_profile: records an event before the launch that follows.
 // `bytes`: what that launch has to read and write once (its inputs plus its outputs).
 void prof_mark(cudaStream_t st, const char* name, double bytes);

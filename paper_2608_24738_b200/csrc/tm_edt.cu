@@ -27,6 +27,33 @@ namespace tmedt {
 static thread_local int g_last_cuda_error = 0;
 static thread_local int g_last_launches = 0;
 
+// Debug and test switches.  The environment is read once, at the first call that needs a switch, and again only
+// when tm_edt_reload_switches() is called (the tests change switches inside one process).
+static Switches g_switches;
+static bool g_switches_loaded = false;
+static std::mutex g_switches_mutex;
+
+static void load_switches_locked() {
+    auto on = [](const char* name) { const char* v = getenv(name); return v && v[0] == '1'; };
+    auto set = [](const char* name) { return getenv(name) != nullptr; };
+    Switches s;
+    s.force_generic = on("TM_EDT_FORCE_GENERIC");
+    s.no_scaled = set("TM_EDT_NO_SCALED");
+    s.old_plane = on("TM_EDT_OLD_PLANE");
+    s.no_value_carry = set("TM_EDT_NO_VALUE_CARRY");
+    s.no_lean = set("TM_EDT_NO_LEAN");
+    s.chunk_voxels = 0;
+    if (const char* lim = getenv("TM_EDT_CHUNK_VOXELS")) { const long long v = atoll(lim); if (v > 0) s.chunk_voxels = v; }
+    g_switches = s;
+    g_switches_loaded = true;
+}
+
+const Switches& switches() {
+    std::lock_guard<std::mutex> lock(g_switches_mutex);
+    if (!g_switches_loaded) load_switches_locked();
+    return g_switches;
+}
+
 // Optional per-kernel timing (tm_edt_profile): an event is recorded on the stream before every launch
 // and once after the last one.
 constexpr int kProfMax = 32;
@@ -48,7 +75,26 @@ void prof_mark(cudaStream_t st, const char* name, double bytes) {
     ++g_prof.count;
 }
 
-static int make_plan(int ndim, const int64_t* shape, const double* sampling, Plan& pl) {
+// Scratch layout of the wide-key and long-line paths: two 32-bit key (or height) buffers, and -- only when an index
+// output is requested -- 16-bit offsets per processed axis; the long-line path adds its block minima.
+struct WideLayout { size_t keysA, offsA, keysB, offsB, offsC, bm, total; };
+
+static WideLayout wide_layout(int64_t N, int E, bool want_idx, bool block_minima) {
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    WideLayout L;
+    size_t o = 0;
+    L.keysA = o; o += up((size_t)N * 4);
+    L.offsA = o; if (want_idx) o += up((size_t)N * 2);
+    L.keysB = o; if (E >= 3) o += up((size_t)N * 4);
+    L.offsB = o; if (E >= 3 && want_idx) o += up((size_t)N * 4);
+    L.offsC = o; if (E == 4 && want_idx) o += up((size_t)N * 8);
+    L.bm = o; if (block_minima) o += up((size_t)N / 4 + 1024);
+    L.total = o;
+    return L;
+}
+
+// want_idx: whether the call asks for the index output (scratch of the wide-key and long-line paths depends on it).
+static int make_plan(int ndim, const int64_t* shape, const double* sampling, Plan& pl, bool want_idx = true) {
     if (!shape || ndim < 1 || ndim > kMaxDims) return TM_EDT_ERR_INVALID_ARG;
     for (int k = 0; k < ndim + 2; ++k)
         if (shape[k] < 0) return TM_EDT_ERR_INVALID_ARG;
@@ -113,28 +159,22 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     const size_t elem = pl.wide ? 2 : 1;
     pl.plane_bytes = (((size_t)pl.N * elem) + 255) & ~(size_t)255;
     pl.ws_bytes = E > 1 ? 2 * (size_t)(E - 1) * pl.plane_bytes : 0;
-    const char* force = getenv("TM_EDT_FORCE_GENERIC");
-    pl.small = nmax <= 8 && !(force && force[0] == '1');
-    pl.fast = !pl.small && nmax <= 128 && E >= 2 && E <= 5 && !(force && force[0] == '1');
+    const Switches& sw = switches();
+    const bool force = sw.force_generic;
+    pl.small = nmax <= 8 && !force;
+    pl.fast = !pl.small && nmax <= 128 && E >= 2 && E <= 5 && !force;
     // unit sampling: integer keys (two axes up to extent 1024, three up to 512); other sampling: float heights
     // integer keys (value << sh | row, sh = 9 row bits up to extent 512, else 10): every real key must stay below the
     // "no site" key 2^31 and "no site" plus the largest addend below 2^32
     const double key_scale = nmax > 512 ? 1024.0 : 512.0;
     const bool keys_fit = sumsq * key_scale < 2147483648.0 && (double)(nmax + 4) * (nmax + 4) * key_scale < 2147483648.0;
     pl.wide_keys = !pl.small && !pl.fast && E >= 2 && E <= 4 && nmax <= 1024 && (!pl.unit || keys_fit) &&
-                   !(force && force[0] == '1');
+                   !force;
     pl.long_lines = !pl.small && !pl.fast && !pl.wide_keys && (E == 2 || E == 3) && nmax <= 8192 &&
-                    !(force && force[0] == '1');
-    if (pl.wide_keys || pl.long_lines) {
-        auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
-        const size_t bm = pl.long_lines ? up((size_t)pl.N / 4 + 1024) : 0;  // block minima of the long path
-        pl.ws_bytes = up((size_t)pl.N * 4) + up((size_t)pl.N * 2);                       // keys + 1 offset
-        if (E >= 3) pl.ws_bytes += up((size_t)pl.N * 4) + up((size_t)pl.N * 4);             // keys + 2 offsets
-        if (E == 4) pl.ws_bytes += up((size_t)pl.N * 8);                                    // 3 offsets, stored as 4
-        pl.ws_bytes += bm;
-    }
+                    !force;
+    if (pl.wide_keys || pl.long_lines) pl.ws_bytes = wide_layout(pl.N, E, want_idx, pl.long_lines).total;
     if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
-    if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !getenv("TM_EDT_NO_SCALED")) {
+    if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !sw.no_scaled) {
         // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
         // the largest possible value below 2^24 (keys are value << 7 | row in 32 bits)
         static const int cand[] = {1, 4, 16, 25, 64, 100, 256, 400, 625, 1024, 2500, 10000};
@@ -213,8 +253,8 @@ static cudaError_t launch_axis_k(const AxisParams& P, const EpilogueParams& ep, 
     while (threads > 32 && per_thread * threads > 64 * 1024) threads >>= 1;
     const size_t smem = per_thread * threads;
     auto kern = axis_pass_kernel<CT, OT, K, FINAL>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    {
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
     }
     const int64_t blocks = (P.lines + threads - 1) / threads;
@@ -280,8 +320,8 @@ static cudaError_t launch_column_tx(const FastParams& P, const EpilogueParams& e
     const size_t eb = (size_t)entry_bytes(K);
     const size_t smem = (size_t)P.n * TX * (4 + eb);
     auto kern = column_kernel<K, FINAL, UNIT, TX>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    {
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
     }
     const int tiles = (int)((P.inner + TX - 1) / TX);
@@ -328,7 +368,8 @@ static cudaError_t launch_column_value(const FastParams& P, const EpilogueParams
 #define TM_LAUNCH_COLUMN_VALUE(TXV)                                                                            \
     do {                                                                                                       \
         auto kern = column_value_kernel<FINAL, VT, SCALED, TXV>;                                               \
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<(unsigned)blocks, 256, smem, st>>>(P, ep, tiles);                                               \
     } while (0)
     if (G == 1) TM_LAUNCH_COLUMN_VALUE(32); else if (G == 2) TM_LAUNCH_COLUMN_VALUE(64); else TM_LAUNCH_COLUMN_VALUE(128);
@@ -358,9 +399,9 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
     // without an index output the passes carry squared distances instead of offsets (unit sampling, tile plane kernel)
     double sumsq = 0.0;
     for (int p = 0; p < pl.E; ++p) sumsq += (double)(pl.ext[p] - 1) * (pl.ext[p] - 1);
-    const char* oldp0 = getenv("TM_EDT_OLD_PLANE");
+    const Switches& sw = switches();
     const bool vc = UNIT && !ep.idx && pl.E >= 3 && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 &&
-                    !(oldp0 && oldp0[0] == '1') && !getenv("TM_EDT_NO_VALUE_CARRY");
+                    !sw.old_plane && !sw.no_value_carry;
     const bool vc16 = vc && sumsq < 65535.0;
     P.value_carry = vc ? (vc16 ? 2 : 4) : 0;
     {
@@ -369,35 +410,36 @@ static cudaError_t run_fast(const Plan& pl, const uint8_t* in, const EpiloguePar
         const size_t smem = (((size_t)pl.ext[1] * tstride + 15) & ~(size_t)15) + (size_t)pl.ext[1] * 32 * 4;
         const bool fin = pl.E == 2;
         prof_mark(st, fin ? "plane_final" : "plane", (double)pl.N * (1.0 + (fin ? out_bpv : (P.value_carry == 4 ? 4.0 : 2.0))));
-        const char* oldp = getenv("TM_EDT_OLD_PLANE");
-        if (UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
+        if (UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !sw.old_plane) {
             // whole-plane key tile; row stride = extent rounded up to 32, 64 or 128 columns
             const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
             const size_t smem_u = (size_t)pl.ext[1] * vs * 4;
 #define TM_LAUNCH_PLANE_UNIT(FIN, VSV, VCV)                                                                    \
     do {                                                                                                       \
         auto kern = plane_unit_kernel<FIN, VSV, VCV>;                                                          \
-        if (smem_u > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_u); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem_u);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<(unsigned)P.outer, threads, smem_u, st>>>(P, ep);                                               \
     } while (0)
 #define TM_LAUNCH_PLANE_UNIT_VS(FIN, VCV)                                                                      \
     do {                                                                                                       \
         if (vs == 32) TM_LAUNCH_PLANE_UNIT(FIN, 32, VCV); else if (vs == 64) TM_LAUNCH_PLANE_UNIT(FIN, 64, VCV); else TM_LAUNCH_PLANE_UNIT(FIN, 128, VCV); \
     } while (0)
-            if (fin && !ep.idx && !getenv("TM_EDT_NO_VALUE_CARRY")) TM_LAUNCH_PLANE_UNIT_VS(true, 4);  // plain values: no site needed
+            if (fin && !ep.idx && !sw.no_value_carry) TM_LAUNCH_PLANE_UNIT_VS(true, 4);  // plain values: no site needed
             else if (fin) TM_LAUNCH_PLANE_UNIT_VS(true, 0);
             else if (P.value_carry == 2) TM_LAUNCH_PLANE_UNIT_VS(false, 2);
             else if (P.value_carry == 4) TM_LAUNCH_PLANE_UNIT_VS(false, 4);
             else TM_LAUNCH_PLANE_UNIT_VS(false, 0);
 #undef TM_LAUNCH_PLANE_UNIT_VS
 #undef TM_LAUNCH_PLANE_UNIT
-        } else if (!UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !(oldp && oldp[0] == '1')) {
+        } else if (!UNIT && pl.ext[0] % 4 == 0 && ((uintptr_t)in & 3u) == 0 && !sw.old_plane) {
             const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
             const size_t smem_s = (size_t)pl.ext[1] * vs * 5;
 #define TM_LAUNCH_PLANE_SAMPLED(FIN, VSV)                                                                      \
     do {                                                                                                       \
         auto kern = plane_sampled_kernel<FIN, VSV>;                                                            \
-        if (smem_s > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_s); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem_s);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<(unsigned)P.outer, 512, smem_s, st>>>(P, ep, tab);                                              \
     } while (0)
             if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SAMPLED(true, 32); else if (vs == 64) TM_LAUNCH_PLANE_SAMPLED(true, 64); else TM_LAUNCH_PLANE_SAMPLED(true, 128); }
@@ -443,7 +485,8 @@ static cudaError_t launch_column_scaled(const FastParams& P, const EpilogueParam
 #define TM_LAUNCH_COLUMN_SCALED(TXV)                                                                           \
     do {                                                                                                       \
         auto kern = column_scaled_kernel<K, FINAL, TXV>;                                                       \
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<(unsigned)blocks, 256, smem, st>>>(P, ep, tiles);                                               \
     } while (0)
     if (G == 1) TM_LAUNCH_COLUMN_SCALED(32); else if (G == 2) TM_LAUNCH_COLUMN_SCALED(64); else TM_LAUNCH_COLUMN_SCALED(128);
@@ -469,21 +512,23 @@ static cudaError_t run_scaled(const Plan& pl, const uint8_t* in, const EpilogueP
     fill(P, 1);
     P.in = in; P.out = bufA; P.n0 = pl.ext[0];
     // without an index output the passes carry the scaled squared distance (32 bits) instead of offsets
-    const bool vc = !ep.idx && pl.E >= 3 && !getenv("TM_EDT_NO_VALUE_CARRY");
+    const Switches& sw = switches();
+    const bool vc = !ep.idx && pl.E >= 3 && !sw.no_value_carry;
     P.value_carry = vc ? 4 : 0;
     {
         const bool fin = pl.E == 2;
         const int vs = pl.ext[0] <= 32 ? 32 : (pl.ext[0] <= 64 ? 64 : 128);
-        const bool plain_fin = fin && !ep.idx && ep.dist && !getenv("TM_EDT_NO_VALUE_CARRY");
+        const bool plain_fin = fin && !ep.idx && ep.dist && !sw.no_value_carry;
         const size_t smem = (size_t)pl.ext[1] * vs * (((vc && !fin) || plain_fin) ? 4 : 5);  // keys, plus a byte tile of first-axis offsets
         prof_mark(st, fin ? "plane_scaled_final" : "plane_scaled", (double)pl.N * (1.0 + (fin ? out_bpv : (vc ? 4.0 : 2.0))));
 #define TM_LAUNCH_PLANE_SCALED(FIN, VSV, VCV)                                                                  \
     do {                                                                                                       \
         auto kern = plane_scaled_kernel<FIN, VSV, VCV>;                                                        \
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<(unsigned)P.outer, 512, smem, st>>>(P, ep);                                                     \
     } while (0)
-        if (fin && !ep.idx && ep.dist && !getenv("TM_EDT_NO_VALUE_CARRY")) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, true); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, true); else TM_LAUNCH_PLANE_SCALED(true, 128, true); }
+        if (plain_fin) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, true); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, true); else TM_LAUNCH_PLANE_SCALED(true, 128, true); }
         else if (fin) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(true, 32, false); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(true, 64, false); else TM_LAUNCH_PLANE_SCALED(true, 128, false); }
         else if (vc) { if (vs == 32) TM_LAUNCH_PLANE_SCALED(false, 32, true); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(false, 64, true); else TM_LAUNCH_PLANE_SCALED(false, 128, true); }
         else { if (vs == 32) TM_LAUNCH_PLANE_SCALED(false, 32, false); else if (vs == 64) TM_LAUNCH_PLANE_SCALED(false, 64, false); else TM_LAUNCH_PLANE_SCALED(false, 128, false); }
@@ -555,7 +600,8 @@ static cudaError_t run_small(const Plan& pl, const uint8_t* in, const EpiloguePa
 #define TM_SMALL_LAUNCH3(FIRST, FIN, NM)                                                                         \
     do {                                                                                                         \
         auto kern = small_group_kernel<SITE, FIRST, FIN, NM>;                                                    \
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        const cudaError_t ea = ensure_smem(reinterpret_cast<const void*>(kern), smem);                           \
+        if (ea != cudaSuccess) return ea;                                                                      \
         kern<<<blocks, threads, smem, st>>>(P, ep);                                                        \
     } while (0)
 #define TM_SMALL_LAUNCH(FIRST, FIN)                                                                              \
@@ -591,8 +637,8 @@ static cudaError_t launch_wide_axis_cw(const WideAxisParams& A, const EpiloguePa
     auto kern = sh < 0 ? wide_axis_kernel<K, FINAL, -1, CW>
                        : (sh == 0 ? wide_axis_kernel<K, FINAL, 0, CW>
                                   : (sh == 10 ? wide_axis_kernel<K, FINAL, 10, CW> : wide_axis_kernel<K, FINAL, 9, CW>));
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    {
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
     }
     // few strips (a single large image): several blocks share a strip, each taking a range of its rows, until
@@ -619,10 +665,11 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
                               int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* w = static_cast<char*>(ws);
-    uint32_t* keysA = reinterpret_cast<uint32_t*>(w);
-    int16_t* offsA = reinterpret_cast<int16_t*>(w + up((size_t)pl.N * 4));
-    uint32_t* keysB = reinterpret_cast<uint32_t*>(w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
-    int16_t* offsB = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
+    const WideLayout L = wide_layout(pl.N, pl.E, ep.idx != nullptr, false);
+    uint32_t* keysA = reinterpret_cast<uint32_t*>(w + L.keysA);
+    int16_t* offsA = reinterpret_cast<int16_t*>(w + L.offsA);
+    uint32_t* keysB = reinterpret_cast<uint32_t*>(w + L.keysB);
+    int16_t* offsB = reinterpret_cast<int16_t*>(w + L.offsB);
     const bool carry = ep.idx != nullptr;  // offsets are carried only for the index output
     WideParams P;
     P.in = in; P.keys = keysA; P.offs = carry ? offsA : nullptr;
@@ -657,7 +704,7 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     ++launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    int16_t* offsC = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2) + up((size_t)pl.N * 4));
+    int16_t* offsC = reinterpret_cast<int16_t*>(w + L.offsC);
     WideAxisParams A;
     memset(&A, 0, sizeof(A));
     A.n0 = pl.ext[0]; A.n1 = pl.ext[1];
@@ -691,12 +738,12 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
                             int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* w = static_cast<char*>(ws);
-    uint32_t* hA = reinterpret_cast<uint32_t*>(w);
-    int16_t* offsA = reinterpret_cast<int16_t*>(w + up((size_t)pl.N * 4));
-    uint32_t* hB = reinterpret_cast<uint32_t*>(w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
-    int16_t* offsB = reinterpret_cast<int16_t*>(w + 2 * up((size_t)pl.N * 4) + up((size_t)pl.N * 2));
-    uint32_t* blockmin = reinterpret_cast<uint32_t*>(
-        w + up((size_t)pl.N * 4) + up((size_t)pl.N * 2) + (pl.E == 3 ? 2 * up((size_t)pl.N * 4) : 0));
+    const WideLayout L = wide_layout(pl.N, pl.E, ep.idx != nullptr, true);
+    uint32_t* hA = reinterpret_cast<uint32_t*>(w + L.keysA);
+    int16_t* offsA = reinterpret_cast<int16_t*>(w + L.offsA);
+    uint32_t* hB = reinterpret_cast<uint32_t*>(w + L.keysB);
+    int16_t* offsB = reinterpret_cast<int16_t*>(w + L.offsB);
+    uint32_t* blockmin = reinterpret_cast<uint32_t*>(w + L.bm);
     WideParams P;
     const bool carry = ep.idx != nullptr;  // offsets are carried only for the index output
     P.in = in; P.keys = hA; P.offs = carry ? offsA : nullptr;
@@ -821,7 +868,9 @@ static int check_call(const uint8_t* input, int ndim, const int64_t* shape, cons
     if (!input) return TM_EDT_ERR_INVALID_ARG;
     if (flags & ~(unsigned)(TM_EDT_FLAG_VIRTUAL_BACKGROUND | TM_EDT_FLAG_FLAT_INDEX | TM_EDT_FLAG_DIST_F64))
         return TM_EDT_ERR_INVALID_ARG;
-    const int rc = make_plan(ndim, shape, sampling, pl);
+    // the float64 variant obtains the site of every voxel first, so it plans like a call with index output
+    const bool want_idx = out_idx != nullptr || ((flags & TM_EDT_FLAG_DIST_F64) && out_dist != nullptr);
+    const int rc = make_plan(ndim, shape, sampling, pl, want_idx);
     if (rc != TM_EDT_OK) return rc;
     pl.flags = flags;
     for (int a = 0; a < ndim; ++a) { pl.shape_sp[a] = shape[2 + a]; pl.w_sp[a] = sampling ? sampling[a] : 1.0; }
@@ -845,7 +894,7 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     if (pl.wide_keys) return run_wide(pl, input, ep, ws, st, launches);
     if (pl.long_lines)
         return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
-    if (!getenv("TM_EDT_NO_LEAN") && lean_ok(pl, input, ep)) return run_lean(pl, input, ep, ws, st, launches);
+    if (!switches().no_lean && lean_ok(pl, input, ep)) return run_lean(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)
         return pl.unit ? run_fast<true>(pl, input, ep, ws, st, launches) : run_fast<false>(pl, input, ep, ws, st, launches);
@@ -861,10 +910,8 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
 static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int64_t* out_sq, int64_t* out_idx,
                       void* ws, cudaStream_t st) {
     int64_t max_voxels = INT32_MAX;
-    if (const char* lim = getenv("TM_EDT_CHUNK_VOXELS")) {  // test hook: smaller image ranges
-        const long long v = atoll(lim);
-        if (v > 0 && v < max_voxels) max_voxels = v;
-    }
+    const long long lim = switches().chunk_voxels;  // test hook: smaller image ranges
+    if (lim > 0 && lim < max_voxels) max_voxels = lim;
     const int64_t max_images = std::max<int64_t>(1, max_voxels / pl.V);
     int launches = 0;
     for (int64_t first = 0; first < pl.images; first += max_images) {
@@ -906,10 +953,30 @@ using namespace tmedt;
 
 extern "C" {
 
-size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape) {
+// Largest scratch any call on this shape can need with / without index output: the planner may pick different kernel
+// families for unit and for other sampling, so both plans are made and the larger one reported.
+static size_t worst_case_workspace(int ndim, const int64_t* shape, bool want_idx) {
+    Plan unit_plan, sampled_plan;
+    double other[kMaxDims];
+    for (int k = 0; k < kMaxDims; ++k) other[k] = 1.37;
+    if (make_plan(ndim, shape, nullptr, unit_plan, want_idx) != TM_EDT_OK) return (size_t)-1;
+    if (make_plan(ndim, shape, other, sampled_plan, want_idx) != TM_EDT_OK) return (size_t)-1;
+    return std::max(unit_plan.ws_bytes, sampled_plan.ws_bytes);
+}
+
+size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape) { return worst_case_workspace(ndim, shape, true); }
+
+size_t tm_edt_workspace_bytes_for(int ndim, const int64_t* shape, const double* sampling, int want_dist, int want_sqdist,
+                                  int want_indices) {
+    (void)want_dist; (void)want_sqdist;  // distances and squared distances need no scratch of their own
     Plan pl;
-    if (make_plan(ndim, shape, nullptr, pl) != TM_EDT_OK) return (size_t)-1;
+    if (make_plan(ndim, shape, sampling, pl, want_indices != 0) != TM_EDT_OK) return (size_t)-1;
     return pl.ws_bytes;
+}
+
+void tm_edt_reload_switches(void) {
+    std::lock_guard<std::mutex> lock(g_switches_mutex);
+    load_switches_locked();
 }
 
 int tm_edt_ws(const uint8_t* input, int ndim, const int64_t* shape, const double* sampling, float* out_dist,
@@ -984,6 +1051,8 @@ size_t tm_edt_ex_workspace_bytes(int ndim, const int64_t* shape, const int64_t* 
                                  int with_distances, int with_indices) {
     Plan pl;
     if (make_plan(ndim, shape, nullptr, pl) != TM_EDT_OK) return (size_t)-1;
+    const bool want_idx = with_indices != 0 || ((flags & TM_EDT_FLAG_DIST_F64) && with_distances != 0);
+    pl.ws_bytes = worst_case_workspace(ndim, shape, want_idx);
     int64_t st[kMaxDims + 2];
     bool strided = false;
     size_t span = 0;

@@ -27,6 +27,42 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+class _Switches:
+    """Sets the library's debug switches (environment variables it reads once) and makes it read them again."""
+
+    def __init__(self):
+        self._saved = {}
+
+    def set(self, name, value):
+        from paper_2608_24738_b200 import binding
+
+        self._saved.setdefault(name, os.environ.get(name))
+        if value is None:
+            os.environ.pop(name, None)
+        else:
+            os.environ[name] = str(value)
+        binding.tm_edt_reload_switches()
+
+    def restore(self):
+        from paper_2608_24738_b200 import binding
+
+        for name, old in self._saved.items():
+            if old is None:
+                os.environ.pop(name, None)
+            else:
+                os.environ[name] = old
+        if self._saved:
+            binding.tm_edt_reload_switches()
+        self._saved = {}
+
+
+@pytest.fixture
+def switches():
+    s = _Switches()
+    yield s
+    s.restore()
+
+
 def read_golden(path):
     """Parse tests/golden/*.txt blocks into dicts (name, shape, sampling, mask, sq)."""
     import numpy as np

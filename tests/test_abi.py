@@ -28,8 +28,9 @@ def test_header_symbols_are_exported(L):
 
 def test_version_and_strerror(L):
     assert "sm_100a" in binding.tm_edt_version()
-    for s in range(6):
-        assert binding.tm_edt_strerror(s)
+    texts = [binding.tm_edt_strerror(s) for s in range(7)]  # TM_EDT_OK .. TM_EDT_ERR_TOO_LARGE
+    assert all(texts) and "unknown status" not in texts and len(set(texts)) == 7
+    assert "tm_edt_noalloc" in binding.tm_edt_strerror(binding.ERR_TOO_LARGE)
     assert binding.tm_edt_strerror(99) == "unknown status"
 
 
@@ -139,6 +140,35 @@ def test_workspace_bytes(L):
     assert binding.tm_edt_workspace_bytes((1, 1, 300, 300)) >= 2 * 300 * 300  # generic path: 16-bit offset planes
     assert binding.tm_edt_workspace_bytes((1, 1, 1024, 1024)) == 6 * 1024 * 1024  # wide path, two axes: key + offset
     assert binding.tm_edt_workspace_bytes((1, 1, 256, 256, 256)) == 14 * 256 ** 3  # three axes: 2 keys + 1 + 2 offsets
+    # one particular call: without an index output no offsets are carried
+    assert binding.tm_edt_workspace_bytes_for((1, 1, 256, 256, 256), want_indices=True) == 14 * 256 ** 3
+    assert binding.tm_edt_workspace_bytes_for((1, 1, 256, 256, 256), want_indices=False) == 8 * 256 ** 3
+    assert binding.tm_edt_workspace_bytes_for((1, 1, 1024, 1024), want_indices=False) == 4 * 1024 * 1024
+    assert binding.tm_edt_workspace_bytes_for((2, 1, 128, 128, 128), (2.5, 0.8, 1.0)) == 4 * 2 * 128 ** 3
+
+
+def test_workspace_bytes_cover_every_sampling(L):
+    """tm_edt_workspace_bytes(shape) suffices whatever the sampling: the planner may choose another kernel family
+    for non-unit sampling (shapes on both sides of the limit up to which integer keys fit 31 bits), and a call with a
+    workspace of the reported size must never be refused as too small.  No GPU: the call stops at the pointer check,
+    which comes after the size check."""
+    shapes = [(1, 1, 2, 66, 1024, 1024), (1, 1, 2, 60, 520, 516), (1, 1, 4, 4, 600, 600), (1, 1, 900, 900, 8),
+              (1, 1, 1024, 1024), (1, 1, 300, 300, 300), (2, 1, 128, 128, 128), (1, 1, 16, 128, 128, 128),
+              (1, 1, 5, 200, 40, 520)]
+    for shape in shapes:
+        ndim = len(shape) - 2
+        need = binding.tm_edt_workspace_bytes(shape)
+        shp = (ctypes.c_int64 * len(shape))(*shape)
+        for sampling in (None, tuple(1.0 + 0.37 * k for k in range(ndim)), (2.5,) * ndim):
+            smp = (ctypes.c_double * ndim)(*sampling) if sampling is not None else None
+            assert binding.tm_edt_workspace_bytes_for(shape, sampling, want_indices=True) <= need
+            fake = lambda v: ctypes.c_void_p((v << 42) + 4096)  # far apart (no overlap), never dereferenced: the pointer check refuses them
+            rc = L.tm_edt_ws(fake(1), ndim, shp, smp, fake(2), None, fake(3), fake(4), ctypes.c_size_t(need), None)
+            assert rc == binding.ERR_BAD_POINTER, (shape, sampling, rc)
+            if need > 0:
+                rc = L.tm_edt_ws(fake(1), ndim, shp, smp, fake(2), None, fake(3), fake(4),
+                                 ctypes.c_size_t(binding.tm_edt_workspace_bytes_for(shape, sampling, want_indices=True) - 1), None)
+                assert rc == binding.ERR_ALLOC or binding.tm_edt_workspace_bytes_for(shape, sampling, want_indices=True) == 0
     with pytest.raises(binding.TmEdtError):
         binding.tm_edt_workspace_bytes((1, 1, binding.MAX_EXTENT + 1))
 

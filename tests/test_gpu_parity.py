@@ -20,13 +20,12 @@ def _built():
     binding.lib()
 
 
-@pytest.fixture(params=["default", "generic"])
-def path(request, monkeypatch):
-    """Both kernel families: the planner's own choice, and the rank-/extent-generic kernels forced."""
-    if request.param == "generic":
-        monkeypatch.setenv("TM_EDT_FORCE_GENERIC", "1")
-    else:
-        monkeypatch.delenv("TM_EDT_FORCE_GENERIC", raising=False)
+@pytest.fixture(params=["default", "generic", "no_lean"])
+def path(request, switches):
+    """Every kernel family: the planner's own choice, the rank-/extent-generic kernels forced, and the
+    one-voxel-per-lane packed-entry kernels in place of the quad kernels."""
+    switches.set("TM_EDT_FORCE_GENERIC", "1" if request.param == "generic" else None)
+    switches.set("TM_EDT_NO_LEAN", "1" if request.param == "no_lean" else None)
     return request.param
 
 
@@ -186,14 +185,25 @@ def test_mixed_batch_with_image_without_background(path):
 
 
 def test_half_space_and_far_sites(path):
+    """Far sites are checked against the closed forms directly as well, not only against the oracle."""
     mask = np.ones((1, 1, 128, 96), dtype=np.uint8)
     mask[0, 0, :3] = 0
-    full_check(mask, None)
-    full_check(mask, (0.3, 1.9))
+    rows = np.maximum(np.arange(128.0) - 2.0, 0.0)[:, None] * np.ones((1, 96))  # distance in rows to row 2
+    res, _ = full_check(mask, None)
+    assert np.array_equal(res["sq"][0, 0], (rows ** 2).astype(np.int64))
+    res, _ = full_check(mask, (0.3, 1.9))
+    np.testing.assert_allclose(res["dist"][0, 0], 0.3 * rows, rtol=1e-5, atol=1e-5)
     mask = np.ones((1, 1, 100, 128, 128), dtype=np.uint8)
-    mask[0, 0, 99, 127, 0] = 0
-    full_check(mask, None)  # largest offsets an int8 carry can hold
-    full_check(mask, (2.5, 0.8, 1.0))
+    site = (99, 127, 0)
+    mask[(0, 0) + site] = 0
+    g = np.meshgrid(np.arange(100.0), np.arange(128.0), np.arange(128.0), indexing="ij", sparse=True)
+    res, _ = full_check(mask, None)  # largest offsets an int8 carry can hold
+    assert np.array_equal(res["sq"][0, 0], sum((g[k] - site[k]) ** 2 for k in range(3)).astype(np.int64))
+    for k in range(3):
+        assert (res["idx"][0, 0, k] == site[k]).all()
+    res, _ = full_check(mask, (2.5, 0.8, 1.0))
+    closed = np.sqrt(sum((w * (g[k] - site[k])) ** 2 for k, w in enumerate((2.5, 0.8, 1.0))))
+    assert (np.abs(res["dist"][0, 0] - closed) <= 1e-5 * np.maximum(1.0, closed)).all()
 
 
 @pytest.mark.parametrize("n", [512, 513, 1024, 1100, 2048])
@@ -305,15 +315,15 @@ def test_unaligned_input_pointer():
             checker.check_indices(r["idx"].cpu().numpy(), mask, ref, samp)
 
 
-def test_large_batches_run_as_image_ranges(monkeypatch):
+def test_large_batches_run_as_image_ranges(switches):
     """A batch that does not fit one grid is cut into image ranges; a test hook makes the ranges tiny."""
-    monkeypatch.setenv("TM_EDT_CHUNK_VOXELS", str(2 * 12 * 16 * 20 + 5))  # two images per range
+    switches.set("TM_EDT_CHUNK_VOXELS", str(2 * 12 * 16 * 20 + 5))  # two images per range
     mask = workloads.random_mask(21, (5, 1, 12, 16, 20), 0.85)
     mask[3] = 1
     res, ref = full_check(mask, None)
     assert binding.tm_edt_last_launch_count() == 3 * 2  # three ranges, two kernels each
     full_check(mask, (1.5, 0.7, 1.0))
-    monkeypatch.setenv("TM_EDT_FORCE_GENERIC", "1")
+    switches.set("TM_EDT_FORCE_GENERIC", "1")
     full_check(mask, None)
 
 
@@ -584,7 +594,7 @@ VALUE_SHAPES = [(2, 1, 12, 20, 24), (1, 2, 33, 17, 40), (1, 1, 128, 20, 48), (2,
 
 @pytest.mark.parametrize("shape", VALUE_SHAPES, ids=["x".join(map(str, s)) for s in VALUE_SHAPES])
 @pytest.mark.parametrize("kind", ["unit", "decimal", "sampled"])
-def test_outputs_without_indices(shape, kind, monkeypatch):
+def test_outputs_without_indices(shape, kind, switches):
     """Without an index output the packed-entry path carries squared distances instead of offsets (16-bit values up to
     four axes, 32-bit beyond and in scaled-integer mode).  Distances and exact squared distances against the oracle,
     and bit-identical to what the offset-carrying kernels give."""
@@ -601,8 +611,8 @@ def test_outputs_without_indices(shape, kind, monkeypatch):
         if unit:
             only_sq = run_gpu(mask, sampling, dist=False, sq=True, idx=False)
             checker.check_sq_exact(only_sq["sq"], ref["sq"])
-        monkeypatch.setenv("TM_EDT_NO_VALUE_CARRY", "1")
+        switches.set("TM_EDT_NO_VALUE_CARRY", "1")
         old = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
-        monkeypatch.delenv("TM_EDT_NO_VALUE_CARRY")
+        switches.set("TM_EDT_NO_VALUE_CARRY", None)
         if kind != "sampled":  # integer paths: the same values either way
             assert np.array_equal(res["dist"], old["dist"])

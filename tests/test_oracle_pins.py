@@ -288,6 +288,62 @@ def test_virtual_background_convention(shape, samp, kind):
     np.testing.assert_array_equal(r["idx"][1, 0], plain["idx"][1, 0])
 
 
+# ---- far sites: the outward scan of the separable oracle walks tens to hundreds of rows before its cut-off ends it
+
+@pytest.mark.parametrize("samp", [None, (2.5, 0.8, 1.0)], ids=["unit", "sampled"])
+def test_far_single_site_closed_form(samp):
+    """One background voxel in a 90 x 70 x 110 volume: every voxel's answer is the distance to that voxel, up to
+    about 150 rows away, so a cut-off that stops a scan one row early (or a sign error far from the site) shows."""
+    shape = (90, 70, 110)
+    site = (71, 5, 93)
+    mask = np.ones((1, 1) + shape, dtype=np.uint8)
+    mask[(0, 0) + site] = 0
+    r = oracle.sep(mask, samp)
+    w = np.ones(3) if samp is None else np.asarray(samp, dtype=np.float64)
+    grid = np.meshgrid(*[np.arange(n, dtype=np.float64) for n in shape], indexing="ij", sparse=True)
+    sq = sum((w[k] * (grid[k] - site[k])) ** 2 for k in range(3))
+    np.testing.assert_allclose(r["sqf"][0, 0], sq, rtol=1e-14, atol=0)
+    np.testing.assert_allclose(r["dist"][0, 0], np.sqrt(sq), rtol=1e-14, atol=0)
+    if samp is None:
+        assert np.array_equal(r["sq"][0, 0], sq.astype(np.int64))
+    for k in range(3):
+        assert (r["idx"][0, 0, k] == site[k]).all()
+
+
+def test_few_far_sites_against_brute_force_and_scipy():
+    """Six background voxels in 60 x 50 x 70: scans of up to 70 rows whose winner changes along the way."""
+    ndimage = pytest.importorskip("scipy.ndimage")
+    rng = np.random.default_rng(424738)
+    shape = (60, 50, 70)
+    mask = np.ones((1, 1) + shape, dtype=np.uint8)
+    for _ in range(6):
+        mask[(0, 0) + tuple(int(rng.integers(0, n)) for n in shape)] = 0
+    for samp in (None, (2.5, 0.8, 1.0)):
+        s = oracle.sep(mask, samp)
+        b = oracle.brute(mask, samp)
+        np.testing.assert_allclose(s["sqf"], b["sqf"], rtol=1e-14, atol=0)
+        ref = ndimage.distance_transform_edt(mask[0, 0], sampling=samp)
+        np.testing.assert_allclose(s["dist"][0, 0], ref, rtol=1e-12, atol=1e-12)
+        checker.check_indices(s["idx"], mask, b, samp)
+
+
+def test_two_far_sites_long_lines_against_scipy():
+    """Two background voxels in a 700 x 900 image: scans of several hundred rows on both axes."""
+    ndimage = pytest.importorskip("scipy.ndimage")
+    mask = np.ones((1, 1, 700, 900), dtype=np.uint8)
+    mask[0, 0, 13, 880] = 0
+    mask[0, 0, 650, 40] = 0
+    for samp in (None, (0.7, 1.3)):
+        s = oracle.sep(mask, samp)
+        ref = ndimage.distance_transform_edt(mask[0, 0], sampling=samp)
+        np.testing.assert_allclose(s["dist"][0, 0], ref, rtol=1e-12, atol=1e-12)
+        w = np.ones(2) if samp is None else np.asarray(samp)
+        yy, xx = np.meshgrid(np.arange(700.0), np.arange(900.0), indexing="ij")
+        closed = np.minimum((w[0] * (yy - 13)) ** 2 + (w[1] * (xx - 880)) ** 2,
+                            (w[0] * (yy - 650)) ** 2 + (w[1] * (xx - 40)) ** 2)
+        np.testing.assert_allclose(s["sqf"][0, 0], closed, rtol=1e-14, atol=0)
+
+
 def test_bad_arguments_are_rejected():
     with pytest.raises(RuntimeError):
         oracle.sep(np.ones((1, 1, 3), dtype=np.uint8), (0.0,))

@@ -1,4 +1,4 @@
-"""The entry point that allocates nothing (tm_edt_noalloc) against the ordinary one (tm_edt).
+"""The entry point that allocates nothing (tm_edt_noalloc) against the ordinary one (tm_edt) and the CPU oracle.
 
 Who needs it: callers that may not allocate device memory once they are running -- a loop with a memory
 budget fixed at start-up, a process whose GPU memory belongs to another allocator.  Its scratch is a
@@ -9,7 +9,9 @@ every other test; it passes alone in a fresh process as well."""
 import numpy as np
 import pytest
 
+import oracle
 from paper_2608_24738_b200 import binding, buildlib, workloads
+from tests import checker
 
 pytestmark = pytest.mark.gpu
 
@@ -21,6 +23,14 @@ def _both(mask_np, sampling, dist, sq, idx):
     a = binding.tm_edt_noalloc(t, sampling, return_distances=dist, return_sqdist=sq, return_indices=idx)
     b = binding.tm_edt(t, sampling, return_distances=dist, return_sqdist=sq, return_indices=idx)
     torch.cuda.synchronize()
+    # and against the oracle, at the bars of the parity tests
+    ref = oracle.sep(mask_np, sampling, want_idx=False)
+    if dist:
+        checker.check_dist(a["dist"].cpu().numpy(), ref["dist"])
+    if sq:
+        checker.check_sq_exact(a["sq"].cpu().numpy(), ref["sq"])
+    if idx:
+        checker.check_indices(a["idx"].cpu().numpy(), mask_np, ref, sampling)
     return a, b
 
 
@@ -61,9 +71,16 @@ def test_noalloc_refuses_what_does_not_fit():
     import torch
 
     buildlib.build()
-    shape = (40, 1, 128, 128, 128)  # 2 bytes of scratch per voxel = 160 MiB
-    assert binding.tm_edt_workspace_bytes(shape) > binding.tm_edt_noalloc_max_scratch()
-    t = torch.ones(shape, dtype=torch.uint8, device="cuda")
+    # three processed axes take 4 bytes of scratch per voxel: two volumes of 128^3 fill the 16 MiB array exactly,
+    # a third one does not fit
+    limit = binding.tm_edt_noalloc_max_scratch()
+    fits, too_large = (2, 1, 128, 128, 128), (3, 1, 128, 128, 128)
+    assert binding.tm_edt_workspace_bytes_for(fits) == 4 * 2 * 128 ** 3 == limit
+    assert binding.tm_edt_workspace_bytes_for(too_large) > limit
+    r = binding.tm_edt_noalloc(torch.zeros(fits, dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert (r["dist"] == 0).all()
+    t = torch.ones(too_large, dtype=torch.uint8, device="cuda")
     with pytest.raises(binding.TmEdtError) as ei:
         binding.tm_edt_noalloc(t)
     assert ei.value.status == binding.ERR_TOO_LARGE
