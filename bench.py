@@ -30,7 +30,18 @@ if ROOT not in sys.path:
 
 METRIC = "edt_gvoxels_per_s"
 UNIT = "Gvoxel/s"
-L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0  # HBM3e figure of the part's data sheet, reported beside the measured copy bandwidth
+_L2_FALLBACK = 126 * 1024 * 1024
+
+
+def l2_bytes(dev=None) -> int:
+    """L2 size of the device, read from its properties."""
+    try:
+        import torch
+
+        return int(torch.cuda.get_device_properties(dev if dev is not None else torch.cuda.current_device()).L2_cache_size)
+    except Exception:
+        return _L2_FALLBACK
 REASON_BITS = {
     0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
     0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
@@ -150,17 +161,45 @@ def sample_images(w, max_voxels: int):
     return flat[:k], k, B * C
 
 
-def time_oracle(w, max_voxels: int, repeats: int = 1):
+def time_oracle(w, max_voxels: int, repeats: int = 1, threads: int = 0):
+    """The oracle on the first images of the workload; threads = 0 keeps its own thread count (all cores)."""
     import oracle
 
     sub, k, total = sample_images(w, max_voxels)
-    best = None
-    for _ in range(repeats):
-        t0 = time.perf_counter()
-        oracle.sep(sub, w.sampling, want_idx=w.want_idx)
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    return sub.size / best / 1e9, best, "%d of %d images (%d voxels), full oracle incl. index decode" % (k, total, sub.size)
+    before = oracle.threads()
+    if threads > 0:
+        oracle.set_threads(threads)
+    try:
+        used = oracle.threads()
+        best = None
+        for _ in range(repeats):
+            t0 = time.perf_counter()
+            oracle.sep(sub, w.sampling, want_idx=w.want_idx)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+    finally:
+        if threads > 0:
+            oracle.set_threads(before)
+    what = "%d of %d images (%d voxels), full oracle incl. index decode" % (k, total, sub.size)
+    if sub.shape[2:] != w.mask.shape[2:]:
+        what = "part of one image (%d voxels)" % sub.size
+    return sub.size / best / 1e9, best, what, used
+
+
+def time_oracle_single_thread(w, seconds_all_cores: float, voxels_all_cores: int, cores: int):
+    """One oracle thread (the protocol of the paper's CPU column) on a sample sized for about ten seconds."""
+    per_voxel = seconds_all_cores * max(cores, 1) / max(voxels_all_cores, 1)
+    want = int(10.0 / max(per_voxel, 1e-12))
+    one = w.voxels // (w.mask.shape[0] * w.mask.shape[1])
+    if want >= one:
+        return time_oracle(w, want, threads=1)
+    # less than one image: the leading slices of the first image along spatial axis 0
+    import copy
+
+    keep = max(2, int(w.mask.shape[2] * want / one))
+    part = copy.copy(w)
+    part.mask = np.ascontiguousarray(w.mask.reshape((-1, 1) + w.mask.shape[2:])[:1, :, :keep])
+    return time_oracle(part, part.mask.size, threads=1)
 
 
 def run_reference(args, w, world, rank):
@@ -203,18 +242,21 @@ def run_reference(args, w, world, rank):
     print(json.dumps(line), flush=True)
 
 
-def load_traffic(workload_number: int, kernel_label: str):
-    """DRAM bytes per launch of a kernel from the committed ncu summary (profiles/traffic.txt), or None."""
+def load_traffic(workload_number: int, kernel_label: str = None):
+    """DRAM bytes per launch from the committed ncu summary (profiles/traffic.txt): of one kernel, or -- without a
+    kernel label -- summed over all kernels of the workload's path.  None if the summary has no such line."""
     try:
-        want = ("C%d" % workload_number, kernel_label.split(":", 1)[1])
+        total, found = 0, False
+        name = kernel_label.split(":", 1)[1] if kernel_label else None
         with open(os.path.join(ROOT, "profiles", "traffic.txt")) as fh:
             for line in fh:
                 parts = line.split()
-                if len(parts) == 3 and (parts[0], parts[1]) == want:
-                    return int(parts[2])
+                if len(parts) == 3 and parts[0] == "C%d" % workload_number and (name is None or parts[1] == name):
+                    total += int(parts[2])
+                    found = True
+        return total if found else None
     except Exception:
-        pass
-    return None
+        return None
 
 
 def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
@@ -225,7 +267,7 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
 
     # buffers: rotate over enough independent sets that one lap exceeds twice the L2
     io = w.io_bytes()
-    sets = max(2, min(16, -(-2 * L2_BYTES // io)))
+    sets = max(2, min(16, -(-2 * l2_bytes(dev) // io)))
     host_mask = torch.from_numpy(w.mask)
     shape = tuple(w.mask.shape)
     calls = []
@@ -262,6 +304,23 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
     clocks = sampler.summary(t0, t1) if sampler is not None else None
     value = whole_job_rate(w.voxels * steps, world, seconds) / 1e9
 
+    # every repetition timed by itself (rotating buffers: cold L2), then one buffer set over and over (warm L2)
+    def each(reps, pick):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i, (a, b) in enumerate(evs):
+            a.record(stream)
+            calls[pick(i)](sp)
+            b.record(stream)
+        torch.cuda.synchronize()
+        return sorted(a.elapsed_time(b) for a, b in evs)
+    reps = max(30, min(steps, 200))
+    cold = each(reps, lambda i: i % sets)
+    each(3, lambda i: 0)
+    warm = each(reps, lambda i: 0)
+    spread = {"repetitions": reps, "ms_median": statistics.median(cold), "ms_min": cold[0],
+              "warm_l2_ms_median": statistics.median(warm), "warm_l2_ms_min": warm[0],
+              "note": "each repetition between its own pair of events; warm = the same buffer set every time"}
+
     # per-kernel times (events between launches), same buffers, right after the timed region
     ksum, korder = {}, []
     for i in range(max(1, profile_steps)):
@@ -284,17 +343,28 @@ def measure_device(w, steps, warmup, profile_steps, dev, world, sampler=None):
         kernels.append({"kernel": "%d:%s" % key, "avg_ms": avg_ms, "bytes": nbytes,
                         "gbs": nbytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else None})
     dom = max(kernels, key=lambda k: k["avg_ms"])
+    # Roofline of the path: the bytes the method cannot avoid (mask in, requested outputs out) over the time of one
+    # whole transform, against the measured copy bandwidth; the kernel with the largest share is reported beside it
+    # with the same algorithmic bytes over its own duration and with its own compulsory bytes (inputs + outputs of
+    # that launch, intermediates included).
     path_gbs = io * steps * 1.0 / seconds / 1e9
+    traffic = load_traffic(w.number)
     roofline = {
-        "bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
-        "frac": dom["gbs"] / peak, "traffic": load_traffic(w.number, dom["kernel"]), "peak_kind": peak_kind + " copy bandwidth",
-        "path": {"io_bytes_per_step": io, "achieved": path_gbs, "frac": path_gbs / peak},
+        "bound": "hbm", "achieved": path_gbs, "peak": peak, "unit": "GB/s", "frac": path_gbs / peak,
+        "peak_kind": peak_kind + " copy bandwidth", "frac_of_nominal_8TBs": path_gbs / NOMINAL_HBM_GBS,
+        "algorithmic_bytes_per_step": io, "bytes_per_voxel": io / w.voxels,
+        "traffic": traffic, "traffic_over_algorithmic": (traffic / io) if traffic else None,
+        "traffic_kind": "dram read + write bytes of every kernel of the path, ncu (profiles/traffic.txt)",
+        "dominant": {"kernel": dom["kernel"], "avg_ms": dom["avg_ms"], "share": dom["avg_ms"] / sum(k["avg_ms"] for k in kernels),
+                     "algorithmic_gbs": io / (dom["avg_ms"] * 1e-3) / 1e9, "algorithmic_frac": io / (dom["avg_ms"] * 1e-3) / 1e9 / peak,
+                     "own_bytes": dom["bytes"], "own_gbs": dom["gbs"], "own_frac": dom["gbs"] / peak,
+                     "traffic": load_traffic(w.number, dom["kernel"])},
         "kernels": kernels,
     }
     del calls
     torch.cuda.empty_cache()
     return {"io": io, "shape": shape, "host_mask": host_mask, "value": value, "seconds": seconds, "clocks": clocks,
-            "roofline": roofline, "launches_per_step": launches_per_step, "sets": sets}
+            "roofline": roofline, "launches_per_step": launches_per_step, "sets": sets, "spread": spread}
 
 
 MORPH_CASES = {
@@ -336,7 +406,7 @@ def run_morph(args):
         fp = np.ones(fps, dtype=bool)
         per_voxel = 2 if binary else 8
         nvox = int(np.prod(shape))
-        sets = max(2, -(-2 * L2_BYTES // (nvox * per_voxel)))
+        sets = max(2, -(-2 * l2_bytes(dev) // (nvox * per_voxel)))
         if binary:
             ins = [torch.from_numpy((rng.random(shape) < 0.8).astype(np.uint8)).to(dev) for _ in range(sets)]
         else:
@@ -416,7 +486,7 @@ def run_cdt(args):
         base = workloads.config2(batch=8, size=size, disks=20 * (size // 512) ** 2 if size >= 512 else 5).mask
         mask = np.concatenate([base] * (batch // 8), axis=0)
         nvox = mask.size
-        sets = max(2, -(-2 * L2_BYTES // (nvox * 5)))
+        sets = max(2, -(-2 * l2_bytes(dev) // (nvox * 5)))
         ins = [torch.from_numpy(mask).to(dev) for _ in range(sets)]
         outs = [torch.empty(mask.shape, dtype=torch.int32, device=dev) for _ in range(sets)]
         for metric in ("chessboard", "taxicab"):
@@ -451,6 +521,97 @@ def run_cdt(args):
                       "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
 
 
+def run_long(args):
+    """Measurement of the paths for extents beyond 128 (wide-key and long-line kernels; a later row of the scope, its
+    own line): the paper's 2-D 1024^2 row at B = 8, one 4096^2 image and one 512^3 volume; blob masks (disks / balls as
+    in workload C2, radii 0.02 .. 0.12 of the extent), unit sampling, float32 distances.  HBM roofline = mask in +
+    distances out once (5 B/voxel); the oracle is timed on a bounded sample of each case."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2608_24738_b200 import binding, buildlib, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(stream.cuda_stream)
+    steps = max(30, args.steps // 4)
+
+    def blobs(seed, shape, count):
+        rng = np.random.default_rng(24738 + seed)
+        grids = np.meshgrid(*[np.arange(n, dtype=np.float32) for n in shape], indexing="ij", sparse=True)
+        fg = np.zeros(shape, dtype=bool)
+        for _ in range(count):
+            c = [rng.uniform(0, n) for n in shape]
+            r = rng.uniform(0.02, 0.12) * min(shape)
+            fg |= sum((g - ci) ** 2 for g, ci in zip(grids, c)) <= r * r
+        if fg.all():
+            fg.flat[0] = False
+        return fg.astype(np.uint8)
+
+    specs = [("edt_2d_1024_b8", (8, 1, 1024, 1024), 20), ("edt_2d_4096_b1", (1, 1, 4096, 4096), 40),
+             ("edt_3d_512_b1", (1, 1, 512, 512, 512), 24)]
+    cases = []
+    for k, (name, shape, count) in enumerate(specs):
+        imgs = [blobs(100 * k + i, shape[2:], count) for i in range(shape[0])]
+        mask = np.stack(imgs)[:, None]
+        nvox = mask.size
+        io = 5 * nvox
+        sets = max(2, min(8, -(-2 * l2_bytes(dev) // io)))
+        calls = [binding.PreparedCall(torch.from_numpy(mask).to(dev), None,
+                                      torch.empty(mask.shape, dtype=torch.float32, device=dev), None, None)
+                 for _ in range(sets)]
+        for i in range(max(3, args.warmup)):
+            calls[i % sets](sp)
+        launches = binding.tm_edt_last_launch_count()
+        torch.cuda.synchronize()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i, (a, b) in enumerate(evs):
+            a.record(stream)
+            calls[i % sets](sp)
+            b.record(stream)
+        torch.cuda.synchronize()
+        times = sorted(a.elapsed_time(b) for a, b in evs)
+        ms = statistics.median(times)
+        c0 = calls[0]
+        _, ks = binding.tm_edt_profile(c0.mask, None, distances=c0.d, workspace=c0.ws, return_distances=True)
+        # the oracle on the first image (its leading rows if the image alone would take minutes)
+        one = mask[:1]
+        rows = one.shape[2]
+        t0 = time.perf_counter()
+        oracle.sep(np.ascontiguousarray(one[:, :, : max(2, rows // 8)]), None, want_idx=False)
+        t_part = time.perf_counter() - t0
+        keep = rows if t_part * 8 < 20 else max(2, int(rows / 8 * 20 / (t_part * 8)))
+        part = np.ascontiguousarray(one[:, :, :keep])
+        t0 = time.perf_counter()
+        oracle.sep(part, None, want_idx=False)
+        cpu_s = time.perf_counter() - t0
+        gbs = io / (ms * 1e-3) / 1e9
+        cases.append({"case": name, "shape": list(mask.shape), "ms_per_step": ms, "ms_min": times[0],
+                      "value": nvox / (ms * 1e-3) / 1e9, "unit": UNIT, "inputs_per_ms": shape[0] / ms,
+                      "gpu_launches_per_step": launches,
+                      "kernels": [(n, round(t, 4)) for n, t, _ in ks],
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                   "peak_kind": peak_kind + " copy bandwidth", "bytes_per_voxel": 5},
+                      "cpu_baseline": {"value": part.size / cpu_s / 1e9, "unit": UNIT, "cores": oracle.threads(),
+                                       "kind": "oracle", "sample": "first %d of %d rows of one image" % (keep, rows)},
+                      "l2": "rotating %d buffer sets" % sets})
+        del calls
+        torch.cuda.empty_cache()
+    head = cases[0]
+    print(json.dumps({"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": 1, "steps": steps,
+                      "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+                      "config": {"workload": head["case"], "shape": head["shape"], "outputs": ["dist_f32"]},
+                      "gpu_launches": head["gpu_launches_per_step"] * steps, "roofline": head["roofline"],
+                      "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -468,8 +629,8 @@ def main():
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
     ap.add_argument("--flat-index", action="store_true",
                     help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
-    ap.add_argument("--workload", default="edt", choices=["edt", "morph", "cdt"],
-                    help="edt: the headline benchmark; morph / cdt: the erosion-dilation kernels and the taxicab / chessboard / brute-force transforms (their own metrics)")
+    ap.add_argument("--workload", default="edt", choices=["edt", "morph", "cdt", "long"],
+                    help="edt: the headline benchmark; long: the same transform on extents beyond 128 (1024^2, 4096^2, 512^3); morph / cdt: the erosion-dilation kernels and the taxicab / chessboard / brute-force transforms (their own metrics)")
     ap.add_argument("--morph-case", default=None, help="with --workload morph: run only this case (profiling aid)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
@@ -478,6 +639,9 @@ def main():
         return
     if args.workload == "cdt":
         run_cdt(args)
+        return
+    if args.workload == "long":
+        run_long(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     world, rank, local = dist_env()
@@ -567,17 +731,20 @@ def main():
             wo = workloads.CONFIGS[num]()
             mo = measure_device(wo, 40, 5, 5, dev, world)
             others.append({"workload": wo.name, "value": mo["value"], "unit": UNIT, "ms_per_step": mo["seconds"] / 40 * 1e3,
-                           "path_frac": mo["roofline"]["path"]["frac"], "dominant": mo["roofline"]["kernel"],
-                           "dominant_frac": mo["roofline"]["frac"],
+                           "ms_median": mo["spread"]["ms_median"], "ms_min": mo["spread"]["ms_min"],
+                           "warm_l2_ms_median": mo["spread"]["warm_l2_ms_median"],
+                           "roofline_frac": mo["roofline"]["frac"], "dominant": mo["roofline"]["dominant"]["kernel"],
                            "kernels": [(k["kernel"], round(k["avg_ms"], 4)) for k in mo["roofline"]["kernels"]]})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
 
-        v, secs, what = time_oracle(w, args.cpu_voxels)
-        cpu = {"value": v, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": what,
-               "seconds": secs}
+        v, secs, what, used = time_oracle(w, args.cpu_voxels)
+        nvox = min(w.voxels, max(args.cpu_voxels, w.voxels // (w.mask.shape[0] * w.mask.shape[1])))
+        v1, secs1, what1, _ = time_oracle_single_thread(w, secs, nvox, used)
+        cpu = {"value": v, "unit": UNIT, "cores": used, "kind": "oracle", "sample": what, "seconds": secs,
+               "single_thread": {"value": v1, "unit": UNIT, "cores": 1, "sample": what1, "seconds": secs1}}
 
     if rank == 0:
         line = {
@@ -588,8 +755,10 @@ def main():
             "config": {"workload": w.name, "shape": list(shape), "sampling": w.sampling,
                        "outputs": [n for n, f in (("dist_f32", w.want_dist), ("sqdist_i64", w.want_sq),
                                                    ("indices_i64", w.want_idx)) if f],
-                       "voxels_per_step": w.voxels, "l2": "rotating %d buffer sets, %d MB per set" % (sets, io >> 20),
+                       "voxels_per_step": w.voxels,
+                       "l2": "rotating %d buffer sets, %d MB per set, L2 %d MB" % (sets, io >> 20, l2_bytes(dev) >> 20),
                        "sha256": w.sha256()[:16]},
+            "timing": m["spread"],
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "other_configs": others,
         }
