@@ -60,7 +60,9 @@ typedef enum {
                                    (or a host buffer of tm_edt_host is device memory) */
     TM_EDT_ERR_ALLOC = 4,       /* scratch allocation failed, or the supplied workspace is too small */
     TM_EDT_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed; see tm_edt_last_cuda_error() */
-    TM_EDT_ERR_TOO_LARGE = 6    /* tm_edt_noalloc only: the problem needs more scratch than its built-in array */
+    TM_EDT_ERR_TOO_LARGE = 6,   /* tm_edt_noalloc only: the problem needs more scratch than its built-in array */
+    TM_EDT_ERR_DEBUG_CHECK = 7  /* debug build only (see tm_edt_debug_build): an index of a kernel left its range;
+                                   the access was skipped, the outputs of the call are not to be trusted */
 } tm_edt_status;
 
 /* The stream argument is a cudaStream_t (NULL = the legacy default stream). */
@@ -145,6 +147,17 @@ TM_EDT_API size_t tm_edt_workspace_bytes(int ndim, const int64_t* shape);
  */
 TM_EDT_API size_t tm_edt_workspace_bytes_for(int ndim, const int64_t* shape, const double* sampling, int want_dist,
                                              int want_sqdist, int want_indices);
+
+/*
+ * Debug build (compiled with -DTM_EDT_DEBUG=1, the stand-in for a device memory checker): the quad kernels check
+ * every shared-memory and global index they use, skip an access that leaves its range and record it; every call
+ * then waits for its own work and returns TM_EDT_ERR_DEBUG_CHECK if anything was recorded.  tm_edt_debug_build()
+ * says whether this library is such a build; tm_edt_debug_last_violation() returns how many violations the calling
+ * thread's last call recorded and, through the optional pointers, the site code, index and bound of the first one.
+ * In a release build the first returns 0 and the second always 0.  (No counterpart in the paper.)
+ */
+TM_EDT_API int tm_edt_debug_build(void);
+TM_EDT_API unsigned long long tm_edt_debug_last_violation(long long* code, long long* index, long long* limit);
 
 /*
  * Debug and test switches (environment variables TM_EDT_FORCE_GENERIC, TM_EDT_NO_SCALED, TM_EDT_OLD_PLANE,

@@ -13,15 +13,16 @@ from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtm_edt.so")
+DEBUG_LIB_PATH = os.path.join(_HERE, "libtm_edt_debug.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_POINTER, ERR_ALLOC, ERR_CUDA, ERR_TOO_LARGE = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_POINTER, ERR_ALLOC, ERR_CUDA, ERR_TOO_LARGE, ERR_DEBUG_CHECK = range(8)
 MAX_DIMS = 8
 MAX_EXTENT = 8192
 
 EXPORTS = (
     "tm_edt", "tm_edt_ws", "tm_edt_ex", "tm_edt_ex_workspace_bytes", "tm_edt_host", "tm_edt_noalloc", "tm_edt_noalloc_max_scratch", "tm_edt_profile", "tm_edt_profile_ex", "tm_edt_workspace_bytes", "tm_edt_strerror",
     "tm_edt_last_cuda_error", "tm_edt_version", "tm_edt_last_launch_count", "tm_edt_trim_memory",
-    "tm_edt_workspace_bytes_for", "tm_edt_reload_switches",
+    "tm_edt_workspace_bytes_for", "tm_edt_reload_switches", "tm_edt_debug_build", "tm_edt_debug_last_violation",
     "tm_grey_morph", "tm_binary_morph", "tm_cdt", "tm_bfdt",
 )
 
@@ -35,16 +36,28 @@ class TmEdtError(RuntimeError):
         self.status = status
 
 
+def use_debug_library(on: bool = True) -> None:
+    """Route every later call through the bounds-checked debug build (``buildlib.build(debug=True)``) or back."""
+    global _lib, _use_debug
+    with _lock:
+        _use_debug = bool(on)
+        _lib = None
+
+
+_use_debug = False
+
+
 def lib() -> ctypes.CDLL:
     """Open the CUDA library (once).  Raises if it has not been built: there is no other code path."""
     global _lib
     with _lock:
         if _lib is None:
-            if not os.path.exists(LIB_PATH):
+            path = DEBUG_LIB_PATH if _use_debug else LIB_PATH
+            if not os.path.exists(path):
                 raise RuntimeError(
-                    "CUDA library %s is missing; build it with `python -m paper_2608_24738_b200.buildlib`" % LIB_PATH
+                    "CUDA library %s is missing; build it with `python -m paper_2608_24738_b200.buildlib`" % path
                 )
-            L = ctypes.CDLL(LIB_PATH)
+            L = ctypes.CDLL(path)
             vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
             L.tm_edt.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
             L.tm_edt.restype = i
@@ -68,6 +81,9 @@ def lib() -> ctypes.CDLL:
             L.tm_edt_workspace_bytes_for.argtypes = [i, vp, vp, i, i, i]
             L.tm_edt_workspace_bytes_for.restype = sz
             L.tm_edt_reload_switches.restype = None
+            L.tm_edt_debug_build.restype = i
+            L.tm_edt_debug_last_violation.argtypes = [vp, vp, vp]
+            L.tm_edt_debug_last_violation.restype = ctypes.c_ulonglong
             L.tm_edt_strerror.argtypes = [i]
             L.tm_edt_strerror.restype = ctypes.c_char_p
             L.tm_edt_last_cuda_error.restype = i
@@ -137,6 +153,17 @@ def tm_edt_workspace_bytes_for(shape: Sequence[int], sampling=None, want_dist=Tr
     if n == ctypes.c_size_t(-1).value:
         raise TmEdtError(ERR_INVALID_ARG, "invalid or unsupported shape")
     return n
+
+
+def tm_edt_debug_build() -> bool:
+    return bool(lib().tm_edt_debug_build())
+
+
+def tm_edt_debug_last_violation():
+    """(count, site code, index, bound) of the bounds violations the calling thread's last call recorded."""
+    c, i, l = ctypes.c_longlong(0), ctypes.c_longlong(0), ctypes.c_longlong(0)
+    n = int(lib().tm_edt_debug_last_violation(ctypes.byref(c), ctypes.byref(i), ctypes.byref(l)))
+    return n, int(c.value), int(i.value), int(l.value)
 
 
 def tm_edt_reload_switches() -> None:

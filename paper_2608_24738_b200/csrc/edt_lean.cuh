@@ -15,6 +15,7 @@
 //       value mode     the squared distance so far, times the common scale in scaled-integer mode
 // "No site" is 2^31 in both; every real key and every addend stays below it (checked by the planner).
 #pragma once
+#include "edt_debug.cuh"
 #include "edt_fast.cuh"
 
 namespace tmedt {
@@ -33,11 +34,19 @@ struct LeanParams {
     uint32_t w0;         // plane kernel: integer weight of the contiguous axis
     float inv_scale;     // final value kernels: 1 / common scale (1 under unit sampling)
     int shift[4];        // final entry kernels: log2 of the extent of plane q, or -1 if it is no power of two
+    int64_t in_elems;    // elements behind `in` and `out` (bounds checks of the debug build)
+    int64_t out_elems;
+    int64_t images;      // images behind the final outputs (bounds checks of the debug build)
 };
+
+// A key tile in shared memory: its first word and its size in words (bounds checks of the debug build).
+struct LeanTile { const uint32_t* base; int words; };
 
 __device__ __forceinline__ uint32_t lean_max4(const uint32_t (&b)[4]) { return max(max(b[0], b[1]), max(b[2], b[3])); }
 
-__device__ __forceinline__ void lean_try_row(const uint32_t* __restrict__ row, const uint32_t a, uint32_t (&b)[4]) {
+__device__ __forceinline__ void lean_try_row(const LeanTile& T, const uint32_t* __restrict__ row, const uint32_t a,
+                                             uint32_t (&b)[4]) {
+    if (!TM_EDT_IN_RANGE(row - T.base, T.words - 3, 101)) return;
     const uint4 c = *reinterpret_cast<const uint4*>(row);
     b[0] = __viaddmin_u32(c.x, a, b[0]); b[1] = __viaddmin_u32(c.y, a, b[1]);
     b[2] = __viaddmin_u32(c.z, a, b[2]); b[3] = __viaddmin_u32(c.w, a, b[3]);
@@ -47,8 +56,10 @@ __device__ __forceinline__ void lean_try_row(const uint32_t* __restrict__ row, c
 // Row distance d adds (wk d^2) << SH; a voxel is finished once that addend reaches its best key, so the work of a
 // voxel grows with its distance to the background along the axis and never exceeds the extent.
 template <int PITCH, int SH>
-__device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, const int y, const int n, const uint32_t wk,
-                                          uint32_t (&b)[4]) {
+__device__ __forceinline__ void lean_scan(const LeanTile& T, const uint32_t* __restrict__ own, const int y, const int n,
+                                          const uint32_t wk, uint32_t (&b)[4]) {
+    b[0] = b[1] = b[2] = b[3] = kLeanNone;
+    if (!TM_EDT_IN_RANGE(own - T.base, T.words - 3, 100)) return;
     {
         const uint4 v = *reinterpret_cast<const uint4*>(own);
         b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
@@ -59,8 +70,8 @@ __device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, cons
     for (int s = 1; s <= kLeanPad; ++s) {  // no bounds tests: the tile is padded
         if (s == 3 && ((wk * 9u) << SH) >= mx) return;
         const uint32_t a = (wk * (uint32_t)(s * s)) << SH;
-        lean_try_row(own - s * PITCH, a, b);
-        lean_try_row(own + s * PITCH, a, b);
+        lean_try_row(T, own - s * PITCH, a, b);
+        lean_try_row(T, own + s * PITCH, a, b);
         if (s == 2) mx = lean_max4(b);
     }
     mx = lean_max4(b);
@@ -73,17 +84,17 @@ __device__ __forceinline__ void lean_scan(const uint32_t* __restrict__ own, cons
     // rows that exist on both sides, two distances per stop test
     for (; d + 1 <= both && a < mx; d += 2, plo -= 2 * PITCH, phi += 2 * PITCH) {
         const uint32_t a1 = (wk * (uint32_t)((d + 1) * (d + 1))) << SH;
-        lean_try_row(plo, a, b);
-        lean_try_row(phi, a, b);
-        lean_try_row(plo - PITCH, a1, b);
-        lean_try_row(phi + PITCH, a1, b);
+        lean_try_row(T, plo, a, b);
+        lean_try_row(T, phi, a, b);
+        lean_try_row(T, plo - PITCH, a1, b);
+        lean_try_row(T, phi + PITCH, a1, b);
         mx = lean_max4(b);
         a = (wk * (uint32_t)((d + 2) * (d + 2))) << SH;
     }
     // the rest: one distance at a time, the tile's ends tested
     for (; a < mx && (d <= up || d <= dn); ++d, plo -= PITCH, phi += PITCH) {
-        if (d <= up) lean_try_row(plo, a, b);
-        if (d <= dn) lean_try_row(phi, a, b);
+        if (d <= up) lean_try_row(T, plo, a, b);
+        if (d <= dn) lean_try_row(T, phi, a, b);
         mx = lean_max4(b);
         a = (wk * (uint32_t)((d + 1) * (d + 1))) << SH;
     }
@@ -96,6 +107,7 @@ __device__ __forceinline__ void lean_fill_pad(uint32_t* __restrict__ kt, const i
     for (int t = threadIdx.x; t < 2 * kLeanPad * QPR; t += blockDim.x) {
         const int r = t / QPR, q = t - r * QPR;
         const int row = r < kLeanPad ? r : n + r;
+        if (!TM_EDT_IN_RANGE(row * PITCH + 4 * q, (n + 2 * kLeanPad) * PITCH - 3, 102)) continue;
         *reinterpret_cast<uint4*>(kt + row * PITCH + 4 * q) = make_uint4(kLeanNone, kLeanNone, kLeanNone, kLeanNone);
     }
 }
@@ -110,7 +122,7 @@ __device__ __forceinline__ void lean_fill_pad(uint32_t* __restrict__ kt, const i
 // ---------------------------------------------------------------------------------------------
 template <bool ENT>
 __device__ __forceinline__ uint32_t lean_first_axis(const uint32_t v, const int n0, const int y, const uint32_t w0,
-                                                uint32_t* __restrict__ krow, const int lane) {
+                                                uint32_t* __restrict__ krow, const int krow_words, const int lane) {
     const bool act = 4 * lane < n0;
     const uint32_t m = ~(((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every zero byte
     const unsigned any = __ballot_sync(0xffffffffu, m != 0u);  // lanes beyond the row hold foreground: m == 0
@@ -153,7 +165,7 @@ __device__ __forceinline__ uint32_t lean_first_axis(const uint32_t v, const int 
         }
         keys = make_uint4(kk[0], kk[1], kk[2], kk[3]);
     }
-    if (act) *reinterpret_cast<uint4*>(krow + 4 * lane) = keys;
+    if (act && TM_EDT_IN_RANGE(4 * lane, krow_words - 3, 111)) *reinterpret_cast<uint4*>(krow + 4 * lane) = keys;
     return act ? (keys.x & keys.y & keys.z & keys.w) : 0xffffffffu;
 }
 
@@ -184,12 +196,13 @@ __global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constan
 #pragma unroll
         for (int i = 0; i < MAXR; ++i) {  // all loads of this warp's rows are issued before the first row is processed
             const int y = warp + i * NW;
-            rowv[i] = (act && y < n1) ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
+            rowv[i] = (act && y < n1 && TM_EDT_IN_RANGE(plane * (int64_t)n1 * n0 + y * n0 + 4 * lane, P.in_elems - 3, 110))
+                          ? *reinterpret_cast<const uint32_t*>(src + y * n0 + 4 * lane) : 0x01010101u;
         }
 #pragma unroll
         for (int i = 0; i < MAXR; ++i) {
             const int y = warp + i * NW;
-            if (y < n1) all &= lean_first_axis<ENT>(rowv[i], n0, y, P.w0, kt + (y + kLeanPad) * VS, lane);
+            if (y < n1) all &= lean_first_axis<ENT>(rowv[i], n0, y, P.w0, kt + (y + kLeanPad) * VS, (n1 + kLeanPad - y) * VS, lane);
         }
     }
     // barrier; a plane without any background voxel needs no scan (every result is "no site")
@@ -199,13 +212,15 @@ __global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constan
     const int r = lane >> 3, q4 = 4 * (lane & 7);
     const int64_t base0 = plane * (int64_t)n1 * n0;
     const int patches = ((n1 + 3) >> 2) * CG;
+    const LeanTile T = {kt, (n1 + 2 * kLeanPad) * VS};
     for (int t = warp; t < patches; t += NW) {
         const int y = 4 * (t / CG) + r, c4 = 32 * (t % CG) + q4;
         if (y >= n1 || c4 >= n0) continue;
         uint32_t b[4];
-        if (any_site) lean_scan<VS, SH>(kt + (y + kLeanPad) * VS + c4, y, n1, wk, b);
+        if (any_site) lean_scan<VS, SH>(T, kt + (y + kLeanPad) * VS + c4, y, n1, wk, b);
         else b[0] = b[1] = b[2] = b[3] = kLeanNone;
         const int64_t p = base0 + (int64_t)y * n0 + c4;
+        if (!TM_EDT_IN_RANGE(p, P.out_elems - 3, 112)) continue;
         if (ENT) {
             uint32_t e[4];
 #pragma unroll
@@ -321,6 +336,7 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
         const EI* g = src + (int64_t)y * P.inner + q4;
+        if (!TM_EDT_IN_RANGE(g - reinterpret_cast<const EI*>(P.in), P.in_elems - 3, 120)) continue;
         uint32_t e[4];
         if (sizeof(EI) == 2) {
             const uint2 w = *reinterpret_cast<const uint2*>(g);
@@ -347,15 +363,17 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     constexpr int YSTEP = 4 * (NW / CG);
     if (c4 >= width) return;
     const uint32_t v0 = (uint32_t)(i0 + c4);  // the quad's position among the earlier planes (plane 0 fastest)
+    const LeanTile T = {kt, (n + 2 * kLeanPad) * TX};
     if (!FINAL) {
         uint32_t* out = reinterpret_cast<uint32_t*>(P.out) + slab * (int64_t)n * P.inner + v0;
         for (int y = yfirst; y < n; y += YSTEP) {
             uint32_t b[4], o[4];
-            if (any_site) lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+            if (any_site) lean_scan<TX, 8>(T, kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
             else b[0] = b[1] = b[2] = b[3] = kLeanNone;
+            if (!TM_EDT_IN_RANGE(slab * (int64_t)n * P.inner + v0 + (int64_t)y * P.inner, P.out_elems - 3, 121)) continue;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
-                const uint32_t j = b[v] & 0xffu;
+                const uint32_t j = TM_EDT_IN_RANGE(b[v] & 0xffu, n, 122) ? (b[v] & 0xffu) : 0u;
                 const uint32_t e = (uint32_t)et[j * TX + c4 + v];
                 o[v] = b[v] >= kLeanNone ? 0x80u : (e | (((j - (uint32_t)y) & 0xffu) << (8 * K)));
             }
@@ -372,11 +390,13 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     for (int q = 0; q <= K; ++q) ip[q] = ep.idx + (slab * ep.ndim + ep.axis[q]) * ep.V;
     for (int y = yfirst; y < n; y += YSTEP) {
         uint32_t b[4], e[4];
-        if (any_site) lean_scan<TX, 8>(kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+        if (any_site) lean_scan<TX, 8>(T, kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
         else b[0] = b[1] = b[2] = b[3] = kLeanNone;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) e[v] = (uint32_t)et[(b[v] & 0xffu) * TX + c4 + v];
-        lean_emit_final<K>(b, e, cq, dist, sq, ip, (uint32_t)y * (uint32_t)P.inner + v0);  // inside one image: below 2^31
+        for (int v = 0; v < 4; ++v) e[v] = (uint32_t)et[(TM_EDT_IN_RANGE(b[v] & 0xffu, n, 123) ? (b[v] & 0xffu) : 0u) * TX + c4 + v];
+        const uint32_t p = (uint32_t)y * (uint32_t)P.inner + v0;  // inside one image: below 2^31
+        if (TM_EDT_IN_RANGE(p, ep.V - 3, 124) && TM_EDT_IN_RANGE(slab, P.images, 125))
+            lean_emit_final<K>(b, e, cq, dist, sq, ip, p);
     }
 }
 
@@ -402,6 +422,7 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
         const VT* g = src + (int64_t)y * P.inner + q4;
+        if (!TM_EDT_IN_RANGE(g - reinterpret_cast<const VT*>(P.in), P.in_elems - 3, 130)) continue;
         uint4 k;
         if (sizeof(VT) == 2) {
             const uint2 w = *reinterpret_cast<const uint2*>(g);
@@ -423,11 +444,13 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
     constexpr int YSTEP = 4 * (NW / CG);
     if (c4 >= width) return;
     const int64_t col = slab * (int64_t)n * P.inner + i0 + c4;  // FINAL: the slab is the image
+    const LeanTile T = {kt, (n + 2 * kLeanPad) * TX};
     for (int y = yfirst; y < n; y += YSTEP) {
         uint32_t b[4];
-        if (any_site) lean_scan<TX, 0>(kt + (y + kLeanPad) * TX + c4, y, n, P.wk, b);
+        if (any_site) lean_scan<TX, 0>(T, kt + (y + kLeanPad) * TX + c4, y, n, P.wk, b);
         else b[0] = b[1] = b[2] = b[3] = kLeanNone;
         const int64_t p = col + (int64_t)y * P.inner;
+        if (!TM_EDT_IN_RANGE(p, (FINAL ? P.images * ep.V : P.out_elems) - 3, 131)) continue;
         if (!FINAL) {
             if (sizeof(VT) == 2) {
 #pragma unroll

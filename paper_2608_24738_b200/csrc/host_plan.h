@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "edt_common.cuh"
+#include "edt_debug.cuh"
 
 namespace tmedt {
 
@@ -46,6 +47,7 @@ struct Switches {
     bool no_value_carry = false;  // TM_EDT_NO_VALUE_CARRY: offsets are carried even without an index output
     bool no_lean = false;         // TM_EDT_NO_LEAN: one-voxel-per-lane kernels instead of the quad kernels
     long long chunk_voxels = 0;   // TM_EDT_CHUNK_VOXELS=n: image ranges of at most n voxels (0 = grid limit)
+    bool debug_inject = false;    // TM_EDT_DEBUG_INJECT=1, debug build only: the bounds checks get a bound that is too small
 };
 const Switches& switches();
 
@@ -61,5 +63,8 @@ cudaError_t ensure_smem(const void* kernel, size_t smem);
 // Quad-per-lane kernels (edt_lean.cuh, launched from tm_edt_lean.cu): whether they cover a call, and the call itself.
 bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep);
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches);
+
+// Debug build: what the kernels launched from tm_edt_lean.cu recorded (see edt_debug.cuh).
+cudaError_t lean_debug_collect(cudaStream_t st, DebugRecord* out);
 
 }  // namespace tmedt

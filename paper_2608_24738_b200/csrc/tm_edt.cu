@@ -26,6 +26,7 @@ namespace tmedt {
 
 static thread_local int g_last_cuda_error = 0;
 static thread_local int g_last_launches = 0;
+static thread_local DebugRecord g_last_debug = {0ull, 0, 0, 0};  // debug build: record of this thread's last call
 
 // Debug and test switches.  The environment is read once, at the first call that needs a switch, and again only
 // when tm_edt_reload_switches() is called (the tests change switches inside one process).
@@ -42,6 +43,7 @@ static void load_switches_locked() {
     s.old_plane = on("TM_EDT_OLD_PLANE");
     s.no_value_carry = set("TM_EDT_NO_VALUE_CARRY");
     s.no_lean = set("TM_EDT_NO_LEAN");
+    s.debug_inject = on("TM_EDT_DEBUG_INJECT");
     s.chunk_voxels = 0;
     if (const char* lim = getenv("TM_EDT_CHUNK_VOXELS")) { const long long v = atoll(lim); if (v > 0) s.chunk_voxels = v; }
     g_switches = s;
@@ -944,6 +946,15 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
         if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
     }
     g_last_launches = launches;
+#ifdef TM_EDT_DEBUG
+    {   // debug build: wait for the call and turn a recorded bounds violation into a status
+        DebugRecord rec = {0ull, 0, 0, 0};
+        cudaError_t e = lean_debug_collect(st, &rec);
+        if (e != cudaSuccess) { g_last_cuda_error = (int)e; return TM_EDT_ERR_CUDA; }
+        g_last_debug = rec;
+        if (rec.count != 0ull) return TM_EDT_ERR_DEBUG_CHECK;
+    }
+#endif
     return TM_EDT_OK;
 }
 
@@ -1253,6 +1264,7 @@ const char* tm_edt_strerror(int status) {
         case TM_EDT_ERR_ALLOC: return "scratch allocation failed or workspace too small";
         case TM_EDT_ERR_CUDA: return "CUDA runtime error";
         case TM_EDT_ERR_TOO_LARGE: return "problem needs more scratch than the built-in array of tm_edt_noalloc holds";
+        case TM_EDT_ERR_DEBUG_CHECK: return "debug build: a kernel index left its range (see tm_edt_debug_last_violation)";
     }
     return "unknown status";
 }
@@ -1304,6 +1316,21 @@ int tm_edt_profile_ex(const uint8_t* input, int ndim, const int64_t* shape, cons
     }
     for (int i = 0; i <= kProfMax; ++i) cudaEventDestroy(g_prof.ev[i]);
     return rc;
+}
+
+int tm_edt_debug_build(void) {
+#ifdef TM_EDT_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+unsigned long long tm_edt_debug_last_violation(long long* code, long long* index, long long* limit) {
+    if (code) *code = g_last_debug.code;
+    if (index) *index = g_last_debug.index;
+    if (limit) *limit = g_last_debug.limit;
+    return g_last_debug.count;
 }
 
 int tm_edt_last_cuda_error(void) { return g_last_cuda_error; }

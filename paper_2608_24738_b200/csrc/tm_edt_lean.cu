@@ -120,6 +120,12 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
     LeanParams P;
     memset(&P, 0, sizeof(P));
     P.in = in; P.out = bufA;
+    P.in_elems = pl.N; P.out_elems = pl.N; P.images = pl.images;
+#ifdef TM_EDT_DEBUG
+    // test hook of the debug build: a bound that is too small on purpose, so that the checks fire on valid accesses
+    // (which are then skipped) and the reporting path can be tested without any invalid access
+    if (switches().debug_inject) P.out_elems = 16;
+#endif
     P.n0 = pl.ext[0]; P.n = pl.ext[1]; P.inner = pl.inner[1];
     P.w0 = weight(0); P.wk = weight(1);
     P.inv_scale = (float)(1.0 / pl.scale);
@@ -157,6 +163,17 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
         char* t = src; src = dst; dst = t;
     }
     return cudaSuccess;
+}
+
+// Debug build: violations recorded by the kernels of this translation unit (cleared by the call).
+cudaError_t lean_debug_collect(cudaStream_t st, DebugRecord* out) {
+#ifdef TM_EDT_DEBUG
+    return debug_collect(st, out);
+#else
+    (void)st;
+    out->count = 0;
+    return cudaSuccess;
+#endif
 }
 
 }  // namespace tmedt

@@ -28,8 +28,9 @@ def test_header_symbols_are_exported(L):
 
 def test_version_and_strerror(L):
     assert "sm_100a" in binding.tm_edt_version()
-    texts = [binding.tm_edt_strerror(s) for s in range(7)]  # TM_EDT_OK .. TM_EDT_ERR_TOO_LARGE
-    assert all(texts) and "unknown status" not in texts and len(set(texts)) == 7
+    texts = [binding.tm_edt_strerror(s) for s in range(8)]  # TM_EDT_OK .. TM_EDT_ERR_DEBUG_CHECK
+    assert all(texts) and "unknown status" not in texts and len(set(texts)) == 8
+    assert not binding.tm_edt_debug_build() and binding.tm_edt_debug_last_violation()[0] == 0
     assert "tm_edt_noalloc" in binding.tm_edt_strerror(binding.ERR_TOO_LARGE)
     assert binding.tm_edt_strerror(99) == "unknown status"
 
