@@ -64,6 +64,11 @@ cudaError_t ensure_smem(const void* kernel, size_t smem);
 bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep);
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches);
 
+// One axis pass of the wide-key path on plain integer values with the quad kernels (see tm_edt_lean.cu).
+bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
+cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
+                                cudaStream_t st);
+
 // Debug build: what the kernels launched from tm_edt_lean.cu recorded (see edt_debug.cuh).
 cudaError_t lean_debug_collect(cudaStream_t st, DebugRecord* out);
 

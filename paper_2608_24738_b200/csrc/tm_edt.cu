@@ -725,7 +725,9 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
         const double offs_b = k == 3 ? 8.0 : 2.0 * k;  // bytes of offsets per voxel read by this axis
         if (fin) prof_mark(st, "wide_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? offs_b : 0.0)));
         else prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 4.0 + (carry ? offs_b + (k == 2 ? 8.0 : 4.0) : 0.0)));
-        if (k == 1) e = fin ? launch_wide_axis<1, true>(A, ep, sh, st) : launch_wide_axis<1, false>(A, ep, sh, st);
+        if (sh == 0 && !switches().no_lean && lean_value_axis_ok(pl, k, ep))
+            e = run_lean_value_axis(pl, k, keys_in[k], fin ? nullptr : keys_out[k], ep, fin, st);
+        else if (k == 1) e = fin ? launch_wide_axis<1, true>(A, ep, sh, st) : launch_wide_axis<1, false>(A, ep, sh, st);
         else if (k == 2) e = fin ? launch_wide_axis<2, true>(A, ep, sh, st) : launch_wide_axis<2, false>(A, ep, sh, st);
         else e = launch_wide_axis<3, true>(A, ep, sh, st);
         ++launches;

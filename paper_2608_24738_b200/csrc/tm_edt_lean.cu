@@ -106,6 +106,31 @@ static cudaError_t launch_lean_value(const LeanParams& P, const EpilogueParams& 
     return launch_lean_value_tx<FINAL, VT, 32>(P, ep, outer, st);
 }
 
+// One axis pass of the wide-key path on plain integer values (unit sampling, no index output, extents up to 1024)
+// with the quad kernel lean_value_kernel: `in` / `out` hold one 32-bit value per voxel (2^31 = no site).
+bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
+    if (!pl.unit || ep.idx || pl.ext[0] % 4 != 0) return false;
+    if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
+    const int n = pl.ext[k];
+    const size_t smem = (size_t)(n + 2 * kLeanPad) * 32 * 4;
+    if (smem > 100 * 1024) return false;  // keeps at least two blocks per SM
+    const int64_t blocks = pl.N / ((int64_t)n * pl.inner[k]) * ((pl.inner[k] + 31) / 32);
+    return blocks >= 296;  // few strips (a single image) are split over several blocks by wide_axis_kernel instead
+}
+
+cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
+                                cudaStream_t st) {
+    LeanParams P;
+    memset(&P, 0, sizeof(P));
+    P.in = in; P.out = out;
+    P.in_elems = pl.N; P.out_elems = pl.N; P.images = pl.images;
+    P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
+    P.inv_scale = 1.0f;
+    const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+    return fin ? launch_lean_value_tx<true, uint32_t, 32>(P, ep, outer, st)
+               : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
+}
+
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* bufA = static_cast<char*>(ws);
