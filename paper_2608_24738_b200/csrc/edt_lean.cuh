@@ -252,6 +252,11 @@ __device__ __forceinline__ void lean_store_4xi64(int64_t* p, uint32_t a, uint32_
                  :: "l"(p), "r"(a), "r"(b), "r"(c), "r"(d), "r"(z) : "memory");
 }
 
+// The same int64 (given as its two halves) four times: one 256-bit streaming store (p 32-byte aligned).
+__device__ __forceinline__ void lean_store_4xi64_same(int64_t* p, uint32_t lo, uint32_t hi) {
+    asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %1, %2, %1, %2, %1, %2};" :: "l"(p), "r"(lo), "r"(hi) : "memory");
+}
+
 __device__ __forceinline__ int lean_sext_byte(uint32_t e, int q) {
     // byte q of e, sign-extended: one byte-permute (bit 3 of a selector nibble replicates the sign of the byte)
     const uint32_t sel = (uint32_t)q | ((8u | (uint32_t)q) << 4) | ((8u | (uint32_t)q) << 8) | ((8u | (uint32_t)q) << 12);
@@ -287,7 +292,12 @@ __device__ __forceinline__ void lean_emit_final(const uint32_t (&b)[4], const ui
             lean_store_4xi64(ip[q] + p, s[0], s[1], s[2], s[3]);
         }
         lean_store_4xi64(ip[K] + p, j[0], j[1], j[2], j[3]);
-    } else {  // an image without background: +inf, INT64_MAX, -1 (checked voxel by voxel)
+    } else if ((b[0] & b[1] & b[2] & b[3] & kLeanNone) != 0u) {  // an image without background: +inf, INT64_MAX, -1
+        if (dist) __stcs(reinterpret_cast<float4*>(dist + p), make_float4(TMEDT_INF, TMEDT_INF, TMEDT_INF, TMEDT_INF));
+        if (sq) lean_store_4xi64_same(sq + p, 0xffffffffu, 0x7fffffffu);
+#pragma unroll
+        for (int q = 0; q <= K; ++q) lean_store_4xi64_same(ip[q] + p, 0xffffffffu, 0xffffffffu);
+    } else {  // cannot happen inside one image (all its voxels have a site or none has); kept voxel by voxel
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             const bool none = b[v] >= kLeanNone;
