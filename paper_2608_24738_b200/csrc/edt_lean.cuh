@@ -175,8 +175,9 @@ __device__ __forceinline__ uint32_t lean_first_axis(const uint32_t v, const int 
 //   VT == uint16_t  values:  writes the squared distance so far (all ones = no site)
 //   VT == uint32_t  values:  writes the (scaled) squared distance so far (2^31 = no site)
 // ---------------------------------------------------------------------------------------------
-template <int VS, typename VT>
-__global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constant__ LeanParams P) {
+//   NW  warps per block: 8, or 16 where more resident warps are needed to cover the latencies of long scans
+template <int VS, typename VT, int NW = 8>
+__global__ void __launch_bounds__(32 * NW, 3) lean_plane_kernel(const __grid_constant__ LeanParams P) {
     constexpr bool ENT = sizeof(VT) == 1;
     constexpr int SH = ENT ? 16 : 0;
     extern __shared__ __align__(16) uint8_t sm_lean_p[];
@@ -185,12 +186,11 @@ __global__ void __launch_bounds__(256, 3) lean_plane_kernel(const __grid_constan
     const int64_t plane = blockIdx.x;
     const uint8_t* src = reinterpret_cast<const uint8_t*>(P.in) + plane * (int64_t)n1 * n0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int NW = 8;
     const uint32_t wk = ENT ? 1u : P.wk;
     lean_fill_pad<VS>(kt, n1);
     uint32_t all = 0xffffffffu;  // AND of this thread's keys
     {
-        constexpr int MAXR = 16;  // rows per warp: 128 rows / 8 warps
+        constexpr int MAXR = 128 / NW;  // rows per warp
         uint32_t rowv[MAXR];
         const bool act = 4 * lane < n0;
 #pragma unroll
@@ -415,10 +415,10 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
 //   VT  uint16_t (all ones = no site) or uint32_t (2^31 = no site)
 //   FINAL == false  writes the new value;  FINAL == true  writes float32 distances and / or int64 squared distances
 // ---------------------------------------------------------------------------------------------
-template <bool FINAL, typename VT, int TX>
-__global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__ LeanParams P,
-                                                         const __grid_constant__ EpilogueParams ep) {
-    constexpr int LPR = TX / 4, CG = TX / 32, NW = 8;
+template <bool FINAL, typename VT, int TX, int NW = 8>
+__global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_constant__ LeanParams P,
+                                                            const __grid_constant__ EpilogueParams ep) {
+    constexpr int LPR = TX / 4, CG = TX / 32;
     extern __shared__ __align__(16) uint8_t sm_lean_v[];
     const int n = P.n;
     uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_v);  // [n + 2 kLeanPad][TX]
@@ -428,7 +428,7 @@ __global__ void __launch_bounds__(256) lean_value_kernel(const __grid_constant__
     const VT* src = reinterpret_cast<const VT*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);
     uint32_t all = 0xffffffffu;  // AND of this thread's keys
-    for (int t = threadIdx.x; t < n * LPR; t += 256) {
+    for (int t = threadIdx.x; t < n * LPR; t += 32 * NW) {
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
         const VT* g = src + (int64_t)y * P.inner + q4;

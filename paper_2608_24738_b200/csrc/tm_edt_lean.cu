@@ -47,7 +47,16 @@ bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep) {
 template <int VS, typename VT>
 static cudaError_t launch_lean_plane(const LeanParams& P, int64_t planes, cudaStream_t st) {
     const size_t smem = (size_t)(P.n + 2 * kLeanPad) * VS * 4;
-    auto kern = lean_plane_kernel<VS, VT>;
+    // full-width planes: three blocks per SM fit whatever their size, so each gets 16 warps (more resident warps to
+    // cover the latencies of the first-axis pass and of long scans)
+    if (VS == 128) {
+        auto kern = lean_plane_kernel<VS, VT, 16>;
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)planes, 512, smem, st>>>(P);
+        return cudaGetLastError();
+    }
+    auto kern = lean_plane_kernel<VS, VT, 8>;
     cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
     kern<<<(unsigned)planes, 256, smem, st>>>(P);
@@ -91,6 +100,13 @@ template <bool FINAL, typename VT, int TX>
 static cudaError_t launch_lean_value_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4;
     P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    if (TX == 32 && P.n > 128) {  // long axes: few blocks fit an SM, so each gets 16 warps
+        auto kern = lean_value_kernel<FINAL, VT, TX, 16>;
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)(outer * P.tiles_per_slab), 512, smem, st>>>(P, ep);
+        return cudaGetLastError();
+    }
     auto kern = lean_value_kernel<FINAL, VT, TX>;
     cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
