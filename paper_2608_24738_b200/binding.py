@@ -393,6 +393,42 @@ class PreparedCall:
 MORPH_MODES = {"constant": 0, "reflect": 1, "nearest": 2, "mirror": 3, "wrap": 4}
 
 
+class PreparedMorph:
+    """A tm_grey_morph / tm_binary_morph call with its arguments marshalled once, for callers that repeat it."""
+
+    def __init__(self, image, footprint, structure=None, op="erosion", mode="reflect", cval=0.0, origin=None, out=None,
+                 border_value=0):
+        import numpy as np
+        import torch
+
+        L = lib()
+        binary = image.dtype in (torch.uint8, torch.bool)
+        if image.dtype == torch.bool:
+            image = image.view(torch.uint8)
+        if not image.is_cuda or image.dim() < 3 or not image.is_contiguous():
+            raise ValueError("image must be a contiguous CUDA tensor shaped (B, C, spatial...)")
+        ndim = image.dim() - 2
+        fp, fps = _element(footprint, ndim)
+        st = None if structure is None else np.ascontiguousarray(structure, dtype=np.float32)
+        self.image, self.out = image, (torch.empty_like(image) if out is None else out)
+        self._keep = (fp, fps, st, _shape_array(tuple(image.shape)), _origin(origin, ndim))
+        opc = {"erosion": 0, "dilation": 1}[op]
+        if binary:
+            self._fn = L.tm_binary_morph
+            self._args = (_p(image), ndim, self._keep[3], fp.ctypes.data_as(ctypes.c_void_p), fps, self._keep[4], opc,
+                          int(bool(border_value)), _p(self.out))
+        else:
+            self._fn = L.tm_grey_morph
+            self._args = (_p(image), ndim, self._keep[3], fp.ctypes.data_as(ctypes.c_void_p),
+                          None if st is None else st.ctypes.data_as(ctypes.c_void_p), fps, self._keep[4], opc,
+                          MORPH_MODES[mode], ctypes.c_float(cval), _p(self.out))
+
+    def __call__(self, stream_ptr):
+        rc = self._fn(*self._args, stream_ptr)
+        if rc != OK:
+            _check(rc)
+
+
 def _element(footprint, ndim):
     import numpy as np
 

@@ -1,0 +1,146 @@
+// Binary erosion / dilation on bit-packed lines (paper, Section 2.3.1: the binary form of the fused kernel combines
+// the neighbourhood with AND / OR and a single border value).  A mask needs one bit per voxel, so the combine of 32
+// voxels with one neighbour position is one funnel shift and one logic instruction on 32-bit words:
+//   1. binary_pack_kernel     mask bytes -> one bit per voxel (bit b of word w of a line = voxel 32 w + b is nonzero);
+//                             a lane takes 32 consecutive voxels (two 16-byte loads), N / 8 bytes of scratch.
+//   2. binary_lines_kernel    the host groups the element's active positions by their offsets along all axes but the
+//                             contiguous one; a group is a neighbouring line plus a 64-bit mask of offsets along
+//                             the line.  A lane produces one output word: per group it reads three words of the
+//                             neighbouring line (or takes the border value if that line lies outside the image), and
+//                             per offset of the group shifts the 96-bit window into place and combines it; the result
+//                             is expanded to bytes and leaves as one 32-byte store.
+// Requires at most 4 axes, a contiguous extent that is a multiple of 32, offsets along it within +-31, and 32-byte
+// aligned buffers;
+// everything else runs on the byte kernels of morph.cuh.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "morph.cuh"
+
+namespace tmmorph {
+
+struct LineGroup {
+    int16_t off[kMaxDims];  // offsets along the axes before the contiguous one (entry ndim - 1 unused)
+    int64_t line_offset;    // the same as a number of lines inside one image
+    uint64_t mask;          // bit (dx + 31) set: offset dx along the line is active
+};
+
+constexpr int kMaxLineGroups = 96;  // groups travel as kernel arguments (no copy to the device, no extra latency)
+
+struct BitsParams {
+    const uint8_t* in;
+    uint8_t* out;
+    uint32_t* bits;          // (lines, words) packed mask
+    LineGroup groups[kMaxLineGroups];
+    int n_groups;
+    int ndim;
+    int64_t lines;           // images * lines per image
+    int64_t lines_per_image;
+    int words;               // words per line = last extent / 32
+    int ext[kMaxDims];
+    int border_value;
+};
+
+__device__ __forceinline__ uint32_t nonzero_bits4(uint32_t v) {
+    // bit i = byte i of v is nonzero
+    const uint32_t m = (((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every nonzero byte
+    return (((m >> 7) * 0x00204081u) >> 21) & 0xfu;
+}
+
+__global__ void __launch_bounds__(256) binary_pack_kernel(const __grid_constant__ BitsParams P) {
+    const int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // word index over the whole batch
+    if (w >= P.lines * P.words) return;
+    uint32_t v[8];  // one 256-bit load: a warp reads 1 KB in one request
+    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(P.in + w * 32));
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) bits |= nonzero_bits4(v[i]) << (4 * i);
+    P.bits[w] = bits;
+}
+
+// Block = 8 x 32 lanes (threadIdx.y, threadIdx.x); a lane produces word w of L consecutive lines, which differ only in
+// their coordinate along the axis before the contiguous one (the host picks L = 4 when that extent is a multiple of
+// 4), so that a group's offsets are decoded once for L words.  Blocks enumerate (group of 8 L lines, chunk of 32
+// words).  ND: number of axes (1 .. 4).
+template <bool MIN, int L, int ND>
+__global__ void __launch_bounds__(256) binary_lines_kernel(const __grid_constant__ BitsParams P, const unsigned chunks) {
+    const unsigned lb = blockIdx.x / chunks, ch = blockIdx.x - lb * chunks;
+    const int64_t line0 = ((int64_t)lb * 8 + threadIdx.y) * L;
+    const int w = (int)(ch * 32 + threadIdx.x);
+    if (line0 >= P.lines || w >= P.words) return;
+    // coordinates of the first line along the axes before the contiguous one (fewer than 2^31 lines per image)
+    int x[ND > 1 ? ND - 1 : 1];
+    x[0] = 0;
+    {
+        uint32_t rr = (uint32_t)(line0 % P.lines_per_image);
+#pragma unroll
+        for (int a = ND - 2; a >= 0; --a) {
+            const uint32_t n = (uint32_t)P.ext[a], q = rr / n;
+            x[a] = (int)(rr - q * n);
+            rr = q;
+        }
+    }
+    const uint32_t fill = P.border_value ? 0xffffffffu : 0u;
+    uint32_t acc[L];
+#pragma unroll
+    for (int j = 0; j < L; ++j) acc[j] = MIN ? 0xffffffffu : 0u;
+    for (int g = 0; g < P.n_groups; ++g) {
+        const LineGroup& G = P.groups[g];
+        bool in_outer = true;
+#pragma unroll
+        for (int a = 0; a < ND - 2; ++a) in_outer = in_outer && (unsigned)(x[a] + G.off[a]) < (unsigned)P.ext[a];
+        const uint32_t* row = P.bits + (line0 + G.line_offset) * P.words + w;
+        uint32_t lo[L], mid[L], hi[L];  // words w - 1, w, w + 1 of the neighbouring lines
+#pragma unroll
+        for (int j = 0; j < L; ++j) {
+            const bool inside = in_outer && (ND < 2 || (unsigned)(x[ND > 1 ? ND - 2 : 0] + j + G.off[ND > 1 ? ND - 2 : 0]) < (unsigned)P.ext[ND > 1 ? ND - 2 : 0]);
+            lo[j] = fill; mid[j] = fill; hi[j] = fill;
+            if (inside) {
+                const uint32_t* r = row + (int64_t)j * P.words;
+                mid[j] = r[0];
+                if (w > 0) lo[j] = r[-1];
+                if (w + 1 < P.words) hi[j] = r[1];
+            }
+        }
+        // output bit i takes input bit i + dx: offsets to the left (dx = b - 31 <= 0), then to the right
+        for (uint32_t m = (uint32_t)G.mask; m; m &= m - 1) {
+            const int sh = 31 - (__ffs((int)m) - 1);  // -dx (a shift of 0 returns mid)
+#pragma unroll
+            for (int j = 0; j < L; ++j) {
+                const uint32_t v = __funnelshift_l(lo[j], mid[j], sh);
+                acc[j] = MIN ? acc[j] & v : acc[j] | v;
+            }
+        }
+        for (uint32_t m = (uint32_t)(G.mask >> 32); m; m &= m - 1) {
+            const int sh = __ffs((int)m);  // dx = bit + 1
+#pragma unroll
+            for (int j = 0; j < L; ++j) {
+                const uint32_t v = __funnelshift_r(mid[j], hi[j], sh);
+                acc[j] = MIN ? acc[j] & v : acc[j] | v;
+            }
+        }
+        uint32_t all = acc[0];
+#pragma unroll
+        for (int j = 1; j < L; ++j) all = MIN ? all | acc[j] : all & acc[j];
+        if (all == (MIN ? 0u : 0xffffffffu)) break;  // decided for every voxel of the lane
+    }
+    // expand 32 bits to 32 bytes (0 / 1): one 256-bit store per line
+#pragma unroll
+    for (int j = 0; j < L; ++j) {
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t nib = (acc[j] >> (4 * i)) & 0xfu;
+            o[i] = (nib * 0x00204081u) & 0x01010101u;
+        }
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(P.out + ((line0 + j) * P.words + w) * 32), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]),
+                        "r"(o[6]), "r"(o[7])
+                     : "memory");
+    }
+}
+
+}  // namespace tmmorph

@@ -11,6 +11,8 @@
 #include "../../include/tm_morph.h"
 #include "host_shared.h"
 #include "morph.cuh"
+#include "morph_bits.cuh"
+#include "morph_box.cuh"
 
 using namespace tmmorph;
 
@@ -131,6 +133,144 @@ int run_box(const T* input, int ndim, const int64_t* shape, const int64_t* fp_sh
     return rc;
 }
 
+// One pass of box_strip_kernel: a window of +-rh along the contiguous axis and +-rv along the walk axis.
+static bool launch_box_strip(bool ero, int rh, int rv, const StripParams& B, unsigned blocks, cudaStream_t s) {
+#define TM_BOX_STRIP(RH, RV)                                                                                     \
+    do {                                                                                                         \
+        if (ero) box_strip_kernel<true, RH, RV, box_strip_len(RV)><<<blocks, dim3(32, 8), 0, s>>>(B);             \
+        else box_strip_kernel<false, RH, RV, box_strip_len(RV)><<<blocks, dim3(32, 8), 0, s>>>(B);                \
+        return true;                                                                                             \
+    } while (0)
+    if (rh == rv) { switch (rh) { case 1: TM_BOX_STRIP(1, 1); case 2: TM_BOX_STRIP(2, 2); case 3: TM_BOX_STRIP(3, 3); case 4: TM_BOX_STRIP(4, 4); } }
+    else if (rv == 0) { switch (rh) { case 1: TM_BOX_STRIP(1, 0); case 2: TM_BOX_STRIP(2, 0); case 3: TM_BOX_STRIP(3, 0); case 4: TM_BOX_STRIP(4, 0); } }
+    else if (rh == 0) { switch (rv) { case 1: TM_BOX_STRIP(0, 1); case 2: TM_BOX_STRIP(0, 2); case 3: TM_BOX_STRIP(0, 3); case 4: TM_BOX_STRIP(0, 4); } }
+#undef TM_BOX_STRIP
+    return false;
+}
+
+// A flat full box of odd extents (at most 9 per axis), centred on its voxel, on a float32 image: passes of
+// box_strip_kernel (morph_box.cuh), the last two axes in one pass when their extents are equal, one further pass per
+// earlier axis; every border rule is applied inside the kernel.  Returns -1 when the shape or the element does not
+// fit, and the caller goes on with the general kernels.
+static int run_box_quads(const float* input, int ndim, const int64_t* fp_shape, const int64_t* origin,
+                         int op, int mode, float cval, float* output, tm_edt_stream_t stream, const Geometry& g) {
+    const int nd = ndim, W = g.ext[nd - 1];
+    if (W % 4 != 0 || ((uintptr_t)input & 15u) || ((uintptr_t)output & 15u)) return -1;
+    int rad[kMaxDims];
+    for (int a = 0; a < nd; ++a) {
+        const int m = (int)fp_shape[a];
+        if (m % 2 == 0 || m > 9 || (origin && origin[a] != 0)) return -1;
+        rad[a] = m / 2;
+    }
+    // passes as (radius along the row, walk axis, radius along it); walk axis -1: no walk
+    struct Pass { int rh, axis, rv; } pass[kMaxDims + 1];
+    int np = 0;
+    const int rh = rad[nd - 1], rv = nd >= 2 ? rad[nd - 2] : 0;
+    if (rh == rv || rh == 0 || rv == 0) { if (rh || rv) pass[np++] = {rh, nd >= 2 ? nd - 2 : -1, rv}; }
+    else { pass[np++] = {rh, nd >= 2 ? nd - 2 : -1, 0}; pass[np++] = {0, nd - 2, rv}; }
+    for (int a = nd - 3; a >= 0; --a)
+        if (rad[a]) pass[np++] = {0, a, rad[a]};
+    if (np == 0) return -1;
+    for (int i = 0; i < np; ++i) {  // every pass must fit a grid before the first one is launched
+        const int n = pass[i].axis >= 0 ? g.ext[pass[i].axis] : 1, T = box_strip_len(pass[i].rv);
+        const int64_t blocks = g.total / ((int64_t)n * W) * (((n + T - 1) / T + 7) / 8) * ((W / 4 + 31) / 32);
+        if (blocks > (int64_t)INT32_MAX) return -1;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t buf = (((size_t)g.total * 4) + 255) & ~(size_t)255;
+    char* ws = nullptr;
+    if (np > 1) {
+        cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, (np > 2 ? 2 : 1) * buf, s);
+        if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    }
+    const float* src = input;
+    int rc = TM_EDT_OK, launches = 0;
+    for (int i = 0; i < np && rc == TM_EDT_OK; ++i) {
+        float* dst = i == np - 1 ? output : reinterpret_cast<float*>(ws + (size_t)(i & 1) * buf);
+        StripParams B;
+        memset(&B, 0, sizeof(B));
+        B.in = src; B.out = dst; B.W = W; B.mode = mode; B.cval = cval;
+        B.chunks = (unsigned)((W / 4 + 31) / 32);
+        if (pass[i].axis >= 0) { B.n = g.ext[pass[i].axis]; B.walk_stride = g.stride[pass[i].axis]; }
+        else { B.n = 1; B.walk_stride = W; }
+        B.inner = (int)(B.walk_stride / W);
+        const int T = box_strip_len(pass[i].rv);
+        B.strip_groups = (unsigned)(((B.n + T - 1) / T + 7) / 8);
+        const int64_t columns = g.total / ((int64_t)B.n * W);
+        const unsigned blocks = (unsigned)(columns * B.strip_groups * B.chunks);
+        if (!launch_box_strip(op == TM_MORPH_EROSION, pass[i].rh, pass[i].rv, B, blocks, s) || cudaGetLastError() != cudaSuccess) {
+            rc = TM_EDT_ERR_CUDA;
+            break;
+        }
+        ++launches;
+        src = dst;
+    }
+    if (ws) cudaFreeAsync(ws, s);
+    if (rc == TM_EDT_OK) tmedt::shared_record(-1, launches);
+    return rc;
+}
+
+// Binary erosion / dilation on bit-packed lines (morph_bits.cuh) when the shape allows it; returns -1 when it does
+// not, and the caller goes on with the byte kernels.
+static int run_binary_bits(const Geometry& g, const std::vector<Entry>& entries, const uint8_t* input, uint8_t* output,
+                           bool erosion, int border_value, cudaStream_t s) {
+    const int nd = g.ndim, W = g.ext[nd - 1];
+    if (nd > 4 || W % 32 != 0 || ((uintptr_t)input & 31u) || ((uintptr_t)output & 31u)) return -1;
+    if ((g.total / W + 7) / 8 * ((W / 32 + 31) / 32) > (int64_t)INT32_MAX) return -1;  // blocks of the line kernel
+    std::vector<LineGroup> groups;
+    for (const Entry& en : entries) {
+        const int dx = en.off[nd - 1];
+        if (dx < -31 || dx > 31) return -1;
+        LineGroup* grp = nullptr;
+        for (LineGroup& c : groups) {
+            bool same = true;
+            for (int a = 0; a < nd - 1; ++a) same = same && c.off[a] == en.off[a];
+            if (same) { grp = &c; break; }
+        }
+        if (!grp) {
+            LineGroup n;
+            memset(&n, 0, sizeof(n));
+            for (int a = 0; a < nd - 1; ++a) { n.off[a] = en.off[a]; n.line_offset += (int64_t)en.off[a] * (g.stride[a] / W); }
+            groups.push_back(n);
+            grp = &groups.back();
+        }
+        grp->mask |= (uint64_t)1 << (dx + 31);
+    }
+    if ((int)groups.size() > kMaxLineGroups) return -1;
+    const int64_t words = g.total / 32;
+    char* dev = nullptr;
+    cudaError_t e = tmedt::shared_scratch_alloc((void**)&dev, (size_t)words * 4, s);
+    if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
+    {
+        BitsParams B;
+        memset(&B, 0, sizeof(B));
+        B.in = input; B.out = output; B.bits = reinterpret_cast<uint32_t*>(dev);
+        for (size_t i = 0; i < groups.size(); ++i) B.groups[i] = groups[i];
+        B.n_groups = (int)groups.size();
+        B.ndim = nd; B.words = W / 32; B.lines = g.total / W; B.lines_per_image = g.V / W;
+        for (int a = 0; a < nd; ++a) B.ext[a] = g.ext[a];
+        B.border_value = border_value ? 1 : 0;
+        const unsigned blocks = (unsigned)((words + 255) / 256);
+        binary_pack_kernel<<<blocks, 256, 0, s>>>(B);
+        const unsigned chunks = (unsigned)((B.words + 31) / 32);
+        const int L = nd >= 2 && g.ext[nd - 2] % 4 == 0 ? 4 : 1;  // lines per lane
+        const unsigned lblocks = (unsigned)((B.lines / L + 7) / 8) * chunks;
+#define TM_BITS_LINES(LL, NDV)                                                                                 \
+    do {                                                                                                       \
+        if (erosion) binary_lines_kernel<true, LL, NDV><<<lblocks, dim3(32, 8), 0, s>>>(B, chunks);             \
+        else binary_lines_kernel<false, LL, NDV><<<lblocks, dim3(32, 8), 0, s>>>(B, chunks);                    \
+    } while (0)
+        if (L == 4) { if (nd == 2) TM_BITS_LINES(4, 2); else if (nd == 3) TM_BITS_LINES(4, 3); else TM_BITS_LINES(4, 4); }
+        else { if (nd == 1) TM_BITS_LINES(1, 1); else if (nd == 2) TM_BITS_LINES(1, 2); else if (nd == 3) TM_BITS_LINES(1, 3); else TM_BITS_LINES(1, 4); }
+#undef TM_BITS_LINES
+        e = cudaGetLastError();
+    }
+    cudaFreeAsync(dev, s);
+    if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
+    tmedt::shared_record(-1, 2);
+    return TM_EDT_OK;
+}
+
 template <typename T, bool BINARY>
 int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const float* st, const int64_t* fp_shape,
         const int64_t* origin, int op, int mode, float cval, int border_value, void* output, tm_edt_stream_t stream,
@@ -152,6 +292,25 @@ int run(const T* input, int ndim, const int64_t* shape, const uint8_t* fp, const
     if (((uintptr_t)input % sizeof(T)) || ((uintptr_t)output % (BINARY ? 1 : 4))) return TM_EDT_ERR_INVALID_ARG;
     if (!tmedt::shared_is_device_ptr(input) || !tmedt::shared_is_device_ptr(output)) return TM_EDT_ERR_BAD_POINTER;
     if (g.total > (int64_t)INT32_MAX * 128) return TM_EDT_ERR_UNSUPPORTED;
+    if (BINARY && allow_separable) {
+        const int rb = run_binary_bits(g, entries, reinterpret_cast<const uint8_t*>(input), static_cast<uint8_t*>(output),
+                                       op == TM_MORPH_EROSION, border_value, (cudaStream_t)stream);
+        if (rb >= 0) return rb;
+    }
+    if (!BINARY && allow_separable) {
+        int64_t box = 1;
+        bool flat = true;
+        for (int a = 0; a < ndim; ++a) box *= fp_shape[a];
+        for (const Entry& en : entries) flat = flat && en.s == 0.0f;
+        if (flat && (int64_t)entries.size() == box && box <= (int64_t)sizeof(uint8_t) * 256 * 9 && box > 1) {
+            int64_t last2 = fp_shape[ndim - 1] * (ndim >= 2 ? fp_shape[ndim - 2] : 1);
+            if (last2 <= 256 * 9) {
+                const int rq = run_box_quads(reinterpret_cast<const float*>(input), ndim, fp_shape, origin, op, mode, cval,
+                                             static_cast<float*>(output), stream, g);
+                if (rq >= 0) return rq;
+            }
+        }
+    }
     if (allow_separable && ndim >= 2 && entries.size() >= 20) {
         int64_t box = 1;
         bool flat = true;
