@@ -145,6 +145,208 @@ __global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ 
     }
 }
 
+// ---- the first two axes on 16-bit values ----
+// Distances along two axes of up to 1024 voxels each stay below 2^14, so the first pass can hand 16-bit values to the
+// second one (half the scratch traffic) and the second pass holds a strip of 32 columns of an axis of 1024 rows in
+// 64 KB of shared memory.  "No background seen" is kNone16 and every value at or above it means the same (adding
+// distances to it stays below 2^16).
+constexpr int kNone16 = 0xC000;
+
+struct Row16Params {
+    const uint8_t* mask;
+    uint16_t* out;
+    int64_t rows;
+    int words;  // 32-voxel words per row (1 .. 32)
+};
+
+__device__ __forceinline__ uint32_t cdt_nonzero_bits4(uint32_t v) {
+    const uint32_t m = (((v & 0x7f7f7f7fu) + 0x7f7f7f7fu) | v) & 0x80808080u;  // 0x80 in every nonzero byte
+    return (((m >> 7) * 0x00204081u) >> 21) & 0xfu;
+}
+
+// First axis, rows of 32 .. 1024 voxels (a multiple of 32).  A lane owns one word of 32 voxels (one 32-byte load,
+// two 32-byte stores); a warp holds 32 / words whole rows.  The nearest background voxel outside the lane's word
+// comes from a ballot over the words that contain one and a shuffle of its position inside that word; inside the word
+// the distances are two running counts over the 32 bits, left to right and right to left.
+__global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ Row16Params P) {
+    const int lane = threadIdx.x & 31;
+    const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int words = P.words, rpw = 32 / words;
+    const int grp = lane / words, w = lane - grp * words;
+    const int64_t row = gw * rpw + grp;
+    const bool valid = grp < rpw && row < P.rows;
+    uint32_t z = 0u;  // bit i: voxel i of the word is background
+    if (valid) {
+        uint32_t v[8];
+        asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "l"(P.mask + (row * words + w) * 32));
+        uint32_t nzb = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) nzb |= cdt_nonzero_bits4(v[i]) << (4 * i);
+        z = ~nzb;
+    }
+    const uint32_t has = __ballot_sync(0xffffffffu, z != 0u);
+    const int g0 = grp * words, g1 = g0 + words;  // lanes of this row
+    const uint32_t in_row = (g1 >= 32 ? 0xffffffffu : (1u << g1) - 1u) & ~((1u << g0) - 1u);
+    const uint32_t left = has & in_row & ((1u << lane) - 1u);
+    const uint32_t right = has & in_row & ~(lane == 31 ? 0xffffffffu : (2u << lane) - 1u);
+    const int hb = 31 - __clz(z), lb = __ffs(z) - 1;  // last / first background voxel of the own word
+    const int wl = left ? 31 - __clz(left) : lane, wr = right ? __ffs(right) - 1 : lane;
+    const int hbl = __shfl_sync(0xffffffffu, hb, wl), lbr = __shfl_sync(0xffffffffu, lb, wr);
+    if (!valid) return;
+    int f = left ? 32 * (lane - wl) - hbl - 1 : kNone16;    // distance of the voxel before the word to the background on its left
+    int d[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        f = (z >> i) & 1u ? 0 : f + 1;
+        d[i] = f;
+    }
+    int b = right ? 32 * (wr - lane) + lbr - 32 : kNone16;  // the same for the voxel after the word, to the right
+#pragma unroll
+    for (int i = 31; i >= 0; --i) {
+        b = (z >> i) & 1u ? 0 : b + 1;
+        d[i] = min(min(d[i], b), kNone16);
+    }
+    uint16_t* dst = P.out + (row * words + w) * 32;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = (uint32_t)d[16 * h + 2 * i] | ((uint32_t)d[16 * h + 2 * i + 1] << 16);
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(dst + 16 * h), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                     : "memory");
+    }
+}
+
+struct Col16Params {
+    const uint16_t* in;  // values of the first pass, view (outer, n, inner)
+    int32_t* out;
+    int64_t inner;       // a multiple of 32
+    int n;               // up to 1024
+    int last;            // last pass: "no background" becomes -1 (else kBig for the next pass)
+};
+
+__device__ __forceinline__ uint32_t cdt_both(int v) { return (uint32_t)v * 0x00010001u; }  // v in both halves
+
+// Second axis on a strip of (n x 32) 16-bit values in shared memory, lane = column, NW warps.
+// Taxicab: g(y) = min_j f(j) + |y - j| is two running minima, g = min(f, g_prev + 1), top to bottom and back.  Each
+// warp runs them over its own segment of rows; what reaches a segment from the rows before (after) it is the value at
+// the end of the previous (start of the next) segment plus the distance, combined over the segments in between.
+// Chessboard: g(y) = min_j max(f(j), |y - j|) by bounded outward scans (a candidate d rows away is worth at least d, so
+// a scan ends once d reaches the minimum): a lane takes eight consecutive rows at a time, their minima as four pairs
+// of 16-bit halves, so that one candidate row fetched from the tile serves eight voxels with two packed instructions
+// per pair (max(f, d + offset) as one add-max, then the minimum).
+template <bool CHESS, int NW>
+__global__ void __launch_bounds__(32 * NW) cdt_col16_kernel(const __grid_constant__ Col16Params P, const int strips_per_slab) {
+    extern __shared__ __align__(16) uint16_t sm_c16[];  // [n][32]
+    __shared__ int s_end[2][NW][32];
+    const int n = P.n;
+    const int64_t slab = blockIdx.x / strips_per_slab;
+    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
+    const int64_t base = slab * (int64_t)n * P.inner + c0;
+#pragma unroll 4
+    for (int t = threadIdx.x; t < n * 4; t += 32 * NW) {  // four lanes copy one row of 64 bytes
+        const int y = t >> 2, ch = t & 3;
+        *reinterpret_cast<int4*>(sm_c16 + y * 32 + 8 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 8 * ch);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t* out = P.out + base + lane;
+    const uint16_t* col = sm_c16 + lane;
+    const int none_out = P.last ? -1 : kBig;
+    if (!CHESS) {
+        const int S = (n + NW - 1) / NW;
+        const int y0 = min(n, warp * S), y1 = min(n, y0 + S);  // rows of this warp's segment
+        uint16_t* mine = sm_c16 + lane;
+        int f = kNone16;
+#pragma unroll 8
+        for (int y = y0; y < y1; ++y) {
+            f = min((int)mine[y * 32], f + 1);
+            mine[y * 32] = (uint16_t)f;
+        }
+        s_end[0][warp][lane] = f;
+        __syncthreads();
+        int cf = kNone16;  // value at the last row before the segment
+        for (int s = 0; s < warp; ++s) cf = min(s_end[0][s][lane], cf + (min(n, (s + 1) * S) - min(n, s * S)));
+        int b = kNone16;
+#pragma unroll 8
+        for (int y = y1 - 1; y >= y0; --y) {
+            b = min(min((int)mine[y * 32], cf + (y - y0 + 1)), b + 1);
+            mine[y * 32] = (uint16_t)b;
+        }
+        s_end[1][warp][lane] = b;
+        __syncthreads();
+        int cb = kNone16;  // value at the first row after the segment
+        for (int s = NW - 1; s > warp; --s) cb = min(s_end[1][s][lane], cb + (min(n, (s + 1) * S) - min(n, s * S)));
+#pragma unroll 8
+        for (int y = y0; y < y1; ++y) {
+            const int g = min((int)mine[y * 32], cb + (y1 - y));
+            out[(int64_t)y * P.inner] = g >= kNone16 ? none_out : g;
+        }
+    } else {
+        for (int y0 = warp * 8; y0 < n; y0 += NW * 8) {
+            int k[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) k[i] = y0 + i < n ? (int)col[(y0 + i) * 32] : kNone16;
+            uint32_t B[4];  // minima of rows (y0 + 2p, y0 + 2p + 1) in the (low, high) halves
+#pragma unroll
+            for (int p = 0; p < 4; ++p) B[p] = (uint32_t)k[2 * p] | ((uint32_t)k[2 * p + 1] << 16);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t V = cdt_both(k[j]);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const int d0 = 2 * p > j ? 2 * p - j : j - 2 * p, d1 = 2 * p + 1 > j ? 2 * p + 1 - j : j - 2 * p - 1;
+                    B[p] = __vminu2(B[p], __vmaxu2(V, (uint32_t)d0 | ((uint32_t)d1 << 16)));
+                }
+            }
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {  // rows beyond the axis: finished from the start
+                if (y0 + 2 * p >= n) B[p] = 0u;
+                else if (y0 + 2 * p + 1 >= n) B[p] &= 0xffffu;
+            }
+            auto largest = [&]() {
+                const uint32_t m = __vmaxu2(__vmaxu2(B[0], B[1]), __vmaxu2(B[2], B[3]));
+                return (int)max(m & 0xffffu, m >> 16);
+            };
+            int mx = largest();
+            int lo = y0 - 1, hi = y0 + 8, d = 1;
+            // candidates on both sides inside the axis
+            for (; d < mx && lo >= 0 && hi < n; ++d, --lo, ++hi) {
+                const uint32_t VL = cdt_both(col[lo * 32]), VH = cdt_both(col[hi * 32]), D = cdt_both(d);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    // row y0 + i is d + i from lo and d + 7 - i from hi
+                    const uint32_t cl = (uint32_t)(2 * p) | ((uint32_t)(2 * p + 1) << 16);
+                    const uint32_t chh = (uint32_t)(7 - 2 * p) | ((uint32_t)(6 - 2 * p) << 16);
+                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, cl, VL));
+                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, chh, VH));
+                }
+                mx = largest();
+            }
+            for (; d < mx && (lo >= 0 || hi < n); ++d, --lo, ++hi) {
+                const uint32_t VL = cdt_both(lo >= 0 ? (int)col[lo * 32] : kNone16);
+                const uint32_t VH = cdt_both(hi < n ? (int)col[hi * 32] : kNone16), D = cdt_both(d);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const uint32_t cl = (uint32_t)(2 * p) | ((uint32_t)(2 * p + 1) << 16);
+                    const uint32_t chh = (uint32_t)(7 - 2 * p) | ((uint32_t)(6 - 2 * p) << 16);
+                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, cl, VL));
+                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, chh, VH));
+                }
+                mx = largest();
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int g = (int)((B[i >> 1] >> (16 * (i & 1))) & 0xffffu);
+                if (y0 + i < n) out[(int64_t)(y0 + i) * P.inner] = g >= kNone16 ? none_out : g;
+            }
+        }
+    }
+}
+
 // ---- brute force ----
 struct BruteParams {
     const uint8_t* mask;

@@ -57,7 +57,39 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
     int32_t* tmp[2] = {reinterpret_cast<int32_t*>(ws), reinterpret_cast<int32_t*>(ws + buf)};
     const int32_t* prev = nullptr;
     cudaError_t e = cudaSuccess;
-    for (int k = 0; k < E && e == cudaSuccess; ++k) {
+    const bool chess = metric == TM_METRIC_CHESSBOARD;
+    int k0 = 0;
+    // The first two axes on 16-bit values (cdt.cuh): rows of a multiple of 32 up to 1024 voxels, a second axis of up
+    // to 1024 rows whose stride is the row length.
+    if (E >= 2 && axes[0] == ndim - 1 && g.ext[axes[0]] % 32 == 0 && g.ext[axes[0]] <= 1024 && g.ext[axes[1]] <= 1024 &&
+        ((uintptr_t)input & 31u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
+        const int n0 = (int)g.ext[axes[0]], n1 = (int)g.ext[axes[1]];
+        Row16Params R;
+        R.mask = input; R.out = reinterpret_cast<uint16_t*>(tmp[0]); R.rows = g.total / n0; R.words = n0 / 32;
+        const int64_t warps = (R.rows + 32 / R.words - 1) / (32 / R.words);
+        cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
+        Col16Params C;
+        C.in = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1]; C.inner = n0; C.n = n1;
+        const int strips = n0 / 32;
+        const size_t smem = (size_t)n1 * 64;
+        const bool wide = n1 > 256;  // 16 warps per block on long axes
+        auto kern = wide ? (chess ? cdt_col16_kernel<true, 16> : cdt_col16_kernel<false, 16>)
+                         : (chess ? cdt_col16_kernel<true, 8> : cdt_col16_kernel<false, 8>);
+        if (smem > 48 * 1024) {
+            static bool raised[2][64];  // per kernel and device: the attribute is set once
+            int dev = 0;
+            cudaGetDevice(&dev);
+            if (dev < 0 || dev >= 64 || !raised[chess][dev]) {
+                cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+                if (dev >= 0 && dev < 64) raised[chess][dev] = true;
+            }
+        }
+        kern<<<(unsigned)(g.total / ((int64_t)n1 * n0) * strips), wide ? 512 : 256, smem, st>>>(C, strips);
+        e = cudaGetLastError();
+        prev = C.out;
+        k0 = 2;
+    }
+    for (int k = k0; k < E && e == cudaSuccess; ++k) {
         PassParams P;
         memset(&P, 0, sizeof(P));
         P.mask = input; P.in = prev; P.total = g.total;
@@ -66,7 +98,6 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
         P.n = (int)g.ext[axes[k]];
         P.inner = 1;
         for (int a = axes[k] + 1; a < ndim; ++a) P.inner *= g.ext[a];
-        const bool chess = metric == TM_METRIC_CHESSBOARD;
         if (k == 0 && P.inner == 1 && P.n <= 8192) {
             // contiguous lines: ballot words, same distance for both metrics
             RowParams R;

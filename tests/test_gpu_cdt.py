@@ -19,7 +19,11 @@ def _built():
 
 SHAPES = [(2, 2, 1), (3, 1, 37), (2, 1, 19, 23), (1, 2, 40, 300), (1, 1, 1, 50, 1), (2, 1, 11, 12, 13), (1, 1, 5, 6, 4, 7),
           (1, 1, 3, 3, 2, 3, 2, 3, 2, 3), (1, 1, 260, 130), (1, 1, 6, 200, 33),
-          (1, 1, 1100, 40), (1, 1, 3, 9000)]  # beyond the shared-memory strip / the ballot-word row kernel
+          (1, 1, 1100, 40), (1, 1, 3, 9000),  # beyond the shared-memory strip / the ballot-word row kernel
+          # rows of a multiple of 32 voxels: the first two axes on 16-bit values (one to 32 words per row, segments of
+          # the second axis that are empty, ragged and full, a third axis after them, an axis of one voxel in between)
+          (2, 1, 64, 64), (3, 1, 5, 96), (1, 1, 300, 1024), (1, 2, 1024, 32), (2, 1, 7, 33, 64), (1, 1, 9, 1, 128),
+          (1, 1, 70, 352), (2, 1, 1, 3, 160)]
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=["x".join(map(str, s)) for s in SHAPES])
