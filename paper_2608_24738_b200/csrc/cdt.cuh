@@ -308,34 +308,32 @@ __global__ void __launch_bounds__(32 * NW) cdt_col16_kernel(const __grid_constan
                 else if (y0 + 2 * p + 1 >= n) B[p] &= 0xffffu;
             }
             auto largest = [&]() {
-                const uint32_t m = __vmaxu2(__vmaxu2(B[0], B[1]), __vmaxu2(B[2], B[3]));
+                const uint32_t m = __vmaxu2(__vimax3_u16x2(B[0], B[1], B[2]), B[3]);
                 return (int)max(m & 0xffffu, m >> 16);
+            };
+            // rows lo and hi, d rows beyond the first and the last of the eight: row y0 + i is d + i from lo and
+            // d + 7 - i from hi
+            auto step = [&](int vlo, int vhi, int d) {
+                const uint32_t VL = cdt_both(vlo), VH = cdt_both(vhi), D = cdt_both(d);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const uint32_t cl = (uint32_t)(2 * p) | ((uint32_t)(2 * p + 1) << 16);
+                    const uint32_t chh = (uint32_t)(7 - 2 * p) | ((uint32_t)(6 - 2 * p) << 16);
+                    B[p] = __vimin3_u16x2(B[p], __viaddmax_u16x2(D, cl, VL), __viaddmax_u16x2(D, chh, VH));
+                }
             };
             int mx = largest();
             int lo = y0 - 1, hi = y0 + 8, d = 1;
-            // candidates on both sides inside the axis
-            for (; d < mx && lo >= 0 && hi < n; ++d, --lo, ++hi) {
-                const uint32_t VL = cdt_both(col[lo * 32]), VH = cdt_both(col[hi * 32]), D = cdt_both(d);
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    // row y0 + i is d + i from lo and d + 7 - i from hi
-                    const uint32_t cl = (uint32_t)(2 * p) | ((uint32_t)(2 * p + 1) << 16);
-                    const uint32_t chh = (uint32_t)(7 - 2 * p) | ((uint32_t)(6 - 2 * p) << 16);
-                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, cl, VL));
-                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, chh, VH));
-                }
+            // two distances per stop test while both sides stay inside the axis (the second one is a true candidate
+            // whether or not it was still needed)
+            for (; d < mx && lo >= 1 && hi + 1 < n; d += 2, lo -= 2, hi += 2) {
+                const int a0 = col[lo * 32], a1 = col[(lo - 1) * 32], b0 = col[hi * 32], b1 = col[(hi + 1) * 32];
+                step(a0, b0, d);
+                step(a1, b1, d + 1);
                 mx = largest();
             }
             for (; d < mx && (lo >= 0 || hi < n); ++d, --lo, ++hi) {
-                const uint32_t VL = cdt_both(lo >= 0 ? (int)col[lo * 32] : kNone16);
-                const uint32_t VH = cdt_both(hi < n ? (int)col[hi * 32] : kNone16), D = cdt_both(d);
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    const uint32_t cl = (uint32_t)(2 * p) | ((uint32_t)(2 * p + 1) << 16);
-                    const uint32_t chh = (uint32_t)(7 - 2 * p) | ((uint32_t)(6 - 2 * p) << 16);
-                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, cl, VL));
-                    B[p] = __vminu2(B[p], __viaddmax_u16x2(D, chh, VH));
-                }
+                step(lo >= 0 ? (int)col[lo * 32] : kNone16, hi < n ? (int)col[hi * 32] : kNone16, d);
                 mx = largest();
             }
 #pragma unroll
