@@ -62,7 +62,7 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
     // The first two axes on 16-bit values (cdt.cuh): rows of a multiple of 32 up to 1024 voxels, a second axis of up
     // to 1024 rows whose stride is the row length.
     if (E >= 2 && axes[0] == ndim - 1 && g.ext[axes[0]] % 32 == 0 && g.ext[axes[0]] <= 1024 && g.ext[axes[1]] <= 1024 &&
-        ((uintptr_t)input & 31u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
+        ((uintptr_t)input & 31u) == 0 && ((uintptr_t)out_dist & 7u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
         const int n0 = (int)g.ext[axes[0]], n1 = (int)g.ext[axes[1]];
         Row16Params R;
         R.mask = input; R.out = reinterpret_cast<uint16_t*>(tmp[0]); R.rows = g.total / n0; R.words = n0 / 32;
@@ -71,20 +71,20 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
         Col16Params C;
         C.in = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1]; C.inner = n0; C.n = n1;
         const int strips = n0 / 32;
-        const size_t smem = (size_t)n1 * 64;
         const bool wide = n1 > 256;  // 16 warps per block on long axes
-        auto kern = wide ? (chess ? cdt_col16_kernel<true, 16> : cdt_col16_kernel<false, 16>)
-                         : (chess ? cdt_col16_kernel<true, 8> : cdt_col16_kernel<false, 8>);
+        const int nw = wide ? 16 : 8;
+        const size_t smem = (size_t)n1 * 64 + (chess ? (size_t)n1 * 8 + (size_t)nw * 64 : 0);
+        auto kern = wide ? (chess ? cdt_chess16_kernel<16, 16> : cdt_taxi16_kernel<16>) : (chess ? cdt_chess16_kernel<8, 8> : cdt_taxi16_kernel<8>);
         if (smem > 48 * 1024) {
             static bool raised[2][64];  // per kernel and device: the attribute is set once
             int dev = 0;
             cudaGetDevice(&dev);
             if (dev < 0 || dev >= 64 || !raised[chess][dev]) {
-                cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+                cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 74 * 1024);
                 if (dev >= 0 && dev < 64) raised[chess][dev] = true;
             }
         }
-        kern<<<(unsigned)(g.total / ((int64_t)n1 * n0) * strips), wide ? 512 : 256, smem, st>>>(C, strips);
+        kern<<<(unsigned)(g.total / ((int64_t)n1 * n0) * strips), 32 * nw, smem, st>>>(C, strips);
         e = cudaGetLastError();
         prev = C.out;
         k0 = 2;
