@@ -156,7 +156,9 @@ struct Row16Params {
     const uint8_t* mask;
     uint16_t* out;
     int64_t rows;
-    int words;  // 32-voxel words per row (1 .. 32)
+    int words;       // 32-voxel words per row (1 .. 32)
+    uint16_t* edge;  // optional (rows, nb, 2): the values of columns 128 k - 1 and 128 k, k = 1 .. nb, for the pinned columns
+    int nb;          // boundaries between groups of 128 columns (words / 4 rounded up, minus 1)
 };
 
 __device__ __forceinline__ uint32_t cdt_nonzero_bits4(uint32_t v) {
@@ -207,6 +209,10 @@ __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ 
     for (int i = 31; i >= 0; --i) {
         b = (z >> i) & 1u ? 0 : b + 1;
         d[i] = min(min(d[i], b), kNone16);
+    }
+    if (P.edge) {  // the last column of a group of 128 and the first one of the next group
+        if ((w & 3) == 3 && w + 1 < words) P.edge[(row * P.nb + (w >> 2)) * 2] = (uint16_t)d[31];
+        if ((w & 3) == 0 && w > 0) P.edge[(row * P.nb + (w >> 2) - 1) * 2 + 1] = (uint16_t)d[0];
     }
     uint16_t* dst = P.out + (row * words + w) * 32;
 #pragma unroll
@@ -459,6 +465,153 @@ __global__ void __launch_bounds__(32 * NW) cdt_chess16_kernel(const __grid_const
         const int hl = on ? (int)hd[y + 1] : kNone16, hr = on ? (int)hd[n + y + 1] : kNone16;
         const uint2 b = relax(prev, f, hl, hr);
         if (on) { put(y, b); prev = b; }
+    }
+}
+
+// ---- second axis as a streaming sweep (no shared-memory tile) ----
+// The same recurrences with the cut voxels computed by kernels of their own, so that the sweep itself only streams:
+// every 32nd row of the axis (and its last row) is pinned, for the chessboard metric also the two columns at every
+// boundary between groups of 128 columns.  cdt_pin_rows_kernel and cdt_pin_cols_kernel find their exact results by
+// bounded scans; cdt_sweep_kernel gives one warp a piece of 31 rows x 128 columns (a lane holds four neighbouring
+// columns as the halves of two registers): down from the pinned row above with the results kept in registers, then
+// up from the piece's own pinned row, writing the int32 output.  Taxicab: a(y) = min(f(y), a(y-1) + 1) needs no
+// neighbouring column and no pinned column.
+constexpr int kSegRows = 32;
+
+struct SweepParams {
+    const uint16_t* f;   // (slabs, n, inner): values of the first pass
+    const uint16_t* edge;// (slabs, n, groups - 1, 2): the same at columns 128 k - 1 and 128 k, written by the first pass
+    uint16_t* pd;        // (slabs, segs, inner): results of the pinned rows
+    uint16_t* hd;        // (slabs, groups - 1, 2, n): results of the pinned columns 128 k - 1 and 128 k
+    int32_t* out;
+    int64_t slabs;
+    int inner, n, segs, groups;
+    int last;            // last pass: "no background" becomes -1 (else kBig for the next pass)
+};
+
+// One lane per pair of neighbouring columns of a pinned row: a bounded outward scan along the axis through global
+// memory (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), four distances per stop test.
+template <bool CHESS>
+__global__ void __launch_bounds__(256) cdt_pin_rows_kernel(const __grid_constant__ SweepParams P) {
+    const int pairs = P.inner >> 1;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= P.slabs * P.segs * pairs) return;
+    const int x2 = (int)(t % pairs), k = (int)((t / pairs) % P.segs);
+    const int64_t slab = t / ((int64_t)pairs * P.segs);
+    const int n = P.n, y = min(n, (k + 1) * kSegRows) - 1;
+    const uint32_t* col = reinterpret_cast<const uint32_t*>(P.f + slab * (int64_t)n * P.inner) + x2;
+    const uint32_t none2 = cdt_both(kNone16);
+    uint32_t best = col[(int64_t)y * pairs];
+    int mx = (int)max(best & 0xffffu, best >> 16);
+    auto cand = [&](uint32_t v, int d) { return CHESS ? __vmaxu2(v, cdt_both(d)) : v + cdt_both(d); };
+    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); d += 4) {  // four distances per stop test: eight loads in flight
+        uint32_t a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            a[i] = y - d - i >= 0 ? col[(int64_t)(y - d - i) * pairs] : none2;
+            b[i] = y + d + i < n ? col[(int64_t)(y + d + i) * pairs] : none2;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) best = __vimin3_u16x2(best, cand(a[i], d + i), cand(b[i], d + i));
+        mx = (int)max(best & 0xffffu, best >> 16);
+    }
+    reinterpret_cast<uint32_t*>(P.pd)[t] = __vminu2(best, none2);
+}
+
+// One block per boundary between groups of 128 columns: the two columns beside it (gathered by the first pass) are
+// staged in shared memory and scanned eight rows per lane.
+__global__ void __launch_bounds__(256) cdt_pin_cols_kernel(const __grid_constant__ SweepParams P) {
+    extern __shared__ __align__(16) uint16_t sm_pc[];  // [2][n]
+    const int n = P.n, nb = P.groups - 1;
+    const int k = (int)(blockIdx.x % nb);
+    const int64_t slab = blockIdx.x / nb;
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(P.edge) + slab * (int64_t)n * nb + k;  // both columns of a row as one word
+#pragma unroll 4
+    for (int y = threadIdx.x; y < n; y += 256) {
+        const uint32_t v = src[(int64_t)y * nb];
+        sm_pc[y] = (uint16_t)(v & 0xffffu);
+        sm_pc[n + y] = (uint16_t)(v >> 16);
+    }
+    __syncthreads();
+    const int groups8 = (n + 7) >> 3;
+    uint16_t* dst = P.hd + (slab * nb + k) * 2 * (int64_t)n;
+    for (int t = threadIdx.x; t < 2 * groups8; t += 256) {
+        const int side = t >= groups8;
+        cdt_chess_scan8(sm_pc + side * n, (t - side * groups8) * 8, n, dst + side * n);
+    }
+}
+
+template <bool CHESS>
+__global__ void __launch_bounds__(128) cdt_sweep_kernel(const __grid_constant__ SweepParams P) {
+    const int lane = threadIdx.x & 31;
+    const int64_t gw = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (gw >= P.slabs * P.segs * P.groups) return;  // the whole warp
+    const int g = (int)(gw % P.groups), k = (int)((gw / P.groups) % P.segs);
+    const int64_t slab = gw / ((int64_t)P.groups * P.segs);
+    const int n = P.n, inner = P.inner, c = 128 * g + 4 * lane;
+    const bool act = c < inner;
+    const int y0 = k * kSegRows, rp = min(n, y0 + kSegRows) - 1, cnt = rp - y0;  // swept rows y0 .. rp - 1
+    const uint2 none2 = make_uint2(cdt_both(kNone16), cdt_both(kNone16));
+    const uint16_t* fcol = P.f + slab * (int64_t)n * inner + (act ? c : 0);
+    const uint16_t* pdk = P.pd + (slab * P.segs + k) * (int64_t)inner + (act ? c : 0);
+    const uint16_t* hl = CHESS && g > 0 ? P.hd + ((slab * (P.groups - 1) + g - 1) * 2 + 0) * (int64_t)n : nullptr;
+    const uint16_t* hr = CHESS && g + 1 < P.groups ? P.hd + ((slab * (P.groups - 1) + g) * 2 + 1) * (int64_t)n : nullptr;
+    int32_t* out = P.out + slab * (int64_t)n * inner + (act ? c : 0);
+    const int none_out = P.last ? -1 : kBig;
+    auto put = [&](int y, uint2 v) {
+        int r[4] = {(int)(v.x & 0xffffu), (int)(v.x >> 16), (int)(v.y & 0xffffu), (int)(v.y >> 16)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r[i] = r[i] >= kNone16 ? none_out : r[i];
+        if (act) *reinterpret_cast<int4*>(out + (int64_t)y * inner) = make_int4(r[0], r[1], r[2], r[3]);
+    };
+    // every row of the piece in flight at once
+    uint2 a[kSegRows - 1];
+#pragma unroll
+    for (int i = 0; i < kSegRows - 1; ++i)
+        a[i] = i < cnt && act ? *reinterpret_cast<const uint2*>(fcol + (int64_t)(y0 + i) * inner) : none2;
+    // results of the pinned columns beside the piece: lane i holds row y0 - 1 + i, row y0 + 31 apart
+    int hlv = kNone16, hrv = kNone16, hl_last = kNone16, hr_last = kNone16;
+    if (CHESS) {
+        const int yh = y0 - 1 + lane;
+        if (hl && yh >= 0 && yh < n) hlv = hl[yh];
+        if (hr && yh >= 0 && yh < n) hrv = hr[yh];
+        if (hl && y0 + 31 < n) hl_last = hl[y0 + 31];
+        if (hr && y0 + 31 < n) hr_last = hr[y0 + 31];
+    }
+    // one row of the recurrence: prev = the row before (after), ih = its place among the rows of the pinned columns
+    auto relax = [&](uint2 prev, uint2 f, int ih) {
+        uint2 r;
+        if (CHESS) {
+            uint32_t pl = __shfl_up_sync(0xffffffffu, prev.y, 1), pr = __shfl_down_sync(0xffffffffu, prev.x, 1);
+            const int l_edge = ih < 32 ? __shfl_sync(0xffffffffu, hlv, ih & 31) : hl_last;
+            const int r_edge = ih < 32 ? __shfl_sync(0xffffffffu, hrv, ih & 31) : hr_last;
+            if (lane == 0) pl = (uint32_t)l_edge << 16;
+            if (lane == 31) pr = (uint32_t)r_edge;
+            const uint32_t L0 = __byte_perm(pl, prev.x, 0x5432), M = __byte_perm(prev.x, prev.y, 0x5432), R1 = __byte_perm(prev.y, pr, 0x5432);
+            r.x = __viaddmin_u16x2(__vimin3_u16x2(L0, prev.x, M), 0x00010001u, f.x);
+            r.y = __viaddmin_u16x2(__vimin3_u16x2(M, prev.y, R1), 0x00010001u, f.y);
+        } else {
+            r.x = __viaddmin_u16x2(prev.x, 0x00010001u, f.x);
+            r.y = __viaddmin_u16x2(prev.y, 0x00010001u, f.y);
+        }
+        return act ? r : none2;  // lanes beyond the row stay "no background" for their neighbours
+    };
+    uint2 prev = act && k > 0 ? *reinterpret_cast<const uint2*>(pdk - inner) : none2;
+#pragma unroll
+    for (int i = 0; i < kSegRows - 1; ++i) {  // down from the pinned row above (row y0 + i - 1: place i)
+        if (i < cnt) {
+            a[i] = relax(prev, a[i], i);
+            prev = a[i];
+        }
+    }
+    prev = act ? *reinterpret_cast<const uint2*>(pdk) : none2;
+    put(rp, prev);
+#pragma unroll
+    for (int i = kSegRows - 2; i >= 0; --i) {  // up from the own pinned row (row y0 + i + 1: place i + 2)
+        if (i < cnt) {
+            prev = relax(prev, a[i], i + 2);
+            put(y0 + i, prev);
+        }
     }
 }
 

@@ -58,33 +58,38 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
     const int32_t* prev = nullptr;
     cudaError_t e = cudaSuccess;
     const bool chess = metric == TM_METRIC_CHESSBOARD;
-    int k0 = 0;
+    int k0 = 0, launches_fast = 0;
     // The first two axes on 16-bit values (cdt.cuh): rows of a multiple of 32 up to 1024 voxels, a second axis of up
     // to 1024 rows whose stride is the row length.
     if (E >= 2 && axes[0] == ndim - 1 && g.ext[axes[0]] % 32 == 0 && g.ext[axes[0]] <= 1024 && g.ext[axes[1]] <= 1024 &&
-        ((uintptr_t)input & 31u) == 0 && ((uintptr_t)out_dist & 7u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
+        ((uintptr_t)input & 31u) == 0 && ((uintptr_t)out_dist & 15u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
         const int n0 = (int)g.ext[axes[0]], n1 = (int)g.ext[axes[1]];
+        const int groups = (n0 + 127) / 128;
+        const int64_t slabs = g.total / ((int64_t)n1 * n0);
+        const int segs = (n1 + kSegRows - 1) / kSegRows;
+        // pinned results and the gathered boundary columns behind the 16-bit values in the first scratch image
+        char* extra = reinterpret_cast<char*>(tmp[0]) + (size_t)g.total * 2;
+        uint16_t* pd = reinterpret_cast<uint16_t*>(extra);
+        uint16_t* hd = reinterpret_cast<uint16_t*>(extra + (size_t)slabs * segs * n0 * 2);
+        uint16_t* edge = hd + (size_t)slabs * (groups - 1) * 2 * n1;
         Row16Params R;
         R.mask = input; R.out = reinterpret_cast<uint16_t*>(tmp[0]); R.rows = g.total / n0; R.words = n0 / 32;
+        R.edge = chess && groups > 1 ? edge : nullptr; R.nb = groups - 1;
         const int64_t warps = (R.rows + 32 / R.words - 1) / (32 / R.words);
         cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
-        Col16Params C;
-        C.in = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1]; C.inner = n0; C.n = n1;
-        const int strips = n0 / 32;
-        const bool wide = n1 > 256;  // 16 warps per block on long axes
-        const int nw = wide ? 16 : 8;
-        const size_t smem = (size_t)n1 * 64 + (chess ? (size_t)n1 * 8 + (size_t)nw * 64 : 0);
-        auto kern = wide ? (chess ? cdt_chess16_kernel<16, 16> : cdt_taxi16_kernel<16>) : (chess ? cdt_chess16_kernel<8, 8> : cdt_taxi16_kernel<8>);
-        if (smem > 48 * 1024) {
-            static bool raised[2][64];  // per kernel and device: the attribute is set once
-            int dev = 0;
-            cudaGetDevice(&dev);
-            if (dev < 0 || dev >= 64 || !raised[chess][dev]) {
-                cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 74 * 1024);
-                if (dev >= 0 && dev < 64) raised[chess][dev] = true;
-            }
-        }
-        kern<<<(unsigned)(g.total / ((int64_t)n1 * n0) * strips), 32 * nw, smem, st>>>(C, strips);
+        SweepParams C;
+        memset(&C, 0, sizeof(C));
+        C.f = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1];
+        C.slabs = slabs; C.inner = n0; C.n = n1; C.segs = segs; C.groups = groups;
+        C.pd = pd; C.hd = hd; C.edge = edge;
+        const int64_t pin_threads = C.slabs * C.segs * (n0 / 2);
+        if (chess) cdt_pin_rows_kernel<true><<<(unsigned)((pin_threads + 255) / 256), 256, 0, st>>>(C);
+        else cdt_pin_rows_kernel<false><<<(unsigned)((pin_threads + 255) / 256), 256, 0, st>>>(C);
+        if (chess && C.groups > 1) cdt_pin_cols_kernel<<<(unsigned)(C.slabs * (C.groups - 1)), 256, (size_t)n1 * 4, st>>>(C);
+        const int64_t pieces = C.slabs * C.segs * C.groups;
+        if (chess) cdt_sweep_kernel<true><<<(unsigned)((pieces + 3) / 4), 128, 0, st>>>(C);
+        else cdt_sweep_kernel<false><<<(unsigned)((pieces + 3) / 4), 128, 0, st>>>(C);
+        launches_fast = 3 + (chess && C.groups > 1 ? 1 : 0);
         e = cudaGetLastError();
         prev = C.out;
         k0 = 2;
@@ -123,7 +128,7 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
     }
     if (ws) cudaFreeAsync(ws, st);
     if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
-    tmedt::shared_record(-1, E);
+    tmedt::shared_record(-1, k0 ? launches_fast + E - 2 : E);
     return TM_EDT_OK;
 }
 
