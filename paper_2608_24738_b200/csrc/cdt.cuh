@@ -146,10 +146,9 @@ __global__ void __launch_bounds__(512) cdt_strip_kernel(const __grid_constant__ 
 }
 
 // ---- the first two axes on 16-bit values ----
-// Distances along two axes of up to 1024 voxels each stay below 2^14, so the first pass can hand 16-bit values to the
-// second one (half the scratch traffic) and the second pass holds a strip of 32 columns of an axis of 1024 rows in
-// 64 KB of shared memory.  "No background seen" is kNone16 and every value at or above it means the same (adding
-// distances to it stays below 2^16).
+// Distances along two axes of up to 1024 voxels each stay below 2^14, so the first pass hands 16-bit values to the
+// second one (half the scratch traffic), and the second pass runs as sweeps in registers (below).  "No background
+// seen" is kNone16 and every value at or above it means the same (adding distances to it stays below 2^16).
 constexpr int kNone16 = 0xC000;
 
 struct Row16Params {
@@ -226,94 +225,11 @@ __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ 
     }
 }
 
-struct Col16Params {
-    const uint16_t* in;  // values of the first pass, view (outer, n, inner); the allocation is read 2 bytes beyond both ends of a strip only inside a row
-    int32_t* out;
-    int64_t inner;       // a multiple of 32
-    int n;               // up to 1024
-    int last;            // last pass: "no background" becomes -1 (else kBig for the next pass)
-};
-
-// Second axis, taxicab metric, on a strip of (n x 32) 16-bit values in shared memory, lane = column, NW warps.
-// g(y) = min_j f(j) + |y - j| is two running minima, g = min(f, g_prev + 1), top to bottom and back.  Each warp runs
-// them over its own segment of rows; what reaches a segment from the rows before (after) it is the value at the end
-// of the previous (start of the next) segment plus the distance, combined over the segments in between.
-template <int NW>
-__global__ void __launch_bounds__(32 * NW) cdt_taxi16_kernel(const __grid_constant__ Col16Params P, const int strips_per_slab) {
-    extern __shared__ __align__(16) uint16_t sm_c16[];  // [n][32]
-    __shared__ int s_end[2][NW][32];
-    const int n = P.n;
-    const int64_t slab = blockIdx.x / strips_per_slab;
-    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
-    const int64_t base = slab * (int64_t)n * P.inner + c0;
-#pragma unroll 4
-    for (int t = threadIdx.x; t < n * 4; t += 32 * NW) {  // four lanes copy one row of 64 bytes
-        const int y = t >> 2, ch = t & 3;
-        *reinterpret_cast<int4*>(sm_c16 + y * 32 + 8 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 8 * ch);
-    }
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int32_t* out = P.out + base + lane;
-    const int none_out = P.last ? -1 : kBig;
-    const int S = (n + NW - 1) / NW;
-    const int y0 = min(n, warp * S), y1 = min(n, y0 + S);  // rows of this warp's segment
-    uint16_t* mine = sm_c16 + lane;
-    int f = kNone16;
-#pragma unroll 8
-    for (int y = y0; y < y1; ++y) {
-        f = min((int)mine[y * 32], f + 1);
-        mine[y * 32] = (uint16_t)f;
-    }
-    s_end[0][warp][lane] = f;
-    __syncthreads();
-    int cf = kNone16;  // value at the last row before the segment
-    for (int s = 0; s < warp; ++s) cf = min(s_end[0][s][lane], cf + (min(n, (s + 1) * S) - min(n, s * S)));
-    int b = kNone16;
-#pragma unroll 8
-    for (int y = y1 - 1; y >= y0; --y) {
-        b = min(min((int)mine[y * 32], cf + (y - y0 + 1)), b + 1);
-        mine[y * 32] = (uint16_t)b;
-    }
-    s_end[1][warp][lane] = b;
-    __syncthreads();
-    int cb = kNone16;  // value at the first row after the segment
-    for (int s = NW - 1; s > warp; --s) cb = min(s_end[1][s][lane], cb + (min(n, (s + 1) * S) - min(n, s * S)));
-#pragma unroll 8
-    for (int y = y0; y < y1; ++y) {
-        const int g = min((int)mine[y * 32], cb + (y1 - y));
-        out[(int64_t)y * P.inner] = g >= kNone16 ? none_out : g;
-    }
-}
-
-// g(y) = min_j max(col[j * stride], |y - j|) for one voxel: a bounded outward scan (a candidate d rows away is worth at
-// least d, so the scan ends once d reaches the minimum).
-__device__ __forceinline__ int cdt_chess_scan(const uint16_t* col, const int stride, const int y, const int n) {
-    int best = col[y * stride];
-    for (int d = 1; d < best && (y - d >= 0 || y + d < n); ++d) {
-        if (y - d >= 0) best = min(best, max((int)col[(y - d) * stride], d));
-        if (y + d < n) best = min(best, max((int)col[(y + d) * stride], d));
-    }
-    return best;
-}
-
 __device__ __forceinline__ uint32_t cdt_both(int v) { return (uint32_t)v * 0x00010001u; }  // v in both halves
 
-// The same for two neighbouring columns of row y at once (their values as the halves of one word, pitch words between
-// rows): the scan ends once d reaches the larger of the two minima.
-__device__ __forceinline__ uint32_t cdt_chess_scan2(const uint32_t* col, const int pitch, const int y, const int n) {
-    uint32_t best = col[y * pitch];
-    int mx = (int)max(best & 0xffffu, best >> 16);
-    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); ++d) {
-        const uint32_t D = cdt_both(d);
-        const uint32_t a = y - d >= 0 ? col[(y - d) * pitch] : cdt_both(kNone16), b = y + d < n ? col[(y + d) * pitch] : cdt_both(kNone16);
-        best = __vimin3_u16x2(best, __vmaxu2(a, D), __vmaxu2(b, D));
-        mx = (int)max(best & 0xffffu, best >> 16);
-    }
-    return best;
-}
-
-// The same for eight consecutive rows y0 .. y0 + 7 of a contiguous column (rows beyond n are left out): their minima
-// as four pairs of 16-bit halves, so that one candidate row serves all eight with two packed instructions per pair
+// g(y) = min_j max(col[j], |y - j|) for eight consecutive rows y0 .. y0 + 7 of a contiguous column (rows beyond n are
+// left out), by a bounded outward scan (a candidate d rows away is worth at least d, so the scan ends once d reaches
+// the largest of the minima): the minima as four pairs of 16-bit halves, so that one candidate row serves all eight with two packed instructions per pair
 // (max(f, d + offset) as one add-max, then a three-input minimum over both sides), two distances per stop test.
 __device__ __forceinline__ void cdt_chess_scan8(const uint16_t* col, const int y0, const int n, uint16_t* res) {
     int k[8];
@@ -367,115 +283,20 @@ __device__ __forceinline__ void cdt_chess_scan8(const uint16_t* col, const int y
         if (y0 + i < n) res[y0 + i] = (uint16_t)((B[i >> 1] >> (16 * (i & 1))) & 0xffffu);
 }
 
-// Second axis, chessboard metric, on the same strip.  g(y) = min_j max(f(j), |y - j|) has no running-minimum form
-// along a column alone (a farther row with a smaller value can take over again later), but because f is a distance
-// along the rows (it changes by at most 1 between neighbouring columns) the result obeys the two-sweep recurrence of
-// the chamfer transform across columns: down the rows, a(y, x) = min(f(y, x), 1 + min(a(y-1, x-1), a(y-1, x),
-// a(y-1, x+1))), then the same upwards starting from a.  A sweep needs its neighbours, so the kernel first computes
-// exact results by bounded scans for the voxels that cut the strip into independent pieces -- the last row of every
-// segment of n / SEGS rows and the two columns beside the strip (8 % of the voxels at 1024 rows) -- and pins them: every
-// shortest path from a background voxel to a voxel of a piece either stays inside the piece or crosses a pinned voxel,
-// whose exact value continues it.  Then (SEGS = 4 NW: every warp stays busy) eight lanes sweep a segment down from the pinned row above and up from the
-// segment's own pinned row: a lane holds four neighbouring columns as the halves of two registers, the columns beside
-// them come from the neighbouring lanes by shuffle and from the pinned columns at the ends.
-template <int NW, int SEGS>
-__global__ void __launch_bounds__(32 * NW) cdt_chess16_kernel(const __grid_constant__ Col16Params P, const int strips_per_slab) {
-    extern __shared__ __align__(16) uint16_t sm_c16[];  // [n][32] values, then hf[2][n], hd[2][n], pd[SEGS][32]
-    const int n = P.n;
-    uint16_t* hf = sm_c16 + n * 32;      // first-axis values of the columns left and right of the strip
-    uint16_t* hd = hf + 2 * n;           // their results
-    uint16_t* pd = hd + 2 * n;           // results of the pinned rows
-    const int64_t slab = blockIdx.x / strips_per_slab;
-    const int64_t c0 = (int64_t)(blockIdx.x - slab * strips_per_slab) * 32;
-    const int64_t base = slab * (int64_t)n * P.inner + c0;
-    const bool has_l = c0 > 0, has_r = c0 + 32 < P.inner;
-#pragma unroll 4
-    for (int t = threadIdx.x; t < n * 4; t += 32 * NW) {  // four lanes copy one row of 64 bytes
-        const int y = t >> 2, ch = t & 3;
-        *reinterpret_cast<int4*>(sm_c16 + y * 32 + 8 * ch) = *reinterpret_cast<const int4*>(P.in + base + (int64_t)y * P.inner + 8 * ch);
-    }
-    for (int y = threadIdx.x; y < n; y += 32 * NW) {
-        hf[y] = has_l ? P.in[base + (int64_t)y * P.inner - 1] : (uint16_t)kNone16;
-        hf[n + y] = has_r ? P.in[base + (int64_t)y * P.inner + 32] : (uint16_t)kNone16;
-    }
-    __syncthreads();
-    const int S = (n + SEGS - 1) / SEGS;   // rows per segment; the last row of a segment is pinned
-    const int segs = (n + S - 1) / S;  // segments that hold rows
-    // pinned columns: eight rows per lane; pinned rows: two neighbouring columns per lane
-    const int groups = (n + 7) >> 3, col_tasks = 2 * groups;
-    for (int t = threadIdx.x; t < col_tasks + segs * 16; t += 32 * NW) {
-        if (t < col_tasks) {
-            const int side = t >= groups, y0 = (t - side * groups) * 8;
-            if (side ? has_r : has_l) cdt_chess_scan8(hf + side * n, y0, n, hd + side * n);
-            else {
-                for (int i = 0; i < 8; ++i)
-                    if (y0 + i < n) hd[side * n + y0 + i] = (uint16_t)kNone16;
-            }
-        } else {
-            const int k = (t - col_tasks) >> 4, x2 = (t - col_tasks) & 15;
-            reinterpret_cast<uint32_t*>(pd)[k * 16 + x2] =
-                cdt_chess_scan2(reinterpret_cast<const uint32_t*>(sm_c16) + x2, 16, min(n, (k + 1) * S) - 1, n);
-        }
-    }
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int quarter = lane >> 3, l = lane & 7;  // eight lanes per segment, four columns per lane
-    const int seg = 4 * warp + quarter;
-    if (4 * warp >= segs) return;                 // the whole warp
-    const bool live = seg < segs;                 // lanes beyond the last segment stay for the shuffles
-    const int y0 = live ? seg * S : 0, rp = live ? min(n, y0 + S) - 1 : 0;
-    const int rows = __shfl_sync(0xffffffffu, rp - y0, 0);  // swept rows of a full segment (the first of a warp is never the shorter one)
-    const uint2 none2 = make_uint2(cdt_both(kNone16), cdt_both(kNone16));
-    const uint2* mine = reinterpret_cast<const uint2*>(sm_c16) + l;  // row pitch: 8 double words
-    uint2* mine_w = reinterpret_cast<uint2*>(sm_c16) + l;
-    const int none_out = P.last ? -1 : kBig;
-    int32_t* out = P.out + base + 4 * l;
-    auto put = [&](int y, uint2 v) {
-        int g[4] = {(int)(v.x & 0xffffu), (int)(v.x >> 16), (int)(v.y & 0xffffu), (int)(v.y >> 16)};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) g[i] = g[i] >= kNone16 ? none_out : g[i];
-        *reinterpret_cast<int4*>(out + (int64_t)y * P.inner) = make_int4(g[0], g[1], g[2], g[3]);
-    };
-    // one row of the recurrence: prev = the row before (after), hl / hr = its pinned neighbours beside the strip
-    auto relax = [&](uint2 prev, uint2 f, int hl, int hr) {
-        uint32_t pl = __shfl_up_sync(0xffffffffu, prev.y, 1, 8), pr = __shfl_down_sync(0xffffffffu, prev.x, 1, 8);
-        if (l == 0) pl = (uint32_t)hl << 16;
-        if (l == 7) pr = (uint32_t)hr;
-        const uint32_t L0 = __byte_perm(pl, prev.x, 0x5432), M = __byte_perm(prev.x, prev.y, 0x5432), R1 = __byte_perm(prev.y, pr, 0x5432);
-        uint2 r;
-        r.x = __viaddmin_u16x2(__vimin3_u16x2(L0, prev.x, M), 0x00010001u, f.x);
-        r.y = __viaddmin_u16x2(__vimin3_u16x2(M, prev.y, R1), 0x00010001u, f.y);
-        return r;
-    };
-    uint2 prev = live && y0 > 0 ? reinterpret_cast<const uint2*>(pd)[(seg - 1) * 8 + l] : none2;
-    for (int i = 0; i < rows; ++i) {  // down from the pinned row above
-        const int y = y0 + i;
-        const bool on = live && y < rp;
-        const uint2 f = on ? mine[y * 8] : none2;
-        const int hl = on && y > 0 ? (int)hd[y - 1] : kNone16, hr = on && y > 0 ? (int)hd[n + y - 1] : kNone16;
-        const uint2 a = relax(prev, f, hl, hr);
-        if (on) { mine_w[y * 8] = a; prev = a; }
-    }
-    prev = live ? reinterpret_cast<const uint2*>(pd)[seg * 8 + l] : none2;
-    if (live) put(rp, prev);
-    for (int i = 0; i < rows; ++i) {  // up from the own pinned row (a shorter last segment waits for its first rows)
-        const int y = y0 + rows - 1 - i;
-        const bool on = live && y < rp;
-        const uint2 f = on ? mine[y * 8] : none2;
-        const int hl = on ? (int)hd[y + 1] : kNone16, hr = on ? (int)hd[n + y + 1] : kNone16;
-        const uint2 b = relax(prev, f, hl, hr);
-        if (on) { put(y, b); prev = b; }
-    }
-}
-
-// ---- second axis as a streaming sweep (no shared-memory tile) ----
-// The same recurrences with the cut voxels computed by kernels of their own, so that the sweep itself only streams:
-// every 32nd row of the axis (and its last row) is pinned, for the chessboard metric also the two columns at every
-// boundary between groups of 128 columns.  cdt_pin_rows_kernel and cdt_pin_cols_kernel find their exact results by
-// bounded scans; cdt_sweep_kernel gives one warp a piece of 31 rows x 128 columns (a lane holds four neighbouring
-// columns as the halves of two registers): down from the pinned row above with the results kept in registers, then
-// up from the piece's own pinned row, writing the int32 output.  Taxicab: a(y) = min(f(y), a(y-1) + 1) needs no
-// neighbouring column and no pinned column.
+// ---- second axis as sweeps between pinned voxels ----
+// Taxicab: g(y) = min_j f(j) + |y - j| is two running minima, a(y) = min(f(y), a(y-1) + 1) down the rows and the same
+// upwards starting from a.  Chessboard: g(y) = min_j max(f(j), |y - j|) has no such form along a column alone (a
+// farther row with a smaller value can take over again later), but because f is a distance along the rows (it changes
+// by at most 1 between neighbouring columns) the result obeys the two-sweep recurrence of the chamfer transform across
+// columns: a(y, x) = min(f(y, x), 1 + min(a(y-1, x-1), a(y-1, x), a(y-1, x+1))) down the rows, then the same upwards.
+// A sweep over a whole axis is sequential, so the image is cut into pieces of 31 rows x 128 columns by voxels whose
+// exact results are computed first, by bounded scans (a candidate d rows away is worth at least d): every 32nd row of
+// the axis and its last row, and for the chessboard metric the two columns at every boundary between groups of 128
+// columns (cdt_pins_kernel; 3 % + 1.6 % of the voxels).  Every shortest path from a background voxel to a voxel of a
+// piece either stays inside the piece or crosses a pinned voxel, whose exact value continues it, so the pieces are
+// independent: cdt_sweep_kernel gives one warp a piece (a lane holds four neighbouring columns as the halves of two
+// registers), loads its 31 rows at once, sweeps down from the pinned row above with the results kept in registers
+// and up from the piece's own pinned row, writing the int32 output.  Work per voxel does not grow with the distances.
 constexpr int kSegRows = 32;
 
 struct SweepParams {
@@ -489,12 +310,11 @@ struct SweepParams {
     int last;            // last pass: "no background" becomes -1 (else kBig for the next pass)
 };
 
-// One lane per pair of neighbouring columns of a pinned row: a bounded outward scan along the axis through global
-// memory (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), four distances per stop test.
+// Pinned rows: one lane per pair of neighbouring columns, a bounded outward scan along the axis through global memory
+// (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), four distances per stop test.
 template <bool CHESS>
-__global__ void __launch_bounds__(256) cdt_pin_rows_kernel(const __grid_constant__ SweepParams P) {
+__device__ __forceinline__ void cdt_pin_rows(const SweepParams& P, const int64_t t) {
     const int pairs = P.inner >> 1;
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= P.slabs * P.segs * pairs) return;
     const int x2 = (int)(t % pairs), k = (int)((t / pairs) % P.segs);
     const int64_t slab = t / ((int64_t)pairs * P.segs);
@@ -504,7 +324,7 @@ __global__ void __launch_bounds__(256) cdt_pin_rows_kernel(const __grid_constant
     uint32_t best = col[(int64_t)y * pairs];
     int mx = (int)max(best & 0xffffu, best >> 16);
     auto cand = [&](uint32_t v, int d) { return CHESS ? __vmaxu2(v, cdt_both(d)) : v + cdt_both(d); };
-    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); d += 4) {  // four distances per stop test: eight loads in flight
+    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); d += 4) {  // eight loads in flight
         uint32_t a[4], b[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -518,13 +338,20 @@ __global__ void __launch_bounds__(256) cdt_pin_rows_kernel(const __grid_constant
     reinterpret_cast<uint32_t*>(P.pd)[t] = __vminu2(best, none2);
 }
 
-// One block per boundary between groups of 128 columns: the two columns beside it (gathered by the first pass) are
-// staged in shared memory and scanned eight rows per lane.
-__global__ void __launch_bounds__(256) cdt_pin_cols_kernel(const __grid_constant__ SweepParams P) {
-    extern __shared__ __align__(16) uint16_t sm_pc[];  // [2][n]
+// Blocks below row_blocks take 256 lanes of the pinned rows each; every further block takes one boundary between
+// groups of 128 columns (chessboard only): the two columns beside it (gathered by the first pass) are staged in shared
+// memory and scanned eight rows per lane.
+template <bool CHESS>
+__global__ void __launch_bounds__(256) cdt_pins_kernel(const __grid_constant__ SweepParams P, const unsigned row_blocks) {
+    extern __shared__ __align__(16) uint16_t sm_pc[];  // [2][n] (column blocks)
+    if (blockIdx.x < row_blocks) {
+        cdt_pin_rows<CHESS>(P, (int64_t)blockIdx.x * 256 + threadIdx.x);
+        return;
+    }
     const int n = P.n, nb = P.groups - 1;
-    const int k = (int)(blockIdx.x % nb);
-    const int64_t slab = blockIdx.x / nb;
+    const unsigned cb = blockIdx.x - row_blocks;
+    const int k = (int)(cb % nb);
+    const int64_t slab = cb / nb;
     const uint32_t* src = reinterpret_cast<const uint32_t*>(P.edge) + slab * (int64_t)n * nb + k;  // both columns of a row as one word
 #pragma unroll 4
     for (int y = threadIdx.x; y < n; y += 256) {

@@ -82,14 +82,14 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
         C.f = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1];
         C.slabs = slabs; C.inner = n0; C.n = n1; C.segs = segs; C.groups = groups;
         C.pd = pd; C.hd = hd; C.edge = edge;
-        const int64_t pin_threads = C.slabs * C.segs * (n0 / 2);
-        if (chess) cdt_pin_rows_kernel<true><<<(unsigned)((pin_threads + 255) / 256), 256, 0, st>>>(C);
-        else cdt_pin_rows_kernel<false><<<(unsigned)((pin_threads + 255) / 256), 256, 0, st>>>(C);
-        if (chess && C.groups > 1) cdt_pin_cols_kernel<<<(unsigned)(C.slabs * (C.groups - 1)), 256, (size_t)n1 * 4, st>>>(C);
+        const int64_t row_blocks = (C.slabs * C.segs * (n0 / 2) + 255) / 256;
+        const int64_t col_blocks = chess ? C.slabs * (groups - 1) : 0;
+        if (chess) cdt_pins_kernel<true><<<(unsigned)(row_blocks + col_blocks), 256, (size_t)n1 * 4, st>>>(C, (unsigned)row_blocks);
+        else cdt_pins_kernel<false><<<(unsigned)row_blocks, 256, 0, st>>>(C, (unsigned)row_blocks);
         const int64_t pieces = C.slabs * C.segs * C.groups;
         if (chess) cdt_sweep_kernel<true><<<(unsigned)((pieces + 3) / 4), 128, 0, st>>>(C);
         else cdt_sweep_kernel<false><<<(unsigned)((pieces + 3) / 4), 128, 0, st>>>(C);
-        launches_fast = 3 + (chess && C.groups > 1 ? 1 : 0);
+        launches_fast = 3;
         e = cudaGetLastError();
         prev = C.out;
         k0 = 2;
