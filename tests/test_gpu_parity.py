@@ -64,6 +64,7 @@ SMALL = [
     (2, 1, 3, 2, 3, 2, 3, 2, 3, 4), (1, 1, 6, 6, 6, 6, 6, 6, 6, 6),
     (1, 1, 128, 128), (2, 1, 127, 128), (1, 1, 128, 100), (1, 2, 50, 128, 64), (1, 1, 128, 20, 48),
     (1, 1, 16, 40, 24, 32), (1, 1, 5, 6, 20, 7, 16), (1, 1, 3, 128, 1, 128),
+    (2, 1, 3, 9, 5, 8), (1, 2, 20, 6, 7, 12), (2, 1, 2, 128, 4, 36),  # four axes on the quad kernels
     (2, 1, 200, 256), (1, 1, 129, 144), (1, 1, 300, 16), (1, 2, 512, 48), (1, 1, 1, 40, 1, 160),
     (1, 1, 1024, 48), (1, 1, 40, 1024), (2, 1, 600, 528), (1, 1, 513, 1008),
     (1, 1, 130, 48, 160), (1, 2, 20, 200, 64), (2, 1, 512, 6, 16), (1, 1, 9, 16, 512), (1, 1, 140, 1, 33, 1, 48),
