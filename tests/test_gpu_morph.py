@@ -108,7 +108,8 @@ QUAD_BOXES = [((2, 1, 19, 24), (3, 3), None), ((1, 2, 11, 12, 16), (3, 3, 3), No
               ((1, 1, 67, 260), (5, 5), None), ((2, 1, 37, 140), (7, 7), None), ((1, 1, 35, 8), (9, 9), None),
               ((1, 1, 2, 4), (9, 9), None), ((1, 1, 3, 300), (7, 3), None), ((1, 1, 130, 12), (3, 1), None),
               ((1, 1, 21, 12), (1, 9), None), ((1, 1, 5, 3, 12), (7, 5, 3), None), ((1, 1, 66, 9, 8), (9, 1, 1), None),
-              ((2, 1, 18, 17, 36), (5, 5, 5), None), ((1, 1, 1, 1, 4), (3, 3, 3), None),
+              ((2, 1, 18, 17, 36), (5, 5, 5), None), ((1, 1, 1, 1, 4), (3, 3, 3), None), ((1, 2, 9, 21, 132), (3, 3, 3), None),
+              ((1, 1, 13, 10, 260), (7, 7, 7), None), ((1, 1, 5, 9, 8), (9, 9, 9), None), ((2, 1, 3, 10, 11, 40), (3, 3, 3, 3), None),
               ((1, 1, 9, 10, 4), (4, 2, 1), (1, 0, 0)), ((1, 1, 6, 33, 8), (2, 6, 3), (0, -2, 0)), ((2, 1, 140, 260), (3, 7), (1, 0))]
 
 
