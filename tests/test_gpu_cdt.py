@@ -56,6 +56,47 @@ def test_cdt_matches_scipy_on_a_larger_image():
             assert np.array_equal(got[b, 0], ndi.distance_transform_cdt(mask[b, 0], metric=metric))
 
 
+def test_cdt_at_the_benchmark_shape_against_scipy():
+    """Two images of the benchmark's 1024^2 disk workload (32 pinned rows, 8 groups of 128 columns per image) and a
+    volume whose third axis follows the two 16-bit passes."""
+    import torch
+
+    ndi = pytest.importorskip("scipy.ndimage")
+    mask = workloads.config2(batch=2, size=1024, disks=80).mask
+    vol = workloads.random_mask(77, (1, 1, 70, 100, 160), 0.97)
+    for metric in ("taxicab", "chessboard"):
+        got = binding.tm_cdt(torch.from_numpy(mask).cuda(), metric).cpu().numpy()
+        for b in range(2):
+            assert np.array_equal(got[b, 0], ndi.distance_transform_cdt(mask[b, 0], metric=metric))
+        got = binding.tm_cdt(torch.from_numpy(vol).cuda(), metric).cpu().numpy()
+        assert np.array_equal(got[0, 0], ndi.distance_transform_cdt(vol[0, 0], metric=metric))
+
+
+@pytest.mark.parametrize("metric", ["taxicab", "chessboard"])
+def test_cdt_structured_masks_on_the_sweep_path(metric):
+    """Masks that stress the pinned rows / columns and the sweeps between them: one background voxel (scans and sweeps
+    over the whole image), a background line, stripes of period 64 along either axis, a checkerboard of 48-voxel
+    squares, and a batch whose second image has no background at all."""
+    import torch
+
+    shape = (2, 1, 200, 288)
+    yy, xx = np.meshgrid(np.arange(shape[2]), np.arange(shape[3]), indexing="ij")
+    cases = []
+    one = np.ones(shape, dtype=np.uint8); one[0, 0, 199, 0] = 0; one[1, 0, 77, 131] = 0
+    cases.append(one)
+    line = np.ones(shape, dtype=np.uint8); line[0, 0, :, 130] = 0; line[1, 0, 63, :] = 0
+    cases.append(line)
+    stripes = np.ones(shape, dtype=np.uint8); stripes[0, 0][yy % 64 == 31] = 0; stripes[1, 0][xx % 64 == 0] = 0
+    cases.append(stripes)
+    board = np.ones(shape, dtype=np.uint8); board[:, 0] = (((yy // 48) + (xx // 48)) % 2).astype(np.uint8)
+    cases.append(board)
+    nobg = np.ones(shape, dtype=np.uint8); nobg[0, 0, 100, 100] = 0
+    cases.append(nobg)
+    for mask in cases:
+        got = binding.tm_cdt(torch.from_numpy(mask).cuda(), metric).cpu().numpy()
+        assert np.array_equal(got, co.separable(mask, metric))
+
+
 BF_SHAPES = [(2, 1, 40), (2, 2, 17, 23), (1, 1, 9, 10, 11), (1, 1, 4, 5, 3, 6), (1, 1, 30, 40)]
 
 
