@@ -665,7 +665,6 @@ static cudaError_t launch_wide_axis(const WideAxisParams& A, const EpilogueParam
 
 static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st,
                               int& launches) {
-    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* w = static_cast<char*>(ws);
     const WideLayout L = wide_layout(pl.N, pl.E, ep.idx != nullptr, false);
     uint32_t* keysA = reinterpret_cast<uint32_t*>(w + L.keysA);
