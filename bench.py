@@ -523,6 +523,77 @@ def run_cdt(args):
                       "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"], "cases": cases}), flush=True)
 
 
+def run_ex(args):
+    """Measurement of the tm_edt_ex variants (a later row of the scope): flat index output on workload C4, float64
+    distances, a strided (z-fastest) mask gathered by the library and the virtual-background convention on workload
+    C3, each beside the default call on the same mask.  HBM roofline = the unavoidable bytes of the variant."""
+    import numpy as np
+    import torch
+
+    from paper_2608_24738_b200 import binding, buildlib, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    buildlib.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak_gbs()
+    stream = torch.cuda.current_stream()
+    steps = max(20, args.steps // 2)
+
+    def timed(call):
+        for _ in range(max(3, args.warmup)):
+            call()
+        torch.cuda.synchronize()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in evs:
+            a.record(stream)
+            call()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in evs)
+
+    c3, c4 = workloads.config3(), workloads.config4()
+    m3, m4 = torch.from_numpy(c3.mask).to(dev), torch.from_numpy(c4.mask).to(dev)
+    n3, n4 = c3.mask.size, c4.mask.size
+    cases = []
+
+    def add(name, mask_t, nvox, bpv, ms, base_ms, note):
+        gbs = nvox * bpv / (ms * 1e-3) / 1e9
+        cases.append({"case": name, "shape": list(mask_t.shape), "ms_per_step": ms, "default_call_ms": base_ms,
+                      "value": nvox / (ms * 1e-3) / 1e9, "unit": "Gvoxel/s", "note": note,
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                   "peak_kind": peak_kind + " copy bandwidth", "bytes_per_voxel": bpv}})
+
+    # workload C4: coordinate planes (the default) against one linear index per voxel
+    d4 = torch.empty(c4.mask.shape, dtype=torch.float32, device=dev)
+    x4 = torch.empty(c4.mask.shape[:2] + (4,) + c4.mask.shape[2:], dtype=torch.int64, device=dev)
+    f4 = torch.empty(c4.mask.shape, dtype=torch.int64, device=dev)
+    base4 = timed(lambda: binding.tm_edt(m4, None, distances=d4, indices=x4, return_indices=True))
+    ms = timed(lambda: binding.tm_edt(m4, None, distances=d4, indices=f4, return_indices=True, flat_index=True))
+    add("c4_flat_index", m4, n4, 13, ms, base4, "dist f32 + one int64 linear index per voxel")
+    del x4, f4
+    # workload C3: float64 distances, a z-fastest mask, the virtual-background convention
+    d3 = torch.empty(c3.mask.shape, dtype=torch.float32, device=dev)
+    base3 = timed(lambda: binding.tm_edt(m3, c3.sampling, distances=d3))
+    d64 = torch.empty(c3.mask.shape, dtype=torch.float64, device=dev)
+    ms = timed(lambda: binding.tm_edt(m3, c3.sampling, distances=d64, dist_f64=True))
+    add("c3_dist_f64", m3, n3, 9, ms, base3, "float64 distances recomputed from the sites")
+    zfast = m3.permute(0, 1, 4, 3, 2).contiguous().permute(0, 1, 4, 3, 2)  # same values, z varies fastest in memory
+    ms = timed(lambda: binding.tm_edt(zfast, c3.sampling, distances=d3, keep_strides=True))
+    add("c3_strided_z_fastest", m3, n3, 5, ms, base3, "byte strides passed, gathered by the library")
+    vb = m3.clone()
+    vb[-1, -1] = 1  # one image without background
+    ms = timed(lambda: binding.tm_edt(vb, c3.sampling, distances=d3, virtual_background=True))
+    add("c3_virtual_background", m3, n3, 5, ms, base3, "one of 16 images without background")
+    head = cases[0]
+    print(json.dumps({"metric": "edt_ex_gvoxels_per_s", "value": head["value"], "unit": "Gvoxel/s", "n_gpus": 1,
+                      "steps": steps, "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_step"],
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": head["case"], "shape": head["shape"]}, "gpu_launches": binding.tm_edt_last_launch_count() * steps,
+                      "roofline": head["roofline"], "cases": cases}), flush=True)
+
+
 def run_long(args):
     """Measurement of the paths for extents beyond 128 (wide-key and long-line kernels; a later row of the scope, its
     own line): the paper's 2-D 1024^2 row at B = 8, one 4096^2 image and one 512^3 volume; blob masks (disks / balls as
@@ -631,13 +702,16 @@ def main():
     ap.add_argument("--outputs", default=None, help="override the requested outputs, e.g. dist,idx or dist,sq,idx")
     ap.add_argument("--flat-index", action="store_true",
                     help="index output as one linear index per voxel (variant of tm_edt_ex; not the headline layout)")
-    ap.add_argument("--workload", default="edt", choices=["edt", "morph", "cdt", "long"],
-                    help="edt: the headline benchmark; long: the same transform on extents beyond 128 (1024^2, 4096^2, 512^3); morph / cdt: the erosion-dilation kernels and the taxicab / chessboard / brute-force transforms (their own metrics)")
+    ap.add_argument("--workload", default="edt", choices=["edt", "morph", "cdt", "long", "ex"],
+                    help="edt: the headline benchmark; long: the same transform on extents beyond 128 (1024^2, 4096^2, 512^3); ex: the tm_edt_ex variants (flat index, float64 distances, strided mask, virtual background); morph / cdt: the erosion-dilation kernels and the taxicab / chessboard / brute-force transforms (their own metrics)")
     ap.add_argument("--morph-case", default=None, help="with --workload morph: run only this case (profiling aid)")
     ap.add_argument("--images", type=int, default=0, help="use only the first K images of the workload (profiling aid)")
     args = ap.parse_args()
     if args.workload == "morph":
         run_morph(args)
+        return
+    if args.workload == "ex":
+        run_ex(args)
         return
     if args.workload == "cdt":
         run_cdt(args)

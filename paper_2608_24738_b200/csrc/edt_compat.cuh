@@ -25,12 +25,13 @@ __device__ __forceinline__ bool image_marked_empty(const EpilogueParams& ep, int
 }
 
 __device__ __forceinline__ void virtual_fill(const VirtualParams& P, const EpilogueParams& ep, int64_t img, int64_t vox) {
-    int64_t rr = vox;
+    uint32_t rr = (uint32_t)vox;  // an image has fewer than 2^31 voxels
     double h = 0.0;
     int64_t s = 0;
     for (int a = P.ndim - 1; a >= 0; --a) {
-        int64_t x = rr % P.shape[a];
-        rr /= P.shape[a];
+        const uint32_t n = (uint32_t)P.shape[a], q = rr / n;
+        int64_t x = rr - q * n;
+        rr = q;
         if (a == 0) x += 1;
         const double t = P.w[a] * (double)x;
         h += t * t;
@@ -44,14 +45,19 @@ __device__ __forceinline__ void virtual_fill(const VirtualParams& P, const Epilo
         for (int a = 0; a < P.ndim; ++a) ep.idx[(img * P.ndim + a) * P.V + vox] = a == 0 ? -1 : 0;
 }
 
-// every voxel but voxel 0 of each image
+// every voxel but voxel 0 of each image: a block takes kVirtualChunk voxels of one image and leaves at once unless
+// the image is marked empty
+constexpr int kVirtualChunk = 256 * 8;
 __global__ void __launch_bounds__(256) virtual_background_kernel(const __grid_constant__ VirtualParams P,
-                                                                 const __grid_constant__ EpilogueParams ep) {
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= P.images * P.V) return;
-    const int64_t img = t / P.V, vox = t - img * P.V;
-    if (vox == 0 || !image_marked_empty(ep, img)) return;
-    virtual_fill(P, ep, img, vox);
+                                                                 const __grid_constant__ EpilogueParams ep,
+                                                                 const unsigned chunks_per_image) {
+    const int64_t img = blockIdx.x / chunks_per_image;
+    if (!image_marked_empty(ep, img)) return;
+    const int64_t v0 = (int64_t)(blockIdx.x - img * chunks_per_image) * kVirtualChunk;
+    for (int i = threadIdx.x; i < kVirtualChunk; i += 256) {
+        const int64_t vox = v0 + i;
+        if (vox != 0 && vox < P.V) virtual_fill(P, ep, img, vox);
+    }
 }
 
 // voxel 0 of each image
@@ -112,24 +118,28 @@ __global__ void __launch_bounds__(256) gather_strided_kernel(const __grid_consta
 // the transform: coordinate planes (images, ndim, V) or one linear index per voxel (flat).  A negative linear
 // index, or -1 in the last coordinate plane, marks an image without background (+inf) unless the virtual-background
 // convention is on, where it names the virtual voxel (-1, 0, .., 0).
+// Blocks enumerate (image, 256 voxels of it); an image has fewer than 2^31 voxels, so positions inside it are split
+// with 32-bit divisions.
 __global__ void __launch_bounds__(256) dist_f64_kernel(const __grid_constant__ VirtualParams P, const int64_t* idx,
-                                                       const int flat, const int virtual_bg, double* out) {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= P.images * P.V) return;
-    const int64_t img = e / P.V, vox = e - img * P.V;
-    int64_t rr = vox;
-    int64_t fs = flat ? idx[e] : 0;
-    const bool neg = flat ? fs < 0 : idx[(img * P.ndim + (P.ndim - 1)) * P.V + vox] == -1 && !virtual_bg;
+                                                       const int flat, const int virtual_bg, double* out,
+                                                       const unsigned blocks_per_image) {
+    const int64_t img = blockIdx.x / blocks_per_image;
+    const uint32_t vox = (blockIdx.x - (uint32_t)img * blocks_per_image) * 256u + threadIdx.x;
+    if ((int64_t)vox >= P.V) return;
+    const int64_t e = img * P.V + vox;
+    const int64_t fs64 = flat ? idx[e] : 0;
+    const bool neg = flat ? fs64 < 0 : idx[(img * P.ndim + (P.ndim - 1)) * P.V + vox] == -1 && !virtual_bg;
     if (neg && !virtual_bg) { out[e] = __longlong_as_double(0x7ff0000000000000ll); return; }
+    uint32_t rr = vox, fs = (uint32_t)fs64;
     double h = 0.0;
     for (int a = P.ndim - 1; a >= 0; --a) {
-        const int64_t q = rr / P.shape[a];
-        const int64_t x = rr - q * P.shape[a];
+        const uint32_t n = (uint32_t)P.shape[a], q = rr / n;
+        const int x = (int)(rr - q * n);
         rr = q;
-        int64_t sa;
-        if (!flat) sa = idx[(img * P.ndim + a) * P.V + vox];
+        int sa;
+        if (!flat) sa = (int)idx[(img * P.ndim + a) * P.V + vox];
         else if (neg) sa = a == 0 ? -1 : 0;
-        else { const int64_t qs = fs / P.shape[a]; sa = fs - qs * P.shape[a]; fs = qs; }
+        else { const uint32_t qs = fs / n; sa = (int)(fs - qs * n); fs = qs; }
         const double t = P.w[a] * (double)(x - sa);
         h += t * t;
     }

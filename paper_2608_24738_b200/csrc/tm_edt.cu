@@ -937,10 +937,10 @@ static int run_device(const Plan& pl, const uint8_t* input, float* out_dist, int
         VP.stride0 = pl.V / pl.shape_sp[0];
         EpilogueParams ep;
         fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
-        const int64_t max_items = (int64_t)INT32_MAX * 128;  // grid limit with 256 threads per block
-        if (pl.N > max_items) return TM_EDT_ERR_UNSUPPORTED;
+        const int64_t cpi = (pl.V + kVirtualChunk - 1) / kVirtualChunk;
+        if (pl.images * cpi > (int64_t)INT32_MAX) return TM_EDT_ERR_UNSUPPORTED;
         prof_mark(st, "virtual_background", 0.0);
-        virtual_background_kernel<<<(unsigned)((pl.N + 255) / 256), 256, 0, st>>>(VP, ep);
+        virtual_background_kernel<<<(unsigned)(pl.images * cpi), 256, 0, st>>>(VP, ep, (unsigned)cpi);
         virtual_background_first_kernel<<<(unsigned)((pl.images + 255) / 256), 256, 0, st>>>(VP, ep);
         launches += 2;
         cudaError_t e = cudaGetLastError();
@@ -1133,16 +1133,17 @@ int tm_edt_ex(const uint8_t* input, int ndim, const int64_t* shape, const int64_
             if (!site) { site = reinterpret_cast<int64_t*>(ws + L.core + L.mask); p2.flags |= TM_EDT_FLAG_FLAT_INDEX; }
             rc = run_device(p2, mask, nullptr, out_sqdist, site, ws, st);
             if (rc == TM_EDT_OK) {
-                if (pl.N > (int64_t)INT32_MAX * 128) rc = TM_EDT_ERR_UNSUPPORTED;
+                const int64_t bpi = (pl.V + 255) / 256;  // blocks per image
+                if (pl.images * bpi > (int64_t)INT32_MAX) rc = TM_EDT_ERR_UNSUPPORTED;
                 else {
                     VirtualParams VP;
                     memset(&VP, 0, sizeof(VP));
                     VP.images = pl.images; VP.V = pl.V; VP.ndim = pl.ndim;
                     for (int a = 0; a < pl.ndim; ++a) { VP.shape[a] = pl.shape_sp[a]; VP.w[a] = pl.w_sp[a]; }
                     prof_mark(st, "dist_f64", (double)pl.N * (8.0 + 8.0 * ((p2.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : pl.ndim)));
-                    dist_f64_kernel<<<(unsigned)((pl.N + 255) / 256), 256, 0, st>>>(
+                    dist_f64_kernel<<<(unsigned)(pl.images * bpi), 256, 0, st>>>(
                         VP, site, (p2.flags & TM_EDT_FLAG_FLAT_INDEX) ? 1 : 0, (flags & TM_EDT_FLAG_VIRTUAL_BACKGROUND) ? 1 : 0,
-                        static_cast<double*>(out_dist));
+                        static_cast<double*>(out_dist), (unsigned)bpi);
                     ++extra_launches;
                     cudaError_t e = cudaGetLastError();
                     if (e != cudaSuccess) { g_last_cuda_error = (int)e; rc = TM_EDT_ERR_CUDA; }
