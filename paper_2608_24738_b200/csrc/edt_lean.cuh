@@ -311,6 +311,49 @@ __device__ __forceinline__ void lean_emit_final(const uint32_t (&b)[4], const ui
     }
 }
 
+// The same with one linear index per voxel (the site's row-major position inside its image) instead of coordinate
+// planes: the quad's own position p + v, moved by the entry's offsets along the K earlier planes (strides ps[q]) and by
+// the site row along this axis (own row y, stride inner).
+template <int K>
+__device__ __forceinline__ void lean_emit_flat(const uint32_t (&b)[4], const uint32_t (&e)[4], float* __restrict__ dist,
+                                               int64_t* __restrict__ sq, int64_t* __restrict__ lin, const uint32_t p,
+                                               const int y, const int inner, const int (&ps)[K]) {
+    const uint32_t any = b[0] | b[1] | b[2] | b[3], every = b[0] & b[1] & b[2] & b[3];
+    if ((any & kLeanNone) == 0u) {
+        if (dist) {
+            float4 d;
+            d.x = fast_sqrt(small_int_to_float((int)(b[0] >> 8))); d.y = fast_sqrt(small_int_to_float((int)(b[1] >> 8)));
+            d.z = fast_sqrt(small_int_to_float((int)(b[2] >> 8))); d.w = fast_sqrt(small_int_to_float((int)(b[3] >> 8)));
+            __stcs(reinterpret_cast<float4*>(dist + p), d);
+        }
+        if (sq) lean_store_4xi64(sq + p, b[0] >> 8, b[1] >> 8, b[2] >> 8, b[3] >> 8);
+        uint32_t s[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            int at = (int)p + v + ((int)(b[v] & 0xffu) - y) * inner;
+#pragma unroll
+            for (int q = 0; q < K; ++q) at += lean_sext_byte(e[v], q) * ps[q];
+            s[v] = (uint32_t)at;
+        }
+        lean_store_4xi64(lin + p, s[0], s[1], s[2], s[3]);
+    } else if ((every & kLeanNone) != 0u) {  // an image without background: +inf, INT64_MAX, -1
+        if (dist) __stcs(reinterpret_cast<float4*>(dist + p), make_float4(TMEDT_INF, TMEDT_INF, TMEDT_INF, TMEDT_INF));
+        if (sq) lean_store_4xi64_same(sq + p, 0xffffffffu, 0x7fffffffu);
+        lean_store_4xi64_same(lin + p, 0xffffffffu, 0xffffffffu);
+    } else {  // cannot happen inside one image; kept voxel by voxel
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const bool none = b[v] >= kLeanNone;
+            if (dist) dist[p + v] = none ? TMEDT_INF : fast_sqrt(small_int_to_float((int)(b[v] >> 8)));
+            if (sq) sq[p + v] = none ? INT64_MAX : (int64_t)(b[v] >> 8);
+            int at = (int)p + v + ((int)(b[v] & 0xffu) - y) * inner;
+#pragma unroll
+            for (int q = 0; q < K; ++q) at += lean_sext_byte(e[v], q) * ps[q];
+            lin[p + v] = none ? (int64_t)-1 : (int64_t)at;
+        }
+    }
+}
+
 // Own coordinates along the K earlier planes of position v0 (plane 0 fastest).
 template <int K>
 __device__ __forceinline__ void lean_decode(uint32_t v0, const LeanParams& P, const EpilogueParams& ep, int (&cq)[K]) {
@@ -391,10 +434,27 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
         }
         return;
     }
-    int cq[K];
-    lean_decode<K>(v0, P, ep, cq);
     float* const dist = ep.dist ? ep.dist + slab * ep.V : nullptr;
     int64_t* const sq = ep.sq ? ep.sq + slab * ep.V : nullptr;
+    if (ep.flat) {  // one linear index per voxel
+        int ps[K];
+#pragma unroll
+        for (int q = 0; q < K; ++q) ps[q] = (int)ep.pstride[q];
+        int64_t* const lin = ep.idx + slab * ep.V;
+        for (int y = yfirst; y < n; y += YSTEP) {
+            uint32_t b[4], e[4];
+            if (any_site) lean_scan<TX, 8>(T, kt + (y + kLeanPad) * TX + c4, y, n, 1u, b);
+            else b[0] = b[1] = b[2] = b[3] = kLeanNone;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) e[v] = (uint32_t)et[(TM_EDT_IN_RANGE(b[v] & 0xffu, n, 126) ? (b[v] & 0xffu) : 0u) * TX + c4 + v];
+            const uint32_t p = (uint32_t)y * (uint32_t)P.inner + v0;  // inside one image: below 2^31
+            if (TM_EDT_IN_RANGE(p, ep.V - 3, 127) && TM_EDT_IN_RANGE(slab, P.images, 128))
+                lean_emit_flat<K>(b, e, dist, sq, lin, p, y, (int)P.inner, ps);
+        }
+        return;
+    }
+    int cq[K];
+    lean_decode<K>(v0, P, ep, cq);
     int64_t* ip[K + 1];
 #pragma unroll
     for (int q = 0; q <= K; ++q) ip[q] = ep.idx + (slab * ep.ndim + ep.axis[q]) * ep.V;

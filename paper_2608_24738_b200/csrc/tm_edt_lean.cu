@@ -36,11 +36,11 @@ cudaError_t ensure_smem(const void* fn, size_t smem) {
 
 // Quad-per-lane kernels (edt_lean.cuh) for the shapes they cover: three or four processed axes, contiguous extent a
 // multiple of 4, outputs aligned for 16-byte (float32) and 32-byte (int64) stores, exact integer keys (unit sampling, or scaled integers without index output),
-// coordinate index layout with every spatial axis processed.
+// index output (coordinate planes or one linear index per voxel) with every spatial axis processed.
 bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep) {
     if (!pl.fast || pl.E < 3 || pl.E > 4 || pl.ext[0] % 4 != 0 || ((uintptr_t)in & 3u) != 0) return false;
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u) || ((uintptr_t)ep.idx & 31u)) return false;
-    if (ep.idx) return pl.unit && pl.ndim == pl.E && !ep.flat;
+    if (ep.idx) return pl.unit && pl.ndim == pl.E;
     return pl.unit || pl.scaled;
 }
 
