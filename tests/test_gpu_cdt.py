@@ -97,6 +97,27 @@ def test_cdt_structured_masks_on_the_sweep_path(metric):
         assert np.array_equal(got, co.separable(mask, metric))
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_cdt_seeded_shapes_around_the_piece_boundaries(seed):
+    """Random shapes whose rows are a multiple of 32 voxels, with second extents around the 32-row pieces and row lengths
+    around the 128-column groups of the sweep kernels, both metrics, against the oracle."""
+    import torch
+
+    rng = np.random.default_rng(4242 + seed)
+    n0 = 32 * int(rng.integers(1, 11))
+    n1 = int(rng.choice([1, 2, 31, 32, 33, 63, 64, 65, 95, 96, 97, int(rng.integers(3, 200))]))
+    lead = [(), (int(rng.integers(2, 5)),)][int(rng.integers(0, 2))] if n0 * n1 < 20000 else ()
+    shape = (int(rng.integers(1, 3)), int(rng.integers(1, 3))) + lead + (n1, n0)
+    p_fg = float(rng.choice([0.5, 0.9, 0.99, 0.999]))
+    mask = workloads.random_mask(int(rng.integers(0, 2**31)), shape, p_fg)
+    if rng.random() < 0.3:
+        mask[-1, -1] = 1  # an image without background
+    t = torch.from_numpy(mask).cuda()
+    for metric in ("taxicab", "chessboard"):
+        got = binding.tm_cdt(t, metric).cpu().numpy()
+        assert np.array_equal(got, co.separable(mask, metric)), (shape, p_fg, metric)
+
+
 BF_SHAPES = [(2, 1, 40), (2, 2, 17, 23), (1, 1, 9, 10, 11), (1, 1, 4, 5, 3, 6), (1, 1, 30, 40)]
 
 

@@ -132,6 +132,38 @@ def test_full_box_elements_on_strip_kernels(shape, fp_shape, origin, mode):
             assert binding.tm_edt_last_launch_count() == passes
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_seeded_boxes_and_masks_on_the_strip_and_bit_kernels(seed):
+    """Random shapes (rows a multiple of 4 for the strip kernels, of 32 for the bit-packed kernels), random odd boxes
+    and border rules, against the oracle."""
+    import torch
+
+    rng = np.random.default_rng(777 + seed)
+    ndim = int(rng.integers(1, 4))
+    bits = bool(rng.integers(0, 2))
+    last = (32 if bits else 4) * int(rng.integers(1, 9 if bits else 40))
+    spatial = tuple(int(rng.integers(1, 40)) for _ in range(ndim - 1)) + (last,)
+    shape = (int(rng.integers(1, 3)), int(rng.integers(1, 3))) + spatial
+    fp_shape = tuple(int(rng.choice([1, 3, 5, 7, 9])) for _ in range(ndim))
+    fp = np.ones(fp_shape, dtype=bool)
+    mode = mo.MODES[int(rng.integers(0, len(mo.MODES)))]
+    if bits:
+        mask = (rng.random(shape) < float(rng.choice([0.3, 0.8, 0.97]))).astype(np.uint8)
+        fp = rng.random(fp_shape) < 0.7
+        fp.flat[int(rng.integers(0, fp.size))] = True
+        b = torch.from_numpy(mask).cuda()
+        for border_value in (0, 1):
+            for op, ref_fn in (("erosion", mo.binary_erosion), ("dilation", mo.binary_dilation)):
+                got = binding.tm_binary_morph(b, fp, op=op, border_value=border_value)
+                assert np.array_equal(got.cpu().numpy(), ref_fn(mask, fp, border_value, None)), (shape, fp_shape, op)
+    else:
+        img = rng.normal(size=shape).astype(np.float32)
+        t = torch.from_numpy(img).cuda()
+        for op, ref_fn in (("erosion", mo.grey_erosion), ("dilation", mo.grey_dilation)):
+            got = binding.tm_grey_morph(t, fp, None, op=op, mode=mode, cval=-1.5)
+            assert np.array_equal(got.cpu().numpy(), ref_fn(img, fp, None, mode, -1.5, None)), (shape, fp_shape, mode, op)
+
+
 @pytest.mark.parametrize("shape,fp_shape,origin", BOXES, ids=["x".join(map(str, c[0])) + "_" + "x".join(map(str, c[1])) for c in BOXES])
 @pytest.mark.parametrize("mode", mo.MODES)
 def test_full_box_elements_run_one_pass_per_axis(shape, fp_shape, origin, mode):
