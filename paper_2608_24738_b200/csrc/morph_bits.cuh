@@ -143,4 +143,97 @@ __global__ void __launch_bounds__(256) binary_lines_kernel(const __grid_constant
     }
 }
 
+// Elements that reach over the last two axes only (every 2-D element): packing and combining in one kernel, without
+// the packed copy of the mask in global memory.  A block takes 32 lines x 32 words; it packs those lines and the
+// lines within reach above and below them (dy_lo .. dy_hi), with one word on either side, into shared memory, then
+// every lane produces word w of four consecutive lines as binary_lines_kernel does.  H: extent of the axis before
+// the contiguous one (1 for a 1-D image).
+constexpr int kFusedReach = 8;  // |dy| of the element, at most
+
+template <bool MIN>
+__global__ void __launch_bounds__(256) binary_fused2d_kernel(const __grid_constant__ BitsParams P, const unsigned chunks,
+                                                             const int H, const int dy_lo, const int dy_hi) {
+    __shared__ uint32_t sbits[32 + 2 * kFusedReach][34];
+    const unsigned lb = blockIdx.x / chunks, ch = blockIdx.x - lb * chunks;
+    const int64_t l0 = (int64_t)lb * 32;
+    const int w0 = (int)ch * 32;
+    const uint32_t fill = P.border_value ? 0xffffffffu : 0u;
+    const int rows = 32 + dy_hi - dy_lo;
+#pragma unroll 3
+    for (int t = threadIdx.x; t < rows * 34; t += 256) {
+        const int r = t / 34, c = t - r * 34;
+        const int64_t line = l0 + dy_lo + r;
+        const int w = w0 - 1 + c;
+        uint32_t bits = fill;  // words beyond the ends of a line hold the border value
+        if (w >= 0 && w < P.words) {
+            bits = 0u;
+            if (line >= 0 && line < P.lines) {
+                uint32_t v[8];
+                asm("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"  // read-only data: free to be scheduled early
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                    : "l"(P.in + (line * P.words + w) * 32));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) bits |= nonzero_bits4(v[i]) << (4 * i);
+            }
+        }
+        sbits[r][c] = bits;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int w = w0 + lane;
+    const int64_t line0 = l0 + 4 * ty;
+    if (w >= P.words || line0 >= P.lines) return;
+    const int y0 = (int)(line0 % H);
+    uint32_t acc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = MIN ? 0xffffffffu : 0u;
+    for (int g = 0; g < P.n_groups; ++g) {
+        const LineGroup& G = P.groups[g];
+        const int dy = P.ndim >= 2 ? G.off[P.ndim - 2] : 0;
+        uint32_t lo[4], mid[4], hi[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int y = y0 + j;
+            if (y >= H) y -= H * (y / H);  // the next image (H < 4: several images further)
+            const bool inside = (unsigned)(y + dy) < (unsigned)H;
+            const uint32_t* row = sbits[4 * ty + j + dy - dy_lo];
+            lo[j] = inside ? row[lane] : fill;
+            mid[j] = inside ? row[lane + 1] : fill;
+            hi[j] = inside ? row[lane + 2] : fill;
+        }
+        for (uint32_t m = (uint32_t)G.mask; m; m &= m - 1) {
+            const int sh = 31 - (__ffs((int)m) - 1);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t v = __funnelshift_l(lo[j], mid[j], sh);
+                acc[j] = MIN ? acc[j] & v : acc[j] | v;
+            }
+        }
+        for (uint32_t m = (uint32_t)(G.mask >> 32); m; m &= m - 1) {
+            const int sh = __ffs((int)m);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t v = __funnelshift_r(mid[j], hi[j], sh);
+                acc[j] = MIN ? acc[j] & v : acc[j] | v;
+            }
+        }
+        const uint32_t all = MIN ? (acc[0] | acc[1] | acc[2] | acc[3]) : (acc[0] & acc[1] & acc[2] & acc[3]);
+        if (all == (MIN ? 0u : 0xffffffffu)) break;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (line0 + j >= P.lines) break;
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t nib = (acc[j] >> (4 * i)) & 0xfu;
+            o[i] = (nib * 0x00204081u) & 0x01010101u;
+        }
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(P.out + ((line0 + j) * P.words + w) * 32), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]),
+                        "r"(o[6]), "r"(o[7])
+                     : "memory");
+    }
+}
+
 }  // namespace tmmorph

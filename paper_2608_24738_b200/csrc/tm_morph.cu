@@ -237,6 +237,35 @@ static int run_binary_bits(const Geometry& g, const std::vector<Entry>& entries,
         grp->mask |= (uint64_t)1 << (dx + 31);
     }
     if ((int)groups.size() > kMaxLineGroups) return -1;
+    // an element that reaches over the last two axes only: packing and combining in one kernel
+    {
+        bool last_two = true;
+        int dy_lo = 0, dy_hi = 0;
+        for (const LineGroup& c : groups) {
+            for (int a = 0; a < nd - 2; ++a) last_two = last_two && c.off[a] == 0;
+            if (nd >= 2) { dy_lo = std::min(dy_lo, (int)c.off[nd - 2]); dy_hi = std::max(dy_hi, (int)c.off[nd - 2]); }
+        }
+        const int64_t lines = g.total / W;
+        const unsigned chunks = (unsigned)((W / 32 + 31) / 32);
+        if (last_two && dy_lo >= -kFusedReach && dy_hi <= kFusedReach && (lines + 31) / 32 * chunks <= (int64_t)INT32_MAX) {
+            BitsParams B;
+            memset(&B, 0, sizeof(B));
+            B.in = input; B.out = output;
+            for (size_t i = 0; i < groups.size(); ++i) B.groups[i] = groups[i];
+            B.n_groups = (int)groups.size();
+            B.ndim = nd; B.words = W / 32; B.lines = lines; B.lines_per_image = g.V / W;
+            for (int a = 0; a < nd; ++a) B.ext[a] = g.ext[a];
+            B.border_value = border_value ? 1 : 0;
+            const unsigned blocks = (unsigned)((lines + 31) / 32) * chunks;
+            const int H = nd >= 2 ? g.ext[nd - 2] : 1;
+            if (erosion) binary_fused2d_kernel<true><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+            else binary_fused2d_kernel<false><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+            const cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
+            tmedt::shared_record(-1, 1);
+            return TM_EDT_OK;
+        }
+    }
     const int64_t words = g.total / 32;
     char* dev = nullptr;
     cudaError_t e = tmedt::shared_scratch_alloc((void**)&dev, (size_t)words * 4, s);
