@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(32 * NW, 3) lean_plane_kernel(const __grid_con
 // One further axis on entries (unit sampling, index output requested).  K earlier axes, K = 2 or 3.
 //   FINAL == false  (K == 2)  writes 4-byte entries
 //   FINAL == true             writes float32 distances and / or int64 squared distances, and the index planes
-//                             (every spatial axis is a processed axis, coordinate layout)
+//                             (every spatial axis is a processed axis; FLAT: one linear index per voxel instead)
 // ---------------------------------------------------------------------------------------------
 // Four zero-extended 32-bit values as four int64: one 256-bit streaming store (p 32-byte aligned).
 __device__ __forceinline__ void lean_store_4xi64(int64_t* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
@@ -370,7 +370,7 @@ __device__ __forceinline__ void lean_decode(uint32_t v0, const LeanParams& P, co
     }
 }
 
-template <int K, bool FINAL, int TX>
+template <int K, bool FINAL, int TX, bool FLAT = false>
 __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const __grid_constant__ LeanParams P,
                                                                          const __grid_constant__ EpilogueParams ep) {
     using EI = typename EntryType<entry_bytes(K)>::type;
@@ -436,7 +436,7 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     }
     float* const dist = ep.dist ? ep.dist + slab * ep.V : nullptr;
     int64_t* const sq = ep.sq ? ep.sq + slab * ep.V : nullptr;
-    if (ep.flat) {  // one linear index per voxel
+    if (FLAT) {  // one linear index per voxel
         int ps[K];
 #pragma unroll
         for (int q = 0; q < K; ++q) ps[q] = (int)ep.pstride[q];

@@ -81,6 +81,13 @@ template <int K, bool FINAL, int TX>
 static cudaError_t launch_lean_column_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4 + (size_t)P.n * TX * entry_bytes(K);
     P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    if (FINAL && ep.flat) {
+        auto kern = lean_column_kernel<K, FINAL, TX, FINAL>;
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)(outer * P.tiles_per_slab), 256, smem, st>>>(P, ep);
+        return cudaGetLastError();
+    }
     auto kern = lean_column_kernel<K, FINAL, TX>;
     cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
