@@ -385,6 +385,7 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);
     uint32_t all = 0xffffffffu;  // AND of this thread's keys
+#pragma unroll 4
     for (int t = threadIdx.x; t < n * LPR; t += 256) {
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
@@ -488,6 +489,7 @@ __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_consta
     const VT* src = reinterpret_cast<const VT*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);
     uint32_t all = 0xffffffffu;  // AND of this thread's keys
+#pragma unroll 4
     for (int t = threadIdx.x; t < n * LPR; t += 32 * NW) {
         const int y = t / LPR, q4 = 4 * (t % LPR);
         if (q4 >= width) continue;
