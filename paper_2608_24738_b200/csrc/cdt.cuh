@@ -198,16 +198,19 @@ __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ 
     if (!valid) return;
     int f = left ? 32 * (lane - wl) - hbl - 1 : kNone16;    // distance of the voxel before the word to the background on its left
     int d[32];
+    const uint32_t fg = ~z;  // bit i: voxel i is foreground; count = fg_i * (count + 1) is one multiply-add
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        f = (z >> i) & 1u ? 0 : f + 1;
+        const int keep = (int)((fg >> i) & 1u);
+        f = keep * f + keep;
         d[i] = f;
     }
     int b = right ? 32 * (wr - lane) + lbr - 32 : kNone16;  // the same for the voxel after the word, to the right
 #pragma unroll
-    for (int i = 31; i >= 0; --i) {
-        b = (z >> i) & 1u ? 0 : b + 1;
-        d[i] = min(min(d[i], b), kNone16);
+    for (int i = 31; i >= 0; --i) {  // a row without background leaves values just above kNone16: "no background" all the same
+        const int keep = (int)((fg >> i) & 1u);
+        b = keep * b + keep;
+        d[i] = min(d[i], b);
     }
     if (P.edge) {  // the last column of a group of 128 and the first one of the next group
         if ((w & 3) == 3 && w + 1 < words) P.edge[(row * P.nb + (w >> 2)) * 2] = (uint16_t)d[31];
