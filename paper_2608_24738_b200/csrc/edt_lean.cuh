@@ -37,6 +37,8 @@ struct LeanParams {
     int64_t in_elems;    // elements behind `in` and `out` (bounds checks of the debug build)
     int64_t out_elems;
     int64_t images;      // images behind the final outputs (bounds checks of the debug build)
+    int dist16;          // value kernels, 16-bit input: the input holds first-axis distances (>= 0xC000: no site in the
+                         // row) instead of squared values; they are squared while the tile is staged
 };
 
 // A key tile in shared memory: its first word and its size in words (bounds checks of the debug build).
@@ -499,10 +501,17 @@ __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_consta
         if (sizeof(VT) == 2) {
             const uint2 w = *reinterpret_cast<const uint2*>(g);
             k = make_uint4(w.x & 0xffffu, w.x >> 16, w.y & 0xffffu, w.y >> 16);
-            if (k.x == 0xffffu) k.x = kLeanNone;
-            if (k.y == 0xffffu) k.y = kLeanNone;
-            if (k.z == 0xffffu) k.z = kLeanNone;
-            if (k.w == 0xffffu) k.w = kLeanNone;
+            if (P.dist16) {
+                k.x = k.x >= 0xC000u ? kLeanNone : k.x * k.x;
+                k.y = k.y >= 0xC000u ? kLeanNone : k.y * k.y;
+                k.z = k.z >= 0xC000u ? kLeanNone : k.z * k.z;
+                k.w = k.w >= 0xC000u ? kLeanNone : k.w * k.w;
+            } else {
+                if (k.x == 0xffffu) k.x = kLeanNone;
+                if (k.y == 0xffffu) k.y = kLeanNone;
+                if (k.z == 0xffffu) k.z = kLeanNone;
+                if (k.w == 0xffffu) k.w = kLeanNone;
+            }
         } else {
             k = *reinterpret_cast<const uint4*>(g);
         }

@@ -67,9 +67,12 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
 // One axis pass of the wide-key path on plain integer values with the quad kernels (see tm_edt_lean.cu).
 bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
-                                cudaStream_t st);
+                                cudaStream_t st, bool dist16 = false);
 
 // Debug build: what the kernels launched from tm_edt_lean.cu recorded (see edt_debug.cuh).
+// First-axis distances as 16-bit values (>= 0xC000: no background in the row) for rows of a multiple of 32 up to 1024
+// voxels and a 32-byte aligned mask: the word-per-lane row kernel of cdt.cuh (defined in tm_cdt.cu).
+cudaError_t launch_row_dist16(const uint8_t* mask, uint16_t* out, int64_t rows, int n0, cudaStream_t st);
 cudaError_t lean_debug_collect(cudaStream_t st, DebugRecord* out);
 
 }  // namespace tmedt

@@ -6,6 +6,8 @@
 #include "cdt.cuh"
 #include "host_shared.h"
 
+namespace tmedt { cudaError_t launch_row_dist16(const uint8_t* mask, uint16_t* out, int64_t rows, int n0, cudaStream_t st); }
+
 using namespace tmcdt;
 
 namespace {
@@ -28,6 +30,19 @@ int geometry(int ndim, const int64_t* shape, int max_ndim, Geo& g) {
 }
 
 }  // namespace
+
+namespace tmedt {
+
+// Used by the Euclidean transform's two-axis path as well: the row distances are the same for every metric.
+cudaError_t launch_row_dist16(const uint8_t* mask, uint16_t* out, int64_t rows, int n0, cudaStream_t st) {
+    Row16Params R;
+    R.mask = mask; R.out = out; R.rows = rows; R.words = n0 / 32; R.edge = nullptr; R.nb = 0;
+    const int64_t warps = (rows + 32 / R.words - 1) / (32 / R.words);
+    cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
+    return cudaGetLastError();
+}
+
+}  // namespace tmedt
 
 extern "C" {
 

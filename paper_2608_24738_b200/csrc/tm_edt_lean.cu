@@ -142,7 +142,7 @@ bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
 }
 
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
-                                cudaStream_t st) {
+                                cudaStream_t st, bool dist16) {
     LeanParams P;
     memset(&P, 0, sizeof(P));
     P.in = in; P.out = out;
@@ -150,6 +150,10 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
     P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
     P.inv_scale = 1.0f;
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+    if (dist16) {  // 16-bit first-axis distances in, final outputs out
+        P.dist16 = 1;
+        return launch_lean_value_tx<true, uint16_t, 32>(P, ep, outer, st);
+    }
     return fin ? launch_lean_value_tx<true, uint32_t, 32>(P, ep, outer, st)
                : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
 }
