@@ -107,6 +107,13 @@ template <bool FINAL, typename VT, int TX>
 static cudaError_t launch_lean_value_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4;
     P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    if (TX == 32 && P.n >= 384) {  // very long axes: two blocks per SM, 32 warps each
+        auto kern = lean_value_kernel<FINAL, VT, TX, 32>;
+        cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)(outer * P.tiles_per_slab), 1024, smem, st>>>(P, ep);
+        return cudaGetLastError();
+    }
     if (TX == 32 && P.n > 128) {  // long axes: few blocks fit an SM, so each gets 16 warps
         auto kern = lean_value_kernel<FINAL, VT, TX, 16>;
         cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
