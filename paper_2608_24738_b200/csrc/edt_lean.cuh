@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_consta
         const int64_t p = col + (int64_t)y * P.inner;
         if (!TM_EDT_IN_RANGE(p, (FINAL ? P.images * ep.V : P.out_elems) - 3, 131)) continue;
         if (!FINAL) {
-            if (sizeof(VT) == 2) {
+            if (sizeof(VT) == 2 && !P.dist16) {  // (16-bit row distances in: 32-bit values out)
 #pragma unroll
                 for (int v = 0; v < 4; ++v) b[v] = min(b[v], 0xffffu);
                 *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(P.out) + p) = make_uint2(b[0] | (b[1] << 16), b[2] | (b[3] << 16));

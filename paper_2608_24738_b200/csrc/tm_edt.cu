@@ -684,8 +684,8 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
     // without an index output no site is needed afterwards: plain values as keys (sh = 0)
     const int sh = !pl.unit ? -1 : (!carry ? 0 : (nmax > 512 ? 10 : 9));
-    // two axes, distances only, unit sampling: the first pass hands 16-bit row distances to the quad value kernel
-    const bool dist16 = sh == 0 && pl.E == 2 && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 && ((uintptr_t)in & 31u) == 0 &&
+    // no index output, unit sampling: the first pass hands 16-bit row distances to the quad value kernel of the second axis
+    const bool dist16 = sh == 0 && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 && ((uintptr_t)in & 31u) == 0 &&
                         !switches().no_lean && lean_value_axis_ok(pl, 1, ep);
     prof_mark(st, "row_keys", (double)pl.N * (1.0 + (dist16 ? 2.0 : 4.0) + (carry ? 2.0 : 0.0)));
     const unsigned row_blocks = (unsigned)((P.rows + 7) / 8);
@@ -728,9 +728,9 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
         A.next_n = fin ? 0 : pl.ext[k + 1];
         A.w2 = (float)(pl.w[k] * pl.w[k]);
         const double offs_b = k == 3 ? 8.0 : 2.0 * k;  // bytes of offsets per voxel read by this axis
-        if (fin) prof_mark(st, "wide_axis_final", (double)pl.N * ((dist16 ? 2.0 : 4.0) + out_bpv + (ep.idx ? offs_b : 0.0)));
-        else prof_mark(st, "wide_axis", (double)pl.N * (4.0 + 4.0 + (carry ? offs_b + (k == 2 ? 8.0 : 4.0) : 0.0)));
-        if (dist16) e = run_lean_value_axis(pl, 1, keysA, nullptr, ep, true, st, true);
+        if (fin) prof_mark(st, "wide_axis_final", (double)pl.N * ((dist16 && k == 1 ? 2.0 : 4.0) + out_bpv + (ep.idx ? offs_b : 0.0)));
+        else prof_mark(st, "wide_axis", (double)pl.N * ((dist16 && k == 1 ? 2.0 : 4.0) + 4.0 + (carry ? offs_b + (k == 2 ? 8.0 : 4.0) : 0.0)));
+        if (dist16 && k == 1) e = run_lean_value_axis(pl, 1, keysA, fin ? nullptr : keys_out[1], ep, fin, st, true);
         else if (sh == 0 && !switches().no_lean && lean_value_axis_ok(pl, k, ep))
             e = run_lean_value_axis(pl, k, keys_in[k], fin ? nullptr : keys_out[k], ep, fin, st);
         else if (k == 1) e = fin ? launch_wide_axis<1, true>(A, ep, sh, st) : launch_wide_axis<1, false>(A, ep, sh, st);

@@ -157,9 +157,10 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
     P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
     P.inv_scale = 1.0f;
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
-    if (dist16) {  // 16-bit first-axis distances in, final outputs out
+    if (dist16) {  // 16-bit first-axis distances in; final outputs or 32-bit values out
         P.dist16 = 1;
-        return launch_lean_value_tx<true, uint16_t, 32>(P, ep, outer, st);
+        return fin ? launch_lean_value_tx<true, uint16_t, 32>(P, ep, outer, st)
+                   : launch_lean_value_tx<false, uint16_t, 32>(P, ep, outer, st);
     }
     return fin ? launch_lean_value_tx<true, uint32_t, 32>(P, ep, outer, st)
                : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
