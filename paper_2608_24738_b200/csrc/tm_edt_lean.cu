@@ -143,9 +143,9 @@ bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
     const int n = pl.ext[k];
     const size_t smem = (size_t)(n + 2 * kLeanPad) * 32 * 4;
-    if (smem > 100 * 1024) return false;  // keeps at least two blocks per SM
+    if (smem > 136 * 1024) return false;  // up to 1024 rows (one block of 32 warps per SM beyond 100 KB)
     const int64_t blocks = pl.N / ((int64_t)n * pl.inner[k]) * ((pl.inner[k] + 31) / 32);
-    return blocks >= 296;  // few strips (a single image) are split over several blocks by wide_axis_kernel instead
+    return blocks >= (smem > 100 * 1024 ? 148 : 296);  // few strips (a single image) are split over several blocks by wide_axis_kernel instead
 }
 
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,

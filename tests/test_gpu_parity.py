@@ -151,7 +151,8 @@ def test_flags_flat_index_and_virtual_background(shape, kind, path):
                           sampling)
 
 
-@pytest.mark.parametrize("shape", [(38, 1, 150, 256), (10, 1, 300, 1024), (2, 1, 140, 40, 160), (1, 2, 30, 520, 96)])
+@pytest.mark.parametrize("shape", [(38, 1, 150, 256), (10, 1, 300, 1024), (2, 1, 140, 40, 160), (1, 2, 30, 520, 96),
+                                   (5, 1, 1000, 1024)])  # the last: one block of 32 warps per SM (132 KB tile)
 def test_16_bit_row_distances_feed_the_value_kernel(shape):
     """Batches large enough for the quad value kernel (at least 296 strips per axis), rows a multiple of 32, no index
     output: the first pass hands 16-bit row distances to it.  Rows without background, an image without background,
