@@ -314,7 +314,7 @@ struct SweepParams {
 };
 
 // Pinned rows: one lane per pair of neighbouring columns, a bounded outward scan along the axis through global memory
-// (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), four distances per stop test.
+// (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), eight distances per stop test.
 template <bool CHESS>
 __device__ __forceinline__ void cdt_pin_rows(const SweepParams& P, const int64_t t) {
     const int pairs = P.inner >> 1;
@@ -327,15 +327,15 @@ __device__ __forceinline__ void cdt_pin_rows(const SweepParams& P, const int64_t
     uint32_t best = col[(int64_t)y * pairs];
     int mx = (int)max(best & 0xffffu, best >> 16);
     auto cand = [&](uint32_t v, int d) { return CHESS ? __vmaxu2(v, cdt_both(d)) : v + cdt_both(d); };
-    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); d += 4) {  // eight loads in flight
-        uint32_t a[4], b[4];
+    for (int d = 1; d < mx && (y - d >= 0 || y + d < n); d += 8) {  // sixteen loads in flight
+        uint32_t a[8], b[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 8; ++i) {
             a[i] = y - d - i >= 0 ? col[(int64_t)(y - d - i) * pairs] : none2;
             b[i] = y + d + i < n ? col[(int64_t)(y + d + i) * pairs] : none2;
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) best = __vimin3_u16x2(best, cand(a[i], d + i), cand(b[i], d + i));
+        for (int i = 0; i < 8; ++i) best = __vimin3_u16x2(best, cand(a[i], d + i), cand(b[i], d + i));
         mx = (int)max(best & 0xffffu, best >> 16);
     }
     reinterpret_cast<uint32_t*>(P.pd)[t] = __vminu2(best, none2);
