@@ -2,16 +2,17 @@
 // the neighbourhood with AND / OR and a single border value).  A mask needs one bit per voxel, so the combine of 32
 // voxels with one neighbour position is one funnel shift and one logic instruction on 32-bit words:
 //   1. binary_pack_kernel     mask bytes -> one bit per voxel (bit b of word w of a line = voxel 32 w + b is nonzero);
-//                             a lane takes 32 consecutive voxels (two 16-byte loads), N / 8 bytes of scratch.
+//                             a lane takes 32 consecutive voxels (one 32-byte load), N / 8 bytes of scratch.
 //   2. binary_lines_kernel    the host groups the element's active positions by their offsets along all axes but the
 //                             contiguous one; a group is a neighbouring line plus a 64-bit mask of offsets along
 //                             the line.  A lane produces one output word: per group it reads three words of the
 //                             neighbouring line (or takes the border value if that line lies outside the image), and
 //                             per offset of the group shifts the 96-bit window into place and combines it; the result
 //                             is expanded to bytes and leaves as one 32-byte store.
+//   3. binary_fused2d_kernel  both steps in one launch for elements that reach over the last two axes only: a block
+//                             packs its lines and those within reach into shared memory and combines from there.
 // Requires at most 4 axes, a contiguous extent that is a multiple of 32, offsets along it within +-31, and 32-byte
-// aligned buffers;
-// everything else runs on the byte kernels of morph.cuh.
+// aligned buffers; everything else runs on the byte kernels of morph.cuh.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
