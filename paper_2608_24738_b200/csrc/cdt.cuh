@@ -155,7 +155,8 @@ struct Row16Params {
     const uint8_t* mask;
     uint16_t* out;
     int64_t rows;
-    int words;       // 32-voxel words per row (1 .. 32)
+    int n0;          // voxels per row: a multiple of 4 (and of 32 unless the rows are at least 64 voxels long)
+    int words;       // 32-voxel words per row, the last one possibly ragged (1 .. 32); the output rows have 32 words voxels
     uint16_t* edge;  // optional (rows, nb, 2): the values of columns 128 k - 1 and 128 k, k = 1 .. nb, for the pinned columns
     int nb;          // boundaries between groups of 128 columns (words / 4 rounded up, minus 1)
 };
@@ -165,8 +166,8 @@ __device__ __forceinline__ uint32_t cdt_nonzero_bits4(uint32_t v) {
     return (((m >> 7) * 0x00204081u) >> 21) & 0xfu;
 }
 
-// First axis, rows of 32 .. 1024 voxels (a multiple of 32).  A lane owns one word of 32 voxels (one 32-byte load,
-// two 32-byte stores); a warp holds 32 / words whole rows.  The nearest background voxel outside the lane's word
+// First axis, rows of up to 1024 voxels (a multiple of 32, or of 4 with a ragged last word).  A lane owns one word of
+// 32 voxels (one 32-byte load, two 32-byte stores into rows padded to whole words); a warp holds 32 / words whole rows.  The nearest background voxel outside the lane's word
 // comes from a ballot over the words that contain one and a shuffle of its position inside that word; inside the word
 // the distances are two running counts over the 32 bits, left to right and right to left.
 __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ Row16Params P) {
@@ -179,9 +180,16 @@ __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ 
     uint32_t z = 0u;  // bit i: voxel i of the word is background
     if (valid) {
         uint32_t v[8];
-        asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                     : "l"(P.mask + (row * words + w) * 32));
+        const uint8_t* src = P.mask + row * P.n0 + 32 * w;
+        if ((P.n0 & 31) == 0 && (reinterpret_cast<uintptr_t>(P.mask) & 31u) == 0) {
+            asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                         : "l"(src));
+        } else {  // rows of a multiple of 4 voxels: 4-byte loads; voxels beyond the row count as foreground
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                v[i] = 32 * w + 4 * i < P.n0 ? __ldg(reinterpret_cast<const uint32_t*>(src) + i) : 0x01010101u;
+        }
         uint32_t nzb = 0u;
 #pragma unroll
         for (int i = 0; i < 8; ++i) nzb |= cdt_nonzero_bits4(v[i]) << (4 * i);
@@ -310,6 +318,7 @@ struct SweepParams {
     int32_t* out;
     int64_t slabs;
     int inner, n, segs, groups;
+    int fpitch;          // voxels per row of f and pd (inner rounded up to a multiple of 32)
     int last;            // last pass: "no background" becomes -1 (else kBig for the next pass)
 };
 
@@ -317,12 +326,12 @@ struct SweepParams {
 // (rows of pairs are contiguous: a warp reads 128 bytes per candidate row), eight distances per stop test.
 template <bool CHESS>
 __device__ __forceinline__ void cdt_pin_rows(const SweepParams& P, const int64_t t) {
-    const int pairs = P.inner >> 1;
+    const int pairs = P.fpitch >> 1;
     if (t >= P.slabs * P.segs * pairs) return;
     const int x2 = (int)(t % pairs), k = (int)((t / pairs) % P.segs);
     const int64_t slab = t / ((int64_t)pairs * P.segs);
     const int n = P.n, y = min(n, (k + 1) * kSegRows) - 1;
-    const uint32_t* col = reinterpret_cast<const uint32_t*>(P.f + slab * (int64_t)n * P.inner) + x2;
+    const uint32_t* col = reinterpret_cast<const uint32_t*>(P.f + slab * (int64_t)n * P.fpitch) + x2;
     const uint32_t none2 = cdt_both(kNone16);
     uint32_t best = col[(int64_t)y * pairs];
     int mx = (int)max(best & 0xffffu, best >> 16);
@@ -382,8 +391,9 @@ __global__ void __launch_bounds__(128) cdt_sweep_kernel(const __grid_constant__ 
     const bool act = c < inner;
     const int y0 = k * kSegRows, rp = min(n, y0 + kSegRows) - 1, cnt = rp - y0;  // swept rows y0 .. rp - 1
     const uint2 none2 = make_uint2(cdt_both(kNone16), cdt_both(kNone16));
-    const uint16_t* fcol = P.f + slab * (int64_t)n * inner + (act ? c : 0);
-    const uint16_t* pdk = P.pd + (slab * P.segs + k) * (int64_t)inner + (act ? c : 0);
+    const int fp = P.fpitch;
+    const uint16_t* fcol = P.f + slab * (int64_t)n * fp + (act ? c : 0);
+    const uint16_t* pdk = P.pd + (slab * P.segs + k) * (int64_t)fp + (act ? c : 0);
     const uint16_t* hl = CHESS && g > 0 ? P.hd + ((slab * (P.groups - 1) + g - 1) * 2 + 0) * (int64_t)n : nullptr;
     const uint16_t* hr = CHESS && g + 1 < P.groups ? P.hd + ((slab * (P.groups - 1) + g) * 2 + 1) * (int64_t)n : nullptr;
     int32_t* out = P.out + slab * (int64_t)n * inner + (act ? c : 0);
@@ -398,7 +408,7 @@ __global__ void __launch_bounds__(128) cdt_sweep_kernel(const __grid_constant__ 
     uint2 a[kSegRows - 1];
 #pragma unroll
     for (int i = 0; i < kSegRows - 1; ++i)
-        a[i] = i < cnt && act ? *reinterpret_cast<const uint2*>(fcol + (int64_t)(y0 + i) * inner) : none2;
+        a[i] = i < cnt && act ? *reinterpret_cast<const uint2*>(fcol + (int64_t)(y0 + i) * fp) : none2;
     // results of the pinned columns beside the piece: lane i holds row y0 - 1 + i, row y0 + 31 apart
     int hlv = kNone16, hrv = kNone16, hl_last = kNone16, hr_last = kNone16;
     if (CHESS) {
@@ -426,7 +436,7 @@ __global__ void __launch_bounds__(128) cdt_sweep_kernel(const __grid_constant__ 
         }
         return act ? r : none2;  // lanes beyond the row stay "no background" for their neighbours
     };
-    uint2 prev = act && k > 0 ? *reinterpret_cast<const uint2*>(pdk - inner) : none2;
+    uint2 prev = act && k > 0 ? *reinterpret_cast<const uint2*>(pdk - fp) : none2;
 #pragma unroll
     for (int i = 0; i < kSegRows - 1; ++i) {  // down from the pinned row above (row y0 + i - 1: place i)
         if (i < cnt) {

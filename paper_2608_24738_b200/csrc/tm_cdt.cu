@@ -36,7 +36,7 @@ namespace tmedt {
 // Used by the Euclidean transform's two-axis path as well: the row distances are the same for every metric.
 cudaError_t launch_row_dist16(const uint8_t* mask, uint16_t* out, int64_t rows, int n0, cudaStream_t st) {
     Row16Params R;
-    R.mask = mask; R.out = out; R.rows = rows; R.words = n0 / 32; R.edge = nullptr; R.nb = 0;
+    R.mask = mask; R.out = out; R.rows = rows; R.n0 = n0; R.words = n0 / 32; R.edge = nullptr; R.nb = 0;
     const int64_t warps = (rows + 32 / R.words - 1) / (32 / R.words);
     cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
     return cudaGetLastError();
@@ -64,40 +64,57 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
     if (E == 0) axes[E++] = ndim - 1;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t buf = (((size_t)g.total * 4) + 255) & ~(size_t)255;
+    // The first two axes on 16-bit values (cdt.cuh): rows of up to 1024 voxels, a multiple of 32 (or of 4 from 64 voxels
+    // on: the last word of a row is then ragged and the 16-bit rows are padded to whole words), a second axis of up to
+    // 1024 rows whose stride is the row length.
+    bool fast = false;
+    size_t fast_bytes = 0;
+    if (E >= 2 && axes[0] == ndim - 1) {
+        const int64_t n0 = g.ext[axes[0]], n1 = g.ext[axes[1]];
+        const bool rows_ok = n0 % 32 == 0 ? ((uintptr_t)input & 31u) == 0 : (n0 % 4 == 0 && n0 >= 64 && ((uintptr_t)input & 3u) == 0);
+        fast = rows_ok && n0 <= 1024 && n1 <= 1024 && ((uintptr_t)out_dist & 15u) == 0 && g.total / (32 * n1) <= (int64_t)INT32_MAX;
+        if (fast) {
+            const int64_t fpitch = (n0 + 31) / 32 * 32, rows = g.total / n0, slabs = rows / n1;
+            const int64_t segs = (n1 + kSegRows - 1) / kSegRows, groups = (n0 + 127) / 128;
+            fast_bytes = (size_t)rows * fpitch * 2 + (size_t)slabs * segs * fpitch * 2 + (size_t)slabs * (groups - 1) * 2 * n1 * 2 +
+                         (size_t)rows * (groups - 1) * 4 + 1024;
+            fast_bytes = (fast_bytes + 255) & ~(size_t)255;
+        }
+    }
     char* ws = nullptr;
+    const size_t later = E > 2 ? 2 * buf : 0;  // the int32 images between the later passes
     if (E > 1) {
-        cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, (E > 2 ? 2 : 1) * buf, st);
+        cudaError_t e = tmedt::shared_scratch_alloc((void**)&ws, fast ? fast_bytes + later : (E > 2 ? 2 : 1) * buf, st);
         if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
     }
-    int32_t* tmp[2] = {reinterpret_cast<int32_t*>(ws), reinterpret_cast<int32_t*>(ws + buf)};
+    char* fast_ws = ws;
+    char* tmp_base = fast ? ws + fast_bytes : ws;
+    int32_t* tmp[2] = {reinterpret_cast<int32_t*>(tmp_base), reinterpret_cast<int32_t*>(tmp_base + buf)};
     const int32_t* prev = nullptr;
     cudaError_t e = cudaSuccess;
     const bool chess = metric == TM_METRIC_CHESSBOARD;
     int k0 = 0, launches_fast = 0;
-    // The first two axes on 16-bit values (cdt.cuh): rows of a multiple of 32 up to 1024 voxels, a second axis of up
-    // to 1024 rows whose stride is the row length.
-    if (E >= 2 && axes[0] == ndim - 1 && g.ext[axes[0]] % 32 == 0 && g.ext[axes[0]] <= 1024 && g.ext[axes[1]] <= 1024 &&
-        ((uintptr_t)input & 31u) == 0 && ((uintptr_t)out_dist & 15u) == 0 && g.total / (32 * g.ext[axes[1]]) <= (int64_t)INT32_MAX) {
+    if (fast) {
         const int n0 = (int)g.ext[axes[0]], n1 = (int)g.ext[axes[1]];
-        const int groups = (n0 + 127) / 128;
+        const int groups = (n0 + 127) / 128, words = (n0 + 31) / 32, fpitch = 32 * words;
         const int64_t slabs = g.total / ((int64_t)n1 * n0);
         const int segs = (n1 + kSegRows - 1) / kSegRows;
-        // pinned results and the gathered boundary columns behind the 16-bit values in the first scratch image
-        char* extra = reinterpret_cast<char*>(tmp[0]) + (size_t)g.total * 2;
-        uint16_t* pd = reinterpret_cast<uint16_t*>(extra);
-        uint16_t* hd = reinterpret_cast<uint16_t*>(extra + (size_t)slabs * segs * n0 * 2);
+        // 16-bit values, pinned results and the gathered boundary columns
+        uint16_t* f = reinterpret_cast<uint16_t*>(fast_ws);
+        uint16_t* pd = f + (size_t)(g.total / n0) * fpitch;
+        uint16_t* hd = pd + (size_t)slabs * segs * fpitch;
         uint16_t* edge = hd + (size_t)slabs * (groups - 1) * 2 * n1;
         Row16Params R;
-        R.mask = input; R.out = reinterpret_cast<uint16_t*>(tmp[0]); R.rows = g.total / n0; R.words = n0 / 32;
+        R.mask = input; R.out = f; R.rows = g.total / n0; R.n0 = n0; R.words = words;
         R.edge = chess && groups > 1 ? edge : nullptr; R.nb = groups - 1;
         const int64_t warps = (R.rows + 32 / R.words - 1) / (32 / R.words);
         cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
         SweepParams C;
         memset(&C, 0, sizeof(C));
         C.f = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1];
-        C.slabs = slabs; C.inner = n0; C.n = n1; C.segs = segs; C.groups = groups;
+        C.slabs = slabs; C.inner = n0; C.n = n1; C.segs = segs; C.groups = groups; C.fpitch = fpitch;
         C.pd = pd; C.hd = hd; C.edge = edge;
-        const int64_t row_blocks = (C.slabs * C.segs * (n0 / 2) + 255) / 256;
+        const int64_t row_blocks = (C.slabs * C.segs * (fpitch / 2) + 255) / 256;
         const int64_t col_blocks = chess ? C.slabs * (groups - 1) : 0;
         if (chess) cdt_pins_kernel<true><<<(unsigned)(row_blocks + col_blocks), 256, (size_t)n1 * 4, st>>>(C, (unsigned)row_blocks);
         else cdt_pins_kernel<false><<<(unsigned)row_blocks, 256, 0, st>>>(C, (unsigned)row_blocks);

@@ -23,7 +23,9 @@ SHAPES = [(2, 2, 1), (3, 1, 37), (2, 1, 19, 23), (1, 2, 40, 300), (1, 1, 1, 50, 
           # rows of a multiple of 32 voxels: the first two axes on 16-bit values (one to 32 words per row, segments of
           # the second axis that are empty, ragged and full, a third axis after them, an axis of one voxel in between)
           (2, 1, 64, 64), (3, 1, 5, 96), (1, 1, 300, 1024), (1, 2, 1024, 32), (2, 1, 7, 33, 64), (1, 1, 9, 1, 128),
-          (1, 1, 70, 352), (2, 1, 1, 3, 160)]
+          (1, 1, 70, 352), (2, 1, 1, 3, 160),
+          # rows of a multiple of 4 from 64 voxels on: a ragged last word, 16-bit rows padded to whole words
+          (2, 1, 100, 1000), (1, 1, 37, 500), (3, 1, 33, 68), (1, 1, 5, 6, 132), (2, 1, 70, 260), (1, 1, 3, 124)]
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=["x".join(map(str, s)) for s in SHAPES])
@@ -104,7 +106,7 @@ def test_cdt_seeded_shapes_around_the_piece_boundaries(seed):
     import torch
 
     rng = np.random.default_rng(4242 + seed)
-    n0 = 32 * int(rng.integers(1, 11))
+    n0 = 32 * int(rng.integers(1, 11)) if seed % 2 == 0 else 4 * int(rng.integers(16, 90))
     n1 = int(rng.choice([1, 2, 31, 32, 33, 63, 64, 65, 95, 96, 97, int(rng.integers(3, 200))]))
     lead = [(), (int(rng.integers(2, 5)),)][int(rng.integers(0, 2))] if n0 * n1 < 20000 else ()
     shape = (int(rng.integers(1, 3)), int(rng.integers(1, 3))) + lead + (n1, n0)
