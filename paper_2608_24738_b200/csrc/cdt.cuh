@@ -170,6 +170,8 @@ __device__ __forceinline__ uint32_t cdt_nonzero_bits4(uint32_t v) {
 // 32 voxels (one 32-byte load, two 32-byte stores into rows padded to whole words); a warp holds 32 / words whole rows.  The nearest background voxel outside the lane's word
 // comes from a ballot over the words that contain one and a shuffle of its position inside that word; inside the word
 // the distances are two running counts over the 32 bits, left to right and right to left.
+// FAST: rows of a multiple of 32 voxels in a 32-byte aligned mask (one 256-bit load per lane).
+template <bool FAST>
 __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ Row16Params P) {
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ 
     if (valid) {
         uint32_t v[8];
         const uint8_t* src = P.mask + row * P.n0 + 32 * w;
-        if ((P.n0 & 31) == 0 && (reinterpret_cast<uintptr_t>(P.mask) & 31u) == 0) {
+        if (FAST) {
             asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                          : "l"(src));

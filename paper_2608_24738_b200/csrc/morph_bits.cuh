@@ -11,8 +11,9 @@
 //                             is expanded to bytes and leaves as one 32-byte store.
 //   3. binary_fused2d_kernel  both steps in one launch for elements that reach over the last two axes only: a block
 //                             packs its lines and those within reach into shared memory and combines from there.
-// Requires at most 4 axes, a contiguous extent that is a multiple of 32, offsets along it within +-31, and 32-byte
-// aligned buffers; everything else runs on the byte kernels of morph.cuh.
+// Requires at most 4 axes, a contiguous extent that is a multiple of 32 with 32-byte aligned buffers (256-bit accesses)
+// or a multiple of 4 from 32 voxels on with 4-byte aligned buffers (the last word of a line is then ragged), and offsets
+// along the line within +-31; everything else runs on the byte kernels of morph.cuh.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -41,6 +42,7 @@ struct BitsParams {
     int words;               // words per line = last extent / 32
     int ext[kMaxDims];
     int border_value;
+    int fast;                // the contiguous extent is a multiple of 32 and both buffers are 32-byte aligned: 256-bit accesses
 };
 
 __device__ __forceinline__ uint32_t nonzero_bits4(uint32_t v) {
@@ -49,17 +51,52 @@ __device__ __forceinline__ uint32_t nonzero_bits4(uint32_t v) {
     return (((m >> 7) * 0x00204081u) >> 21) & 0xfu;
 }
 
-__global__ void __launch_bounds__(256) binary_pack_kernel(const __grid_constant__ BitsParams P) {
-    const int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // word index over the whole batch
-    if (w >= P.lines * P.words) return;
-    uint32_t v[8];  // one 256-bit load: a warp reads 1 KB in one request
-    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                 : "l"(P.in + w * 32));
+// Word w (32 voxels) of a line of W voxels as bits.  W is a multiple of 32 (fast: one 256-bit load; the buffer is
+// 32-byte aligned) or of 4 (4-byte loads; the voxels of a ragged last word beyond the line take the border value, like
+// every other position outside the image).
+__device__ __forceinline__ uint32_t bits_load_word(const uint8_t* line, const int w, const int W, const bool fast,
+                                                   const uint32_t fill) {
+    uint32_t v[8];
+    if (fast) {
+        asm("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"  // read-only data: free to be scheduled early
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+            : "l"(line + 32 * w));
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            v[i] = 32 * w + 4 * i < W ? __ldg(reinterpret_cast<const uint32_t*>(line + 32 * w) + i) : (fill & 0x01010101u);
+    }
     uint32_t bits = 0u;
 #pragma unroll
     for (int i = 0; i < 8; ++i) bits |= nonzero_bits4(v[i]) << (4 * i);
-    P.bits[w] = bits;
+    return bits;
+}
+
+// 32 result bits -> bytes (0 / 1) of word w of a line of W voxels.
+__device__ __forceinline__ void bits_store_word(uint8_t* line, const int w, const int W, const bool fast, const uint32_t acc) {
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t nib = (acc >> (4 * i)) & 0xfu;
+        o[i] = (nib * 0x00204081u) & 0x01010101u;
+    }
+    if (fast) {
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(line + 32 * w), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                     : "memory");
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (32 * w + 4 * i < W) reinterpret_cast<uint32_t*>(line + 32 * w)[i] = o[i];
+    }
+}
+
+__global__ void __launch_bounds__(256) binary_pack_kernel(const __grid_constant__ BitsParams P) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // word index over the whole batch
+    if (t >= P.lines * P.words) return;
+    const int64_t line = t / P.words;
+    const int w = (int)(t - line * P.words), W = P.ext[P.ndim - 1];
+    P.bits[t] = bits_load_word(P.in + line * W, w, W, P.fast, P.border_value ? 0xffffffffu : 0u);
 }
 
 // Block = 8 x 32 lanes (threadIdx.y, threadIdx.x); a lane produces word w of L consecutive lines, which differ only in
@@ -129,19 +166,9 @@ __global__ void __launch_bounds__(256) binary_lines_kernel(const __grid_constant
         if (all == (MIN ? 0u : 0xffffffffu)) break;  // decided for every voxel of the lane
     }
     // expand 32 bits to 32 bytes (0 / 1): one 256-bit store per line
+    const int W = P.ext[P.ndim - 1];
 #pragma unroll
-    for (int j = 0; j < L; ++j) {
-        uint32_t o[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t nib = (acc[j] >> (4 * i)) & 0xfu;
-            o[i] = (nib * 0x00204081u) & 0x01010101u;
-        }
-        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                     :: "l"(P.out + ((line0 + j) * P.words + w) * 32), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]),
-                        "r"(o[6]), "r"(o[7])
-                     : "memory");
-    }
+    for (int j = 0; j < L; ++j) bits_store_word(P.out + (line0 + j) * W, w, W, P.fast, acc[j]);
 }
 
 // Elements that reach over the last two axes only (every 2-D element): packing and combining in one kernel, without
@@ -151,7 +178,7 @@ __global__ void __launch_bounds__(256) binary_lines_kernel(const __grid_constant
 // the contiguous one (1 for a 1-D image).
 constexpr int kFusedReach = 8;  // |dy| of the element, at most
 
-template <bool MIN>
+template <bool MIN, bool FAST>
 __global__ void __launch_bounds__(256) binary_fused2d_kernel(const __grid_constant__ BitsParams P, const unsigned chunks,
                                                              const int H, const int dy_lo, const int dy_hi) {
     __shared__ uint32_t sbits[32 + 2 * kFusedReach][34];
@@ -160,6 +187,7 @@ __global__ void __launch_bounds__(256) binary_fused2d_kernel(const __grid_consta
     const int w0 = (int)ch * 32;
     const uint32_t fill = P.border_value ? 0xffffffffu : 0u;
     const int rows = 32 + dy_hi - dy_lo;
+    const int W = P.ext[P.ndim - 1];
 #pragma unroll 3
     for (int t = threadIdx.x; t < rows * 34; t += 256) {
         const int r = t / 34, c = t - r * 34;
@@ -168,14 +196,7 @@ __global__ void __launch_bounds__(256) binary_fused2d_kernel(const __grid_consta
         uint32_t bits = fill;  // words beyond the ends of a line hold the border value
         if (w >= 0 && w < P.words) {
             bits = 0u;
-            if (line >= 0 && line < P.lines) {
-                uint32_t v[8];
-                asm("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"  // read-only data: free to be scheduled early
-                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                    : "l"(P.in + (line * P.words + w) * 32));
-#pragma unroll
-                for (int i = 0; i < 8; ++i) bits |= nonzero_bits4(v[i]) << (4 * i);
-            }
+            if (line >= 0 && line < P.lines) bits = bits_load_word(P.in + line * W, w, W, FAST, fill);
         }
         sbits[r][c] = bits;
     }
@@ -224,16 +245,7 @@ __global__ void __launch_bounds__(256) binary_fused2d_kernel(const __grid_consta
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         if (line0 + j >= P.lines) break;
-        uint32_t o[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t nib = (acc[j] >> (4 * i)) & 0xfu;
-            o[i] = (nib * 0x00204081u) & 0x01010101u;
-        }
-        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                     :: "l"(P.out + ((line0 + j) * P.words + w) * 32), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]),
-                        "r"(o[6]), "r"(o[7])
-                     : "memory");
+        bits_store_word(P.out + (line0 + j) * W, w, W, FAST, acc[j]);
     }
 }
 

@@ -38,7 +38,7 @@ cudaError_t launch_row_dist16(const uint8_t* mask, uint16_t* out, int64_t rows, 
     Row16Params R;
     R.mask = mask; R.out = out; R.rows = rows; R.n0 = n0; R.words = n0 / 32; R.edge = nullptr; R.nb = 0;
     const int64_t warps = (rows + 32 / R.words - 1) / (32 / R.words);
-    cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
+    cdt_row16_kernel<true><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
     return cudaGetLastError();
 }
 
@@ -108,7 +108,8 @@ int tm_cdt(const uint8_t* input, int ndim, const int64_t* shape, int metric, int
         R.mask = input; R.out = f; R.rows = g.total / n0; R.n0 = n0; R.words = words;
         R.edge = chess && groups > 1 ? edge : nullptr; R.nb = groups - 1;
         const int64_t warps = (R.rows + 32 / R.words - 1) / (32 / R.words);
-        cdt_row16_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
+        if (n0 % 32 == 0) cdt_row16_kernel<true><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
+        else cdt_row16_kernel<false><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(R);
         SweepParams C;
         memset(&C, 0, sizeof(C));
         C.f = R.out; C.last = E == 2; C.out = C.last ? out_dist : tmp[1];

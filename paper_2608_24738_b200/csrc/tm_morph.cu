@@ -215,8 +215,10 @@ static int run_box_quads(const float* input, int ndim, const int64_t* fp_shape, 
 static int run_binary_bits(const Geometry& g, const std::vector<Entry>& entries, const uint8_t* input, uint8_t* output,
                            bool erosion, int border_value, cudaStream_t s) {
     const int nd = g.ndim, W = g.ext[nd - 1];
-    if (nd > 4 || W % 32 != 0 || ((uintptr_t)input & 31u) || ((uintptr_t)output & 31u)) return -1;
-    if ((g.total / W + 7) / 8 * ((W / 32 + 31) / 32) > (int64_t)INT32_MAX) return -1;  // blocks of the line kernel
+    const bool fast = W % 32 == 0 && !((uintptr_t)input & 31u) && !((uintptr_t)output & 31u);
+    if (nd > 4 || (!fast && (W % 4 != 0 || W < 32 || ((uintptr_t)input & 3u) || ((uintptr_t)output & 3u)))) return -1;
+    const int words_per_line = (W + 31) / 32;
+    if ((g.total / W + 7) / 8 * ((words_per_line + 31) / 32) > (int64_t)INT32_MAX) return -1;  // blocks of the line kernel
     std::vector<LineGroup> groups;
     for (const Entry& en : entries) {
         const int dx = en.off[nd - 1];
@@ -246,27 +248,32 @@ static int run_binary_bits(const Geometry& g, const std::vector<Entry>& entries,
             if (nd >= 2) { dy_lo = std::min(dy_lo, (int)c.off[nd - 2]); dy_hi = std::max(dy_hi, (int)c.off[nd - 2]); }
         }
         const int64_t lines = g.total / W;
-        const unsigned chunks = (unsigned)((W / 32 + 31) / 32);
+        const unsigned chunks = (unsigned)((words_per_line + 31) / 32);
         if (last_two && dy_lo >= -kFusedReach && dy_hi <= kFusedReach && (lines + 31) / 32 * chunks <= (int64_t)INT32_MAX) {
             BitsParams B;
             memset(&B, 0, sizeof(B));
             B.in = input; B.out = output;
             for (size_t i = 0; i < groups.size(); ++i) B.groups[i] = groups[i];
             B.n_groups = (int)groups.size();
-            B.ndim = nd; B.words = W / 32; B.lines = lines; B.lines_per_image = g.V / W;
+            B.ndim = nd; B.words = words_per_line; B.lines = lines; B.lines_per_image = g.V / W; B.fast = fast;
             for (int a = 0; a < nd; ++a) B.ext[a] = g.ext[a];
             B.border_value = border_value ? 1 : 0;
             const unsigned blocks = (unsigned)((lines + 31) / 32) * chunks;
             const int H = nd >= 2 ? g.ext[nd - 2] : 1;
-            if (erosion) binary_fused2d_kernel<true><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
-            else binary_fused2d_kernel<false><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+            if (fast) {
+                if (erosion) binary_fused2d_kernel<true, true><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+                else binary_fused2d_kernel<false, true><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+            } else {
+                if (erosion) binary_fused2d_kernel<true, false><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+                else binary_fused2d_kernel<false, false><<<blocks, 256, 0, s>>>(B, chunks, H, dy_lo, dy_hi);
+            }
             const cudaError_t e = cudaGetLastError();
             if (e != cudaSuccess) { tmedt::shared_record((int)e, 0); return TM_EDT_ERR_CUDA; }
             tmedt::shared_record(-1, 1);
             return TM_EDT_OK;
         }
     }
-    const int64_t words = g.total / 32;
+    const int64_t words = g.total / W * words_per_line;
     char* dev = nullptr;
     cudaError_t e = tmedt::shared_scratch_alloc((void**)&dev, (size_t)words * 4, s);
     if (e != cudaSuccess) { cudaGetLastError(); tmedt::shared_record((int)e, 0); return TM_EDT_ERR_ALLOC; }
@@ -276,7 +283,7 @@ static int run_binary_bits(const Geometry& g, const std::vector<Entry>& entries,
         B.in = input; B.out = output; B.bits = reinterpret_cast<uint32_t*>(dev);
         for (size_t i = 0; i < groups.size(); ++i) B.groups[i] = groups[i];
         B.n_groups = (int)groups.size();
-        B.ndim = nd; B.words = W / 32; B.lines = g.total / W; B.lines_per_image = g.V / W;
+        B.ndim = nd; B.words = words_per_line; B.lines = g.total / W; B.lines_per_image = g.V / W; B.fast = fast;
         for (int a = 0; a < nd; ++a) B.ext[a] = g.ext[a];
         B.border_value = border_value ? 1 : 0;
         const unsigned blocks = (unsigned)((words + 255) / 256);

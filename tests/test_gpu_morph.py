@@ -32,6 +32,9 @@ CASES = [
     # the same with four lines per lane (extent before the last a multiple of 4), 1 to 4 axes, and 5 axes (byte kernels)
     ((2, 1, 12, 8, 64), (3, 3, 3), None), ((1, 1, 3, 4, 8, 32), (3, 2, 3, 5), (0, 0, 1, -1)), ((2, 2, 64), (5,), None),
     ((1, 1, 2, 3, 5, 32), (2, 3, 3, 3), None), ((1, 1, 2, 3, 4, 4, 32), (1, 3, 3, 2, 3), None), ((3, 1, 40, 160), (5, 5), (1, -1)),
+    # rows of a multiple of 4 (from 32 voxels on): the last word of a line is ragged
+    ((2, 1, 9, 36), (3, 3), None), ((1, 1, 8, 100), (3, 7), (0, 2)), ((1, 1, 5, 6, 44), (3, 3, 3), None), ((2, 1, 40, 1000), (5, 5), None),
+    ((1, 2, 68), (9,), None),
 ]
 
 
@@ -141,7 +144,7 @@ def test_seeded_boxes_and_masks_on_the_strip_and_bit_kernels(seed):
     rng = np.random.default_rng(777 + seed)
     ndim = int(rng.integers(1, 4))
     bits = bool(rng.integers(0, 2))
-    last = (32 if bits else 4) * int(rng.integers(1, 9 if bits else 40))
+    last = (32 * int(rng.integers(1, 9)) if seed % 3 else 4 * int(rng.integers(8, 70))) if bits else 4 * int(rng.integers(1, 40))
     spatial = tuple(int(rng.integers(1, 40)) for _ in range(ndim - 1)) + (last,)
     shape = (int(rng.integers(1, 3)), int(rng.integers(1, 3))) + spatial
     fp_shape = tuple(int(rng.choice([1, 3, 5, 7, 9])) for _ in range(ndim))
