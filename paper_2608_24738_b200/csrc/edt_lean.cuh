@@ -37,6 +37,9 @@ struct LeanParams {
     int64_t in_elems;    // elements behind `in` and `out` (bounds checks of the debug build)
     int64_t out_elems;
     int64_t images;      // images behind the final outputs (bounds checks of the debug build)
+    int reverse;         // column kernels: walk the blocks backwards (a pass between the plane pass and the last one:
+                         // it starts with what the plane pass wrote last, still in L2, and ends with what the last pass,
+                         // walking forwards, reads first)
     int dist16;          // value kernels, 16-bit input: the input holds first-axis distances (>= 0xC000: no site in the
                          // row) instead of squared values; they are squared while the tile is staged
 };
@@ -381,8 +384,9 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
     const int n = P.n;
     uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_c);                                  // [n + 2 kLeanPad][TX]
     EI* et = reinterpret_cast<EI*>(sm_lean_c + (size_t)(n + 2 * kLeanPad) * TX * 4);        // [n][TX]
-    const int64_t slab = blockIdx.x / P.tiles_per_slab;
-    const int64_t i0 = (int64_t)(blockIdx.x - slab * P.tiles_per_slab) * TX;
+    const unsigned bid = P.reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
+    const int64_t slab = bid / P.tiles_per_slab;
+    const int64_t i0 = (int64_t)(bid - slab * P.tiles_per_slab) * TX;
     const int width = (int)min((int64_t)TX, P.inner - i0);
     const EI* src = reinterpret_cast<const EI*>(P.in) + slab * (int64_t)n * P.inner + i0;
     lean_fill_pad<TX>(kt, n);

@@ -207,6 +207,7 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
         const bool fin = k == pl.E - 1;
         P.in = src; P.out = dst;
         P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = weight(k);
+        P.reverse = fin ? 0 : 1;  // a pass between the plane pass and the last one walks its blocks backwards
         const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
         if (entries) {
             const double eb = (double)entry_bytes(k);
