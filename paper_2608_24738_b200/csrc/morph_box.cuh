@@ -30,6 +30,7 @@ struct StripParams {
     unsigned strip_groups;// groups of 8 strips per column of the walk axis
     int mode;             // border rule of both axes
     float cval;           // value of the constant rule
+    int reverse;          // walk the blocks backwards (every second pass: it starts with what the pass before wrote last)
 };
 
 template <bool MIN> __device__ __forceinline__ float pick(float a, float b) { return MIN ? fminf(a, b) : fmaxf(a, b); }
@@ -139,7 +140,7 @@ __device__ __forceinline__ void box_strip_body(const StripParams& P, const int64
 // chunk fastest.  A column is a pair (index over the axes before the walk axis, row within one position of it).
 template <bool MIN, int RH, int RV, int T>
 __global__ void __launch_bounds__(256) box_strip_kernel(const __grid_constant__ StripParams P) {
-    unsigned b = blockIdx.x;
+    unsigned b = P.reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
     const unsigned ch = b % P.chunks; b /= P.chunks;
     const unsigned sg = b % P.strip_groups;
     const unsigned col = b / P.strip_groups;

@@ -189,7 +189,7 @@ static int run_box_quads(const float* input, int ndim, const int64_t* fp_shape, 
         float* dst = i == np - 1 ? output : reinterpret_cast<float*>(ws + (size_t)(i & 1) * buf);
         StripParams B;
         memset(&B, 0, sizeof(B));
-        B.in = src; B.out = dst; B.W = W; B.mode = mode; B.cval = cval;
+        B.in = src; B.out = dst; B.W = W; B.mode = mode; B.cval = cval; B.reverse = i & 1;
         B.chunks = (unsigned)((W / 4 + 31) / 32);
         if (pass[i].axis >= 0) { B.n = g.ext[pass[i].axis]; B.walk_stride = g.stride[pass[i].axis]; }
         else { B.n = 1; B.walk_stride = W; }
