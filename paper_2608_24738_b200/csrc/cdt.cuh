@@ -172,7 +172,7 @@ __device__ __forceinline__ uint32_t cdt_nonzero_bits4(uint32_t v) {
 // the distances are two running counts over the 32 bits, left to right and right to left.
 // FAST: rows of a multiple of 32 voxels in a 32-byte aligned mask (one 256-bit load per lane).
 template <bool FAST>
-__global__ void __launch_bounds__(256) cdt_row16_kernel(const __grid_constant__ Row16Params P) {
+__global__ void __launch_bounds__(256, 4) cdt_row16_kernel(const __grid_constant__ Row16Params P) {
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int words = P.words, rpw = 32 / words;
