@@ -139,7 +139,7 @@ __device__ __forceinline__ void box_strip_body(const StripParams& P, const int64
 // Block = 8 strips x 32 quads.  Blocks enumerate (column of the walk axis, group of 8 strips, chunk of 128 voxels),
 // chunk fastest.  A column is a pair (index over the axes before the walk axis, row within one position of it).
 template <bool MIN, int RH, int RV, int T>
-__global__ void __launch_bounds__(256) box_strip_kernel(const __grid_constant__ StripParams P) {
+__global__ void __launch_bounds__(256, (RH <= 1 && RV <= 1) ? 3 : 2) box_strip_kernel(const __grid_constant__ StripParams P) {
     unsigned b = P.reverse ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
     const unsigned ch = b % P.chunks; b /= P.chunks;
     const unsigned sg = b % P.strip_groups;
