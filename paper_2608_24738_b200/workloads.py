@@ -134,3 +134,17 @@ def random_mask(seed: int, shape, p_fg: float) -> np.ndarray:
     """Bernoulli(p_fg) foreground mask of the given (B, C, spatial...) shape, for the small parity cases."""
     rng = np.random.default_rng(seed)
     return (rng.random(tuple(shape)) < p_fg).astype(np.uint8)
+
+
+def large_random_mask(seed: int, shape, p_fg: float) -> np.ndarray:
+    """Bernoulli foreground mask for shapes of billions of voxels: one random byte per voxel, drawn in pieces,
+    foreground where the byte is below round(256 p_fg)."""
+    rng = np.random.default_rng(seed)
+    out = np.empty(tuple(shape), dtype=np.uint8)
+    flat = out.reshape(-1)
+    threshold = int(round(256 * p_fg))
+    piece = 1 << 26
+    for start in range(0, flat.size, piece):
+        n = min(piece, flat.size - start)
+        flat[start:start + n] = rng.integers(0, 256, n, dtype=np.uint8) < threshold
+    return out
