@@ -188,3 +188,63 @@ def test_one_image_of_just_under_2_31_voxels(spatial, with_indices, side, near_r
     far = _check_windows_against_the_oracle(mask[0, 0], dist, sq, spatial, pts[-41:], far_radius)
     assert near >= 450 and far >= 30
     assert float(dist[centre]) >= side // 2 - 1
+
+
+def _repeated_batch(first, images):
+    import torch
+
+    distinct = first.shape[0]
+    t = torch.from_numpy(first).cuda()[torch.arange(images, device="cuda") % distinct].contiguous()
+    assert t.numel() > 2**31
+    return t
+
+
+def _every_copy_equals_the_first(out, want, distinct):
+    """out: result of a batch that repeats `distinct` images; want: the oracle's result for those."""
+    assert out.numel() > 2**31
+    for k in range(distinct):
+        copies = out[k::distinct]
+        assert bool((copies == copies[:1]).all()), "image %d: a copy differs" % k
+    assert np.array_equal(out[:distinct].cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("what", ["grey", "binary", "cdt"])
+def test_morphology_and_cdt_on_batches_of_more_than_2_31_voxels(what):
+    """tm_grey_morph, tm_binary_morph and tm_cdt take such a batch in one launch per pass (64-bit offsets)."""
+    import torch
+    from oracle import cdt_oracle as co
+    from oracle import morph_oracle as mo
+
+    _need_memory(40)
+    spatial, distinct = ((256, 1024) if what == "cdt" else (512, 1024)), 3
+    images = 2**31 // int(np.prod(spatial)) + 2 * distinct + 1
+    rng = np.random.default_rng(99)
+    box = np.ones((3, 3), dtype=bool)
+    cross = np.array([[0, 1, 0], [1, 1, 1], [0, 1, 0]], dtype=bool)
+    if what == "grey":
+        first = rng.normal(size=(distinct, 1) + spatial).astype(np.float32)
+        t = _repeated_batch(first, images)
+        got = binding.tm_grey_morph(t, box, None, op="erosion", mode="reflect")
+        _every_copy_equals_the_first(got, mo.grey_erosion(first, box, None, "reflect"), distinct)
+        del got
+        weights = rng.normal(size=(3, 3)).astype(np.float32)
+        got = binding.tm_grey_morph(t, cross, weights, op="dilation", mode="nearest")
+        _every_copy_equals_the_first(got, mo.grey_dilation(first, cross, weights, "nearest"), distinct)
+    elif what == "binary":
+        first = workloads.random_mask(31, (distinct, 1) + spatial, 0.8)
+        t = _repeated_batch(first, images)
+        got = binding.tm_binary_morph(t, box, op="erosion", border_value=1)
+        _every_copy_equals_the_first(got, mo.binary_erosion(first, box, 1), distinct)
+        del got
+        got = binding.tm_binary_morph(t, cross, op="dilation", border_value=0)
+        _every_copy_equals_the_first(got, mo.binary_dilation(first, cross, 0), distinct)
+    else:
+        first = workloads.random_mask(32, (distinct, 1) + spatial, 0.98)
+        first[1] = 1  # an image without background
+        first[2, 0, 100:160, 200:500] = 1
+        t = _repeated_batch(first, images)
+        for metric in ("chessboard", "taxicab"):
+            got = binding.tm_cdt(t, metric)
+            _every_copy_equals_the_first(got, co.separable(first, metric), distinct)
+            del got
+    torch.cuda.synchronize()
