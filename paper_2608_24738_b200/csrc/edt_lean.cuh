@@ -485,7 +485,8 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
 template <bool FINAL, typename VT, int TX, int NW = 8>
 __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_constant__ LeanParams P,
                                                             const __grid_constant__ EpilogueParams ep) {
-    constexpr int LPR = TX / 4, CG = TX / 32;
+    // tiles of 8 or 16 columns (axes beyond 1024 rows): a warp's patch is 16 or 8 rows of the whole tile width
+    constexpr int LPR = TX / 4, CG = TX >= 32 ? TX / 32 : 1, RPW = TX >= 32 ? 4 : 128 / TX;
     extern __shared__ __align__(16) uint8_t sm_lean_v[];
     const int n = P.n;
     uint32_t* kt = reinterpret_cast<uint32_t*>(sm_lean_v);  // [n + 2 kLeanPad][TX]
@@ -524,9 +525,9 @@ __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_consta
     }
     const int any_site = __syncthreads_or((all & kLeanNone) == 0u);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int c4 = 32 * (warp % CG) + 4 * (lane & 7);
-    const int yfirst = 4 * (warp / CG) + (lane >> 3);
-    constexpr int YSTEP = 4 * (NW / CG);
+    const int c4 = TX >= 32 ? 32 * (warp % CG) + 4 * (lane & 7) : 4 * (lane % LPR);
+    const int yfirst = TX >= 32 ? 4 * (warp / CG) + (lane >> 3) : RPW * warp + lane / LPR;
+    constexpr int YSTEP = RPW * (NW / CG);
     if (c4 >= width) return;
     const int64_t col = slab * (int64_t)n * P.inner + i0 + c4;  // FINAL: the slab is the image
     const LeanTile T = {kt, (n + 2 * kLeanPad) * TX};

@@ -66,6 +66,9 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
 
 // One axis pass of the wide-key path on plain integer values with the quad kernels (see tm_edt_lean.cu).
 bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
+bool lean_value_long_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
+cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
+                                     cudaStream_t st);
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
                                 cudaStream_t st, bool dist16 = false);
 

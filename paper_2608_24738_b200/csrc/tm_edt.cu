@@ -787,23 +787,41 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
         ++launches;
         return cudaGetLastError();
     };
-    A.h_in = hA; A.offs_in = offsA; A.h_out = hB; A.offs_out = carry ? offsB : nullptr;
-    unsigned blocks = set_axis(1);
-    e = block_minima();
-    if (e != cudaSuccess) return e;
-    if (pl.E == 2) {
-        prof_mark(st, "long_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
-        long_axis_kernel<1, true, FLT><<<blocks, 256, 0, st>>>(A, ep);
+    // unit sampling without index output: an axis of up to 4096 rows still fits a shared-memory tile (32 columns wide
+    // up to 1024 rows, 16 or 8 beyond), and the quad value kernel takes the pass instead of the scans through the cache
+    auto tile_axis = [&](int k) {
+        if (FLT || carry || switches().no_lean) return 0;
+        return lean_value_axis_ok(pl, k, ep) ? 1 : (lean_value_long_axis_ok(pl, k, ep) ? 2 : 0);
+    };
+    auto run_tile_axis = [&](int k, const void* src, void* dst, bool fin) -> cudaError_t {
+        prof_mark(st, fin ? "long_tile_final" : "long_tile", (double)pl.N * (4.0 + (fin ? out_bpv : 4.0)));
         ++launches;
-        return cudaGetLastError();
+        return tile_axis(k) == 1 ? run_lean_value_axis(pl, k, src, dst, ep, fin, st) : run_lean_value_long_axis(pl, k, src, dst, ep, fin, st);
+    };
+    {
+        const bool fin = pl.E == 2;
+        if (tile_axis(1)) {
+            e = run_tile_axis(1, hA, fin ? nullptr : hB, fin);
+        } else {
+            A.h_in = hA; A.offs_in = offsA; A.h_out = hB; A.offs_out = carry ? offsB : nullptr;
+            const unsigned blocks = set_axis(1);
+            e = block_minima();
+            if (e != cudaSuccess) return e;
+            if (fin) {
+                prof_mark(st, "long_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 2.0 : 0.0)));
+                long_axis_kernel<1, true, FLT><<<blocks, 256, 0, st>>>(A, ep);
+            } else {
+                prof_mark(st, "long_axis", (double)pl.N * (4.0 + 4.0 + (carry ? 2.0 + 4.0 : 0.0)));
+                long_axis_kernel<1, false, FLT><<<blocks, 256, 0, st>>>(A, ep);
+            }
+            ++launches;
+            e = cudaGetLastError();
+        }
+        if (e != cudaSuccess || fin) return e;
     }
-    prof_mark(st, "long_axis", (double)pl.N * (4.0 + 4.0 + (carry ? 2.0 + 4.0 : 0.0)));
-    long_axis_kernel<1, false, FLT><<<blocks, 256, 0, st>>>(A, ep);
-    ++launches;
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (tile_axis(2)) return run_tile_axis(2, hB, nullptr, true);
     A.h_in = hB; A.offs_in = offsB; A.h_out = nullptr; A.offs_out = nullptr;
-    blocks = set_axis(2);
+    const unsigned blocks = set_axis(2);
     e = block_minima();
     if (e != cudaSuccess) return e;
     prof_mark(st, "long_axis_final", (double)pl.N * (4.0 + out_bpv + (ep.idx ? 4.0 : 0.0)));

@@ -166,6 +166,48 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
                : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
 }
 
+// The same pass on axes of 1025 .. 4096 rows: the whole column still fits a shared-memory tile if the tile is only
+// 16 or 8 columns wide (one block of 32 warps per SM); 32-bit values in, values or final outputs out.
+static int lean_value_long_tile(int n) {
+    if ((size_t)(n + 2 * kLeanPad) * 16 * 4 <= 136 * 1024) return 16;
+    if ((size_t)(n + 2 * kLeanPad) * 8 * 4 <= 136 * 1024) return 8;
+    return 0;
+}
+
+bool lean_value_long_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
+    if (!pl.unit || ep.idx || pl.ext[0] % 4 != 0) return false;
+    if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
+    const int n = pl.ext[k], tx = lean_value_long_tile(n);
+    if (n <= 1024 || tx == 0) return false;
+    const int64_t blocks = pl.N / ((int64_t)n * pl.inner[k]) * ((pl.inner[k] + tx - 1) / tx);
+    return blocks >= 148;
+}
+
+template <bool FINAL, int TX>
+static cudaError_t launch_lean_value_long(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
+    const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4;
+    P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
+    auto kern = lean_value_kernel<FINAL, uint32_t, TX, 32>;
+    cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)(outer * P.tiles_per_slab), 1024, smem, st>>>(P, ep);
+    return cudaGetLastError();
+}
+
+cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
+                                     cudaStream_t st) {
+    LeanParams P;
+    memset(&P, 0, sizeof(P));
+    P.in = in; P.out = out;
+    P.in_elems = pl.N; P.out_elems = pl.N; P.images = pl.images;
+    P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
+    P.inv_scale = 1.0f;
+    const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+    if (lean_value_long_tile(P.n) == 16)
+        return fin ? launch_lean_value_long<true, 16>(P, ep, outer, st) : launch_lean_value_long<false, 16>(P, ep, outer, st);
+    return fin ? launch_lean_value_long<true, 8>(P, ep, outer, st) : launch_lean_value_long<false, 8>(P, ep, outer, st);
+}
+
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches) {
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     char* bufA = static_cast<char*>(ws);

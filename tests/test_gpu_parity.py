@@ -279,6 +279,37 @@ def test_long_line_far_sites(pattern, kind):
     full_check(mask[None, None], _sampling(2, kind))
 
 
+NARROW = [((1, 1, 1100, 2400), 2), ((1, 1, 2200, 1188), 2), ((1, 1, 4096, 1184), 2), ((1, 1, 1032, 2404), 2),
+          ((2, 1, 1030, 40, 32), 3), ((1, 1, 1500, 40, 64), 3), ((1, 1, 4340, 1200), 2)]
+
+
+@pytest.mark.parametrize("shape,launches", NARROW, ids=["x".join(map(str, s)) for s, _ in NARROW])
+def test_long_axes_on_narrow_tiles(shape, launches):
+    """Unit sampling without index output: an axis of 1025 .. 4344 rows runs on the quad value kernel with tiles of 16
+    or 8 columns (whole and ragged last tiles, two and three axes, the longest axis that fits).  Dense background,
+    blobs and a handful of sites (scans over thousands of rows), distances and exact squared distances."""
+    import torch
+
+    seed = zlib.crc32(repr(shape).encode())
+    rng = np.random.default_rng(seed)
+    dense = workloads.random_mask(seed, shape, 0.97)
+    blobs = workloads.random_mask(seed + 1, shape, 0.999)
+    sp = shape[2:]
+    for _ in range(6):  # boxes of background
+        lo = [int(rng.integers(0, n)) for n in sp]
+        blobs[(slice(None), slice(None)) + tuple(slice(l, l + max(2, n // 5)) for l, n in zip(lo, sp))] = 0
+    sparse = np.ones(shape, dtype=np.uint8)
+    for _ in range(5):
+        sparse[(0, 0) + tuple(int(rng.integers(0, n)) for n in sp)] = 0
+    if shape[0] > 1:
+        sparse[-1] = 1  # an image without background
+    for mask in (dense, blobs, sparse):
+        ref = oracle.sep(mask, None, want_idx=False)
+        res = run_gpu(mask, None, dist=True, sq=True, idx=False)
+        assert binding.tm_edt_last_launch_count() == launches
+        compare(mask, None, res, ref, True, True, False)
+
+
 def test_sparse_background_long_axis_exactness():
     """Few background voxels and large extents: squared distances up to ~1e7 must stay exact."""
     mask = np.ones((1, 1, 2048, 300), dtype=np.uint8)
