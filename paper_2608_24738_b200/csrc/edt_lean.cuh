@@ -485,7 +485,7 @@ __global__ void __launch_bounds__(256, FINAL ? 6 : 8) lean_column_kernel(const _
 template <bool FINAL, typename VT, int TX, int NW = 8>
 __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_constant__ LeanParams P,
                                                             const __grid_constant__ EpilogueParams ep) {
-    // tiles of 8 or 16 columns (axes beyond 1024 rows): a warp's patch is 16 or 8 rows of the whole tile width
+    // tiles of 4, 8 or 16 columns (axes beyond 1024 rows): a warp's patch is 32, 16 or 8 rows of the whole tile width
     constexpr int LPR = TX / 4, CG = TX >= 32 ? TX / 32 : 1, RPW = TX >= 32 ? 4 : 128 / TX;
     extern __shared__ __align__(16) uint8_t sm_lean_v[];
     const int n = P.n;

@@ -787,8 +787,8 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
         ++launches;
         return cudaGetLastError();
     };
-    // unit sampling without index output: an axis of up to 4096 rows still fits a shared-memory tile (32 columns wide
-    // up to 1024 rows, 16 or 8 beyond), and the quad value kernel takes the pass instead of the scans through the cache
+    // unit sampling without index output: every axis still fits a shared-memory tile (32 columns wide up to 1024
+    // rows, 16, 8 or 4 beyond), and the quad value kernel takes the pass instead of the scans through the cache
     auto tile_axis = [&](int k) {
         if (FLT || carry || switches().no_lean) return 0;
         return lean_value_axis_ok(pl, k, ep) ? 1 : (lean_value_long_axis_ok(pl, k, ep) ? 2 : 0);

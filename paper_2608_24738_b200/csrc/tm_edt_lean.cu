@@ -166,11 +166,15 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
                : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
 }
 
-// The same pass on axes of 1025 .. 4096 rows: the whole column still fits a shared-memory tile if the tile is only
-// 16 or 8 columns wide (one block of 32 warps per SM); 32-bit values in, values or final outputs out.
+// The same pass on axes beyond 1024 rows: the whole column still fits a shared-memory tile if the tile is only 16, 8
+// or 4 columns wide (one block of 32 warps per SM); 32-bit values in, values or final outputs out.
 static int lean_value_long_tile(int n) {
-    if ((size_t)(n + 2 * kLeanPad) * 16 * 4 <= 136 * 1024) return 16;
-    if ((size_t)(n + 2 * kLeanPad) * 8 * 4 <= 136 * 1024) return 8;
+    const size_t rows = (size_t)(n + 2 * kLeanPad);
+    // one block per SM; narrower tiles that would let two blocks share an SM are not faster (4096 rows: 0.408 ms with
+    // 4 columns and two blocks against 0.400 ms with 8 columns and one)
+    if (rows * 16 * 4 <= 136 * 1024) return 16;
+    if (rows * 8 * 4 <= 136 * 1024) return 8;
+    if (rows * 4 * 4 <= 136 * 1024) return 4;
     return 0;
 }
 
@@ -203,9 +207,12 @@ cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void
     P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
     P.inv_scale = 1.0f;
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
-    if (lean_value_long_tile(P.n) == 16)
+    const int tx = lean_value_long_tile(P.n);
+    if (tx == 16)
         return fin ? launch_lean_value_long<true, 16>(P, ep, outer, st) : launch_lean_value_long<false, 16>(P, ep, outer, st);
-    return fin ? launch_lean_value_long<true, 8>(P, ep, outer, st) : launch_lean_value_long<false, 8>(P, ep, outer, st);
+    if (tx == 8)
+        return fin ? launch_lean_value_long<true, 8>(P, ep, outer, st) : launch_lean_value_long<false, 8>(P, ep, outer, st);
+    return fin ? launch_lean_value_long<true, 4>(P, ep, outer, st) : launch_lean_value_long<false, 4>(P, ep, outer, st);
 }
 
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches) {

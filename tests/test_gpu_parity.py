@@ -280,13 +280,15 @@ def test_long_line_far_sites(pattern, kind):
 
 
 NARROW = [((1, 1, 1100, 2400), 2), ((1, 1, 2200, 1188), 2), ((1, 1, 4096, 1184), 2), ((1, 1, 1032, 2404), 2),
-          ((2, 1, 1030, 40, 32), 3), ((1, 1, 1500, 40, 64), 3), ((1, 1, 4340, 1200), 2)]
+          ((2, 1, 1030, 40, 32), 3), ((1, 1, 1500, 40, 64), 3), ((1, 1, 4344, 1200), 2), ((1, 1, 4345, 600), 2),
+          ((1, 1, 8192, 592), 2)]
 
 
 @pytest.mark.parametrize("shape,launches", NARROW, ids=["x".join(map(str, s)) for s, _ in NARROW])
 def test_long_axes_on_narrow_tiles(shape, launches):
-    """Unit sampling without index output: an axis of 1025 .. 4344 rows runs on the quad value kernel with tiles of 16
-    or 8 columns (whole and ragged last tiles, two and three axes, the longest axis that fits).  Dense background,
+    """Unit sampling without index output: an axis beyond 1024 rows runs on the quad value kernel with tiles of 16, 8
+    or 4 columns (whole and ragged last tiles, two and three axes, the extents at which the tile width changes, the
+    longest axis of the interface).  Dense background,
     blobs and a handful of sites (scans over thousands of rows), distances and exact squared distances."""
     import torch
 
