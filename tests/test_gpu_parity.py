@@ -281,7 +281,7 @@ def test_long_line_far_sites(pattern, kind):
 
 NARROW = [((1, 1, 1100, 2400), 2), ((1, 1, 2200, 1188), 2), ((1, 1, 4096, 1184), 2), ((1, 1, 1032, 2404), 2),
           ((2, 1, 1030, 40, 32), 3), ((1, 1, 1500, 40, 64), 3), ((1, 1, 4344, 1200), 2), ((1, 1, 4345, 600), 2),
-          ((1, 1, 8192, 592), 2)]
+          ((1, 1, 8192, 592), 2), ((1, 1, 2168, 2368), 2), ((1, 1, 2169, 1184), 2)]
 
 
 @pytest.mark.parametrize("shape,launches", NARROW, ids=["x".join(map(str, s)) for s, _ in NARROW])
