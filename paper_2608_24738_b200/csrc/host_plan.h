@@ -46,6 +46,7 @@ struct Switches {
     bool old_plane = false;       // TM_EDT_OLD_PLANE=1: byte-load plane kernel
     bool no_value_carry = false;  // TM_EDT_NO_VALUE_CARRY: offsets are carried even without an index output
     bool no_lean = false;         // TM_EDT_NO_LEAN: one-voxel-per-lane kernels instead of the quad kernels
+    bool no_narrow_tiles = false; // TM_EDT_NO_NARROW_TILES: a single image with few columns stays on wide_axis_kernel
     long long chunk_voxels = 0;   // TM_EDT_CHUNK_VOXELS=n: image ranges of at most n voxels (0 = grid limit)
     bool debug_inject = false;    // TM_EDT_DEBUG_INJECT=1, debug build only: the bounds checks get a bound that is too small
 };

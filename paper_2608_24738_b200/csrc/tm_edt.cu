@@ -43,6 +43,7 @@ static void load_switches_locked() {
     s.old_plane = on("TM_EDT_OLD_PLANE");
     s.no_value_carry = set("TM_EDT_NO_VALUE_CARRY");
     s.no_lean = set("TM_EDT_NO_LEAN");
+    s.no_narrow_tiles = set("TM_EDT_NO_NARROW_TILES");
     s.debug_inject = on("TM_EDT_DEBUG_INJECT");
     s.chunk_voxels = 0;
     if (const char* lim = getenv("TM_EDT_CHUNK_VOXELS")) { const long long v = atoll(lim); if (v > 0) s.chunk_voxels = v; }

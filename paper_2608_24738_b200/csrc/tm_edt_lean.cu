@@ -107,7 +107,7 @@ template <bool FINAL, typename VT, int TX>
 static cudaError_t launch_lean_value_tx(LeanParams P, const EpilogueParams& ep, int64_t outer, cudaStream_t st) {
     const size_t smem = (size_t)(P.n + 2 * kLeanPad) * TX * 4;
     P.tiles_per_slab = (int)((P.inner + TX - 1) / TX);
-    if (TX == 32 && P.n >= 384) {  // very long axes: two blocks per SM, 32 warps each
+    if (TX < 32 || P.n >= 384) {  // very long axes, narrow tiles: two blocks per SM, 32 warps each
         auto kern = lean_value_kernel<FINAL, VT, TX, 32>;
         cudaError_t e = ensure_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) return e;
@@ -138,14 +138,26 @@ static cudaError_t launch_lean_value(const LeanParams& P, const EpilogueParams& 
 
 // One axis pass of the wide-key path on plain integer values (unit sampling, no index output, extents up to 1024)
 // with the quad kernel lean_value_kernel: `in` / `out` hold one 32-bit value per voxel (2^31 = no site).
+// Columns per tile on axis k: 32 where that gives every SM its blocks; with few columns (a single image) and 384
+// rows or more, tiles of 16 or 8 columns; 0 = too few tiles even so (wide_axis_kernel splits its strips over several
+// blocks instead) or too many rows.
+static int lean_value_tile(const Plan& pl, int k) {
+    const int n = pl.ext[k];
+    const size_t smem = (size_t)(n + 2 * kLeanPad) * 32 * 4;
+    if (smem > 136 * 1024) return 0;  // up to 1024 rows (one block of 32 warps per SM beyond 100 KB)
+    const int64_t outer = pl.N / ((int64_t)n * pl.inner[k]);
+    auto blocks = [&](int tx) { return outer * ((pl.inner[k] + tx - 1) / tx); };
+    if (blocks(32) >= (smem > 100 * 1024 ? 148 : 296)) return 32;
+    if (n < 384 || switches().no_narrow_tiles) return 0;
+    if (blocks(16) >= 148) return 16;
+    if (blocks(8) >= 96) return 8;
+    return 0;
+}
+
 bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
     if (!pl.unit || ep.idx || pl.ext[0] % 4 != 0) return false;
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
-    const int n = pl.ext[k];
-    const size_t smem = (size_t)(n + 2 * kLeanPad) * 32 * 4;
-    if (smem > 136 * 1024) return false;  // up to 1024 rows (one block of 32 warps per SM beyond 100 KB)
-    const int64_t blocks = pl.N / ((int64_t)n * pl.inner[k]) * ((pl.inner[k] + 31) / 32);
-    return blocks >= (smem > 100 * 1024 ? 148 : 296);  // few strips (a single image) are split over several blocks by wide_axis_kernel instead
+    return lean_value_tile(pl, k) != 0;
 }
 
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
@@ -157,11 +169,20 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
     P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
     P.inv_scale = 1.0f;
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
+    const int tx = lean_value_tile(pl, k);
     if (dist16) {  // 16-bit first-axis distances in; final outputs or 32-bit values out
         P.dist16 = 1;
+        if (tx == 16) return fin ? launch_lean_value_tx<true, uint16_t, 16>(P, ep, outer, st)
+                                 : launch_lean_value_tx<false, uint16_t, 16>(P, ep, outer, st);
+        if (tx == 8) return fin ? launch_lean_value_tx<true, uint16_t, 8>(P, ep, outer, st)
+                                : launch_lean_value_tx<false, uint16_t, 8>(P, ep, outer, st);
         return fin ? launch_lean_value_tx<true, uint16_t, 32>(P, ep, outer, st)
                    : launch_lean_value_tx<false, uint16_t, 32>(P, ep, outer, st);
     }
+    if (tx == 16) return fin ? launch_lean_value_tx<true, uint32_t, 16>(P, ep, outer, st)
+                             : launch_lean_value_tx<false, uint32_t, 16>(P, ep, outer, st);
+    if (tx == 8) return fin ? launch_lean_value_tx<true, uint32_t, 8>(P, ep, outer, st)
+                            : launch_lean_value_tx<false, uint32_t, 8>(P, ep, outer, st);
     return fin ? launch_lean_value_tx<true, uint32_t, 32>(P, ep, outer, st)
                : launch_lean_value_tx<false, uint32_t, 32>(P, ep, outer, st);
 }

@@ -312,6 +312,37 @@ def test_long_axes_on_narrow_tiles(shape, launches):
         compare(mask, None, res, ref, True, True, False)
 
 
+FEW_COLUMNS = [(1, 1, 1024, 1024), (1, 1, 600, 800), (1, 1, 400, 2400), (1, 1, 384, 772), (1, 1, 500, 1000),
+               (1, 1, 400, 24, 32), (1, 1, 2, 500, 800), (2, 1, 1000, 512)]
+
+
+@pytest.mark.parametrize("shape", FEW_COLUMNS, ids=["x".join(map(str, s)) for s in FEW_COLUMNS])
+def test_single_images_on_narrow_tiles(shape, switches):
+    """A single image has too few columns to give every SM a 32-column tile of the value kernel: axes of 384 rows and
+    more then run on tiles of 16 or 8 columns (16-bit row distances or 32-bit values in, final outputs or values out,
+    ragged last tiles).  Distances and exact squared distances against the oracle, and squared distances bit-identical
+    to the strip kernel such shapes ran on before."""
+    seed = zlib.crc32(repr(shape).encode())
+    rng = np.random.default_rng(seed)
+    blobs = workloads.random_mask(seed, shape, 0.998)
+    sp = shape[2:]
+    for _ in range(5):
+        lo = [int(rng.integers(0, n)) for n in sp]
+        blobs[(slice(None), slice(None)) + tuple(slice(l, l + max(2, n // 4)) for l, n in zip(lo, sp))] = 0
+    sparse = np.ones(shape, dtype=np.uint8)
+    for _ in range(4):
+        sparse[(0, 0) + tuple(int(rng.integers(0, n)) for n in sp)] = 0
+    for mask in (workloads.random_mask(seed + 1, shape, 0.95), blobs, sparse):
+        ref = oracle.sep(mask, None, want_idx=False)
+        res = run_gpu(mask, None, dist=True, sq=True, idx=False)
+        assert binding.tm_edt_last_launch_count() == len(sp)
+        compare(mask, None, res, ref, True, True, False)
+        switches.set("TM_EDT_NO_NARROW_TILES", "1")
+        old = run_gpu(mask, None, dist=False, sq=True, idx=False)
+        switches.set("TM_EDT_NO_NARROW_TILES", None)
+        assert np.array_equal(old["sq"], res["sq"])
+
+
 def test_sparse_background_long_axis_exactness():
     """Few background voxels and large extents: squared distances up to ~1e7 must stay exact."""
     mask = np.ones((1, 1, 2048, 300), dtype=np.uint8)
