@@ -33,7 +33,7 @@ struct SmallParams {
 };
 
 template <bool SITE, bool FIRST, bool FINAL, int NMAX>
-__global__ void __launch_bounds__(kSmallThreads) small_group_kernel(const __grid_constant__ SmallParams P,
+__global__ void __launch_bounds__(kSmallThreads, (!SITE && NMAX <= 6) ? 4 : 1) small_group_kernel(const __grid_constant__ SmallParams P,
                                                           const __grid_constant__ EpilogueParams ep) {
     extern __shared__ __align__(16) unsigned char small_smem[];
     float* sv = reinterpret_cast<float*>(small_smem);
