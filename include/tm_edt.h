@@ -161,8 +161,10 @@ TM_EDT_API unsigned long long tm_edt_debug_last_violation(long long* code, long 
 
 /*
  * Debug and test switches (environment variables TM_EDT_FORCE_GENERIC, TM_EDT_NO_SCALED, TM_EDT_OLD_PLANE,
- * TM_EDT_NO_VALUE_CARRY, TM_EDT_NO_LEAN, TM_EDT_CHUNK_VOXELS; none changes any result) are read from the
- * environment once, at the first call that plans a transform.  This call reads them again.
+ * TM_EDT_NO_VALUE_CARRY, TM_EDT_NO_LEAN, TM_EDT_NO_NARROW_TILES, TM_EDT_CHUNK_VOXELS; they select kernel families
+ * and change no exact result -- squared distances and sites stay the same, a float32 distance can differ in its last
+ * bit between families) are read from the environment once, at the first call that plans a transform.  This call
+ * reads them again.
  */
 TM_EDT_API void tm_edt_reload_switches(void);
 
