@@ -604,6 +604,42 @@ def test_random_large_extents(chunk):
             raise AssertionError("shape %r sampling %r p_fg %r seed %r: %s" % (shape, samp, p_fg, seed, exc))
 
 
+def _value_path_cases(count, seed):
+    """Unit sampling without index output: shapes that take the value kernel on tiles of 32, 16, 8 or 4 columns."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    for _ in range(count):
+        kind = int(rng.integers(0, 4))
+        if kind == 0:    # one image, few columns, up to 1024 rows
+            spatial = (int(rng.integers(384, 1025)), 4 * int(rng.integers(192, 600)))
+        elif kind == 1:  # beyond 1024 rows
+            n = int(rng.integers(1025, 8193))
+            spatial = (n, 4 * int(rng.integers(148, max(149, min(700, 5_000_000 // (4 * n))))))
+        elif kind == 2:  # three axes, the long one outermost or in the middle
+            n = int(rng.integers(384, 3000))
+            rest = (4 * int(rng.integers(2, 10)), 4 * int(rng.integers(8, 40)))
+            spatial = (n,) + rest if rng.random() < 0.5 else (rest[0], n, rest[1])
+        else:            # a batch of medium images
+            spatial = (int(rng.integers(384, 700)), 32 * int(rng.integers(4, 17)))
+        batch = int(rng.integers(2, 6)) if kind == 3 else 1
+        cases.append(((batch, 1) + spatial, float(rng.choice([0.5, 0.9, 0.99, 0.9995])), int(rng.integers(0, 2**31))))
+    return cases
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_random_shapes_without_indices_beyond_128(chunk):
+    """Seeded fuzzing of the value-carrying passes beyond extent 128 (the tile width follows the shape)."""
+    for shape, p_fg, seed in _value_path_cases(6, 3000 + chunk):
+        mask = workloads.random_mask(seed, shape, p_fg)
+        mask[0, 0].flat[seed % mask[0, 0].size] = 0
+        ref = oracle.sep(mask, None, want_idx=False)
+        res = run_gpu(mask, None, dist=True, sq=True, idx=False)
+        try:
+            compare(mask, None, res, ref, True, True, False)
+        except AssertionError as exc:  # name the case
+            raise AssertionError("shape %r p_fg %r seed %r: %s" % (shape, p_fg, seed, exc))
+
+
 F64_SHAPES = [(2, 1, 7), (2, 1, 40, 36), (2, 1, 12, 20, 24), (2, 1, 140, 150), (2, 1, 6, 5, 4, 7), (2, 1, 9, 9, 9, 9, 9, 9)]
 
 
