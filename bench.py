@@ -597,7 +597,7 @@ def run_ex(args):
 def run_long(args):
     """Measurement of the paths for extents beyond 128 (wide-key and long-line kernels; a later row of the scope, its
     own line): the paper's 2-D 1024^2 row at B = 8, one 4096^2 image and one 512^3 volume; blob masks (disks / balls as
-    in workload C2, radii 0.02 .. 0.12 of the extent), unit sampling, float32 distances.  HBM roofline = mask in +
+    in workload C2, radii 0.02 .. 0.12 of the extent), unit sampling (and one case with decimal sampling), float32 distances.  HBM roofline = mask in +
     distances out once (5 B/voxel); the oracle is timed on a bounded sample of each case."""
     import numpy as np
     import torch
@@ -627,16 +627,17 @@ def run_long(args):
             fg.flat[0] = False
         return fg.astype(np.uint8)
 
-    specs = [("edt_2d_1024_b8", (8, 1, 1024, 1024), 20), ("edt_2d_4096_b1", (1, 1, 4096, 4096), 40),
-             ("edt_3d_512_b1", (1, 1, 512, 512, 512), 24)]
+    specs = [("edt_2d_1024_b8", (8, 1, 1024, 1024), 20, None), ("edt_2d_4096_b1", (1, 1, 4096, 4096), 40, None),
+             ("edt_3d_512_b1", (1, 1, 512, 512, 512), 24, None),
+             ("edt_3d_512_b1_sampling_2.5_0.8_1", (1, 1, 512, 512, 512), 24, (2.5, 0.8, 1.0))]
     cases = []
-    for k, (name, shape, count) in enumerate(specs):
+    for k, (name, shape, count, samp) in enumerate(specs):
         imgs = [blobs(100 * k + i, shape[2:], count) for i in range(shape[0])]
         mask = np.stack(imgs)[:, None]
         nvox = mask.size
         io = 5 * nvox
         sets = max(2, min(8, -(-2 * l2_bytes(dev) // io)))
-        calls = [binding.PreparedCall(torch.from_numpy(mask).to(dev), None,
+        calls = [binding.PreparedCall(torch.from_numpy(mask).to(dev), samp,
                                       torch.empty(mask.shape, dtype=torch.float32, device=dev), None, None)
                  for _ in range(sets)]
         for i in range(max(3, args.warmup)):
@@ -652,20 +653,20 @@ def run_long(args):
         times = sorted(a.elapsed_time(b) for a, b in evs)
         ms = statistics.median(times)
         c0 = calls[0]
-        _, ks = binding.tm_edt_profile(c0.mask, None, distances=c0.d, workspace=c0.ws, return_distances=True)
+        _, ks = binding.tm_edt_profile(c0.mask, samp, distances=c0.d, workspace=c0.ws, return_distances=True)
         # the oracle on the first image (its leading rows if the image alone would take minutes)
         one = mask[:1]
         rows = one.shape[2]
         t0 = time.perf_counter()
-        oracle.sep(np.ascontiguousarray(one[:, :, : max(2, rows // 8)]), None, want_idx=False)
+        oracle.sep(np.ascontiguousarray(one[:, :, : max(2, rows // 8)]), samp, want_idx=False)
         t_part = time.perf_counter() - t0
         keep = rows if t_part * 8 < 20 else max(2, int(rows / 8 * 20 / (t_part * 8)))
         part = np.ascontiguousarray(one[:, :, :keep])
         t0 = time.perf_counter()
-        oracle.sep(part, None, want_idx=False)
+        oracle.sep(part, samp, want_idx=False)
         cpu_s = time.perf_counter() - t0
         gbs = io / (ms * 1e-3) / 1e9
-        cases.append({"case": name, "shape": list(mask.shape), "ms_per_step": ms, "ms_min": times[0],
+        cases.append({"case": name, "shape": list(mask.shape), "sampling": samp, "ms_per_step": ms, "ms_min": times[0],
                       "value": nvox / (ms * 1e-3) / 1e9, "unit": UNIT, "inputs_per_ms": shape[0] / ms,
                       "gpu_launches_per_step": launches,
                       "kernels": [(n, round(t, 4)) for n, t, _ in ks],

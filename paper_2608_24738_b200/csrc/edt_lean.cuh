@@ -507,10 +507,10 @@ __global__ void __launch_bounds__(32 * NW) lean_value_kernel(const __grid_consta
             const uint2 w = *reinterpret_cast<const uint2*>(g);
             k = make_uint4(w.x & 0xffffu, w.x >> 16, w.y & 0xffffu, w.y >> 16);
             if (P.dist16) {
-                k.x = k.x >= 0xC000u ? kLeanNone : k.x * k.x;
-                k.y = k.y >= 0xC000u ? kLeanNone : k.y * k.y;
-                k.z = k.z >= 0xC000u ? kLeanNone : k.z * k.z;
-                k.w = k.w >= 0xC000u ? kLeanNone : k.w * k.w;
+                k.x = k.x >= 0xC000u ? kLeanNone : k.x * k.x * P.w0;  // (w0: 1, or the integer weight of scaled sampling)
+                k.y = k.y >= 0xC000u ? kLeanNone : k.y * k.y * P.w0;
+                k.z = k.z >= 0xC000u ? kLeanNone : k.z * k.z * P.w0;
+                k.w = k.w >= 0xC000u ? kLeanNone : k.w * k.w * P.w0;
             } else {
                 if (k.x == 0xffffu) k.x = kLeanNone;
                 if (k.y == 0xffffu) k.y = kLeanNone;

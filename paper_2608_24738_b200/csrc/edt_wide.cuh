@@ -25,6 +25,7 @@ struct WideParams {
     int64_t rows;        // images * n1
     int n0, n1;
     float w2x;           // squared sampling of the contiguous axis (float-height variant)
+    uint32_t w0i;        // its integer weight (plain integer heights of the long-line path; 1 under unit sampling)
 };
 
 // SH > 0: integer keys (off^2 << SH | row).  SH == 0: the plain integer off^2 (no site is needed afterwards: no index

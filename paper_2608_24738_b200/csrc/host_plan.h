@@ -34,6 +34,9 @@ struct Plan {
     bool scaled = false;      // fast path in exact integers: scale * w^2 is an integer for every processed axis
     int si[kMaxDims];         // those integers
     double scale = 1.0;
+    bool vscaled = false;     // wide-key / long-line shapes, distances only: the value kernels in exact scaled integers
+    int vsi[kMaxDims];        // scale * w^2 per processed axis
+    double vscale = 1.0;
     bool wide_keys = false;      // unit sampling, contiguous extent % 16 == 0: two axes <= 1024 or three axes <= 512
     size_t ws_bytes = 0;
     size_t plane_bytes = 0;   // bytes of one offset plane, rounded up to 256
@@ -68,6 +71,7 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
 // One axis pass of the wide-key path on plain integer values with the quad kernels (see tm_edt_lean.cu).
 bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
 bool lean_value_long_axis_ok(const Plan& pl, int k, const EpilogueParams& ep);
+bool lean_value_all_axes_ok(const Plan& pl, const EpilogueParams& ep);
 cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,
                                      cudaStream_t st);
 cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out, const EpilogueParams& ep, bool fin,

@@ -177,10 +177,27 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
                     !force;
     if (pl.wide_keys || pl.long_lines) pl.ws_bytes = wide_layout(pl.N, E, want_idx, pl.long_lines).total;
     if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
+    static const int cand[] = {1, 4, 16, 25, 64, 100, 256, 400, 625, 1024, 2500, 10000};
+    if ((pl.wide_keys || pl.long_lines) && !pl.unit && !want_idx && pl.ext[0] % 4 == 0 && !sw.no_scaled) {
+        // the same search for the value kernels of the longer extents (no index output): plain 32-bit values, so the
+        // largest value and the largest addend of a scan (a few rows beyond the extent) must stay below 2^31
+        for (int S : cand) {
+            bool ok = true;
+            double total = 0.0, edge = 0.0;
+            for (int p = 0; p < E && ok; ++p) {
+                const double v = pl.w[p] * pl.w[p] * S, r = nearbyint(v);
+                if (r < 1.0 || r > 1048576.0 || fabs(v - r) > 1e-9 * v) { ok = false; break; }
+                pl.vsi[p] = (int)r;
+                total += r * (double)(pl.ext[p] - 1) * (double)(pl.ext[p] - 1);
+                const double e2 = r * (double)(pl.ext[p] + 8) * (double)(pl.ext[p] + 8);
+                edge = e2 > edge ? e2 : edge;
+            }
+            if (ok && total < 2147483648.0 && edge < 2147483648.0) { pl.vscaled = true; pl.vscale = S; break; }
+        }
+    }
     if (pl.fast && !pl.unit && pl.ext[0] % 4 == 0 && !sw.no_scaled) {
         // sampling given with a few decimals: look for a scale that makes every w^2 an integer and keeps
         // the largest possible value below 2^24 (keys are value << 7 | row in 32 bits)
-        static const int cand[] = {1, 4, 16, 25, 64, 100, 256, 400, 625, 1024, 2500, 10000};
         for (int S : cand) {
             bool ok = true;
             double total = 0.0, edge = 0.0;
@@ -678,13 +695,18 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     P.w2x = (float)(pl.w[0] * pl.w[0]);
+    P.w0i = 1u;
     const double out_bpv = out_bytes_per_voxel(ep);
     // integer keys carry 9 row bits up to extent 512 and 10 up to 1024 (two axes only); general sampling uses float
     // heights.  A lane of the row kernel takes 16 voxels (rows up to 512) or 32.
     int nmax = 1;
     for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
     // without an index output no site is needed afterwards: plain values as keys (sh = 0)
-    const int sh = !pl.unit ? -1 : (!carry ? 0 : (nmax > 512 ? 10 : 9));
+    // sampling whose squares share an integer scale, distances only: the value kernels run in exact scaled integers if
+    // the first pass can hand them 16-bit row distances and every axis pass fits them
+    const bool vs = !pl.unit && pl.vscaled && !carry && !switches().no_lean && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 &&
+                    ((uintptr_t)in & 31u) == 0 && lean_value_all_axes_ok(pl, ep);
+    const int sh = vs ? 0 : (!pl.unit ? -1 : (!carry ? 0 : (nmax > 512 ? 10 : 9)));
     // no index output, unit sampling: the first pass hands 16-bit row distances to the quad value kernel of the second axis
     const bool dist16 = sh == 0 && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 && ((uintptr_t)in & 31u) == 0 &&
                         !switches().no_lean && lean_value_axis_ok(pl, 1, ep);
@@ -761,6 +783,7 @@ static cudaError_t run_long(const Plan& pl, const uint8_t* in, const EpiloguePar
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     P.w2x = (float)(pl.w[0] * pl.w[0]);
+    P.w0i = pl.unit ? 1u : (uint32_t)pl.vsi[0];  // (integer heights under sampling: the scaled-integer value passes)
     const double out_bpv = out_bytes_per_voxel(ep);
     prof_mark(st, "long_row", (double)pl.N * (1.0 + 4.0 + (carry ? 2.0 : 0.0)));
     if (pl.ext[0] % 16 == 0 && ((uintptr_t)in & 15u) == 0) long_row_kernel<FLT><<<(unsigned)((P.rows + 7) / 8), 256, 0, st>>>(P);
@@ -921,8 +944,11 @@ static cudaError_t run_images(const Plan& pl, const uint8_t* input, float* out_d
     fill_epilogue(pl, out_dist, out_sq, out_idx, ep);
     if (pl.small) return ep.idx ? run_small<true>(pl, input, ep, ws, st, launches) : run_small<false>(pl, input, ep, ws, st, launches);
     if (pl.wide_keys) return run_wide(pl, input, ep, ws, st, launches);
-    if (pl.long_lines)
-        return pl.unit ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
+    if (pl.long_lines) {
+        // sampling with an integer scale, distances only, every axis pass on the value kernels: integer heights too
+        const bool ints = pl.unit || (pl.vscaled && !ep.idx && !switches().no_lean && lean_value_all_axes_ok(pl, ep));
+        return ints ? run_long<false>(pl, input, ep, ws, st, launches) : run_long<true>(pl, input, ep, ws, st, launches);
+    }
     if (!switches().no_lean && lean_ok(pl, input, ep)) return run_lean(pl, input, ep, ws, st, launches);
     if (pl.fast && pl.scaled && ((uintptr_t)input & 3u) == 0) return run_scaled(pl, input, ep, ws, st, launches);
     if (pl.fast)

@@ -160,7 +160,7 @@ static int lean_value_tile(const Plan& pl, int k) {
 }
 
 bool lean_value_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
-    if (!pl.unit || ep.idx || pl.ext[0] % 4 != 0) return false;
+    if ((!pl.unit && !pl.vscaled) || ep.idx || pl.ext[0] % 4 != 0) return false;
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
     return lean_value_tile(pl, k) != 0;
 }
@@ -171,8 +171,9 @@ cudaError_t run_lean_value_axis(const Plan& pl, int k, const void* in, void* out
     memset(&P, 0, sizeof(P));
     P.in = in; P.out = out;
     P.in_elems = pl.N; P.out_elems = pl.N; P.images = pl.images;
-    P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
-    P.inv_scale = 1.0f;
+    P.n = pl.ext[k]; P.inner = pl.inner[k];
+    P.wk = pl.unit ? 1u : (uint32_t)pl.vsi[k]; P.w0 = pl.unit ? 1u : (uint32_t)pl.vsi[0];  // (scaled sampling: integer weights)
+    P.inv_scale = pl.unit ? 1.0f : (float)(1.0 / pl.vscale);
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
     const int tx = lean_value_tile(pl, k);
     if (dist16) {  // 16-bit first-axis distances in; final outputs or 32-bit values out
@@ -205,7 +206,7 @@ static int lean_value_long_tile(int n) {
 }
 
 bool lean_value_long_axis_ok(const Plan& pl, int k, const EpilogueParams& ep) {
-    if (!pl.unit || ep.idx || pl.ext[0] % 4 != 0) return false;
+    if ((!pl.unit && !pl.vscaled) || ep.idx || pl.ext[0] % 4 != 0) return false;
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u)) return false;
     const int n = pl.ext[k], tx = lean_value_long_tile(n);
     if (n <= 1024 || tx == 0) return false;
@@ -230,8 +231,9 @@ cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void
     memset(&P, 0, sizeof(P));
     P.in = in; P.out = out;
     P.in_elems = pl.N; P.out_elems = pl.N; P.images = pl.images;
-    P.n = pl.ext[k]; P.inner = pl.inner[k]; P.wk = 1u; P.w0 = 1u;
-    P.inv_scale = 1.0f;
+    P.n = pl.ext[k]; P.inner = pl.inner[k];
+    P.wk = pl.unit ? 1u : (uint32_t)pl.vsi[k]; P.w0 = pl.unit ? 1u : (uint32_t)pl.vsi[0];  // (scaled sampling: integer weights)
+    P.inv_scale = pl.unit ? 1.0f : (float)(1.0 / pl.vscale);
     const int64_t outer = pl.N / ((int64_t)pl.ext[k] * pl.inner[k]);
     const int tx = lean_value_long_tile(P.n);
     if (tx == 16)
@@ -239,6 +241,13 @@ cudaError_t run_lean_value_long_axis(const Plan& pl, int k, const void* in, void
     if (tx == 8)
         return fin ? launch_lean_value_long<true, 8>(P, ep, outer, st) : launch_lean_value_long<false, 8>(P, ep, outer, st);
     return fin ? launch_lean_value_long<true, 4>(P, ep, outer, st) : launch_lean_value_long<false, 4>(P, ep, outer, st);
+}
+
+// every axis pass after the first on one of the two forms above
+bool lean_value_all_axes_ok(const Plan& pl, const EpilogueParams& ep) {
+    for (int k = 1; k < pl.E; ++k)
+        if (!lean_value_axis_ok(pl, k, ep) && !lean_value_long_axis_ok(pl, k, ep)) return false;
+    return pl.E >= 2;
 }
 
 cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep, void* ws, cudaStream_t st, int& launches) {

@@ -343,6 +343,42 @@ def test_single_images_on_narrow_tiles(shape, switches):
         assert np.array_equal(old["sq"], res["sq"])
 
 
+DECIMAL = [((4, 1, 512, 512), (0.8, 1.0), 2), ((2, 1, 300, 1024), (2.5, 1.0), 2), ((1, 1, 140, 40, 160), (2.5, 0.8, 1.0), 3),
+           ((1, 1, 400, 24, 32), (1.25, 0.5, 2.0), 3), ((1, 1, 1024, 1024), (1.5, 0.5), 2), ((1, 1, 1100, 2400), (1.5, 0.5), 2),
+           ((1, 1, 4096, 1184), (0.8, 1.0), 2), ((1, 1, 8192, 592), (1.0, 2.5), 2), ((1, 1, 1500, 40, 64), (2.0, 1.0, 0.5), 3),
+           ((1, 1, 8192, 592), (1.0, 0.3), 3), ((2, 1, 200, 1000), (0.8, 1.0), 2)]
+
+
+@pytest.mark.parametrize("shape,sampling,launches", DECIMAL,
+                         ids=["x".join(map(str, s)) + "_" + "_".join(map(str, w)) for s, w, _ in DECIMAL])
+def test_decimal_sampling_beyond_128_without_indices(shape, sampling, launches, switches):
+    """Sampling whose squares share an integer scale, distances only, extents beyond 128: the value kernels run in exact
+    scaled integers (16-bit row distances or integer heights first), on every tile width; a scale that would overflow 32
+    bits (the last but one case) and rows that are no multiple of 32 voxels (the last) stay on float heights.  Against the
+    oracle, and against the float-height path."""
+    seed = zlib.crc32(repr((shape, sampling)).encode())
+    rng = np.random.default_rng(seed)
+    blobs = workloads.random_mask(seed, shape, 0.998)
+    sp = shape[2:]
+    for _ in range(5):
+        lo = [int(rng.integers(0, n)) for n in sp]
+        blobs[(slice(None), slice(None)) + tuple(slice(l, l + max(2, n // 4)) for l, n in zip(lo, sp))] = 0
+    sparse = np.ones(shape, dtype=np.uint8)
+    for _ in range(4):
+        sparse[(0, 0) + tuple(int(rng.integers(0, n)) for n in sp)] = 0
+    if shape[0] > 1:
+        sparse[-1] = 1  # an image without background
+    for mask in (workloads.random_mask(seed + 1, shape, 0.9), blobs, sparse):
+        ref = oracle.sep(mask, sampling, want_idx=False)
+        res = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
+        assert binding.tm_edt_last_launch_count() == launches
+        checker.check_dist(res["dist"], ref["dist"])
+        switches.set("TM_EDT_NO_SCALED", "1")
+        old = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
+        switches.set("TM_EDT_NO_SCALED", None)
+        checker.check_dist(old["dist"], ref["dist"])
+
+
 def test_sparse_background_long_axis_exactness():
     """Few background voxels and large extents: squared distances up to ~1e7 must stay exact."""
     mask = np.ones((1, 1, 2048, 300), dtype=np.uint8)
