@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(256) long_row_any_kernel(const __grid_constant
             if (P.offs) P.offs[row * n0 + x] = row_has_zero ? (int16_t)(dl <= dr ? -a : a) : (int16_t)-32768;
             P.keys[row * n0 + x] = !row_has_zero ? (FLT ? kLongNoneFlt : kLongNoneInt)
                                                  : (FLT ? __float_as_uint(__fmul_rn(P.w2x, (float)(a * a)))
-                                                        : ((((uint32_t)(a * a) * (SH == -2 ? P.w0i : 1u)) << (SH > 0 ? SH : 0)) | yrow));
+                                                        : ((((uint32_t)(a * a) * (SH == -2 || SH == 0 ? P.w0i : 1u)) << (SH > 0 ? SH : 0)) | yrow));
         }
         if (word) carry_l = 32 * b + 31 - __clz(word);
     }

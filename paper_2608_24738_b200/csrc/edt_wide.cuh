@@ -25,7 +25,7 @@ struct WideParams {
     int64_t rows;        // images * n1
     int n0, n1;
     float w2x;           // squared sampling of the contiguous axis (float-height variant)
-    uint32_t w0i;        // its integer weight (plain integer heights of the long-line path; 1 under unit sampling)
+    uint32_t w0i;        // its integer weight (plain integer values, SH == 0 or the long-line path; 1 under unit sampling)
 };
 
 // SH > 0: integer keys (off^2 << SH | row).  SH == 0: the plain integer off^2 (no site is needed afterwards: no index
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(256) row_keys_kernel(const __grid_constant__ W
             const int dr = cur - (x0 + b);
             const int a = min(dl[b], dr);
             offs[b] = (int16_t)(dl[b] <= dr ? -a : a);
-            keys[b] = SH < 0 ? __float_as_uint(P.w2x * (float)(a * a)) : (SH == 0 ? (uint32_t)(a * a) : (((uint32_t)(a * a) << (SH < 0 ? 0 : SH)) | (uint32_t)y));
+            keys[b] = SH < 0 ? __float_as_uint(P.w2x * (float)(a * a)) : (SH == 0 ? (uint32_t)(a * a) * P.w0i : (((uint32_t)(a * a) << (SH < 0 ? 0 : SH)) | (uint32_t)y));
         }
     }
 #pragma unroll

@@ -695,7 +695,7 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     P.n0 = pl.ext[0]; P.n1 = pl.ext[1];
     P.rows = pl.N / pl.ext[0];
     P.w2x = (float)(pl.w[0] * pl.w[0]);
-    P.w0i = 1u;
+    P.w0i = 1u;  // (set below for scaled sampling)
     const double out_bpv = out_bytes_per_voxel(ep);
     // integer keys carry 9 row bits up to extent 512 and 10 up to 1024 (two axes only); general sampling uses float
     // heights.  A lane of the row kernel takes 16 voxels (rows up to 512) or 32.
@@ -703,10 +703,10 @@ static cudaError_t run_wide(const Plan& pl, const uint8_t* in, const EpiloguePar
     for (int p = 0; p < pl.E; ++p) nmax = pl.ext[p] > nmax ? pl.ext[p] : nmax;
     // without an index output no site is needed afterwards: plain values as keys (sh = 0)
     // sampling whose squares share an integer scale, distances only: the value kernels run in exact scaled integers if
-    // the first pass can hand them 16-bit row distances and every axis pass fits them
-    const bool vs = !pl.unit && pl.vscaled && !carry && !switches().no_lean && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 &&
-                    ((uintptr_t)in & 31u) == 0 && lean_value_all_axes_ok(pl, ep);
+    // every axis pass fits them (the first pass hands them 16-bit row distances or weighted integer values)
+    const bool vs = !pl.unit && pl.vscaled && !carry && !switches().no_lean && lean_value_all_axes_ok(pl, ep);
     const int sh = vs ? 0 : (!pl.unit ? -1 : (!carry ? 0 : (nmax > 512 ? 10 : 9)));
+    if (vs) P.w0i = (uint32_t)pl.vsi[0];
     // no index output, unit sampling: the first pass hands 16-bit row distances to the quad value kernel of the second axis
     const bool dist16 = sh == 0 && pl.ext[0] % 32 == 0 && pl.ext[0] <= 1024 && ((uintptr_t)in & 31u) == 0 &&
                         !switches().no_lean && lean_value_axis_ok(pl, 1, ep);

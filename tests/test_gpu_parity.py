@@ -346,7 +346,8 @@ def test_single_images_on_narrow_tiles(shape, switches):
 DECIMAL = [((4, 1, 512, 512), (0.8, 1.0), 2), ((2, 1, 300, 1024), (2.5, 1.0), 2), ((1, 1, 140, 40, 160), (2.5, 0.8, 1.0), 3),
            ((1, 1, 400, 24, 32), (1.25, 0.5, 2.0), 3), ((1, 1, 1024, 1024), (1.5, 0.5), 2), ((1, 1, 1100, 2400), (1.5, 0.5), 2),
            ((1, 1, 4096, 1184), (0.8, 1.0), 2), ((1, 1, 8192, 592), (1.0, 2.5), 2), ((1, 1, 1500, 40, 64), (2.0, 1.0, 0.5), 3),
-           ((1, 1, 8192, 592), (1.0, 0.3), 3), ((2, 1, 200, 1000), (0.8, 1.0), 2)]
+           ((1, 1, 8192, 592), (1.0, 0.3), 3), ((2, 1, 200, 1000), (0.8, 1.0), 2),
+           ((12, 1, 300, 1000), (0.8, 1.0), 2), ((12, 1, 300, 1008), (2.5, 1.0), 2), ((12, 1, 300, 496), (1.0, 0.5), 2)]
 
 
 @pytest.mark.parametrize("shape,sampling,launches", DECIMAL,
@@ -354,8 +355,9 @@ DECIMAL = [((4, 1, 512, 512), (0.8, 1.0), 2), ((2, 1, 300, 1024), (2.5, 1.0), 2)
 def test_decimal_sampling_beyond_128_without_indices(shape, sampling, launches, switches):
     """Sampling whose squares share an integer scale, distances only, extents beyond 128: the value kernels run in exact
     scaled integers (16-bit row distances or integer heights first), on every tile width; a scale that would overflow 32
-    bits (the last but one case) and rows that are no multiple of 32 voxels (the last) stay on float heights.  Against the
-    oracle, and against the float-height path."""
+    bits, or too few tiles for the value kernel, stay on float heights; rows that are no multiple of 32 voxels get their
+    weighted integer values from the other first-axis kernels (the last three cases).  Against the oracle, and against
+    the float-height path."""
     seed = zlib.crc32(repr((shape, sampling)).encode())
     rng = np.random.default_rng(seed)
     blobs = workloads.random_mask(seed, shape, 0.998)
