@@ -178,9 +178,10 @@ static int make_plan(int ndim, const int64_t* shape, const double* sampling, Pla
     if (pl.wide_keys || pl.long_lines) pl.ws_bytes = wide_layout(pl.N, E, want_idx, pl.long_lines).total;
     if (pl.small) pl.ws_bytes = E > 1 ? 4 * ((((size_t)pl.N * 4) + 255) & ~(size_t)255) : 0;  // 2 value + 2 site buffers
     static const int cand[] = {1, 4, 16, 25, 64, 100, 256, 400, 625, 1024, 2500, 10000};
-    if ((pl.wide_keys || pl.long_lines) && !pl.unit && !want_idx && pl.ext[0] % 4 == 0 && !sw.no_scaled) {
-        // the same search for the value kernels of the longer extents (no index output): plain 32-bit values, so the
-        // largest value and the largest addend of a scan (a few rows beyond the extent) must stay below 2^31
+    if ((pl.wide_keys || pl.long_lines || pl.fast) && !pl.unit && !want_idx && pl.ext[0] % 4 == 0 && !sw.no_scaled) {
+        // a scale for the value-carrying kernels (no index output; the longer extents, and the quad kernels of the
+        // packed-entry shapes when the narrower search below fails): plain 32-bit values, so the largest value and the
+        // largest addend of a scan (a few rows beyond the extent) must stay below 2^31
         for (int S : cand) {
             bool ok = true;
             double total = 0.0, edge = 0.0;

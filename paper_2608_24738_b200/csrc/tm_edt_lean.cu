@@ -41,7 +41,7 @@ bool lean_ok(const Plan& pl, const uint8_t* in, const EpilogueParams& ep) {
     if (!pl.fast || pl.E < 3 || pl.E > 4 || pl.ext[0] % 4 != 0 || ((uintptr_t)in & 3u) != 0) return false;
     if (((uintptr_t)ep.dist & 15u) || ((uintptr_t)ep.sq & 31u) || ((uintptr_t)ep.idx & 31u)) return false;
     if (ep.idx) return pl.unit && pl.ndim == pl.E;
-    return pl.unit || pl.scaled;
+    return pl.unit || pl.scaled || pl.vscaled;  // (vscaled: a scale that fits plain 32-bit values, no index output)
 }
 
 template <int VS, typename VT>
@@ -260,7 +260,7 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
     for (int p = 0; p < pl.E; ++p) sumsq += (double)(pl.ext[p] - 1) * (pl.ext[p] - 1);
     const bool v16 = !entries && pl.unit && sumsq < 65535.0;
     const double carry = entries ? 2.0 : (v16 ? 2.0 : 4.0);  // bytes per voxel the plane kernel writes
-    auto weight = [&](int p) { return pl.unit ? 1u : (uint32_t)pl.si[p]; };
+    auto weight = [&](int p) { return pl.unit ? 1u : (uint32_t)(pl.scaled ? pl.si[p] : pl.vsi[p]); };
     LeanParams P;
     memset(&P, 0, sizeof(P));
     P.in = in; P.out = bufA;
@@ -272,7 +272,7 @@ cudaError_t run_lean(const Plan& pl, const uint8_t* in, const EpilogueParams& ep
 #endif
     P.n0 = pl.ext[0]; P.n = pl.ext[1]; P.inner = pl.inner[1];
     P.w0 = weight(0); P.wk = weight(1);
-    P.inv_scale = (float)(1.0 / pl.scale);
+    P.inv_scale = (float)(1.0 / (pl.unit || pl.scaled ? pl.scale : pl.vscale));
     for (int q = 0; q < 4; ++q) {
         P.shift[q] = -1;
         if (q < pl.E)

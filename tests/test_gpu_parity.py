@@ -748,13 +748,17 @@ VALUE_SHAPES = [(2, 1, 12, 20, 24), (1, 2, 33, 17, 40), (1, 1, 128, 20, 48), (2,
 
 
 @pytest.mark.parametrize("shape", VALUE_SHAPES, ids=["x".join(map(str, s)) for s in VALUE_SHAPES])
-@pytest.mark.parametrize("kind", ["unit", "decimal", "sampled"])
+@pytest.mark.parametrize("kind", ["unit", "decimal", "two_decimals", "sampled"])
 def test_outputs_without_indices(shape, kind, switches):
     """Without an index output the packed-entry path carries squared distances instead of offsets (16-bit values up to
     four axes, 32-bit beyond and in scaled-integer mode).  Distances and exact squared distances against the oracle,
     and bit-identical to what the offset-carrying kernels give."""
     ndim = len(shape) - 2
-    sampling = None if kind == "unit" else (tuple([2.5, 0.8, 1.0, 1.25, 0.5][:ndim]) if kind == "decimal" else _sampling(ndim, "sampled"))
+    # "two_decimals": squares with a common scale of 10000, beyond the 24 bits of the index-carrying keys but within
+    # the 31 bits of plain values
+    sampling = None if kind == "unit" else (tuple([2.5, 0.8, 1.0, 1.25, 0.5][:ndim]) if kind == "decimal" else
+                                            (tuple([0.37, 0.8, 3.3, 1.25, 0.48][:ndim]) if kind == "two_decimals"
+                                             else _sampling(ndim, "sampled")))
     unit = sampling is None
     for p_fg in (0.6, 0.98):
         mask = workloads.random_mask(zlib.crc32(repr((shape, kind, p_fg, "val")).encode()), shape, p_fg)
@@ -769,5 +773,7 @@ def test_outputs_without_indices(shape, kind, switches):
         switches.set("TM_EDT_NO_VALUE_CARRY", "1")
         old = run_gpu(mask, sampling, dist=True, sq=False, idx=False)
         switches.set("TM_EDT_NO_VALUE_CARRY", None)
-        if kind != "sampled":  # integer paths: the same values either way
+        if kind in ("unit", "decimal"):  # integer paths: the same values either way
             assert np.array_equal(res["dist"], old["dist"])
+        else:
+            checker.check_dist(old["dist"], ref["dist"])
